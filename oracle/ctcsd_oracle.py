@@ -1,0 +1,348 @@
+"""CPU oracle for the CTC-drafted draft-and-verify step.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, fp64/int64 restatement of what one decoding step computes, written from
+the paper's definitions so that it can be checked against them by eye.  It shares no
+code with the CUDA path and must never be imported by it: only the tests, the smoke
+check and the benchmark's CPU-baseline leg may call into this file.
+
+Each function names the passage it follows.  Notation is the paper's: T draft slots
+("places"), blank symbol (the paper's epsilon) with id V, alignment a = (a_1..a_T),
+beta^{-1} the collapse map, Y the collapsed candidate.
+
+Pins (see tests/test_oracle_pins.py): every function below is pinned by something other
+than itself - hand-worked collapse cases, the total-mass closed form, the Graves forward
+recursion (torch's ctc_loss and an independent alpha recursion), library matmul /
+log-softmax / top-k / scaled-dot-product attention in fp64, and brute-force tries and
+acceptance definitions.  The finite-beam prefix search is a heuristic the paper does not
+specify ("a group of the most valuable combinations are reserved", Sec. 3.3): with a beam
+that never prunes it is pinned to exact enumeration; with a pruning beam it is pinned only
+by bounds (candidate subset, score <= exact) - beyond that: parity unpinned.
+"""
+from __future__ import annotations
+
+import itertools
+import math
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+NEG_INF = float("-inf")
+
+
+# --------------------------------------------------------------------------------------
+# S1  draft head: per-slot logits (Sec. 3.2, "Softmax(LmHead(F_hat))" gives one
+#     distribution per place; here the projection is a linear head over V+1 classes)
+# --------------------------------------------------------------------------------------
+def draft_logits(x: np.ndarray, Wd: np.ndarray, blank_bias: Optional[np.ndarray] = None,
+                 row_seq: Optional[np.ndarray] = None) -> np.ndarray:
+    """z[m,t,v] = sum_h x[m,h] * Wd[t,v,h]; the blank class v = V additionally gets
+    blank_bias[row_seq[m]].  x [M,H], Wd [T,V+1,H] -> z [M,T,V+1] in fp64."""
+    x64 = np.asarray(x, dtype=np.float64)
+    M = x64.shape[0]
+    T, V1, _ = Wd.shape
+    z = np.empty((M, T, V1), dtype=np.float64)
+    for t in range(T):
+        z[:, t, :] = x64 @ np.asarray(Wd[t], dtype=np.float64).T
+    if blank_bias is not None:
+        for m in range(M):
+            s = m if row_seq is None else int(row_seq[m])
+            z[m, :, V1 - 1] += float(blank_bias[s])
+    return z
+
+
+# --------------------------------------------------------------------------------------
+# S2  per-slot log-softmax (Sec. 3.2: P_hat = Softmax(...), one distribution per place)
+# --------------------------------------------------------------------------------------
+def log_softmax_slots(z: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """lse[m,t] = log sum_v exp z[m,t,v];  lp = z - lse."""
+    z = np.asarray(z, dtype=np.float64)
+    mx = z.max(axis=-1, keepdims=True)
+    lse = mx + np.log(np.exp(z - mx).sum(axis=-1, keepdims=True))
+    return lse[..., 0], z - lse
+
+
+# --------------------------------------------------------------------------------------
+# S3  per-slot top-k (Sec. 3.3: "For every position, the top k tokens are selected in
+#     descending order of probability"); blank is eligible; ties go to the lower id
+# --------------------------------------------------------------------------------------
+def topk_slots(z: np.ndarray, k: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Returns (topk_id [M,T,k] int64, topk_lp [M,T,k] fp64) with lp = z - lse."""
+    z = np.asarray(z, dtype=np.float64)
+    lse, _ = log_softmax_slots(z)
+    order = np.argsort(-z, axis=-1, kind="stable")[..., :k]   # stable: equal values keep id order
+    vals = np.take_along_axis(z, order, axis=-1)
+    return order.astype(np.int64), vals - lse[..., None]
+
+
+# --------------------------------------------------------------------------------------
+# S5  CTC collapse beta^{-1} (Sec. 2.3: "merging adjacent, repeated tokens and removing
+#     blanks"; Sec. 3.1: "removes consecutive duplicate tokens and blank character")
+# --------------------------------------------------------------------------------------
+def ctc_collapse(a: Sequence[int], blank: int) -> Tuple[int, ...]:
+    out: List[int] = []
+    prev = None
+    for s in a:
+        s = int(s)
+        if s != prev and s != blank:      # compared with the previous RAW symbol, blank included
+            out.append(s)
+        prev = s
+    return tuple(out)
+
+
+def _logaddexp(a: float, b: float) -> float:
+    if a == NEG_INF:
+        return b
+    if b == NEG_INF:
+        return a
+    hi, lo = (a, b) if a >= b else (b, a)
+    return hi + math.log1p(math.exp(lo - hi))
+
+
+# --------------------------------------------------------------------------------------
+# S4 + S6  enumerate every slot path, score it (Eq. 6: P(A) = prod_t p(a_t)), collapse it,
+#          and give each distinct collapsed sequence the sum over its alignments
+#          (Eq. 1 / Eq. 5: P(Y) = sum_{A in beta(Y)} P(A))
+# --------------------------------------------------------------------------------------
+def enumerate_candidates(topk_id: np.ndarray, topk_lp: np.ndarray, blank: int,
+                         score_mode: int = 0) -> Dict[Tuple[int, ...], float]:
+    """topk_id, topk_lp: [T,k] for one drafting row.  Returns {collapsed sequence: log score},
+    the empty sequence included.  score_mode 0: log sum exp over alignments; 1: best alignment."""
+    T, k = topk_id.shape
+    groups: Dict[Tuple[int, ...], List[float]] = {}
+    for a in itertools.product(range(k), repeat=T):
+        s = 0.0
+        for t in range(T):
+            s += float(topk_lp[t, a[t]])
+        y = ctc_collapse([int(topk_id[t, a[t]]) for t in range(T)], blank)
+        groups.setdefault(y, []).append(s)
+    out: Dict[Tuple[int, ...], float] = {}
+    for y, ss in groups.items():
+        m = max(ss)
+        if score_mode == 1:
+            out[y] = m
+        else:
+            out[y] = m + math.log(sum(math.exp(s - m) for s in ss))
+    return out
+
+
+def order_o1(item: Tuple[Tuple[int, ...], float]):
+    """Total order on candidates: score descending, then shorter first, then token ids
+    lexicographically ascending (the paper is silent on ties)."""
+    y, score = item
+    return (-score, len(y), y)
+
+
+# --------------------------------------------------------------------------------------
+# S7  keep the N best non-empty candidates (Sec. 3.3: "a group of the most valuable
+#     combinations are reserved")
+# --------------------------------------------------------------------------------------
+def select_top_n(cands: Dict[Tuple[int, ...], float], N: int) -> List[Tuple[Tuple[int, ...], float]]:
+    items = [(y, s) for y, s in cands.items() if len(y) > 0]
+    items.sort(key=order_o1)
+    return items[:N]
+
+
+def selection_margin(cands: Dict[Tuple[int, ...], float], N: int) -> float:
+    """Smallest score gap that the top-N selection relied on: between adjacent kept
+    candidates and between the last kept and the first dropped one (inf if none)."""
+    items = [(y, s) for y, s in cands.items() if len(y) > 0]
+    items.sort(key=order_o1)
+    gaps = [items[i][1] - items[i + 1][1] for i in range(min(N, len(items) - 1))]
+    return min(gaps) if gaps else float("inf")
+
+
+# --------------------------------------------------------------------------------------
+# S4'  CTC prefix beam search restricted to each slot's top-k symbols.  The paper gives no
+#      pruning rule; this is the textbook prefix search (probability mass of a prefix split
+#      into alignments ending in blank / ending in its last token), pruned to `beam`
+#      prefixes after every slot.
+# --------------------------------------------------------------------------------------
+def prefix_beam_candidates(topk_id: np.ndarray, topk_lp: np.ndarray, blank: int, beam: int,
+                           stats: Optional[dict] = None) -> Dict[Tuple[int, ...], float]:
+    """Returns {prefix: log(pb + pnb)} for the prefixes alive after the last slot."""
+    T, k = topk_id.shape
+    cur: Dict[Tuple[int, ...], Tuple[float, float]] = {(): (0.0, NEG_INF)}   # (log pb, log pnb)
+    min_cut_gap = float("inf")
+    for t in range(T):
+        nxt: Dict[Tuple[int, ...], List[float]] = {}
+
+        def acc(prefix, which, val):
+            if val == NEG_INF:                              # no alignment reaches it: not a prefix
+                return
+            e = nxt.setdefault(prefix, [NEG_INF, NEG_INF])
+            e[which] = _logaddexp(e[which], val)
+
+        for prefix, (pb, pnb) in cur.items():
+            tot = _logaddexp(pb, pnb)
+            for j in range(k):
+                s = int(topk_id[t, j])
+                p = float(topk_lp[t, j])
+                if s == blank:
+                    acc(prefix, 0, tot + p)                 # stays, now ends in blank
+                elif len(prefix) > 0 and s == prefix[-1]:
+                    acc(prefix, 1, pnb + p)                 # repeat merges into the same prefix
+                    acc(prefix + (s,), 1, pb + p)           # a blank in between starts a new token
+                else:
+                    acc(prefix + (s,), 1, tot + p)
+        ranked = sorted(((y, _logaddexp(e[0], e[1])) for y, e in nxt.items()),
+                        key=lambda it: (-it[1], len(it[0]), it[0]))
+        if len(ranked) > beam:
+            min_cut_gap = min(min_cut_gap, ranked[beam - 1][1] - ranked[beam][1])
+        cur = {y: (nxt[y][0], nxt[y][1]) for y, _ in ranked[:beam]}
+    if stats is not None:
+        stats["min_cut_gap"] = min_cut_gap
+    return {y: _logaddexp(pb, pnb) for y, (pb, pnb) in cur.items()}
+
+
+def topk_collapse(topk_id: np.ndarray, topk_lp: np.ndarray, blank: int, T: int, N: int,
+                  beam: int = 0, score_mode: int = 0, sel_row: Optional[np.ndarray] = None,
+                  B: Optional[int] = None, stats: Optional[dict] = None):
+    """S4-S7 for a batch.  topk_id/topk_lp: [M,T,k]; sequence b drafts from row sel_row[b]
+    (default b).  Returns cand_tok [B,N,T] (pad -1), cand_len [B,N], cand_score [B,N]
+    (pad -inf), n_cand [B]."""
+    M = topk_id.shape[0]
+    B = M if B is None else B
+    cand_tok = np.full((B, N, T), -1, dtype=np.int64)
+    cand_len = np.zeros((B, N), dtype=np.int64)
+    cand_score = np.full((B, N), NEG_INF, dtype=np.float64)
+    n_cand = np.zeros((B,), dtype=np.int64)
+    margins = []
+    for b in range(B):
+        r = b if sel_row is None else int(sel_row[b])
+        st: dict = {}
+        if beam > 0:
+            cands = prefix_beam_candidates(topk_id[r], topk_lp[r], blank, beam, st)
+        else:
+            cands = enumerate_candidates(topk_id[r], topk_lp[r], blank, score_mode)
+        margins.append(min(selection_margin(cands, N), st.get("min_cut_gap", float("inf"))))
+        kept = select_top_n(cands, N)
+        n_cand[b] = len(kept)
+        for c, (y, s) in enumerate(kept):
+            cand_len[b, c] = len(y)
+            cand_tok[b, c, :len(y)] = y
+            cand_score[b, c] = s
+    if stats is not None:
+        stats["margin"] = margins
+    return cand_tok, cand_len, cand_score, n_cand
+
+
+# --------------------------------------------------------------------------------------
+# S8  token tree (Sec. 2.2: candidates are root-to-leaf paths of a tree verified in one
+#     pass under a tree attention mask; Sec. 3.3: the base token precedes the drafts)
+# --------------------------------------------------------------------------------------
+def build_tree(base_tok: np.ndarray, kv_len: np.ndarray, cand_tok: np.ndarray,
+               cand_len: np.ndarray, n_cand: np.ndarray, n_max: int):
+    """Prefix trie of the ranked candidates under a root that holds the base token.
+    Nodes are numbered in order of first appearance while walking candidates by rank and
+    each candidate left to right; a new node is made only while fewer than n_max exist.
+    mask bit j of row i is set iff j is i or an ancestor of i."""
+    B, N, T = cand_tok.shape
+    W = (n_max + 63) // 64
+    node_tok = np.full((B, n_max), -1, dtype=np.int64)
+    parent = np.full((B, n_max), -1, dtype=np.int64)
+    depth = np.zeros((B, n_max), dtype=np.int64)
+    pos = np.zeros((B, n_max), dtype=np.int64)
+    mask = np.zeros((B, n_max, W), dtype=np.uint64)
+    retrieve = np.full((B, N, T), -1, dtype=np.int64)
+    n_nodes = np.zeros((B,), dtype=np.int64)
+    for b in range(B):
+        node_of: Dict[Tuple[int, ...], int] = {(): 0}
+        node_tok[b, 0] = int(base_tok[b])
+        n = 1
+        for c in range(int(n_cand[b])):
+            for l in range(1, int(cand_len[b, c]) + 1):
+                pre = tuple(int(v) for v in cand_tok[b, c, :l])
+                if pre not in node_of:
+                    if pre[:-1] not in node_of or n >= n_max:
+                        break                                  # budget hit: rest of this candidate is dropped
+                    node_of[pre] = n
+                    node_tok[b, n] = pre[-1]
+                    parent[b, n] = node_of[pre[:-1]]
+                    depth[b, n] = l
+                    n += 1
+                retrieve[b, c, l - 1] = node_of[pre]
+        n_nodes[b] = n
+        for i in range(n):
+            pos[b, i] = int(kv_len[b]) + depth[b, i]
+            j = i
+            while j >= 0:
+                mask[b, i, j // 64] |= np.uint64(1) << np.uint64(j % 64)
+                j = int(parent[b, j])
+    return node_tok, parent, depth, pos, mask, retrieve, n_nodes
+
+
+# --------------------------------------------------------------------------------------
+# S9  tree attention: plain softmax(q k^T / sqrt(d)) v over the cached prefix (all
+#     visible) and the tree nodes allowed by the ancestor mask (Sec. 2.2, Sec. 3.3)
+# --------------------------------------------------------------------------------------
+def tree_attention(Q: np.ndarray, K: np.ndarray, Vc: np.ndarray, kv_len: np.ndarray,
+                   n_nodes: np.ndarray, mask: np.ndarray, scale: float) -> np.ndarray:
+    """Q [B,n_max,Hq,D]; K,Vc [B,Hkv,Lcap,D] with node j's key/value at row kv_len[b]+j.
+    Query head h reads kv head h // (Hq/Hkv).  Returns O [B,n_max,Hq,D] fp64 (dead rows 0)."""
+    B, n_max, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    grp = Hq // Hkv
+    O = np.zeros((B, n_max, Hq, D), dtype=np.float64)
+    for b in range(B):
+        L, n = int(kv_len[b]), int(n_nodes[b])
+        for h in range(Hq):
+            Kh = np.asarray(K[b, h // grp, :L + n], dtype=np.float64)
+            Vh = np.asarray(Vc[b, h // grp, :L + n], dtype=np.float64)
+            for i in range(n):
+                q = np.asarray(Q[b, i, h], dtype=np.float64)
+                s = (Kh @ q) * scale
+                vis = np.ones(L + n, dtype=bool)
+                for j in range(n):
+                    bit = (int(mask[b, i, j // 64]) >> (j % 64)) & 1
+                    vis[L + j] = bool(bit)
+                s = np.where(vis, s, NEG_INF)
+                p = np.exp(s - s.max())
+                p /= p.sum()
+                O[b, i, h] = p @ Vh
+    return O
+
+
+# --------------------------------------------------------------------------------------
+# S10  LM head and greedy token at every tree node (Eq. 3-4 form: argmax Softmax(LmHead(F)))
+# --------------------------------------------------------------------------------------
+def lm_head_argmax(hn: np.ndarray, Wl: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """y[m,v] = sum_h hn[m,h] Wl[v,h]; am[m] = argmax_v y[m,v] (lowest id on ties)."""
+    y = np.asarray(hn, dtype=np.float64) @ np.asarray(Wl, dtype=np.float64).T
+    return y, np.argmax(y, axis=1).astype(np.int64)
+
+
+def argmax_rows(y: np.ndarray) -> np.ndarray:
+    return np.argmax(np.asarray(y, dtype=np.float64), axis=1).astype(np.int64)
+
+
+# --------------------------------------------------------------------------------------
+# S11  greedy acceptance (Sec. 2.2: only sequences matching the target model's greedy
+#      output are accepted; Sec. 3.3: the longest such sequence is the step's output)
+# --------------------------------------------------------------------------------------
+def greedy_accept(node_tok: np.ndarray, parent: np.ndarray, n_nodes: np.ndarray,
+                  am: np.ndarray, T: int):
+    """am [B,n_max]: base model's greedy token after each node.  Walk down from the root:
+    move to the child whose token equals am[current]; stop when no child matches.
+    Returns acc_len [B], acc_nodes [B,T] (pad -1), acc_tok [B,T] (pad -1), next_tok [B]."""
+    B = node_tok.shape[0]
+    acc_len = np.zeros((B,), dtype=np.int64)
+    acc_nodes = np.full((B, T), -1, dtype=np.int64)
+    acc_tok = np.full((B, T), -1, dtype=np.int64)
+    next_tok = np.zeros((B,), dtype=np.int64)
+    for b in range(B):
+        cur = 0
+        while True:
+            want = int(am[b, cur])
+            nxt = -1
+            for c in range(int(n_nodes[b])):
+                if int(parent[b, c]) == cur and int(node_tok[b, c]) == want:
+                    nxt = c
+                    break
+            if nxt < 0 or acc_len[b] >= T:
+                break
+            acc_nodes[b, acc_len[b]] = nxt
+            acc_tok[b, acc_len[b]] = want
+            acc_len[b] += 1
+            cur = nxt
+        next_tok[b] = int(am[b, cur])
+    return acc_len, acc_nodes, acc_tok, next_tok

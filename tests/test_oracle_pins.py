@@ -1,0 +1,426 @@
+"""Pins for the CPU oracle: each part is checked against something the paper or the
+mathematics fixes (hand-worked cases, closed forms, library routines, a different
+algorithm for the same quantity), never against a retyping of its own formula."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ctcsd_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+BLANK = 99
+
+
+def _rand_topk(rng, T, k, V, blank_rate=0.5, repeat_rate=0.5):
+    """Random per-slot top-k lists over tokens 0..V-1 plus blank id V, built so that blanks
+    and repeats across neighbouring slots are common."""
+    ids = np.zeros((T, k), dtype=np.int64)
+    lps = np.zeros((T, k), dtype=np.float64)
+    for t in range(T):
+        pool = list(range(V + 1))
+        rng.shuffle(pool)
+        row = []
+        if rng.random() < blank_rate:
+            row.append(V)
+        if t > 0 and rng.random() < repeat_rate:
+            for s in ids[t - 1]:
+                if s not in row and len(row) < k and rng.random() < 0.7:
+                    row.append(int(s))
+        for s in pool:
+            if len(row) >= k:
+                break
+            if s not in row:
+                row.append(s)
+        rng.shuffle(row)
+        p = rng.dirichlet(np.ones(k + 1))[:k]           # leaves some mass outside the top-k
+        order = np.argsort(-p)
+        ids[t] = np.asarray(row)[order]
+        lps[t] = np.log(p[order])
+    return ids, lps
+
+
+# ------------------------------------------------------------------ S5 collapse
+def test_collapse_golden_cases():
+    sym = {"_": BLANK}
+    n = 0
+    with open(os.path.join(GOLDEN, "ctc_collapse_cases.txt")) as f:
+        for line in f:
+            line = line.rstrip("\n")
+            if not line.strip() or line.startswith("#"):
+                continue
+            lhs, rhs = line.split("->")
+            a = [sym.setdefault(s, len(sym)) for s in lhs.split()]
+            want = tuple(sym[s] for s in rhs.split())
+            assert orc.ctc_collapse(a, BLANK) == want, line
+            n += 1
+    assert n >= 8
+
+
+def test_collapse_properties():
+    rng = np.random.default_rng(0)
+    for _ in range(300):
+        T = int(rng.integers(1, 9))
+        a = rng.integers(0, 4, size=T).tolist()
+        a = [BLANK if s == 3 else s for s in a]
+        y = orc.ctc_collapse(a, BLANK)
+        assert len(y) <= T and BLANK not in y
+        # a blank-free, repeat-free alignment is its own image
+        if BLANK not in a and all(a[i] != a[i + 1] for i in range(T - 1)):
+            assert y == tuple(a)
+        # two-step form: run-length merge first, blank removal second
+        merged = [s for i, s in enumerate(a) if i == 0 or s != a[i - 1]]
+        assert y == tuple(s for s in merged if s != BLANK)
+
+
+# ------------------------------------------------------------------ S4/S6 scores
+def _alpha_score(lp_t, y, blank, semiring="sum"):
+    """Graves et al. forward recursion over the blank-interleaved label sequence
+    (the dynamic programme the paper points to for Eq. 5).  lp_t[t][symbol] -> log prob
+    (missing symbols have probability 0).  semiring 'max' gives the best alignment."""
+    add = (lambda a, b: max(a, b)) if semiring == "max" else (lambda a, b: np.logaddexp(a, b))
+    ext = [blank]
+    for s in y:
+        ext += [s, blank]
+    S, T = len(ext), len(lp_t)
+    get = lambda t, s: lp_t[t].get(s, -np.inf)
+    alpha = np.full((T, S), -np.inf)
+    alpha[0, 0] = get(0, blank)
+    if S > 1:
+        alpha[0, 1] = get(0, ext[1])
+    for t in range(1, T):
+        for s in range(S):
+            v = alpha[t - 1, s]
+            if s >= 1:
+                v = add(v, alpha[t - 1, s - 1])
+            if s >= 2 and ext[s] != blank and ext[s] != ext[s - 2]:
+                v = add(v, alpha[t - 1, s - 2])
+            alpha[t, s] = v + get(t, ext[s])
+    out = alpha[T - 1, S - 1]
+    if S > 1:
+        out = add(out, alpha[T - 1, S - 2])
+    return float(out)
+
+
+@pytest.mark.parametrize("T,k,V", [(4, 3, 6), (5, 4, 9), (3, 2, 3), (6, 3, 5)])
+def test_sum_score_is_graves_forward_and_ctc_loss(T, k, V):
+    rng = np.random.default_rng(T * 100 + k)
+    deduped = False
+    for trial in range(4):
+        ids, lps = _rand_topk(rng, T, k, V)
+        cands = orc.enumerate_candidates(ids, lps, blank=V)
+        lp_t = [{int(ids[t, j]): float(lps[t, j]) for j in range(k)} for t in range(T)]
+        dense = torch.full((T, 1, V + 1), -float("inf"), dtype=torch.float64)
+        for t in range(T):
+            for j in range(k):
+                dense[t, 0, ids[t, j]] = lps[t, j]
+        deduped = deduped or len(cands) < k ** T
+        for y, score in cands.items():
+            assert score == pytest.approx(_alpha_score(lp_t, y, V), abs=1e-10)
+            if len(y) > 0:
+                loss = torch.nn.functional.ctc_loss(
+                    dense, torch.tensor([list(y)]), torch.tensor([T]), torch.tensor([len(y)]),
+                    blank=V, reduction="sum")
+                assert score == pytest.approx(-float(loss), abs=1e-9)
+        # sequences that were NOT produced have no alignment inside the top-k lists
+        toks = sorted({int(s) for s in ids.reshape(-1) if s != V})
+        for y in itertools.product(toks, repeat=2):
+            if y not in cands:
+                assert _alpha_score(lp_t, y, V) == -np.inf
+    assert deduped                                        # several alignments really merged
+
+
+def test_max_score_is_best_alignment():
+    rng = np.random.default_rng(7)
+    for trial in range(5):
+        ids, lps = _rand_topk(rng, 5, 3, 6)
+        mx = orc.enumerate_candidates(ids, lps, blank=6, score_mode=1)
+        sm = orc.enumerate_candidates(ids, lps, blank=6, score_mode=0)
+        lp_t = [{int(ids[t, j]): float(lps[t, j]) for j in range(3)} for t in range(5)]
+        assert mx.keys() == sm.keys()
+        for y in mx:
+            assert mx[y] == pytest.approx(_alpha_score(lp_t, y, 6, "max"), abs=1e-10)
+            assert mx[y] <= sm[y] + 1e-12
+
+
+def test_total_mass_closed_form():
+    # sum over all collapsed sequences of exp(score) = prod_t sum_j exp(lp[t,j])   (Eq. 1 + Eq. 6)
+    rng = np.random.default_rng(3)
+    for T, k, V in [(4, 3, 1000), (5, 4, 50), (2, 5, 7)]:
+        ids, lps = _rand_topk(rng, T, k, V)
+        cands = orc.enumerate_candidates(ids, lps, blank=V)
+        total = sum(math.exp(s) for s in cands.values())
+        want = float(np.prod(np.exp(lps).sum(axis=1)))
+        assert total == pytest.approx(want, rel=1e-12)
+    # k = V+1 on a toy vocabulary: the lists hold whole distributions, total mass is 1
+    V, T = 3, 4
+    z = rng.normal(size=(1, T, V + 1))
+    ids, lps = orc.topk_slots(z, V + 1)
+    cands = orc.enumerate_candidates(ids[0], lps[0], blank=V)
+    assert sum(math.exp(s) for s in cands.values()) == pytest.approx(1.0, abs=1e-12)
+
+
+def test_top_n_order_and_empty_dropped():
+    cands = {(): -0.1, (5,): -1.0, (4,): -1.0, (4, 1): -1.0, (3, 9): -0.5, (7,): -3.0}
+    kept = orc.select_top_n(cands, 4)
+    # score desc; ties: shorter first, then lexicographic tokens; empty sequence never kept
+    assert kept == [((3, 9), -0.5), ((4,), -1.0), ((5,), -1.0), ((4, 1), -1.0)]
+    assert orc.selection_margin(cands, 4) == 0.0
+    assert orc.selection_margin({(1,): -1.0, (2,): -1.5, (3,): -4.0}, 2) == pytest.approx(0.5)
+
+
+# ------------------------------------------------------------------ S4' prefix beam
+@pytest.mark.parametrize("T,k,V", [(4, 3, 6), (6, 4, 8)])
+def test_prefix_beam_without_pruning_equals_enumeration(T, k, V):
+    rng = np.random.default_rng(11 + T)
+    for trial in range(3):
+        ids, lps = _rand_topk(rng, T, k, V)
+        exact = orc.enumerate_candidates(ids, lps, blank=V)
+        beam = orc.prefix_beam_candidates(ids, lps, blank=V, beam=10 ** 6)
+        assert beam.keys() == exact.keys()
+        for y in exact:
+            assert beam[y] == pytest.approx(exact[y], abs=1e-12)
+
+
+def test_prefix_beam_pruned_bounds():
+    rng = np.random.default_rng(5)
+    for trial in range(5):
+        ids, lps = _rand_topk(rng, 6, 4, 8)
+        exact = orc.enumerate_candidates(ids, lps, blank=8)
+        st = {}
+        beam = orc.prefix_beam_candidates(ids, lps, blank=8, beam=8, stats=st)
+        assert len(beam) <= 8 and st["min_cut_gap"] >= 0.0
+        for y, s in beam.items():
+            assert y in exact and s <= exact[y] + 1e-12
+        # the best exact candidate's mass is concentrated enough to survive a beam of 8
+        best = max((y for y in exact), key=lambda y: exact[y])
+        assert best in beam
+
+
+# ------------------------------------------------------------------ S1-S3
+def test_draft_logits_against_library_and_bias_placement():
+    rng = np.random.default_rng(2)
+    M, H, T, V = 3, 32, 4, 10
+    x = rng.normal(size=(M, H)).astype(np.float32)
+    Wd = rng.normal(size=(T, V + 1, H)).astype(np.float32)
+    bias = np.array([0.5, -1.0], dtype=np.float32)
+    row_seq = np.array([1, 0, 1])
+    z = orc.draft_logits(x, Wd, bias, row_seq)
+    ref = torch.einsum("mh,tvh->mtv", torch.tensor(x, dtype=torch.float64),
+                       torch.tensor(Wd, dtype=torch.float64)).numpy()
+    ref[:, :, V] += bias[row_seq][:, None]
+    np.testing.assert_allclose(z, ref, rtol=0, atol=1e-12)
+    # hand case: H = 1, x = 2 -> logits are twice the weights, blank gets +bias
+    z1 = orc.draft_logits(np.array([[2.0]]), np.array([[[1.0], [3.0], [-1.0]]]), np.array([0.25]))
+    np.testing.assert_array_equal(z1, [[[2.0, 6.0, -1.75]]])
+
+
+def test_log_softmax_and_topk_against_library():
+    rng = np.random.default_rng(4)
+    z = rng.normal(size=(2, 3, 501)) * 3.0
+    lse, lp = orc.log_softmax_slots(z)
+    np.testing.assert_allclose(np.exp(lp).sum(-1), 1.0, atol=1e-12)
+    np.testing.assert_allclose(lp, torch.log_softmax(torch.tensor(z), -1).numpy(), atol=1e-12)
+    np.testing.assert_allclose(lse, torch.logsumexp(torch.tensor(z), -1).numpy(), atol=1e-12)
+    ids, lps = orc.topk_slots(z, 5)
+    tv, ti = torch.topk(torch.tensor(lp), 5, dim=-1)
+    np.testing.assert_array_equal(ids, ti.numpy())
+    np.testing.assert_allclose(lps, tv.numpy(), atol=1e-12)
+    # ties go to the lower id, blank (last id) is eligible
+    zt = np.array([[[1.0, 5.0, 5.0, 0.0, 5.0]]])
+    ids, _ = orc.topk_slots(zt, 4)
+    assert ids.tolist() == [[[1, 2, 4, 0]]]
+
+
+# ------------------------------------------------------------------ S8 tree
+def _pack(cands, N, T):
+    tok = np.full((1, N, T), -1, dtype=np.int64)
+    ln = np.zeros((1, N), dtype=np.int64)
+    for c, y in enumerate(cands):
+        tok[0, c, :len(y)] = y
+        ln[0, c] = len(y)
+    return tok, ln, np.array([len(cands)])
+
+
+def test_tree_hand_example_and_truncation():
+    tok, ln, nc = _pack([(5, 6), (5, 7), (8,)], 4, 3)
+    node_tok, parent, depth, pos, mask, retrieve, n = orc.build_tree(
+        np.array([1]), np.array([10]), tok, ln, nc, n_max=8)
+    assert n[0] == 5
+    assert node_tok[0, :5].tolist() == [1, 5, 6, 7, 8]
+    assert parent[0, :5].tolist() == [-1, 0, 1, 1, 0]
+    assert depth[0, :5].tolist() == [0, 1, 2, 2, 1]
+    assert pos[0, :5].tolist() == [10, 11, 12, 12, 11]
+    assert [int(m) for m in mask[0, :5, 0]] == [0b1, 0b11, 0b111, 0b1011, 0b10001]
+    assert retrieve[0, :3].tolist() == [[1, 2, -1], [1, 3, -1], [4, -1, -1]]
+    # node budget 4 (root included): ids >= 4 are dropped, earlier prefixes still resolve
+    node_tok, parent, depth, pos, mask, retrieve, n = orc.build_tree(
+        np.array([1]), np.array([10]), tok, ln, nc, n_max=4)
+    assert n[0] == 4 and node_tok[0].tolist() == [1, 5, 6, 7]
+    assert retrieve[0, :3].tolist() == [[1, 2, -1], [1, 3, -1], [-1, -1, -1]]
+
+
+def test_tree_invariants_against_bruteforce_trie():
+    rng = np.random.default_rng(9)
+    for trial in range(40):
+        N, T = int(rng.integers(1, 9)), int(rng.integers(1, 6))
+        n_max = int(rng.integers(2, 70))
+        seen, cands = set(), []
+        for _ in range(N):
+            y = tuple(rng.integers(0, 3, size=int(rng.integers(1, T + 1))).tolist())
+            if y not in seen:
+                seen.add(y)
+                cands.append(y)
+        tok, ln, nc = _pack(cands, N, T)
+        node_tok, parent, depth, pos, mask, retrieve, n = orc.build_tree(
+            np.array([42]), np.array([100]), tok, ln, nc, n_max=n_max)
+        n = int(n[0])
+        prefixes = []                                     # distinct prefixes in first-seen order
+        for y in cands:
+            for l in range(1, len(y) + 1):
+                if y[:l] not in prefixes:
+                    prefixes.append(y[:l])
+        assert n == min(n_max, 1 + len(prefixes))
+        path = {0: ()}
+        for i in range(1, n):
+            assert 0 <= parent[0, i] < i
+            path[i] = path[int(parent[0, i])] + (int(node_tok[0, i]),)
+            assert path[i] == prefixes[i - 1]
+            assert depth[0, i] == len(path[i]) and pos[0, i] == 100 + len(path[i])
+        for i in range(n):                                # mask == ancestor-or-self relation
+            anc, j = set(), i
+            while j >= 0:
+                anc.add(j)
+                j = int(parent[0, j])
+            bits = {j for j in range(n_max) if (int(mask[0, i, j // 64]) >> (j % 64)) & 1}
+            assert bits == anc and len(bits) == depth[0, i] + 1
+        for i in range(1, n):                             # siblings carry distinct tokens
+            sib = [int(node_tok[0, c]) for c in range(1, n) if parent[0, c] == parent[0, i]]
+            assert len(sib) == len(set(sib))
+        for c, y in enumerate(cands):                     # retrieve round-trips
+            for l in range(len(y)):
+                r = int(retrieve[0, c, l])
+                want = prefixes.index(y[:l + 1]) + 1
+                assert r == (want if want < n_max else -1)
+            assert all(retrieve[0, c, len(y):] == -1)
+
+
+# ------------------------------------------------------------------ S9 attention
+def _sdpa_ref(Q, K, V, kv_len, n_nodes, mask, scale):
+    B, n_max, Hq, D = Q.shape
+    grp = Hq // K.shape[1]
+    O = np.zeros((B, n_max, Hq, D))
+    for b in range(B):
+        L, n = int(kv_len[b]), int(n_nodes[b])
+        allow = torch.ones((n, L + n), dtype=torch.bool)
+        for i in range(n):
+            for j in range(n):
+                allow[i, L + j] = bool((int(mask[b, i, j // 64]) >> (j % 64)) & 1)
+        q = torch.tensor(Q[b, :n], dtype=torch.float64).permute(1, 0, 2)          # [Hq,n,D]
+        k = torch.tensor(K[b, :, :L + n], dtype=torch.float64).repeat_interleave(grp, 0)
+        v = torch.tensor(V[b, :, :L + n], dtype=torch.float64).repeat_interleave(grp, 0)
+        o = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=allow, scale=scale)
+        O[b, :n] = o.permute(1, 0, 2).numpy()
+    return O
+
+
+def _random_tree(rng, n, n_max):
+    parent = np.full(n_max, -1, dtype=np.int64)
+    for i in range(1, n):
+        parent[i] = rng.integers(0, i)
+    W = (n_max + 63) // 64
+    mask = np.zeros((n_max, W), dtype=np.uint64)
+    for i in range(n):
+        j = i
+        while j >= 0:
+            mask[i, j // 64] |= np.uint64(1) << np.uint64(j % 64)
+            j = int(parent[j])
+    return parent, mask
+
+
+def test_attention_against_sdpa_and_special_cases():
+    rng = np.random.default_rng(6)
+    B, n_max, Hq, Hkv, D, Lcap = 2, 70, 4, 2, 16, 120
+    Q = rng.normal(size=(B, n_max, Hq, D))
+    K = rng.normal(size=(B, Hkv, Lcap, D))
+    V = rng.normal(size=(B, Hkv, Lcap, D))
+    kv_len = np.array([37, 5])
+    n_nodes = np.array([70, 9])
+    mask = np.zeros((B, n_max, 2), dtype=np.uint64)
+    for b in range(B):
+        _, mask[b] = _random_tree(rng, int(n_nodes[b]), n_max)
+    scale = 1.0 / math.sqrt(D)
+    O = orc.tree_attention(Q, K, V, kv_len, n_nodes, mask, scale)
+    np.testing.assert_allclose(O, _sdpa_ref(Q, K, V, kv_len, n_nodes, mask, scale), atol=1e-12)
+    assert np.all(O[1, 9:] == 0)
+    # GQA == MHA with the kv heads repeated
+    O2 = orc.tree_attention(Q, np.repeat(K, 2, axis=1), np.repeat(V, 2, axis=1), kv_len, n_nodes, mask, scale)
+    np.testing.assert_allclose(O, O2, atol=1e-13)
+    # chain tree == causal attention over prefix + chain; single node == plain decode attention
+    n = 6
+    chain = np.zeros((1, n_max, 2), dtype=np.uint64)
+    for i in range(n):
+        chain[0, i, 0] = np.uint64((1 << (i + 1)) - 1)
+    Oc = orc.tree_attention(Q[:1], K[:1], V[:1], np.array([20]), np.array([n]), chain, scale)
+    for i in range(n):
+        k = torch.tensor(K[0, 0, :20 + i + 1])
+        v = torch.tensor(V[0, 0, :20 + i + 1])
+        p = torch.softmax(k @ torch.tensor(Q[0, i, 0]) * scale, 0)
+        np.testing.assert_allclose(Oc[0, i, 0], (p @ v).numpy(), atol=1e-12)
+
+
+# ------------------------------------------------------------------ S10 / S11
+def test_lm_head_argmax_against_library_and_ties():
+    rng = np.random.default_rng(8)
+    hn = rng.normal(size=(5, 16)).astype(np.float32)
+    Wl = rng.normal(size=(40, 16)).astype(np.float32)
+    y, am = orc.lm_head_argmax(hn, Wl)
+    ref = torch.tensor(hn, dtype=torch.float64) @ torch.tensor(Wl, dtype=torch.float64).T
+    np.testing.assert_allclose(y, ref.numpy(), atol=1e-12)
+    np.testing.assert_array_equal(am, ref.argmax(1).numpy())
+    assert orc.argmax_rows(np.array([[1.0, 7.0, 7.0, 2.0]])).tolist() == [1]
+
+
+def test_greedy_accept_against_candidate_definition():
+    """Definition used as the pin: the accepted length is the longest candidate prefix whose
+    every token equals the base model's greedy token at the node before it."""
+    rng = np.random.default_rng(10)
+    for trial in range(60):
+        N, T = int(rng.integers(1, 7)), int(rng.integers(1, 6))
+        cands = list({tuple(rng.integers(0, 3, size=int(rng.integers(1, T + 1))).tolist()) for _ in range(N)})
+        tok, ln, nc = _pack(cands, len(cands), T)
+        node_tok, parent, depth, pos, mask, retrieve, n = orc.build_tree(
+            np.array([1]), np.array([0]), tok, ln, nc, n_max=64)
+        am = rng.integers(0, 3, size=(1, 64))
+        acc_len, acc_nodes, acc_tok, next_tok = orc.greedy_accept(node_tok, parent, n, am, T)
+        best = 0
+        for c, y in enumerate(cands):
+            l, prev = 0, 0
+            while l < len(y) and am[0, prev] == y[l]:
+                prev = int(retrieve[0, c, l])
+                l += 1
+            best = max(best, l)
+        assert acc_len[0] == best <= int(depth[0, :n[0]].max()) <= T
+        cur = 0
+        for l in range(best):                             # accepted nodes form a root path
+            nd = int(acc_nodes[0, l])
+            assert parent[0, nd] == cur and node_tok[0, nd] == acc_tok[0, l] == am[0, cur]
+            cur = nd
+        assert next_tok[0] == am[0, cur]
+        assert all(acc_nodes[0, best:] == -1) and all(acc_tok[0, best:] == -1)
+
+
+def test_greedy_accept_chain_extremes():
+    tok, ln, nc = _pack([(3, 4, 5, 6)], 1, 4)
+    node_tok, parent, depth, pos, mask, retrieve, n = orc.build_tree(
+        np.array([2]), np.array([0]), tok, ln, nc, n_max=16)
+    am = np.zeros((1, 16), dtype=np.int64)
+    am[0, :5] = [3, 4, 5, 6, 9]                           # full agreement along the chain
+    acc_len, acc_nodes, acc_tok, next_tok = orc.greedy_accept(node_tok, parent, n, am, 4)
+    assert acc_len[0] == 4 and acc_tok[0].tolist() == [3, 4, 5, 6] and next_tok[0] == 9
+    am[0, 0] = 7                                          # no agreement at the root
+    acc_len, acc_nodes, acc_tok, next_tok = orc.greedy_accept(node_tok, parent, n, am, 4)
+    assert acc_len[0] == 0 and next_tok[0] == 7
