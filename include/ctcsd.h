@@ -1,0 +1,201 @@
+/*
+ * ctcsd - the per-step draft-and-verify pass of CTC-drafted speculative decoding,
+ * as CUDA kernels for NVIDIA B200 (sm_100a) behind a plain C ABI.
+ *
+ * One decoding step (paper Sec. 3.3, "Inference"): the base model has produced a hidden
+ * state and a greedy base token; a draft head turns the hidden state into one distribution
+ * per draft slot over the vocabulary plus the CTC blank; the k best symbols per slot are
+ * combined into slot paths; each path is collapsed by beta^{-1} (Sec. 2.3), duplicates are
+ * merged and scored by the sum over their alignments (Eq. 1 / Eq. 5, with Eq. 6 for one
+ * alignment); the N best candidates become a token tree (Sec. 2.2) that the base model
+ * verifies in one pass (tree attention + LM head), and the longest candidate that agrees
+ * with the base model's greedy choice is accepted (Sec. 2.2, Sec. 3.3).
+ *
+ * Conventions
+ *  - Every function returns an int status: CTCSD_OK (0) or a negative CTCSD_ERR_* code.
+ *    Nothing throws; arguments are validated on the host before any launch.
+ *  - Unless a parameter is marked [host], every pointer is a DEVICE pointer owned by the
+ *    caller; inputs are read-only, outputs are the parameters named out_*.  The library
+ *    never allocates device memory: all scratch lives in the workspace given to
+ *    ctcsd_create.  Buffers must not alias unless stated.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *    enqueue work on it and return without synchronising.  Two calls on the same handle
+ *    must not overlap on the device (they share the workspace).
+ *  - Problems found by a kernel (for example a bounded wait that ran out) are recorded in a
+ *    device status word that ctcsd_poll_status reads.
+ *  - dtype: 0 = float32, 1 = bfloat16 for activations, weights, Q/K/V and the attention
+ *    output; logits, log-probabilities and scores are always float32 on the device.
+ *  - Tensors are dense, row-major, last index fastest, in the shapes given.
+ */
+#ifndef CTCSD_H_
+#define CTCSD_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CTCSD_OK                0
+#define CTCSD_ERR_INVALID_ARG  -1   /* null pointer, bad shape, value out of the documented range */
+#define CTCSD_ERR_UNSUPPORTED  -2   /* a legal request this build has no kernel for */
+#define CTCSD_ERR_WORKSPACE    -3   /* workspace missing, misaligned or too small */
+#define CTCSD_ERR_CUDA         -4   /* a CUDA runtime/driver call failed (see ctcsd_last_cuda_error) */
+#define CTCSD_ERR_TIMEOUT      -5   /* a bounded device-side wait ran out */
+#define CTCSD_ERR_INTERNAL     -6
+
+#define CTCSD_DTYPE_F32   0
+#define CTCSD_DTYPE_BF16  1
+
+#define CTCSD_SCORE_SUM   0   /* candidate score = log sum over alignments (Eq. 1 / Eq. 5) */
+#define CTCSD_SCORE_MAX   1   /* candidate score = best single alignment (enumeration only) */
+
+#define CTCSD_MAX_T        8    /* draft slots */
+#define CTCSD_MAX_K        8    /* symbols kept per slot */
+#define CTCSD_MAX_NODES    128  /* tree nodes per sequence, root included */
+#define CTCSD_MAX_TOPN     64   /* candidates kept */
+#define CTCSD_MAX_PATHS    4096 /* k^T limit for exhaustive enumeration */
+#define CTCSD_MAX_BEAM     128
+
+/* Problem shape, fixed per handle.  Notation follows the paper: T draft slots, blank id = V. */
+typedef struct ctcsd_config {
+    int B;          /* sequences per step (>= 1) */
+    int H;          /* hidden size, multiple of 8 */
+    int V;          /* vocabulary size; the draft head has V+1 classes, blank = V */
+    int T;          /* draft slots, 1..CTCSD_MAX_T */
+    int k;          /* symbols kept per slot, 1..CTCSD_MAX_K, T*k <= 64 */
+    int beam;       /* 0: enumerate all k^T slot paths (k^T <= CTCSD_MAX_PATHS);
+                       >0: CTC prefix beam search of this width (<= CTCSD_MAX_BEAM) */
+    int topN;       /* candidates kept, 1..CTCSD_MAX_TOPN */
+    int max_nodes;  /* tree node budget per sequence including the root, 2..CTCSD_MAX_NODES */
+    int Hq;         /* query heads */
+    int Hkv;        /* key/value heads, divides Hq */
+    int D;          /* head dimension: 64 or 128 */
+    int dtype;      /* CTCSD_DTYPE_* */
+    int score_mode; /* CTCSD_SCORE_* */
+    int max_draft_rows; /* largest M passed to ctcsd_draft_logits; 0 means B */
+} ctcsd_config;
+
+typedef struct ctcsd_handle ctcsd_handle;
+
+/* Bytes of device workspace a handle for `cfg` needs.  [host] cfg, [host] out_bytes. */
+int ctcsd_workspace_bytes(const ctcsd_config* cfg, size_t* out_bytes);
+
+/* Creates a handle on the current CUDA device.  `workspace` is device memory, 256-byte
+ * aligned, at least ctcsd_workspace_bytes() large, owned by the caller and kept alive until
+ * ctcsd_destroy; its first bytes are cleared here (synchronously).  [host] out_handle, cfg. */
+int ctcsd_create(ctcsd_handle** out_handle, const ctcsd_config* cfg, void* workspace, size_t workspace_bytes);
+
+/* Frees the host-side handle.  The workspace stays with the caller. */
+int ctcsd_destroy(ctcsd_handle* h);
+
+/* Synchronises `stream`, then reads and clears the device status word.  [host] out_status
+ * receives CTCSD_OK or the first error a kernel recorded. */
+int ctcsd_poll_status(ctcsd_handle* h, void* stream, int* out_status);
+
+/* Text for a status code; never NULL.  The string is static. */
+const char* ctcsd_strerror(int status);
+
+/* cudaError_t value of the most recent failing CUDA call made through handle `h` (0 if none). */
+int ctcsd_last_cuda_error(const ctcsd_handle* h);
+
+/* Number of kernels this handle has launched since creation (for launch accounting). */
+long long ctcsd_launch_count(const ctcsd_handle* h);
+
+/*
+ * Draft head, per-slot log-softmax and per-slot top-k (Sec. 3.2: one probability
+ * distribution per place from the projected hidden state; Sec. 3.3: "the top k tokens are
+ * selected in descending order of probability").
+ *   z[m,t,v]   = sum_h x[m,h] * Wd[t,v,h]  (+ blank_bias[row_seq[m]] when v == V)
+ *   lse[m,t]   = log sum_v exp z[m,t,v]
+ *   top-k      = the k largest z[m,t,:] over all V+1 classes, descending, ties to the lower id;
+ *                out_topk_lp = z - lse.
+ * M          rows of x, 1 <= M <= max_draft_rows.
+ * x          [M,H] dtype.            Wd  [T,V+1,H] dtype (hidden axis contiguous).
+ * row_seq    [M] int32 sequence index of each row, or NULL for the identity (needs M <= B).
+ * blank_bias [B] float32, or NULL for no bias.
+ * out_topk_id [M,T,k] int32;  out_topk_lp [M,T,k] float32;  out_lse [M,T] float32.
+ * out_logits_dbg  NULL, or [M,T,V+1] float32 receiving every logit exactly as the kernel
+ *                 computed it (for checking the selection against the kernel's own values).
+ */
+int ctcsd_draft_logits(ctcsd_handle* h, void* stream, int M, const void* x, const void* Wd,
+                       const int* row_seq, const float* blank_bias,
+                       int* out_topk_id, float* out_topk_lp, float* out_lse, float* out_logits_dbg);
+
+/*
+ * Slot paths -> collapsed, deduplicated, scored candidates -> the topN best (Sec. 3.3: the
+ * slot tokens are combined and "the most valuable combinations are reserved"; Sec. 2.3 /
+ * Sec. 3.1: beta^{-1} merges adjacent repeats, then removes blanks; Eq. 6: a path's
+ * probability is the product over slots; Eq. 1 / Eq. 5: a candidate's probability is the sum
+ * over the paths that collapse to it).
+ * With beam == 0 all k^T paths are enumerated; with beam > 0 a CTC prefix beam search over
+ * the same per-slot lists keeps the `beam` most probable prefixes after every slot.
+ * Candidates are ordered by score descending, then shorter first, then token ids
+ * lexicographically ascending; the empty candidate is never returned.  Scores are formed in
+ * float64 from the float32 inputs and returned as float32.
+ * M          rows in topk_id/topk_lp.    topk_id [M,T,k] int32;  topk_lp [M,T,k] float32.
+ * sel_row    [B] int32: sequence b drafts from row sel_row[b]; NULL means row b.
+ * out_cand_tok [B,topN,T] int32 (-1 padded);  out_cand_len [B,topN] int32 (0 when unused);
+ * out_cand_score [B,topN] float32 (-inf when unused);  out_n_cand [B] int32.
+ */
+int ctcsd_topk_collapse(ctcsd_handle* h, void* stream, int M, const int* topk_id, const float* topk_lp,
+                        const int* sel_row,
+                        int* out_cand_tok, int* out_cand_len, float* out_cand_score, int* out_n_cand);
+
+/*
+ * Packs the ranked candidates into a token tree (Sec. 2.2: candidates are the root-to-leaf
+ * paths of a tree verified under a tree attention mask; Sec. 3.3: the greedy base token
+ * comes first).  Node 0 is the root holding base_tok[b]; further nodes are the distinct
+ * candidate prefixes in order of first appearance (candidates by rank, each left to right);
+ * prefixes that would get an id >= max_nodes are dropped.
+ * base_tok [B] int32;  kv_len [B] int32 (cached tokens before the tree);
+ * cand_tok [B,topN,T], cand_len [B,topN], n_cand [B] as produced by ctcsd_topk_collapse.
+ * out_node_tok/out_parent/out_depth/out_pos [B,max_nodes] int32 (parent of the root = -1,
+ *   pos = kv_len + depth; entries of unused nodes: token -1, parent -1, depth 0, pos 0);
+ * out_mask [B,max_nodes,W] uint64 with W = ceil(max_nodes/64): bit j of row i is set iff
+ *   node j is node i or one of its ancestors;
+ * out_retrieve [B,topN,T] int32: node id of candidate c's prefix of length l+1, or -1;
+ * out_n_nodes [B] int32.
+ */
+int ctcsd_build_tree(ctcsd_handle* h, void* stream, const int* base_tok, const int* kv_len,
+                     const int* cand_tok, const int* cand_len, const int* n_cand,
+                     int* out_node_tok, int* out_parent, int* out_depth, int* out_pos,
+                     unsigned long long* out_mask, int* out_retrieve, int* out_n_nodes);
+
+/*
+ * Tree attention (Sec. 2.2 / Sec. 3.3: all candidates are verified in one pass of the base
+ * model; a node attends to the cached prefix and to its own ancestors):
+ *   O[b,i,h,:] = softmax_j( scale * q[b,i,h,:] . k[b,g,j,:] ) v[b,g,j,:],  g = h / (Hq/Hkv),
+ *   j over cache rows 0..kv_len[b]-1 and rows kv_len[b]+j' for every node j' whose mask bit
+ *   is set in row i.
+ * Q [B,max_nodes,Hq,D] dtype;  K, V [B,Hkv,Lcap,D] dtype, the caller having written node j's
+ * key/value at cache row kv_len[b]+j;  Lcap >= max_b(kv_len[b]) + max_nodes.
+ * kv_len, n_nodes [B] int32;  mask as produced by ctcsd_build_tree.
+ * out_O [B,max_nodes,Hq,D] dtype; rows i >= n_nodes[b] are written as zero.
+ */
+int ctcsd_tree_attention(ctcsd_handle* h, void* stream, const void* Q, const void* K, const void* V,
+                         int Lcap, const int* kv_len, const int* n_nodes,
+                         const unsigned long long* mask, float scale, void* out_O);
+
+/*
+ * LM head with row arg-max at every tree node, then greedy acceptance (Eq. 3-4 form:
+ * argmax of the LM head's distribution; Sec. 2.2: a draft is accepted only where it matches
+ * the base model's greedy output; Sec. 3.3: the longest such candidate is the step's output).
+ *   y[m,v] = sum_h hn[m,h] * Wl[v,h];  am[m] = argmax_v y[m,v], ties to the lower id.
+ *   Walk: cur = root; while some child c of cur has node_tok[c] == am[cur]: accept c.
+ * hn [B*max_nodes,H] dtype (row b*max_nodes+i is node i of sequence b; rows of unused nodes
+ *   are computed but ignored);  Wl [V,H] dtype;  node_tok, parent [B,max_nodes], n_nodes [B].
+ * out_argmax [B,max_nodes] int32;  out_acc_len [B] int32 (accepted draft tokens, root and
+ *   bonus token excluded);  out_acc_nodes, out_acc_tok [B,T] int32 (-1 padded);
+ *   out_next_tok [B] int32 = am at the last accepted node (the bonus token);
+ * out_logits_dbg  NULL or [B*max_nodes,V] float32 receiving every logit as computed.
+ */
+int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const void* Wl,
+                        const int* node_tok, const int* parent, const int* n_nodes,
+                        int* out_argmax, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
+                        int* out_next_tok, float* out_logits_dbg);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CTCSD_H_ */

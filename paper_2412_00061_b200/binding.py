@@ -1,0 +1,214 @@
+"""ctypes binding of libctcsd.so: argument marshalling only.
+
+Every step of the draft-and-verify pass runs inside the CUDA library; this module turns
+torch tensors (used purely as device-memory owners) into raw pointers, checks shapes and
+dtypes, and forwards to the C entry points of the same names.  There is no CPU fallback:
+if the library cannot be loaded, or a call reports an error, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libctcsd.so")
+
+DTYPE_F32, DTYPE_BF16 = 0, 1
+SCORE_SUM, SCORE_MAX = 0, 1
+
+EXPORTS = [
+    "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
+    "ctcsd_last_cuda_error", "ctcsd_launch_count",
+    "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
+    "ctcsd_verify_accept",
+]
+
+
+class CtcsdError(RuntimeError):
+    pass
+
+
+class CConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "B", "H", "V", "T", "k", "beam", "topN", "max_nodes", "Hq", "Hkv", "D", "dtype", "score_mode",
+        "max_draft_rows")]
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads libctcsd.so (built in-tree by paper_2412_00061_b200.build).  Raises if absent."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise CtcsdError("CUDA library %s is missing: run `python -m paper_2412_00061_b200.build`" % p)
+    lib = ctypes.CDLL(p)
+    vp, ci, cs = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.ctcsd_workspace_bytes.argtypes = [ctypes.POINTER(CConfig), ctypes.POINTER(cs)]
+    lib.ctcsd_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(CConfig), vp, cs]
+    lib.ctcsd_destroy.argtypes = [vp]
+    lib.ctcsd_poll_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
+    lib.ctcsd_strerror.argtypes = [ci]
+    lib.ctcsd_strerror.restype = ctypes.c_char_p
+    lib.ctcsd_last_cuda_error.argtypes = [vp]
+    lib.ctcsd_launch_count.argtypes = [vp]
+    lib.ctcsd_launch_count.restype = ctypes.c_longlong
+    lib.ctcsd_draft_logits.argtypes = [vp, vp, ci] + [vp] * 8
+    lib.ctcsd_topk_collapse.argtypes = [vp, vp, ci] + [vp] * 7
+    lib.ctcsd_build_tree.argtypes = [vp, vp] + [vp] * 12
+    lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
+    lib.ctcsd_verify_accept.argtypes = [vp, vp] + [vp] * 11
+    for name in EXPORTS:
+        if name not in ("ctcsd_strerror", "ctcsd_launch_count"):
+            getattr(lib, name).restype = ci
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, numel: Optional[int] = None, name: str = "") -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise CtcsdError("%s must be a contiguous CUDA tensor" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise CtcsdError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    if numel is not None and t.numel() != numel:
+        raise CtcsdError("%s must have %d elements, got %d" % (name, numel, t.numel()))
+    return t.data_ptr()
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+class Handle:
+    """Owns a ctcsd handle and its device workspace (a torch uint8 tensor)."""
+
+    def __init__(self, B, H, V, T, k, beam, topN, max_nodes, Hq, Hkv, D, dtype, score_mode=SCORE_SUM,
+                 max_draft_rows=0, device="cuda:0"):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise CtcsdError("ctcsd needs a CUDA device (B200); there is no CPU path")
+        self.cfg = CConfig(B, H, V, T, k, beam, topN, max_nodes, Hq, Hkv, D, dtype, score_mode, max_draft_rows)
+        self.device = torch.device(device)
+        self.act_dtype = torch.bfloat16 if dtype == DTYPE_BF16 else torch.float32
+        self.M_draft_max = max_draft_rows or B
+        nbytes = ctypes.c_size_t(0)
+        self._check(self.lib.ctcsd_workspace_bytes(ctypes.byref(self.cfg), ctypes.byref(nbytes)), "workspace_bytes")
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            h = ctypes.c_void_p()
+            self._check(self.lib.ctcsd_create(ctypes.byref(h), ctypes.byref(self.cfg), self._ws_ptr, nbytes.value),
+                        "create")
+        self._h = h
+
+    def _check(self, rc: int, what: str):
+        if rc != 0:
+            extra = ""
+            if rc == -4 and getattr(self, "_h", None):
+                extra = " (cudaError %d)" % self.lib.ctcsd_last_cuda_error(self._h)
+            raise CtcsdError("ctcsd_%s failed: %s%s" % (what, self.lib.ctcsd_strerror(rc).decode(), extra))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.ctcsd_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def launch_count(self) -> int:
+        return int(self.lib.ctcsd_launch_count(self._h))
+
+    def poll_status(self, stream=None) -> int:
+        st = ctypes.c_int(0)
+        self._check(self.lib.ctcsd_poll_status(self._h, _stream_ptr(stream), ctypes.byref(st)), "poll_status")
+        return st.value
+
+    # ---- the five calls of the hot path ------------------------------------------------
+    def draft_logits(self, x, Wd, row_seq, blank_bias, out_topk_id, out_topk_lp, out_lse,
+                     out_logits_dbg=None, stream=None):
+        c = self.cfg
+        M = x.shape[0]
+        i32, f32 = torch.int32, torch.float32
+        rc = self.lib.ctcsd_draft_logits(
+            self._h, _stream_ptr(stream), M,
+            _ptr(x, self.act_dtype, M * c.H, "x"), _ptr(Wd, self.act_dtype, c.T * (c.V + 1) * c.H, "Wd"),
+            _ptr(row_seq, i32, M, "row_seq"), _ptr(blank_bias, f32, c.B, "blank_bias"),
+            _ptr(out_topk_id, i32, M * c.T * c.k, "out_topk_id"), _ptr(out_topk_lp, f32, M * c.T * c.k, "out_topk_lp"),
+            _ptr(out_lse, f32, M * c.T, "out_lse"),
+            _ptr(out_logits_dbg, f32, M * c.T * (c.V + 1), "out_logits_dbg"))
+        self._check(rc, "draft_logits")
+
+    def topk_collapse(self, topk_id, topk_lp, sel_row, out_cand_tok, out_cand_len, out_cand_score, out_n_cand,
+                      stream=None):
+        c = self.cfg
+        M = topk_id.shape[0]
+        i32, f32 = torch.int32, torch.float32
+        rc = self.lib.ctcsd_topk_collapse(
+            self._h, _stream_ptr(stream), M,
+            _ptr(topk_id, i32, M * c.T * c.k, "topk_id"), _ptr(topk_lp, f32, M * c.T * c.k, "topk_lp"),
+            _ptr(sel_row, i32, c.B, "sel_row"),
+            _ptr(out_cand_tok, i32, c.B * c.topN * c.T, "out_cand_tok"), _ptr(out_cand_len, i32, c.B * c.topN, "out_cand_len"),
+            _ptr(out_cand_score, f32, c.B * c.topN, "out_cand_score"), _ptr(out_n_cand, i32, c.B, "out_n_cand"))
+        self._check(rc, "topk_collapse")
+
+    def build_tree(self, base_tok, kv_len, cand_tok, cand_len, n_cand, out_node_tok, out_parent, out_depth,
+                   out_pos, out_mask, out_retrieve, out_n_nodes, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        W = (c.max_nodes + 63) // 64
+        nn = c.B * c.max_nodes
+        rc = self.lib.ctcsd_build_tree(
+            self._h, _stream_ptr(stream),
+            _ptr(base_tok, i32, c.B, "base_tok"), _ptr(kv_len, i32, c.B, "kv_len"),
+            _ptr(cand_tok, i32, c.B * c.topN * c.T, "cand_tok"), _ptr(cand_len, i32, c.B * c.topN, "cand_len"),
+            _ptr(n_cand, i32, c.B, "n_cand"),
+            _ptr(out_node_tok, i32, nn, "out_node_tok"), _ptr(out_parent, i32, nn, "out_parent"),
+            _ptr(out_depth, i32, nn, "out_depth"), _ptr(out_pos, i32, nn, "out_pos"),
+            _ptr(out_mask, torch.int64, nn * W, "out_mask"),
+            _ptr(out_retrieve, i32, c.B * c.topN * c.T, "out_retrieve"), _ptr(out_n_nodes, i32, c.B, "out_n_nodes"))
+        self._check(rc, "build_tree")
+
+    def tree_attention(self, Q, K, V, kv_len, n_nodes, mask, scale, out_O, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        Lcap = K.shape[2]
+        W = (c.max_nodes + 63) // 64
+        rc = self.lib.ctcsd_tree_attention(
+            self._h, _stream_ptr(stream),
+            _ptr(Q, self.act_dtype, c.B * c.max_nodes * c.Hq * c.D, "Q"),
+            _ptr(K, self.act_dtype, c.B * c.Hkv * Lcap * c.D, "K"), _ptr(V, self.act_dtype, c.B * c.Hkv * Lcap * c.D, "V"),
+            Lcap, _ptr(kv_len, i32, c.B, "kv_len"), _ptr(n_nodes, i32, c.B, "n_nodes"),
+            _ptr(mask, torch.int64, c.B * c.max_nodes * W, "mask"), float(scale),
+            _ptr(out_O, self.act_dtype, c.B * c.max_nodes * c.Hq * c.D, "out_O"))
+        self._check(rc, "tree_attention")
+
+    def verify_accept(self, hn, Wl, node_tok, parent, n_nodes, out_argmax, out_acc_len, out_acc_nodes,
+                      out_acc_tok, out_next_tok, out_logits_dbg=None, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        nn = c.B * c.max_nodes
+        rc = self.lib.ctcsd_verify_accept(
+            self._h, _stream_ptr(stream),
+            _ptr(hn, self.act_dtype, nn * c.H, "hn"), _ptr(Wl, self.act_dtype, c.V * c.H, "Wl"),
+            _ptr(node_tok, i32, nn, "node_tok"), _ptr(parent, i32, nn, "parent"), _ptr(n_nodes, i32, c.B, "n_nodes"),
+            _ptr(out_argmax, i32, nn, "out_argmax"), _ptr(out_acc_len, i32, c.B, "out_acc_len"),
+            _ptr(out_acc_nodes, i32, c.B * c.T, "out_acc_nodes"), _ptr(out_acc_tok, i32, c.B * c.T, "out_acc_tok"),
+            _ptr(out_next_tok, i32, c.B, "out_next_tok"),
+            _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
+        self._check(rc, "verify_accept")

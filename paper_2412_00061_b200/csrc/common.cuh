@@ -1,0 +1,142 @@
+// Shared host/device declarations for the ctcsd kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "ctcsd.h"
+
+namespace ctcsd {
+
+// ---------------------------------------------------------------------------------------
+// Workspace layout.  Everything the kernels need beyond their inputs and outputs lives in
+// the caller's workspace at the offsets computed here.
+// ---------------------------------------------------------------------------------------
+constexpr int kTopSlots = CTCSD_MAX_K;          // every partial top-k list keeps 8 entries
+
+// Partial result of one chunk of vocabulary rows for one (row m, slot t):
+// running max, sum of exp(z - max), and the chunk's best kTopSlots logits with their ids.
+struct alignas(16) DraftPartial {
+    float mx;
+    float sum;
+    float val[kTopSlots];
+    int   id[kTopSlots];
+    int   pad[2];
+};
+static_assert(sizeof(DraftPartial) == 80, "DraftPartial is copied as five 16-byte words");
+
+struct ArgmaxPartial {
+    float val;
+    int   idx;
+};
+
+struct Layout {
+    size_t status_off;        // int[16]: [0] status word, [1] detail
+    size_t counter_off;       // unsigned[kCounters]: "chunks finished" tickets, zero between calls
+    size_t draft_part_off;    // DraftPartial[4][gemv_grid_max][2]  (weight-streaming GEMV partials)
+    size_t part_slot_off;     // int[gemv_grid_max][2]
+    size_t lm_part_off;       // ArgmaxPartial[lm_tiles_max][B*max_nodes]  (tensor-core LM head partials)
+    size_t attn_part_off;     // float[B][Hq][max_nodes][kv_splits][D+2]
+    size_t total;
+    int gemv_grid_max;        // largest grid the GEMV may use
+    int lm_tiles_max;
+    int kv_splits;            // KV-axis splits in tree attention
+};
+
+constexpr int kCounters = 64;
+
+struct Handle {
+    ctcsd_config cfg;
+    Layout lay;
+    char* ws;
+    int device;
+    int num_sms;
+    int last_cuda_error;
+    long long launches;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+Layout make_layout(const ctcsd_config& cfg, int num_sms);
+int validate_config(const ctcsd_config& cfg);
+
+#define CTCSD_CUDA_CHECK(h, expr)                                   \
+    do {                                                            \
+        cudaError_t e__ = (expr);                                   \
+        if (e__ != cudaSuccess) {                                   \
+            (h)->last_cuda_error = (int)e__;                        \
+            return CTCSD_ERR_CUDA;                                  \
+        }                                                           \
+    } while (0)
+
+#define CTCSD_LAUNCH_CHECK(h)                                       \
+    do {                                                            \
+        (h)->launches++;                                            \
+        CTCSD_CUDA_CHECK(h, cudaGetLastError());                    \
+    } while (0)
+
+inline int* status_ptr(const Handle* h) { return reinterpret_cast<int*>(h->ws + h->lay.status_off); }
+inline unsigned* counter_ptr(const Handle* h) { return reinterpret_cast<unsigned*>(h->ws + h->lay.counter_off); }
+
+// ---------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// 16-byte streaming load that does not allocate in L1 (weights are read exactly once).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+// A 32-bit word holding two bfloat16 -> two floats (low half first).
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// "a ranks before b" for (logit, id) pairs: larger logit first, equal logits -> lower id.
+__device__ __forceinline__ bool ranks_before(float va, int ia, float vb, int ib) {
+    return va > vb || (va == vb && ia < ib);
+}
+
+// Insert (v, id) into a descending list of kTopSlots entries held in registers.
+__device__ __forceinline__ void topk_insert(float (&val)[kTopSlots], int (&id)[kTopSlots], float v, int i) {
+    if (!ranks_before(v, i, val[kTopSlots - 1], id[kTopSlots - 1])) return;
+#pragma unroll
+    for (int s = kTopSlots - 1; s >= 0; --s) {
+        bool shift = (s > 0) && ranks_before(v, i, val[s - 1], id[s - 1]);
+        bool here = !shift && ranks_before(v, i, val[s], id[s]);
+        float pv = (s > 0) ? val[s - 1] : 0.f;
+        int pi = (s > 0) ? id[s - 1] : 0;
+        if (shift) { val[s] = pv; id[s] = pi; }
+        else if (here) { val[s] = v; id[s] = i; }
+    }
+}
+
+__device__ __forceinline__ void report_error(int* status, int code, int detail) {
+    if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace ctcsd
+
+// The opaque handle of the C ABI wraps the C++ state.
+struct ctcsd_handle {
+    ctcsd::Handle h;
+};

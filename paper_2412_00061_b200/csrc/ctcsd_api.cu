@@ -1,0 +1,137 @@
+// Handle management, configuration checks and workspace layout for the ctcsd C ABI.
+#include "common.cuh"
+
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+
+namespace ctcsd {
+
+int validate_config(const ctcsd_config& c) {
+    if (c.B < 1 || c.H < 8 || c.H % 8 != 0 || c.V < 1) return CTCSD_ERR_INVALID_ARG;
+    if (c.T < 1 || c.T > CTCSD_MAX_T || c.k < 1 || c.k > CTCSD_MAX_K) return CTCSD_ERR_INVALID_ARG;
+    if (c.k > c.V + 1 || c.T * c.k > 64) return CTCSD_ERR_INVALID_ARG;
+    if (c.beam < 0 || c.beam > CTCSD_MAX_BEAM) return CTCSD_ERR_INVALID_ARG;
+    if (c.beam == 0) {
+        long long paths = 1;
+        for (int t = 0; t < c.T; ++t) paths *= c.k;
+        if (paths > CTCSD_MAX_PATHS) return CTCSD_ERR_INVALID_ARG;
+    }
+    if (c.topN < 1 || c.topN > CTCSD_MAX_TOPN) return CTCSD_ERR_INVALID_ARG;
+    if (c.max_nodes < 2 || c.max_nodes > CTCSD_MAX_NODES) return CTCSD_ERR_INVALID_ARG;
+    if (c.Hq < 1 || c.Hkv < 1 || c.Hq % c.Hkv != 0) return CTCSD_ERR_INVALID_ARG;
+    if (c.D != 64 && c.D != 128) return CTCSD_ERR_INVALID_ARG;
+    if (c.dtype != CTCSD_DTYPE_F32 && c.dtype != CTCSD_DTYPE_BF16) return CTCSD_ERR_INVALID_ARG;
+    if (c.score_mode != CTCSD_SCORE_SUM && c.score_mode != CTCSD_SCORE_MAX) return CTCSD_ERR_INVALID_ARG;
+    if (c.score_mode == CTCSD_SCORE_MAX && c.beam != 0) return CTCSD_ERR_UNSUPPORTED;
+    if (c.max_draft_rows < 0) return CTCSD_ERR_INVALID_ARG;
+    if ((long long)c.B * c.max_nodes > (1 << 20)) return CTCSD_ERR_INVALID_ARG;
+    return CTCSD_OK;
+}
+
+Layout make_layout(const ctcsd_config& c, int num_sms) {
+    Layout l;
+    memset(&l, 0, sizeof(l));
+    size_t off = 0;
+    l.status_off = off;      off = align_up(off + 16 * sizeof(int), 256);
+    l.counter_off = off;     off = align_up(off + kCounters * sizeof(unsigned), 256);
+    l.gemv_grid_max = num_sms * 8 > 64 ? num_sms * 8 : 64;
+    l.draft_part_off = off;  off = align_up(off + sizeof(DraftPartial) * 4 * (size_t)l.gemv_grid_max * 2, 256);
+    l.part_slot_off = off;   off = align_up(off + sizeof(int) * (size_t)l.gemv_grid_max * 2, 256);
+    l.lm_tiles_max = (c.V + 15) / 16 + 8;
+    l.lm_part_off = off;     off = align_up(off + sizeof(ArgmaxPartial) * (size_t)l.lm_tiles_max * c.B * c.max_nodes, 256);
+    int units = c.B * c.Hkv;
+    int splits = (2 * num_sms + units - 1) / units;
+    if (splits < 1) splits = 1;
+    if (splits > 16) splits = 16;
+    l.kv_splits = splits;
+    l.attn_part_off = off;
+    off = align_up(off + sizeof(float) * (size_t)c.B * c.Hq * c.max_nodes * splits * (c.D + 2), 256);
+    l.total = off;
+    return l;
+}
+
+}  // namespace ctcsd
+
+using namespace ctcsd;
+
+// The workspace size depends on the SM count only through upper bounds; 160 covers every
+// B200 configuration and lets the size be queried without a device.
+static const int kLayoutSms = 160;
+
+extern "C" int ctcsd_workspace_bytes(const ctcsd_config* cfg, size_t* out_bytes) {
+    if (!cfg || !out_bytes) return CTCSD_ERR_INVALID_ARG;
+    int rc = validate_config(*cfg);
+    if (rc != CTCSD_OK) return rc;
+    *out_bytes = make_layout(*cfg, kLayoutSms).total;
+    return CTCSD_OK;
+}
+
+extern "C" int ctcsd_create(ctcsd_handle** out_handle, const ctcsd_config* cfg, void* workspace, size_t workspace_bytes) {
+    if (!out_handle || !cfg) return CTCSD_ERR_INVALID_ARG;
+    *out_handle = nullptr;
+    int rc = validate_config(*cfg);
+    if (rc != CTCSD_OK) return rc;
+    Layout lay = make_layout(*cfg, kLayoutSms);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < lay.total)
+        return CTCSD_ERR_WORKSPACE;
+    ctcsd_handle* hh = new (std::nothrow) ctcsd_handle;
+    if (!hh) return CTCSD_ERR_INTERNAL;
+    Handle* h = &hh->h;
+    memset(h, 0, sizeof(*h));
+    h->cfg = *cfg;
+    if (h->cfg.max_draft_rows == 0) h->cfg.max_draft_rows = cfg->B;
+    h->lay = lay;
+    h->ws = static_cast<char*>(workspace);
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+    int major = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, h->device);
+    if (e == cudaSuccess && major != 10) { delete hh; return CTCSD_ERR_UNSUPPORTED; }
+    if (e == cudaSuccess && h->num_sms > kLayoutSms) { delete hh; return CTCSD_ERR_UNSUPPORTED; }
+    // status word and ticket counters start at zero
+    if (e == cudaSuccess) e = cudaMemset(workspace, 0, lay.draft_part_off);
+    if (e != cudaSuccess) { delete hh; return CTCSD_ERR_CUDA; }
+    *out_handle = hh;
+    return CTCSD_OK;
+}
+
+extern "C" int ctcsd_destroy(ctcsd_handle* h) {
+    if (!h) return CTCSD_ERR_INVALID_ARG;
+    delete h;
+    return CTCSD_OK;
+}
+
+extern "C" int ctcsd_poll_status(ctcsd_handle* hh, void* stream, int* out_status) {
+    if (!hh || !out_status) return CTCSD_ERR_INVALID_ARG;
+    Handle* h = &hh->h;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int st[2] = {0, 0};
+    CTCSD_CUDA_CHECK(h, cudaMemcpyAsync(st, status_ptr(h), sizeof(st), cudaMemcpyDeviceToHost, s));
+    CTCSD_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    if (st[0] != 0) {
+        CTCSD_CUDA_CHECK(h, cudaMemsetAsync(status_ptr(h), 0, 16 * sizeof(int), s));
+        // a kernel that gave up may have left its ticket counters mid-count
+        CTCSD_CUDA_CHECK(h, cudaMemsetAsync(counter_ptr(h), 0, kCounters * sizeof(unsigned), s));
+        CTCSD_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    }
+    *out_status = st[0];
+    return CTCSD_OK;
+}
+
+extern "C" const char* ctcsd_strerror(int status) {
+    switch (status) {
+        case CTCSD_OK: return "ok";
+        case CTCSD_ERR_INVALID_ARG: return "invalid argument";
+        case CTCSD_ERR_UNSUPPORTED: return "unsupported configuration";
+        case CTCSD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CTCSD_ERR_CUDA: return "CUDA call failed";
+        case CTCSD_ERR_TIMEOUT: return "device-side wait timed out";
+        case CTCSD_ERR_INTERNAL: return "internal error";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int ctcsd_last_cuda_error(const ctcsd_handle* h) { return h ? h->h.last_cuda_error : 0; }
+
+extern "C" long long ctcsd_launch_count(const ctcsd_handle* h) { return h ? h->h.launches : 0; }

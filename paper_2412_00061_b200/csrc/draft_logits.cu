@@ -1,0 +1,38 @@
+// ctcsd_draft_logits: draft-head projection, per-slot log-softmax and per-slot top-k.
+#include "gemv_stream.cuh"
+
+using namespace ctcsd;
+
+extern "C" int ctcsd_draft_logits(ctcsd_handle* hh, void* stream, int M, const void* x, const void* Wd,
+                                  const int* row_seq, const float* blank_bias,
+                                  int* out_topk_id, float* out_topk_lp, float* out_lse, float* out_logits_dbg) {
+    if (!hh || !x || !Wd || !out_topk_id || !out_topk_lp || !out_lse) return CTCSD_ERR_INVALID_ARG;
+    Handle* h = &hh->h;
+    const ctcsd_config& c = h->cfg;
+    if (M < 1 || M > c.max_draft_rows) return CTCSD_ERR_INVALID_ARG;
+    if (!row_seq && blank_bias && M > c.B) return CTCSD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(Wd)) & 15) return CTCSD_ERR_INVALID_ARG;
+
+    GemvParams p;
+    p.x = x;
+    p.W = Wd;
+    p.row_seq = row_seq;
+    p.blank_bias = blank_bias;
+    p.m0 = 0;
+    p.mcount = 0;
+    p.H = c.H;
+    p.slots = c.T;
+    p.rows_per_slot = c.V + 1;
+    p.grid = 0;
+    p.part = nullptr;
+    p.part_slot = nullptr;
+    p.counter = nullptr;
+    p.mode = 0;
+    p.k = c.k;
+    p.out_topk_id = out_topk_id;
+    p.out_topk_lp = out_topk_lp;
+    p.out_lse = out_lse;
+    p.out_argmax = nullptr;
+    p.logits_dbg = out_logits_dbg;
+    return launch_gemv_stream(h, static_cast<cudaStream_t>(stream), c.dtype, M, p);
+}

@@ -1,0 +1,16 @@
+// Tensor-core (tcgen05 / TMEM) LM head with fused row arg-max.
+#pragma once
+
+#include "common.cuh"
+
+namespace ctcsd {
+
+// True when the handle's shape and dtype are served by the tensor-core kernel.
+bool lm_head_tc_supported(const Handle* h);
+
+// y = hn . Wl^T on the 5th-generation tensor cores with the row arg-max folded into the
+// epilogue.  Returns CTCSD_ERR_UNSUPPORTED when the shape is not covered.
+int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, const void* Wl,
+                      int* out_argmax, float* out_logits_dbg);
+
+}  // namespace ctcsd

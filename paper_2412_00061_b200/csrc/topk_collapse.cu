@@ -1,0 +1,381 @@
+// ctcsd_topk_collapse: slot paths -> CTC collapse -> dedup + alignment-sum score -> top-N.
+//
+// One CTA per sequence.  The at most T*k <= 64 distinct tokens of the per-slot lists get
+// local ids in ascending token order, so a collapsed sequence packs into one 64-bit key
+// (length in the top bits, then 6 bits per position) whose unsigned order is exactly
+// "shorter first, then token ids lexicographically ascending".  Keys are deduplicated in a
+// shared-memory hash table.  Scores are formed in float64; the sum over a candidate's
+// alignments is accumulated in 64-bit fixed point relative to the candidate's best
+// alignment, which makes it independent of the order in which threads arrive.
+#include "common.cuh"
+
+#include <math.h>
+
+namespace ctcsd {
+namespace {
+
+constexpr int kThreads = 512;
+constexpr unsigned long long kEmpty = ~0ull;
+constexpr int kBlankMark = 255;
+constexpr double kFix = 1125899906842624.0;          // 2^50
+constexpr int kBeamCap = 2048;                       // hash capacity for one beam step
+
+struct CollapseParams {
+    const int* topk_id;      // [M,T,k]
+    const float* topk_lp;    // [M,T,k]
+    const int* sel_row;      // [B] or null
+    int M, T, k, V, topN, beam, score_mode;
+    int npaths;              // k^T (enumeration)
+    int cap;                 // hash capacity (power of two)
+    int* out_cand_tok;       // [B,topN,T]
+    int* out_cand_len;       // [B,topN]
+    float* out_cand_score;   // [B,topN]
+    int* out_n_cand;         // [B]
+    int* status;
+};
+
+__device__ __forceinline__ int key_len(unsigned long long key) { return (int)(key >> 48); }
+__device__ __forceinline__ int key_tok(unsigned long long key, int i) { return (int)((key >> (6 * (7 - i))) & 63ull); }
+__device__ __forceinline__ unsigned long long key_append(unsigned long long key, int lid) {
+    int len = key_len(key);
+    return (key & 0x0000ffffffffffffull) | ((unsigned long long)(len + 1) << 48) |
+           ((unsigned long long)lid << (6 * (7 - len)));
+}
+
+__device__ __forceinline__ unsigned hash_key(unsigned long long key, int cap) {
+    unsigned long long h = key * 0x9E3779B97F4A7C15ull;
+    return (unsigned)(h >> 40) & (unsigned)(cap - 1);
+}
+
+// Finds or claims the slot of `key`.  The table never fills (capacity >= 2x the entries).
+__device__ __forceinline__ int table_insert(unsigned long long* keys, int cap, unsigned long long key) {
+    unsigned s = hash_key(key, cap);
+    for (int probe = 0; probe < cap; ++probe) {
+        unsigned long long cur = keys[s];
+        if (cur == key) return (int)s;
+        if (cur == kEmpty) {
+            unsigned long long old = atomicCAS(&keys[s], kEmpty, key);
+            if (old == kEmpty || old == key) return (int)s;
+        }
+        s = (s + 1) & (unsigned)(cap - 1);
+    }
+    return -1;
+}
+
+__device__ __forceinline__ long long dbl_sortable(double d) {
+    long long v = __double_as_longlong(d);
+    return v ^ ((v >> 63) & 0x7fffffffffffffffll);
+}
+__device__ __forceinline__ double sortable_dbl(long long v) {
+    return __longlong_as_double(v ^ ((v >> 63) & 0x7fffffffffffffffll));
+}
+
+__device__ __forceinline__ double logadd(double a, double b) {
+    if (a == -INFINITY) return b;
+    if (b == -INFINITY) return a;
+    double hi = fmax(a, b), lo = fmin(a, b);
+    return hi + log1p(exp(lo - hi));
+}
+
+// (score, key) a precedes b: higher score; equal scores -> smaller key (shorter, then lexicographic)
+__device__ __forceinline__ bool precedes(double sa, unsigned long long ka, double sb, unsigned long long kb) {
+    return sa > sb || (sa == sb && ka < kb);
+}
+
+// Shared bookkeeping common to both modes: the slot lists and the local token ids.
+struct SlotLists {
+    int tok[CTCSD_MAX_T * CTCSD_MAX_K];        // token id of (t, j)
+    double lp[CTCSD_MAX_T * CTCSD_MAX_K];
+    unsigned char lid[CTCSD_MAX_T * CTCSD_MAX_K];   // local id, kBlankMark for the blank
+    int sorted_tok[64];                        // local id -> token id
+};
+
+__device__ void load_slot_lists(const CollapseParams& p, int row, SlotLists& sl) {
+    const int n = p.T * p.k;
+    const int tid = threadIdx.x;
+    if (tid < n) {
+        sl.tok[tid] = p.topk_id[(size_t)row * n + tid];
+        sl.lp[tid] = (double)p.topk_lp[(size_t)row * n + tid];
+    }
+    __syncthreads();
+    if (tid < n) {
+        int me = sl.tok[tid];
+        if (me == p.V) {
+            sl.lid[tid] = kBlankMark;
+        } else {
+            // local id = number of distinct non-blank tokens smaller than mine
+            int cnt = 0;
+            for (int j = 0; j < n; ++j) {
+                int tj = sl.tok[j];
+                if (tj == p.V || tj >= me) continue;
+                bool first = true;
+                for (int q = 0; q < j; ++q) if (sl.tok[q] == tj) { first = false; break; }
+                cnt += first ? 1 : 0;
+            }
+            sl.lid[tid] = (unsigned char)cnt;
+            sl.sorted_tok[cnt] = me;
+        }
+    }
+    __syncthreads();
+}
+
+// Ranks the table entries and writes the best topN non-empty candidates.
+__device__ void emit_top_candidates(const CollapseParams& p, int b, const SlotLists& sl,
+                                    const unsigned long long* keys, const double* score, int cap) {
+    __shared__ int s_count;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_count = 0;
+    int* ctok = p.out_cand_tok + (size_t)b * p.topN * p.T;
+    int* clen = p.out_cand_len + (size_t)b * p.topN;
+    float* cscore = p.out_cand_score + (size_t)b * p.topN;
+    for (int i = tid; i < p.topN * p.T; i += kThreads) ctok[i] = -1;
+    for (int i = tid; i < p.topN; i += kThreads) { clen[i] = 0; cscore[i] = -INFINITY; }
+    __syncthreads();
+    for (int i = tid; i < cap; i += kThreads) {
+        unsigned long long ki = keys[i];
+        if (ki == kEmpty || key_len(ki) == 0) continue;
+        double si = score[i];
+        int rank = 0;
+        for (int j = 0; j < cap; ++j) {
+            unsigned long long kj = keys[j];
+            if (kj == kEmpty || key_len(kj) == 0) continue;
+            rank += precedes(score[j], kj, si, ki) ? 1 : 0;
+        }
+        atomicAdd(&s_count, 1);
+        if (rank < p.topN) {
+            int len = key_len(ki);
+            clen[rank] = len;
+            cscore[rank] = (float)si;
+            for (int l = 0; l < len; ++l) ctok[rank * p.T + l] = sl.sorted_tok[key_tok(ki, l)];
+        }
+    }
+    __syncthreads();
+    if (tid == 0) p.out_n_cand[b] = s_count < p.topN ? s_count : p.topN;
+}
+
+// ---------------------------------------------------------------------------------------
+// Exhaustive enumeration of the k^T slot paths
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams p) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);             // [cap]
+    long long* best = reinterpret_cast<long long*>(keys + p.cap);                      // [cap] sortable max, then score
+    unsigned long long* fsum = reinterpret_cast<unsigned long long*>(best + p.cap);    // [cap] fixed-point sum
+    unsigned short* path_slot = reinterpret_cast<unsigned short*>(fsum + p.cap);       // [npaths]
+    __shared__ SlotLists sl;
+
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int row = p.sel_row ? p.sel_row[b] : b;
+    if (row < 0 || row >= p.M) {
+        if (tid == 0) { report_error(p.status, CTCSD_ERR_INVALID_ARG, b); p.out_n_cand[b] = 0; }
+        return;
+    }
+    load_slot_lists(p, row, sl);
+    const long long neg_inf_sortable = dbl_sortable(-INFINITY);
+    for (int i = tid; i < p.cap; i += kThreads) { keys[i] = kEmpty; best[i] = neg_inf_sortable; fsum[i] = 0ull; }
+    __syncthreads();
+
+    // pass 1: collapse every path, claim a table slot, track the best alignment
+    for (int path = tid; path < p.npaths; path += kThreads) {
+        int rem = path;
+        int digit[CTCSD_MAX_T];
+#pragma unroll
+        for (int t = CTCSD_MAX_T - 1; t >= 0; --t) {
+            if (t < p.T) { digit[t] = rem % p.k; rem /= p.k; } else digit[t] = 0;
+        }
+        double s = 0.0;
+        unsigned long long key = 0ull;
+        int prev = -1;
+#pragma unroll
+        for (int t = 0; t < CTCSD_MAX_T; ++t) {
+            if (t < p.T) {
+                int e = t * p.k + digit[t];
+                s += sl.lp[e];
+                int m = sl.lid[e];
+                if (m != prev && m != kBlankMark) key = key_append(key, m);
+                prev = m;
+            }
+        }
+        int slot = table_insert(keys, p.cap, key);
+        if (slot < 0) { report_error(p.status, CTCSD_ERR_INTERNAL, 1); slot = 0; }
+        path_slot[path] = (unsigned short)slot;
+        atomicMax(&best[slot], dbl_sortable(s));
+    }
+    __syncthreads();
+
+    // pass 2: sum exp(s - best) per candidate in fixed point (order independent)
+    if (p.score_mode == CTCSD_SCORE_SUM) {
+        for (int path = tid; path < p.npaths; path += kThreads) {
+            int rem = path;
+            double s = 0.0;
+            int digit[CTCSD_MAX_T];
+#pragma unroll
+            for (int t = CTCSD_MAX_T - 1; t >= 0; --t) {
+                if (t < p.T) { digit[t] = rem % p.k; rem /= p.k; } else digit[t] = 0;
+            }
+#pragma unroll
+            for (int t = 0; t < CTCSD_MAX_T; ++t)
+                if (t < p.T) s += sl.lp[t * p.k + digit[t]];
+            int slot = path_slot[path];
+            double mx = sortable_dbl(best[slot]);
+            double term = exp(s - mx) * kFix;
+            atomicAdd(&fsum[slot], __double2ull_rn(term));
+        }
+    }
+    __syncthreads();
+    double* score = reinterpret_cast<double*>(best);
+    for (int i = tid; i < p.cap; i += kThreads) {
+        if (keys[i] == kEmpty) continue;
+        double mx = sortable_dbl(best[i]);
+        double sc = mx;
+        if (p.score_mode == CTCSD_SCORE_SUM) sc = mx + log((double)fsum[i] * (1.0 / kFix));
+        score[i] = sc;
+    }
+    __syncthreads();
+    emit_top_candidates(p, b, sl, keys, score, p.cap);
+}
+
+// ---------------------------------------------------------------------------------------
+// CTC prefix beam search over the per-slot lists
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams p) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);   // [kBeamCap]
+    double* t_pb = reinterpret_cast<double*>(keys + kBeamCap);    // mass ending in blank (one contributor: the prefix itself)
+    double* t_stay = t_pb + kBeamCap;        // ending in the last token, from the prefix itself (repeat)
+    double* t_ext = t_stay + kBeamCap;       // ending in the last token, from the parent prefix (extension)
+    __shared__ unsigned long long bm_key[CTCSD_MAX_BEAM];
+    __shared__ double bm_pb[CTCSD_MAX_BEAM], bm_pnb[CTCSD_MAX_BEAM];
+    __shared__ int s_nbeam, s_next;
+    __shared__ SlotLists sl;
+
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int row = p.sel_row ? p.sel_row[b] : b;
+    if (row < 0 || row >= p.M) {
+        if (tid == 0) { report_error(p.status, CTCSD_ERR_INVALID_ARG, b); p.out_n_cand[b] = 0; }
+        return;
+    }
+    load_slot_lists(p, row, sl);
+    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 0.0; bm_pnb[0] = -INFINITY; s_nbeam = 1; }
+    __syncthreads();
+
+    for (int t = 0; t < p.T; ++t) {
+        for (int i = tid; i < kBeamCap; i += kThreads) {
+            keys[i] = kEmpty; t_pb[i] = -INFINITY; t_stay[i] = -INFINITY; t_ext[i] = -INFINITY;
+        }
+        if (tid == 0) s_next = 0;
+        __syncthreads();
+        const int nbeam = s_nbeam;
+        for (int w = tid; w < nbeam * p.k; w += kThreads) {
+            const int e = w / p.k, j = w - e * p.k;
+            const unsigned long long key = bm_key[e];
+            const double pb = bm_pb[e], pnb = bm_pnb[e];
+            const double tot = logadd(pb, pnb);
+            const int m = sl.lid[t * p.k + j];
+            const double lp = sl.lp[t * p.k + j];
+            const int len = key_len(key);
+            const int last = len > 0 ? key_tok(key, len - 1) : -1;
+            if (m == kBlankMark) {
+                int s = table_insert(keys, kBeamCap, key);
+                if (s >= 0) t_pb[s] = tot + lp;
+            } else if (m == last) {
+                if (pnb != -INFINITY) {
+                    int s = table_insert(keys, kBeamCap, key);
+                    if (s >= 0) t_stay[s] = pnb + lp;
+                }
+                if (pb != -INFINITY) {
+                    int s = table_insert(keys, kBeamCap, key_append(key, m));
+                    if (s >= 0) t_ext[s] = pb + lp;
+                }
+            } else {
+                int s = table_insert(keys, kBeamCap, key_append(key, m));
+                if (s >= 0) t_ext[s] = tot + lp;
+            }
+        }
+        __syncthreads();
+        // total mass per prefix, then keep the best `beam` in ranked order
+        for (int i = tid; i < kBeamCap; i += kThreads) {
+            if (keys[i] == kEmpty) continue;
+            double pnb = logadd(t_stay[i], t_ext[i]);
+            t_stay[i] = pnb;
+            t_ext[i] = logadd(t_pb[i], pnb);
+        }
+        __syncthreads();
+        for (int i = tid; i < kBeamCap; i += kThreads) {
+            unsigned long long ki = keys[i];
+            if (ki == kEmpty) continue;
+            double si = t_ext[i];
+            int rank = 0;
+            for (int j = 0; j < kBeamCap; ++j) {
+                unsigned long long kj = keys[j];
+                if (kj == kEmpty) continue;
+                rank += precedes(t_ext[j], kj, si, ki) ? 1 : 0;
+            }
+            atomicAdd(&s_next, 1);
+            if (rank < p.beam) { bm_key[rank] = ki; bm_pb[rank] = t_pb[i]; bm_pnb[rank] = t_stay[i]; }
+        }
+        __syncthreads();
+        if (tid == 0) s_nbeam = s_next < p.beam ? s_next : p.beam;
+        __syncthreads();
+    }
+    // after the last slot the table still holds every surviving prefix with its total mass;
+    // entries pruned by the beam cut must not be candidates, so rebuild the table from the beam
+    const int nbeam = s_nbeam;
+    for (int i = tid; i < kBeamCap; i += kThreads) keys[i] = kEmpty;
+    __syncthreads();
+    for (int e = tid; e < nbeam; e += kThreads) {
+        int s = table_insert(keys, kBeamCap, bm_key[e]);
+        if (s >= 0) t_ext[s] = logadd(bm_pb[e], bm_pnb[e]);
+    }
+    __syncthreads();
+    emit_top_candidates(p, b, sl, keys, t_ext, kBeamCap);
+}
+
+}  // namespace
+}  // namespace ctcsd
+
+using namespace ctcsd;
+
+extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const int* topk_id, const float* topk_lp,
+                                   const int* sel_row,
+                                   int* out_cand_tok, int* out_cand_len, float* out_cand_score, int* out_n_cand) {
+    if (!hh || !topk_id || !topk_lp || !out_cand_tok || !out_cand_len || !out_cand_score || !out_n_cand)
+        return CTCSD_ERR_INVALID_ARG;
+    Handle* h = &hh->h;
+    const ctcsd_config& c = h->cfg;
+    if (M < 1) return CTCSD_ERR_INVALID_ARG;
+    if (!sel_row && M < c.B) return CTCSD_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    CollapseParams p;
+    p.topk_id = topk_id;
+    p.topk_lp = topk_lp;
+    p.sel_row = sel_row;
+    p.M = M; p.T = c.T; p.k = c.k; p.V = c.V; p.topN = c.topN; p.beam = c.beam; p.score_mode = c.score_mode;
+    p.npaths = 0; p.cap = 0;
+    p.out_cand_tok = out_cand_tok;
+    p.out_cand_len = out_cand_len;
+    p.out_cand_score = out_cand_score;
+    p.out_n_cand = out_n_cand;
+    p.status = status_ptr(h);
+
+    if (c.beam > 0) {
+        const size_t smem = (size_t)kBeamCap * 32;
+        CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_beam_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        collapse_beam_kernel<<<c.B, kThreads, smem, s>>>(p);
+        CTCSD_LAUNCH_CHECK(h);
+        return CTCSD_OK;
+    }
+    int npaths = 1;
+    for (int t = 0; t < c.T; ++t) npaths *= c.k;
+    int cap = 64;
+    while (cap < 2 * npaths) cap <<= 1;
+    p.npaths = npaths;
+    p.cap = cap;
+    size_t smem = (size_t)cap * 24 + (size_t)npaths * 2;
+    if (smem > 48 * 1024)
+        CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_enum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    collapse_enum_kernel<<<c.B, kThreads, smem, s>>>(p);
+    CTCSD_LAUNCH_CHECK(h);
+    return CTCSD_OK;
+}

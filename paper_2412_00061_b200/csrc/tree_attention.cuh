@@ -1,0 +1,21 @@
+// Parameters shared by the tree-attention kernels.
+#pragma once
+
+#include "common.cuh"
+
+namespace ctcsd {
+
+struct AttnParams {
+    const void* Q;      // [B,max_nodes,Hq,D]
+    const void* K;      // [B,Hkv,Lcap,D]
+    const void* V;      // [B,Hkv,Lcap,D]
+    void* O;            // [B,max_nodes,Hq,D]
+    const int* kv_len;  // [B]
+    const int* n_nodes; // [B]
+    const unsigned long long* mask;   // [B,max_nodes,ceil(max_nodes/64)]
+    int B, Hq, Hkv, D, max_nodes, Lcap;
+    float scale;
+    int* status;
+};
+
+}  // namespace ctcsd

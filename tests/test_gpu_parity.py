@@ -1,0 +1,94 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, stage by stage.
+
+Tolerances (written out here as the acceptance bar): integer outputs bit-exact when the oracle
+is fed the CUDA path's previous-stage output; logits and attention outputs within 2e-2 max-abs
+for bf16 inputs with fp32 accumulation (2e-4 for fp32 inputs); fp32 log-probabilities within
+1e-4 relative."""
+import numpy as np
+import pytest
+
+from paper_2412_00061_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+C = synth.CONFIGS
+
+# scaled-down instances of the five workloads: several tiles, ragged tails, odd V+1
+SMALL = {
+    "c2s": C["c2"].replace(name="c2s", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200),
+    "c3s": C["c3"].replace(name="c3s", B=3, H=512, V=1777, Hq=4, Hkv=4, kv_lo=70, kv_hi=300, beam=16),
+    "c4s": C["c4"].replace(name="c4s", B=2, H=640, V=2500, Hq=4, Hkv=4, kv_lo=333, kv_hi=333),
+    "c5s": C["c5"].replace(name="c5s", B=5, H=1024, V=1200, Hq=8, Hkv=2, kv_lo=100, kv_hi=500),
+    "c1d64": C["c1"].replace(name="c1d64", B=2, H=264, V=777, kv_lo=1, kv_hi=90, dtype="bf16"),
+}
+
+
+def _run(cfg, **kw):
+    from tests.parity_util import run_parity
+    return run_parity(cfg, **kw)
+
+
+def test_c1_tiny_fp32_full():
+    r = _run(C["c1"], seed=0, require_certified=True)
+    assert r["n_nodes"][0] >= 2
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+@pytest.mark.parametrize("seed", [0, 1])
+def test_small_shapes(name, seed):
+    _run(SMALL[name], seed=seed)
+
+
+def test_forced_repeats_make_real_duplicates():
+    r = _run(SMALL["c2s"], seed=3, force_repeats=True)
+    assert r["n_nodes"][0] >= 2
+
+
+def test_many_draft_rows_with_row_and_sel_maps():
+    # draft head on 11 rows (three passes of the row-blocked kernel), 3 sequences pick rows 9, 0, 4
+    cfg = SMALL["c3s"]
+    row_seq = np.array([0, 1, 2, 0, 1, 2, 0, 1, 2, 0, 1], dtype=np.int32)
+    sel_row = np.array([9, 0, 4], dtype=np.int32)
+    _run(cfg, seed=2, M=11, row_seq=row_seq, sel_row=sel_row)
+
+
+def test_enumeration_limits_and_max_score_mode():
+    # 4096 paths (T=6, k=4) enumerated exhaustively; best-alignment scoring variant
+    _run(C["c1"].replace(name="enum4096", T=6, k=4, topN=64, max_nodes=128), seed=0)
+    _run(C["c1"].replace(name="maxmode", score_mode=1), seed=0)
+    # k = V + 1: the lists hold the whole distribution (tiny vocabulary)
+    _run(C["c1"].replace(name="tinyV", V=4, k=5, T=3, H=64), seed=0)
+
+
+def test_only_blank_paths_leave_just_the_root():
+    # a huge blank bias with k = 1 makes every slot pick the blank: no candidate, tree = root
+    cfg = C["c1"].replace(name="allblank", k=1, blank_bias=(50.0,))
+    r = _run(cfg, seed=0)
+    assert r["n_nodes"][0] == 1 and r["acc_len"][0] == 0
+
+
+def test_c2_full_size_sampled():
+    """The headline workload at full size, in the launch configuration the benchmark times.
+    The definition-mode oracle checks one draft row in full, sampled LM-head rows and sampled
+    attention (sequence, head) pairs; all integer stages are compared in full."""
+    r = _run(C["c2"], seed=0, require_certified=True, attention_rows=4, lm_rows=8)
+    assert 2 <= r["n_nodes"][0] <= 64
+
+
+def test_invalid_arguments_are_rejected_on_the_host():
+    import ctypes
+    from paper_2412_00061_b200 import binding
+    lib = binding.load_library()
+    bad = binding.CConfig(1, 250, 100, 4, 3, 0, 8, 32, 4, 4, 64, 0, 0, 0)     # H not a multiple of 8
+    n = ctypes.c_size_t(0)
+    assert lib.ctcsd_workspace_bytes(ctypes.byref(bad), ctypes.byref(n)) == -1
+    too_many = binding.CConfig(1, 256, 100, 7, 4, 0, 8, 32, 4, 4, 64, 0, 0, 0)  # 4^7 paths > 4096
+    assert lib.ctcsd_workspace_bytes(ctypes.byref(too_many), ctypes.byref(n)) == -1
+    h = ctypes.c_void_p()
+    ok = binding.CConfig(1, 256, 100, 4, 3, 0, 8, 32, 4, 4, 64, 0, 0, 0)
+    assert lib.ctcsd_create(ctypes.byref(h), ctypes.byref(ok), None, 0) == -3   # no workspace
+    with pytest.raises(binding.CtcsdError):
+        import torch
+        hd = binding.Handle(1, 256, 100, 4, 3, 0, 8, 32, 4, 4, 64, 0)
+        x = torch.zeros(1, 256, device="cuda")
+        hd.draft_logits(x, x, None, None, x, x, x)          # wrong sizes and dtypes
