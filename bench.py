@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-and-verify step (the five C-ABI calls back to back on one stream).
+
+Default workload: the Vicuna-7B-shaped step (batch 1, hidden 4096, vocab 32000 + blank, T=5,
+top-k 4, top-N 16, <= 64-node tree, 32 heads x 128 over 1024 cached tokens, bf16).  One
+"step" is one pass S1..S11 over synthetic, seeded inputs that are resident in HBM.  With
+N > 1 GPUs every rank runs its own replica of the step on its own sequences (the path is
+independent per sequence: no collective on the data path), so the aggregate is N x.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "draft+verify steps/s at 7B shape (batch 1, 64-node tree)"
+UNIT = "steps/s"
+
+
+def algorithmic_bytes(cfg, mean_kv_len, n_live):
+    """Bytes the method must move per step: every draft-head and LM-head weight once, every
+    live key/value row once (activations, lists and tree arrays are < 0.1 %)."""
+    esz = 2 if cfg.dtype == "bf16" else 4
+    draft = cfg.T * (cfg.V + 1) * cfg.H * esz
+    lm = cfg.V * cfg.H * esz
+    kv = 2 * cfg.B * cfg.Hkv * (mean_kv_len + n_live) * cfg.D * esz
+    return draft, lm, kv
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        clocks, reasons, mx = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                clocks.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nme, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        self.f.close()
+        os.unlink(self.f.name)
+        if clocks:
+            out["sm_mhz"] = float(np.median(clocks))
+            out["sm_max_mhz"] = mx
+            out["reasons"] = sorted(reasons)
+            out["samples"] = len(clocks)
+        return out
+
+
+def oracle_step(cfg, inp, sample_slots=None):
+    """One pass of the CPU oracle over the step (definition mode, fp64).  Returns nothing:
+    it is only timed."""
+    import math
+
+    from oracle import ctcsd_oracle as orc
+    from paper_2412_00061_b200 import synth
+    z = orc.draft_logits(inp["x"], inp["Wd"], inp["blank_bias"])
+    ids, lps = orc.topk_slots(z, cfg.k)
+    ctok, clen, cscore, nc = orc.topk_collapse(ids, lps, cfg.V, cfg.T, cfg.topN, cfg.beam, cfg.score_mode)
+    tree = orc.build_tree(inp["base_tok"], inp["kv_len"], ctok, clen, nc, cfg.max_nodes)
+    node_tok, parent, depth, pos, mask, retrieve, n_nodes = tree
+    orc.tree_attention(inp["Q"], inp["K"], inp["V"], inp["kv_len"], n_nodes, mask, 1.0 / math.sqrt(cfg.D))
+    if "hn" not in inp:
+        inp["hn"], _ = synth.gen_node_hidden(cfg, 0, inp["Wl"], node_tok, parent, n_nodes)
+    _, am = orc.lm_head_argmax(inp["hn"], inp["Wl"])
+    orc.greedy_accept(node_tok, parent, n_nodes, am.reshape(cfg.B, cfg.max_nodes), cfg.T)
+
+
+def host_inputs(cfg, seed):
+    from paper_2412_00061_b200 import synth
+    x, Wd, bb = synth.gen_draft(cfg, seed)
+    base_tok, kv_len = synth.gen_base(cfg, seed)
+    Q, K, V = synth.gen_attention(cfg, seed)
+    Wl = synth.gen_lm_head(cfg, seed)
+    return dict(x=x, Wd=Wd, blank_bias=bb, base_tok=base_tok, kv_len=kv_len, Q=Q, K=K, V=V, Wl=Wl)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(cfg, inp, steps, warmup):
+    for _ in range(warmup):
+        oracle_step(cfg, inp)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(cfg, inp)
+    return (time.perf_counter() - t0) / steps
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores.  Each step is one full pass of
+    the oracle over the same workload (about two seconds at the 7B shape)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2412_00061_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    inp = host_inputs(cfg, 0)
+    steps = max(1, min(args.steps, 20))
+    warmup = max(1, min(args.warmup, 2))
+    sec = time_oracle(cfg, inp, steps, warmup)
+    val = 1.0 / sec
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "sample": "whole step, all stages"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "%d full steps of the fp64 oracle (numpy, BLAS threads = cores)" % steps},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(cfg):
+    return ("%s: B=%d H=%d V=%d+blank T=%d k=%d %s topN=%d nodes<=%d heads=%d/%d x%d kv=%d..%d %s"
+            % (cfg.name, cfg.B, cfg.H, cfg.V, cfg.T, cfg.k,
+               "enumerate" if cfg.beam == 0 else "beam=%d" % cfg.beam, cfg.topN, cfg.max_nodes,
+               cfg.Hq, cfg.Hkv, cfg.D, cfg.kv_lo, cfg.kv_hi, cfg.dtype))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_00061_b200 import binding, build, synth
+    from paper_2412_00061_b200.step import DraftVerifyStep, to_device
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    build.build()
+    binding.load_library()
+
+    cfg = synth.CONFIGS[args.config]
+    seed = rank                                    # every rank drafts for its own sequences
+    inp = host_inputs(cfg, seed)
+    step = DraftVerifyStep(cfg, device=str(dev))
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    step.set_inputs(x=to_device(inp["x"], cfg.dtype, dev), Wd=to_device(inp["Wd"], cfg.dtype, dev),
+                    blank_bias=torch.from_numpy(inp["blank_bias"]).to(dev),
+                    base_tok=i32(inp["base_tok"]), kv_len=i32(inp["kv_len"]),
+                    Q=to_device(inp["Q"], cfg.dtype, dev), K=to_device(inp["K"], cfg.dtype, dev),
+                    V=to_device(inp["V"], cfg.dtype, dev), Wl=to_device(inp["Wl"], cfg.dtype, dev))
+    # tree-node hidden states need the tree: build it once on the GPU, outside the timed loop
+    step.draft(); step.collapse(); step.tree()
+    step.check_status()
+    node_tok, parent, n_nodes = step.host("node_tok"), step.host("parent"), step.host("n_nodes")
+    hn, _ = synth.gen_node_hidden(cfg, seed, inp["Wl"], node_tok, parent, n_nodes)
+    inp["hn"] = hn
+    step.set_inputs(hn=to_device(hn, cfg.dtype, dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K, Wm = args.steps, max(3, args.warmup)
+    for _ in range(Wm):
+        step.run()
+    step.check_status()
+
+    # ---- device-timed region: inputs resident in HBM -----------------------------------
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_beg, t_end = ev(), ev()
+    d_beg = [ev() for _ in range(K)]
+    d_end = [ev() for _ in range(K)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = step.h.launch_count
+    barrier()
+    t_beg.record()
+    for i in range(K):
+        d_beg[i].record()
+        step.draft()
+        d_end[i].record()
+        step.collapse()
+        step.tree()
+        step.attention()
+        step.verify()
+    t_end.record()
+    barrier()
+    launches = step.h.launch_count - launches0
+    clocks = sampler.stop() if sampler else None
+    step.check_status()
+    ms = t_beg.elapsed_time(t_end)
+    draft_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(d_beg, d_end)]))
+
+    # ---- end to end: per-step inputs come from pinned host memory, results go back ------
+    act = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    pin = lambda t: t.cpu().pin_memory()
+    h_in = {k: pin(step.inp[k]) for k in ("x", "base_tok", "kv_len", "Q", "hn")}
+    h_out = {k: torch.empty_like(step.out[k], device="cpu").pin_memory() for k in ("acc_len", "acc_tok", "next_tok")}
+    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+
+    def e2e_step():
+        for k, t in h_in.items():
+            step.inp[k].copy_(t, non_blocking=True)
+        step.run()
+        for k, t in h_out.items():
+            t.copy_(step.out[k], non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e_beg, e_end = ev(), ev()
+    e_beg.record()
+    for _ in range(K):
+        e2e_step()
+    e_end.record()
+    barrier()
+    e2e_ms = e_beg.elapsed_time(e_end)
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms, draft_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms, draft_ms = [float(v) for v in t.tolist()]
+        tl = torch.tensor([launches], device=dev, dtype=torch.int64)
+        dist.all_reduce(tl)
+        launches = int(tl.item())
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        mean_kv = float(np.mean(inp["kv_len"]))
+        n_live = float(np.mean(n_nodes))
+        draft_b, lm_b, kv_b = algorithmic_bytes(cfg, mean_kv, n_live)
+        achieved = draft_b / (draft_ms * 1e-3) / 1e9
+        step_bytes = draft_b + lm_b + kv_b
+        value = world * K / (ms * 1e-3)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (weights %.0f MB)" % (
+                (draft_b + lm_b) / 1e6), "parallelism": "replicas x%d" % world,
+                "tree_nodes": n_live, "step_bytes": step_bytes,
+                "step_hbm_frac_of_%s_peak" % peak_kind: step_bytes / (ms / K * 1e-3) / 1e9 / peak},
+            "clocks": clocks,
+            "e2e": {"value": world * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches,
+            "roofline": {"kernel": "gemv_stream_kernel (draft head)", "bound": "hbm", "achieved": achieved,
+                         "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": args.traffic},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            n_or = 5
+            sec = time_oracle(cfg, inp, n_or, 1)
+            line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                    "sample": "%d full steps of the fp64 oracle on the same inputs" % n_or}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture (recorded in profiles/)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
