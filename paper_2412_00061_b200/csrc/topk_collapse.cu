@@ -119,38 +119,69 @@ __device__ void load_slot_lists(const CollapseParams& p, int row, SlotLists& sl)
     __syncthreads();
 }
 
-// Ranks the table entries and writes the best topN non-empty candidates.
-__device__ void emit_top_candidates(const CollapseParams& p, int b, const SlotLists& sl,
-                                    const unsigned long long* keys, const double* score, int cap) {
-    __shared__ int s_count;
+// Block-wide bitonic sort of n2 (a power of two) entries into "best first" order:
+// higher score first, equal scores -> smaller key.  ix is an optional payload.
+__device__ void bitonic_sort_best_first(double* sc, unsigned long long* ky, int* ix, int n2) {
     const int tid = threadIdx.x;
-    if (tid == 0) s_count = 0;
+    for (int k = 2; k <= n2; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = tid; t < (n2 >> 1); t += kThreads) {
+                const int lo = t & (j - 1);
+                const int i = ((t - lo) << 1) | lo;
+                const int q = i | j;
+                const bool up = (i & k) == 0;
+                const double si = sc[i], sq = sc[q];
+                const unsigned long long ki = ky[i], kq = ky[q];
+                const bool swap = up ? precedes(sq, kq, si, ki) : precedes(si, ki, sq, kq);
+                if (swap) {
+                    sc[i] = sq; sc[q] = si;
+                    ky[i] = kq; ky[q] = ki;
+                    if (ix) { int a = ix[i]; ix[i] = ix[q]; ix[q] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// Writes the first topN non-empty entries of a best-first list as the candidates.
+__device__ void emit_candidates(const CollapseParams& p, int b, const SlotLists& sl, const double* sc,
+                                const unsigned long long* ky, int count) {
+    __shared__ int s_empty_at;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_empty_at = 0x7fffffff;
     int* ctok = p.out_cand_tok + (size_t)b * p.topN * p.T;
     int* clen = p.out_cand_len + (size_t)b * p.topN;
     float* cscore = p.out_cand_score + (size_t)b * p.topN;
     for (int i = tid; i < p.topN * p.T; i += kThreads) ctok[i] = -1;
     for (int i = tid; i < p.topN; i += kThreads) { clen[i] = 0; cscore[i] = -INFINITY; }
     __syncthreads();
-    for (int i = tid; i < cap; i += kThreads) {
-        unsigned long long ki = keys[i];
-        if (ki == kEmpty || key_len(ki) == 0) continue;
-        double si = score[i];
-        int rank = 0;
-        for (int j = 0; j < cap; ++j) {
-            unsigned long long kj = keys[j];
-            if (kj == kEmpty || key_len(kj) == 0) continue;
-            rank += precedes(score[j], kj, si, ki) ? 1 : 0;
-        }
-        atomicAdd(&s_count, 1);
-        if (rank < p.topN) {
-            int len = key_len(ki);
-            clen[rank] = len;
-            cscore[rank] = (float)si;
-            for (int l = 0; l < len; ++l) ctok[rank * p.T + l] = sl.sorted_tok[key_tok(ki, l)];
-        }
-    }
+    const int look = count < p.topN + 1 ? count : p.topN + 1;      // the empty sequence occurs at most once
+    for (int e = tid; e < look; e += kThreads)
+        if (key_len(ky[e]) == 0) s_empty_at = e;
     __syncthreads();
-    if (tid == 0) p.out_n_cand[b] = s_count < p.topN ? s_count : p.topN;
+    const int empty_at = s_empty_at;
+    for (int e = tid; e < look; e += kThreads) {
+        if (e == empty_at) continue;
+        const int rank = e - (empty_at < e ? 1 : 0);
+        if (rank >= p.topN) continue;
+        const unsigned long long key = ky[e];
+        const int len = key_len(key);
+        clen[rank] = len;
+        cscore[rank] = (float)sc[e];
+        for (int l = 0; l < len; ++l) ctok[rank * p.T + l] = sl.sorted_tok[key_tok(key, l)];
+    }
+    if (tid == 0) {
+        int nonempty = count - (empty_at < count ? 1 : 0);
+        if (empty_at == 0x7fffffff && count > look) nonempty = count;     // not among the first topN+1
+        p.out_n_cand[b] = nonempty < p.topN ? nonempty : p.topN;
+    }
+}
+
+__device__ __forceinline__ int next_pow2(int v) {
+    int n = 2;
+    while (n < v) n <<= 1;
+    return n;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -163,6 +194,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     unsigned long long* fsum = reinterpret_cast<unsigned long long*>(best + p.cap);    // [cap] fixed-point sum
     unsigned short* path_slot = reinterpret_cast<unsigned short*>(fsum + p.cap);       // [npaths]
     __shared__ SlotLists sl;
+    __shared__ int s_count;
 
     const int b = blockIdx.x, tid = threadIdx.x;
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -173,6 +205,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     load_slot_lists(p, row, sl);
     const long long neg_inf_sortable = dbl_sortable(-INFINITY);
     for (int i = tid; i < p.cap; i += kThreads) { keys[i] = kEmpty; best[i] = neg_inf_sortable; fsum[i] = 0ull; }
+    if (tid == 0) s_count = 0;
     __syncthreads();
 
     // pass 1: collapse every path, claim a table slot, track the best alignment
@@ -232,7 +265,25 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
         score[i] = sc;
     }
     __syncthreads();
-    emit_top_candidates(p, b, sl, keys, score, p.cap);
+
+    // compact the distinct candidates into the (now free) sum array and sort them best first
+    double* c_sc = reinterpret_cast<double*>(fsum);                     // [cap/2]
+    unsigned long long* c_ky = fsum + (p.cap >> 1);                     // [cap/2]
+    for (int i = tid; i < p.cap; i += kThreads) {
+        const unsigned long long ki = keys[i];
+        if (ki == kEmpty) continue;
+        const double si = score[i];
+        const int at = atomicAdd(&s_count, 1);
+        c_sc[at] = si;
+        c_ky[at] = ki;
+    }
+    __syncthreads();
+    const int count = s_count;
+    const int n2 = next_pow2(count);
+    for (int i = count + tid; i < n2; i += kThreads) { c_sc[i] = -INFINITY; c_ky[i] = kEmpty; }
+    __syncthreads();
+    bitonic_sort_best_first(c_sc, c_ky, nullptr, n2);
+    emit_candidates(p, b, sl, c_sc, c_ky, count);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -244,8 +295,11 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     double* t_pb = reinterpret_cast<double*>(keys + kBeamCap);    // mass ending in blank (one contributor: the prefix itself)
     double* t_stay = t_pb + kBeamCap;        // ending in the last token, from the prefix itself (repeat)
     double* t_ext = t_stay + kBeamCap;       // ending in the last token, from the parent prefix (extension)
+    double* c_sc = t_ext + kBeamCap;                                          // [kBeamCap] sort keys
+    unsigned long long* c_ky = reinterpret_cast<unsigned long long*>(c_sc + kBeamCap);
+    int* c_ix = reinterpret_cast<int*>(c_ky + kBeamCap);                      // [kBeamCap] table slot
     __shared__ unsigned long long bm_key[CTCSD_MAX_BEAM];
-    __shared__ double bm_pb[CTCSD_MAX_BEAM], bm_pnb[CTCSD_MAX_BEAM];
+    __shared__ double bm_pb[CTCSD_MAX_BEAM], bm_pnb[CTCSD_MAX_BEAM], bm_tot[CTCSD_MAX_BEAM];
     __shared__ int s_nbeam, s_next;
     __shared__ SlotLists sl;
 
@@ -256,7 +310,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         return;
     }
     load_slot_lists(p, row, sl);
-    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 0.0; bm_pnb[0] = -INFINITY; s_nbeam = 1; }
+    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 0.0; bm_pnb[0] = -INFINITY; bm_tot[0] = 0.0; s_nbeam = 1; }
     __syncthreads();
 
     for (int t = 0; t < p.T; ++t) {
@@ -270,7 +324,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
             const int e = w / p.k, j = w - e * p.k;
             const unsigned long long key = bm_key[e];
             const double pb = bm_pb[e], pnb = bm_pnb[e];
-            const double tot = logadd(pb, pnb);
+            const double tot = bm_tot[e];
             const int m = sl.lid[t * p.k + j];
             const double lp = sl.lp[t * p.k + j];
             const int len = key_len(key);
@@ -293,42 +347,38 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
             }
         }
         __syncthreads();
-        // total mass per prefix, then keep the best `beam` in ranked order
+        // total mass per prefix; compact into the sort arrays
         for (int i = tid; i < kBeamCap; i += kThreads) {
-            if (keys[i] == kEmpty) continue;
-            double pnb = logadd(t_stay[i], t_ext[i]);
-            t_stay[i] = pnb;
-            t_ext[i] = logadd(t_pb[i], pnb);
-        }
-        __syncthreads();
-        for (int i = tid; i < kBeamCap; i += kThreads) {
-            unsigned long long ki = keys[i];
+            const unsigned long long ki = keys[i];
             if (ki == kEmpty) continue;
-            double si = t_ext[i];
-            int rank = 0;
-            for (int j = 0; j < kBeamCap; ++j) {
-                unsigned long long kj = keys[j];
-                if (kj == kEmpty) continue;
-                rank += precedes(t_ext[j], kj, si, ki) ? 1 : 0;
-            }
-            atomicAdd(&s_next, 1);
-            if (rank < p.beam) { bm_key[rank] = ki; bm_pb[rank] = t_pb[i]; bm_pnb[rank] = t_stay[i]; }
+            const double pnb = logadd(t_stay[i], t_ext[i]);
+            const double tot = logadd(t_pb[i], pnb);
+            t_stay[i] = pnb;
+            t_ext[i] = tot;
+            const int at = atomicAdd(&s_next, 1);
+            c_sc[at] = tot;
+            c_ky[at] = ki;
+            c_ix[at] = i;
         }
         __syncthreads();
-        if (tid == 0) s_nbeam = s_next < p.beam ? s_next : p.beam;
+        const int count = s_next;
+        const int n2 = next_pow2(count);
+        for (int i = count + tid; i < n2; i += kThreads) { c_sc[i] = -INFINITY; c_ky[i] = kEmpty; c_ix[i] = 0; }
+        __syncthreads();
+        bitonic_sort_best_first(c_sc, c_ky, c_ix, n2);
+        const int keep = count < p.beam ? count : p.beam;
+        for (int r = tid; r < keep; r += kThreads) {
+            const int slot = c_ix[r];
+            bm_key[r] = c_ky[r];
+            bm_pb[r] = t_pb[slot];
+            bm_pnb[r] = t_stay[slot];
+            bm_tot[r] = c_sc[r];
+        }
+        if (tid == 0) s_nbeam = keep;
         __syncthreads();
     }
-    // after the last slot the table still holds every surviving prefix with its total mass;
-    // entries pruned by the beam cut must not be candidates, so rebuild the table from the beam
-    const int nbeam = s_nbeam;
-    for (int i = tid; i < kBeamCap; i += kThreads) keys[i] = kEmpty;
-    __syncthreads();
-    for (int e = tid; e < nbeam; e += kThreads) {
-        int s = table_insert(keys, kBeamCap, bm_key[e]);
-        if (s >= 0) t_ext[s] = logadd(bm_pb[e], bm_pnb[e]);
-    }
-    __syncthreads();
-    emit_top_candidates(p, b, sl, keys, t_ext, kBeamCap);
+    // the beam is already ranked best first by total mass
+    emit_candidates(p, b, sl, bm_tot, bm_key, s_nbeam);
 }
 
 }  // namespace
@@ -360,7 +410,7 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     p.status = status_ptr(h);
 
     if (c.beam > 0) {
-        const size_t smem = (size_t)kBeamCap * 32;
+        const size_t smem = (size_t)kBeamCap * 52;
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_beam_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         collapse_beam_kernel<<<c.B, kThreads, smem, s>>>(p);
         CTCSD_LAUNCH_CHECK(h);

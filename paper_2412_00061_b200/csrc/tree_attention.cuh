@@ -18,4 +18,7 @@ struct AttnParams {
     int* status;
 };
 
+// bf16 tensor-core path (flash-style, KV split across CTAs, GQA head grouping).
+int launch_tree_attention_mma(Handle* h, cudaStream_t s, const AttnParams& p);
+
 }  // namespace ctcsd

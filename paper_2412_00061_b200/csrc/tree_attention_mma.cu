@@ -1,0 +1,314 @@
+// Tree attention for bf16 on tensor cores: a flash-style kernel that streams the KV cache
+// once per (sequence, kv head), split along the KV axis, plus a small merge kernel.
+//
+// Work decomposition: CTA = (64 query rows, one KV split, kv head g, sequence b).  Query row
+// r of kv head g is (node i = r / grp, query head g*grp + r % grp), so all query heads that
+// share a kv head read its keys and values from the same shared-memory tile (GQA grouping).
+// Each of the 4 warps owns 16 rows: S = Q K^T with mma.m16n8k16 (bf16 in, fp32 out), the
+// ancestor mask is applied to the columns that are tree nodes, an online softmax keeps the
+// running max and sum, and O += P V reuses the S accumulators as the A operand.  K and V
+// tiles of 64 keys are double buffered with cp.async into XOR-swizzled shared memory.
+// Every CTA writes (max, sum, unnormalised O) per row; the merge kernel combines the splits.
+#include "tree_attention.cuh"
+
+#include <math.h>
+
+namespace ctcsd {
+namespace {
+
+constexpr int kRows = 64;          // query rows per CTA
+constexpr int kKeys = 64;          // keys per tile
+constexpr int kThreads = 128;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
+    const int bytes = valid ? 16 : 0;                 // 0 source bytes -> the 16 bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// byte offset of 16-byte chunk `chunk` of row `row` in a tile with D bf16 per row, swizzled
+template <int D> __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+    return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams p, float* part, int splits) {
+    constexpr int CH = D / 8;                  // 16-byte chunks per row
+    constexpr int KS = D / 16;                 // k-steps of the QK^T product
+    constexpr int DT = D / 8;                  // 8-wide output tiles of O
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* Qs = smem;                                  // [64][D]
+    unsigned char* Ks = Qs + kRows * D * 2;                    // [2][64][D]
+    unsigned char* Vs = Ks + 2 * kKeys * D * 2;                // [2][64][D]
+
+    const int grp = p.Hq / p.Hkv;
+    const int qtile = blockIdx.x / splits, split = blockIdx.x - qtile * splits;
+    const int g = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+
+    int n = p.n_nodes[b];
+    const int L = p.kv_len[b];
+    if (n < 0 || n > p.max_nodes || L < 0 || L + n > p.Lcap) {
+        if (tid == 0) report_error(p.status, CTCSD_ERR_INVALID_ARG, b);
+        n = 0;
+    }
+    const int Ltot = L + n;
+    const int nblk = (Ltot + kKeys - 1) / kKeys;
+    const int bps = (nblk + splits - 1) / splits;
+    const int blk0 = split * bps;
+    const int blk1 = (blk0 + bps < nblk) ? blk0 + bps : nblk;
+
+    const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q);
+    const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(p.K) + ((size_t)b * p.Hkv + g) * (size_t)p.Lcap * D;
+    const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(p.V) + ((size_t)b * p.Hkv + g) * (size_t)p.Lcap * D;
+
+    // rows of this thread: r0 = first row of the pair (gid), r1 = r0 + 8
+    const int row_base = qtile * kRows + warp * 16;
+    const int rA = row_base + gid, rB = rA + 8;
+    const int iA = rA / grp, iB = rB / grp;                     // tree node of each row
+    const bool liveA = iA < n, liveB = iB < n;
+    const int W = (p.max_nodes + 63) / 64;
+    unsigned long long mA0 = 0, mA1 = 0, mB0 = 0, mB1 = 0;
+    if (liveA) { const unsigned long long* m = p.mask + ((size_t)b * p.max_nodes + iA) * W; mA0 = m[0]; if (W > 1) mA1 = m[1]; }
+    if (liveB) { const unsigned long long* m = p.mask + ((size_t)b * p.max_nodes + iB) * W; mB0 = m[0]; if (W > 1) mB1 = m[1]; }
+
+    auto load_kv = [&](int blk, int buf) {
+        const int key0 = blk * kKeys;
+        unsigned char* kd = Ks + buf * (kKeys * D * 2);
+        unsigned char* vd = Vs + buf * (kKeys * D * 2);
+        for (int c = tid; c < kKeys * CH; c += kThreads) {
+            const int row = c / CH, ch = c - row * CH;
+            const int key = key0 + row;
+            const bool ok = key < Ltot;
+            const size_t src = (size_t)(ok ? key : 0) * D + ch * 8;
+            cp_async16(kd + tile_off<D>(row, ch), Kg + src, ok);
+            cp_async16(vd + tile_off<D>(row, ch), Vg + src, ok);
+        }
+    };
+
+    // Q tile (rows past the live rows are zero-filled) and the first KV tile
+    for (int c = tid; c < kRows * CH; c += kThreads) {
+        const int row = c / CH, ch = c - row * CH;
+        const int r = qtile * kRows + row;
+        const int i = r / grp, hq = g * grp + (r - i * grp);
+        const bool ok = i < n;
+        const size_t src = (((size_t)b * p.max_nodes + (ok ? i : 0)) * p.Hq + hq) * D + ch * 8;
+        cp_async16(Qs + tile_off<D>(row, ch), Qg + src, ok);
+    }
+    if (blk0 < blk1) load_kv(blk0, 0);
+    cp_async_commit();
+
+    float o[DT][4];
+#pragma unroll
+    for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+    float mxA = -INFINITY, mxB = -INFINITY, sumA = 0.f, sumB = 0.f;
+    const float sl2 = p.scale * 1.4426950408889634f;          // scores are kept in log2 units
+    uint32_t qf[KS][4];
+
+    for (int blk = blk0; blk < blk1; ++blk) {
+        const int buf = (blk - blk0) & 1;
+        if (blk + 1 < blk1) load_kv(blk + 1, buf ^ 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        if (blk == blk0) {
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {
+                const int row = warp * 16 + (lane & 15), ch = 2 * kk + (lane >> 4);
+                ldmatrix_x4(qf[kk], smem_u32(Qs + tile_off<D>(row, ch)));
+            }
+        }
+        const unsigned char* kb = Ks + buf * (kKeys * D * 2);
+        const unsigned char* vb = Vs + buf * (kKeys * D * 2);
+
+        // S = Q K^T for 16 rows x 64 keys
+        float s[kKeys / 8][4];
+#pragma unroll
+        for (int t = 0; t < kKeys / 8; ++t) { s[t][0] = s[t][1] = s[t][2] = s[t][3] = 0.f; }
+#pragma unroll
+        for (int kk = 0; kk < KS; ++kk) {
+#pragma unroll
+            for (int pr = 0; pr < kKeys / 16; ++pr) {
+                uint32_t kf[4];
+                const int mi = lane >> 3, rin = lane & 7;
+                const int key = 16 * pr + (mi >> 1) * 8 + rin, ch = 2 * kk + (mi & 1);
+                ldmatrix_x4(kf, smem_u32(kb + tile_off<D>(key, ch)));
+                mma_bf16(s[2 * pr], qf[kk], kf[0], kf[1]);
+                mma_bf16(s[2 * pr + 1], qf[kk], kf[2], kf[3]);
+            }
+        }
+
+        // scale, mask, online softmax
+        const int key0 = blk * kKeys;
+        const bool need_mask = key0 + kKeys > L;
+        float bmA = -INFINITY, bmB = -INFINITY;
+#pragma unroll
+        for (int t = 0; t < kKeys / 8; ++t) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float v = s[t][e] * sl2;
+                const bool second = e >= 2;                     // c2,c3 belong to row gid+8
+                bool vis = second ? liveB : liveA;
+                if (need_mask) {
+                    const int key = key0 + 8 * t + 2 * tig + (e & 1);
+                    if (key >= L) {
+                        const int tn = key - L;
+                        const unsigned long long w0 = second ? mB0 : mA0, w1 = second ? mB1 : mA1;
+                        const unsigned long long w = tn < 64 ? w0 : w1;
+                        vis = vis && key < Ltot && ((w >> (tn & 63)) & 1ull);
+                    }
+                }
+                v = vis ? v : -INFINITY;
+                s[t][e] = v;
+                if (second) bmB = fmaxf(bmB, v); else bmA = fmaxf(bmA, v);
+            }
+        }
+        bmA = fmaxf(bmA, __shfl_xor_sync(0xffffffffu, bmA, 1));
+        bmA = fmaxf(bmA, __shfl_xor_sync(0xffffffffu, bmA, 2));
+        bmB = fmaxf(bmB, __shfl_xor_sync(0xffffffffu, bmB, 1));
+        bmB = fmaxf(bmB, __shfl_xor_sync(0xffffffffu, bmB, 2));
+        const float nmA = fmaxf(mxA, bmA), nmB = fmaxf(mxB, bmB);
+        const float refA = nmA == -INFINITY ? 0.f : nmA, refB = nmB == -INFINITY ? 0.f : nmB;
+        const float corrA = exp2f(mxA - refA), corrB = exp2f(mxB - refB);   // exp2(-inf) = 0
+        mxA = nmA; mxB = nmB;
+        float psA = 0.f, psB = 0.f;
+        uint32_t pf[kKeys / 16][4];
+#pragma unroll
+        for (int t = 0; t < kKeys / 8; ++t) {
+            const float p0 = exp2f(s[t][0] - refA), p1 = exp2f(s[t][1] - refA);
+            const float p2 = exp2f(s[t][2] - refB), p3 = exp2f(s[t][3] - refB);
+            psA += p0 + p1;
+            psB += p2 + p3;
+            pf[t >> 1][(t & 1) * 2 + 0] = pack_bf16(p0, p1);
+            pf[t >> 1][(t & 1) * 2 + 1] = pack_bf16(p2, p3);
+        }
+        sumA = sumA * corrA + psA;
+        sumB = sumB * corrB + psB;
+#pragma unroll
+        for (int t = 0; t < DT; ++t) { o[t][0] *= corrA; o[t][1] *= corrA; o[t][2] *= corrB; o[t][3] *= corrB; }
+
+        // O += P V
+#pragma unroll
+        for (int kk = 0; kk < kKeys / 16; ++kk) {
+#pragma unroll
+            for (int pr = 0; pr < DT / 2; ++pr) {
+                uint32_t vf[4];
+                const int mi = lane >> 3, rin = lane & 7;
+                const int key = 16 * kk + (mi & 1) * 8 + rin, ch = 2 * pr + (mi >> 1);
+                ldmatrix_x4_trans(vf, smem_u32(vb + tile_off<D>(key, ch)));
+                mma_bf16(o[2 * pr], pf[kk], vf[0], vf[1]);
+                mma_bf16(o[2 * pr + 1], pf[kk], vf[2], vf[3]);
+            }
+        }
+        __syncthreads();                                        // the other buffer may be overwritten next
+    }
+    cp_async_wait<0>();
+
+    // per-row partials: [b][hq][node][split][D+2] = (max in log2 units, sum, unnormalised O)
+    sumA += __shfl_xor_sync(0xffffffffu, sumA, 1);
+    sumA += __shfl_xor_sync(0xffffffffu, sumA, 2);
+    sumB += __shfl_xor_sync(0xffffffffu, sumB, 1);
+    sumB += __shfl_xor_sync(0xffffffffu, sumB, 2);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int r = half ? rB : rA;
+        const int i = half ? iB : iA;
+        if (i >= n) continue;                                   // dead rows are zeroed by the merge kernel
+        const int hq = g * grp + (r - i * grp);
+        float* dst = part + ((((size_t)b * p.Hq + hq) * p.max_nodes + i) * splits + split) * (D + 2);
+        if (tig == 0) { dst[0] = half ? mxB : mxA; dst[1] = half ? sumB : sumA; }
+#pragma unroll
+        for (int t = 0; t < DT; ++t) {
+            float2 v = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
+            *reinterpret_cast<float2*>(dst + 2 + 8 * t + 2 * tig) = v;
+        }
+    }
+}
+
+// One warp per (sequence, node, query head): combine the KV splits and write bf16.
+template <int D>
+__global__ void __launch_bounds__(128) tree_attention_merge_kernel(AttnParams p, const float* part, int splits) {
+    const int lane = threadIdx.x & 31;
+    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    const long long total = (long long)p.B * p.max_nodes * p.Hq;
+    if (wid >= total) return;
+    const int hq = (int)(wid % p.Hq);
+    const int i = (int)((wid / p.Hq) % p.max_nodes);
+    const int b = (int)(wid / ((long long)p.Hq * p.max_nodes));
+    const float* src = part + (((size_t)b * p.Hq + hq) * p.max_nodes + i) * splits * (D + 2);
+    int n = p.n_nodes[b];
+    const int L = p.kv_len[b];
+    if (n < 0 || n > p.max_nodes || L < 0 || L + n > p.Lcap) n = 0;
+    float gm = -INFINITY;
+    if (i < n)
+        for (int s = 0; s < splits; ++s) gm = fmaxf(gm, src[(size_t)s * (D + 2)]);
+    constexpr int PER = D / 32;
+    float acc[PER], tot = 0.f;
+#pragma unroll
+    for (int d = 0; d < PER; ++d) acc[d] = 0.f;
+    if (gm != -INFINITY) {
+        for (int s = 0; s < splits; ++s) {
+            const float* ps = src + (size_t)s * (D + 2);
+            const float m = ps[0];
+            if (m == -INFINITY) continue;
+            const float w = exp2f(m - gm);
+            tot += w * ps[1];
+#pragma unroll
+            for (int d = 0; d < PER; ++d) acc[d] += w * ps[2 + lane + 32 * d];
+        }
+    }
+    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.O) + (((size_t)b * p.max_nodes + i) * p.Hq + hq) * D;
+#pragma unroll
+    for (int d = 0; d < PER; ++d) out[lane + 32 * d] = __float2bfloat16_rn(acc[d] * inv);
+}
+
+template <int D>
+int launch_d(Handle* h, cudaStream_t s, const AttnParams& p) {
+    const int grp = p.Hq / p.Hkv;
+    const int qtiles = (p.max_nodes * grp + kRows - 1) / kRows;
+    const int splits = h->lay.kv_splits;
+    float* part = reinterpret_cast<float*>(h->ws + h->lay.attn_part_off);
+    const size_t smem = (size_t)kRows * D * 2 + 4 * (size_t)kKeys * D * 2;
+    auto kern = tree_attention_mma_kernel<D>;
+    if (smem > 48 * 1024)
+        CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid(qtiles * splits, p.Hkv, p.B);
+    kern<<<grid, kThreads, smem, s>>>(p, part, splits);
+    CTCSD_LAUNCH_CHECK(h);
+    const long long warps = (long long)p.B * p.max_nodes * p.Hq;
+    tree_attention_merge_kernel<D><<<(unsigned)((warps + 3) / 4), 128, 0, s>>>(p, part, splits);
+    CTCSD_LAUNCH_CHECK(h);
+    return CTCSD_OK;
+}
+
+}  // namespace
+
+int launch_tree_attention_mma(Handle* h, cudaStream_t s, const AttnParams& p) {
+    if (p.D == 64) return launch_d<64>(h, s, p);
+    return launch_d<128>(h, s, p);
+}
+
+}  // namespace ctcsd
