@@ -97,11 +97,19 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
-// 16-byte streaming load that does not allocate in L1 (weights are read exactly once).
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+// L2 policy "evict first": a stream that is read once must not push the step's small,
+// reused data (K/V cache, activations, code) out of L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+// 16-byte streaming load: no L1 allocation, L2 eviction priority given by `policy`.
+__device__ __forceinline__ uint4 ld_stream16(const void* p, uint64_t policy) {
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(policy));
     return r;
 }
 

@@ -148,6 +148,7 @@ __global__ void __launch_bounds__(kThreads) gemv_stream_kernel(GemvParams p) {
     const long long r1 = R * (blockIdx.x + 1) / gridDim.x;
     const int slot0 = (int)(r0 / rps);
     const uint4* Wbase = reinterpret_cast<const uint4*>(p.W);
+    const uint64_t policy = l2_policy_evict_first();
 
     for (int seg = 0; seg < 2; ++seg) {
         const int slot = slot0 + seg;
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(kThreads) gemv_stream_kernel(GemvParams p) {
             for (int ch = lane; ch < nch; ch += 32) {
                 uint4 w[kRW];
 #pragma unroll
-                for (int r = 0; r < kRW; ++r) w[r] = ld_stream16(wp[r] + ch);
+                for (int r = 0; r < kRW; ++r) w[r] = ld_stream16(wp[r] + ch, policy);
 #pragma unroll
                 for (int m = 0; m < MROWS; ++m) {
                     uint4 xv = xs[m * nch + ch];

@@ -26,6 +26,7 @@ struct CollapseParams {
     const int* sel_row;      // [B] or null
     int M, T, k, V, topN, beam, score_mode;
     int npaths;              // k^T (enumeration)
+    unsigned k_magic;        // floor(2^32 / k) + 1: x / k == umulhi(x, k_magic) for x < 2^16
     int cap;                 // hash capacity (power of two)
     int* out_cand_tok;       // [B,topN,T]
     int* out_cand_len;       // [B,topN]
@@ -91,6 +92,7 @@ struct SlotLists {
 };
 
 __device__ void load_slot_lists(const CollapseParams& p, int row, SlotLists& sl) {
+    __shared__ unsigned char s_first[CTCSD_MAX_T * CTCSD_MAX_K];
     const int n = p.T * p.k;
     const int tid = threadIdx.x;
     if (tid < n) {
@@ -98,22 +100,22 @@ __device__ void load_slot_lists(const CollapseParams& p, int row, SlotLists& sl)
         sl.lp[tid] = (double)p.topk_lp[(size_t)row * n + tid];
     }
     __syncthreads();
+    if (tid < n) {                                   // is (t, j) the first occurrence of its token?
+        const int me = sl.tok[tid];
+        bool first = me != p.V;
+        for (int q = 0; q < tid; ++q) first = first && (sl.tok[q] != me);
+        s_first[tid] = first ? 1 : 0;
+    }
+    __syncthreads();
     if (tid < n) {
-        int me = sl.tok[tid];
+        const int me = sl.tok[tid];
         if (me == p.V) {
             sl.lid[tid] = kBlankMark;
         } else {
-            // local id = number of distinct non-blank tokens smaller than mine
-            int cnt = 0;
-            for (int j = 0; j < n; ++j) {
-                int tj = sl.tok[j];
-                if (tj == p.V || tj >= me) continue;
-                bool first = true;
-                for (int q = 0; q < j; ++q) if (sl.tok[q] == tj) { first = false; break; }
-                cnt += first ? 1 : 0;
-            }
+            int cnt = 0;                             // local id = number of distinct smaller tokens
+            for (int j = 0; j < n; ++j) cnt += (s_first[j] && sl.tok[j] < me) ? 1 : 0;
             sl.lid[tid] = (unsigned char)cnt;
-            sl.sorted_tok[cnt] = me;
+            if (s_first[tid]) sl.sorted_tok[cnt] = me;
         }
     }
     __syncthreads();
@@ -144,9 +146,154 @@ __device__ void bitonic_sort_best_first(double* sc, unsigned long long* ky, int*
     }
 }
 
-// Writes the first topN non-empty entries of a best-first list as the candidates.
+constexpr int kSelMax = 256;     // most near-threshold entries the exact tie-break handles
+
+struct SelectScratch {
+    unsigned hist[256];
+    int win[CTCSD_MAX_BEAM + 8];   // indices of selected entries (unordered)
+    int cand[kSelMax];             // indices of entries on the threshold
+    unsigned fmax, fmin, thr;
+    int lo, need, nwin, ncand, ccnt;
+};
+
+// float32 image of a score as an unsigned integer whose order matches the score's
+__device__ __forceinline__ unsigned sortable_f32(double v) {
+    unsigned u = __float_as_uint((float)v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ int next_pow2(int v) {
+    int n = 2;
+    while (n < v) n <<= 1;
+    return n;
+}
+
+// Selects the `need` (<= CTCSD_MAX_BEAM) best of `count` entries and writes their indices,
+// best first, to sel[]; returns how many were selected.  A radix select on the float32 image
+// of the scores finds the threshold in O(count) work; entries on the threshold are ranked
+// exactly (float64 score, then key).  If more than kSelMax entries sit on the threshold the
+// arrays (padded to a power of two, capacity >= next_pow2(count)) are sorted in place instead
+// and sel[] becomes the identity.
+__device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int count, int need, int* sel,
+                                SelectScratch& S) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    if (need > count) need = count;
+    if (tid == 0) { S.fmax = 0u; S.fmin = 0xffffffffu; S.nwin = 0; S.ncand = 0; S.ccnt = 0; }
+    __syncthreads();
+    if (count > need) {
+        unsigned lmax = 0u, lmin = 0xffffffffu;
+        for (int i = tid; i < count; i += kThreads) {
+            const unsigned f = sortable_f32(sc[i]);
+            lmax = max(lmax, f);
+            lmin = min(lmin, f);
+        }
+        lmax = __reduce_max_sync(0xffffffffu, lmax);
+        lmin = __reduce_min_sync(0xffffffffu, lmin);
+        if (lane == 0) { atomicMax(&S.fmax, lmax); atomicMin(&S.fmin, lmin); }
+        __syncthreads();
+        const unsigned diff = S.fmax ^ S.fmin;
+        // bits above `hb` agree for all entries; walk down 8 bits at a time
+        int lo = diff ? (31 - __clz(diff)) + 1 : 0;
+        unsigned thr = lo < 32 ? (S.fmax >> lo) : 0u;
+        int remaining = need;
+        int ncand = count;
+        while (lo > 0 && ncand > remaining) {
+            const int nlo = lo > 8 ? lo - 8 : 0;
+            const int width = lo - nlo;
+            if (tid < 256) S.hist[tid] = 0u;
+            __syncthreads();
+            for (int i = tid; i < count; i += kThreads) {
+                const unsigned f = sortable_f32(sc[i]);
+                const unsigned top = lo < 32 ? (f >> lo) : 0u;
+                if (top == thr) atomicAdd(&S.hist[(f >> nlo) & ((1u << width) - 1u)], 1u);
+            }
+            __syncthreads();
+            if (tid < 32) {
+                // lane owns digits [8*lane, 8*lane+8); find the digit where the count from the top reaches `remaining`
+                unsigned h[8], mine = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { h[q] = S.hist[8 * lane + q]; mine += h[q]; }
+                unsigned suf = mine;                      // suffix sum: entries in this lane and above
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    unsigned v = __shfl_down_sync(0xffffffffu, suf, o);
+                    if (lane + o < 32) suf += v;
+                }
+                const unsigned above = suf - mine;
+                if (above < (unsigned)remaining && above + mine >= (unsigned)remaining) {
+                    unsigned acc = above;
+#pragma unroll
+                    for (int q = 7; q >= 0; --q) {
+                        if (acc < (unsigned)remaining && acc + h[q] >= (unsigned)remaining) {
+                            S.thr = (thr << width) | (unsigned)(8 * lane + q);
+                            S.need = remaining - (int)acc;
+                            S.ncand = (int)h[q];
+                        }
+                        acc += h[q];
+                    }
+                }
+            }
+            __syncthreads();
+            thr = S.thr; remaining = S.need; ncand = S.ncand;
+            lo = nlo;
+            __syncthreads();
+            if (ncand <= kSelMax) break;
+        }
+        if (ncand > remaining && ncand > kSelMax) {
+            // too many entries share the threshold even at full float32 resolution: sort everything
+            const int n2 = next_pow2(count);
+            for (int i = count + tid; i < n2; i += kThreads) { sc[i] = -INFINITY; ky[i] = kEmpty; if (ix) ix[i] = 0; }
+            __syncthreads();
+            bitonic_sort_best_first(sc, ky, ix, n2);
+            for (int r = tid; r < need; r += kThreads) sel[r] = r;
+            __syncthreads();
+            return need;
+        }
+        // gather definite winners (above the threshold) and the entries on it
+        for (int i = tid; i < count; i += kThreads) {
+            const unsigned f = sortable_f32(sc[i]);
+            const unsigned top = lo < 32 ? (f >> lo) : 0u;
+            if (top > thr) S.win[atomicAdd(&S.nwin, 1)] = i;
+            else if (top == thr) S.cand[atomicAdd(&S.ccnt, 1)] = i;
+        }
+        __syncthreads();
+        // exact ranking among the threshold entries
+        for (int c = tid; c < ncand; c += kThreads) {
+            const int i = S.cand[c];
+            const double si = sc[i];
+            const unsigned long long ki = ky[i];
+            int rank = 0;
+            for (int d = 0; d < ncand; ++d) {
+                const int j = S.cand[d];
+                rank += precedes(sc[j], ky[j], si, ki) ? 1 : 0;
+            }
+            if (rank < remaining) S.win[atomicAdd(&S.nwin, 1)] = i;
+        }
+        __syncthreads();
+    } else {
+        for (int i = tid; i < count; i += kThreads) S.win[i] = i;
+        __syncthreads();
+    }
+    // order the winners
+    for (int w = tid; w < need; w += kThreads) {
+        const int i = S.win[w];
+        const double si = sc[i];
+        const unsigned long long ki = ky[i];
+        int rank = 0;
+        for (int d = 0; d < need; ++d) {
+            const int j = S.win[d];
+            rank += precedes(sc[j], ky[j], si, ki) ? 1 : 0;
+        }
+        sel[rank] = i;
+    }
+    __syncthreads();
+    return need;
+}
+
+// Writes the candidates: the selected entries in ranked order, the empty sequence skipped.
+// `total_nonempty` is the number of distinct non-empty sequences that exist.
 __device__ void emit_candidates(const CollapseParams& p, int b, const SlotLists& sl, const double* sc,
-                                const unsigned long long* ky, int count) {
+                                const unsigned long long* ky, const int* sel, int nsel, int total_nonempty) {
     __shared__ int s_empty_at;
     const int tid = threadIdx.x;
     if (tid == 0) s_empty_at = 0x7fffffff;
@@ -156,32 +303,57 @@ __device__ void emit_candidates(const CollapseParams& p, int b, const SlotLists&
     for (int i = tid; i < p.topN * p.T; i += kThreads) ctok[i] = -1;
     for (int i = tid; i < p.topN; i += kThreads) { clen[i] = 0; cscore[i] = -INFINITY; }
     __syncthreads();
-    const int look = count < p.topN + 1 ? count : p.topN + 1;      // the empty sequence occurs at most once
-    for (int e = tid; e < look; e += kThreads)
-        if (key_len(ky[e]) == 0) s_empty_at = e;
+    for (int e = tid; e < nsel; e += kThreads)
+        if (key_len(ky[sel[e]]) == 0) s_empty_at = e;
     __syncthreads();
     const int empty_at = s_empty_at;
-    for (int e = tid; e < look; e += kThreads) {
+    for (int e = tid; e < nsel; e += kThreads) {
         if (e == empty_at) continue;
         const int rank = e - (empty_at < e ? 1 : 0);
         if (rank >= p.topN) continue;
-        const unsigned long long key = ky[e];
+        const unsigned long long key = ky[sel[e]];
         const int len = key_len(key);
         clen[rank] = len;
-        cscore[rank] = (float)sc[e];
+        cscore[rank] = (float)sc[sel[e]];
         for (int l = 0; l < len; ++l) ctok[rank * p.T + l] = sl.sorted_tok[key_tok(key, l)];
     }
     if (tid == 0) {
-        int nonempty = count - (empty_at < count ? 1 : 0);
-        if (empty_at == 0x7fffffff && count > look) nonempty = count;     // not among the first topN+1
+        const int nonempty = total_nonempty >= 0 ? total_nonempty : nsel - (empty_at != 0x7fffffff ? 1 : 0);
         p.out_n_cand[b] = nonempty < p.topN ? nonempty : p.topN;
     }
 }
 
-__device__ __forceinline__ int next_pow2(int v) {
-    int n = 2;
-    while (n < v) n <<= 1;
-    return n;
+// Decodes path index -> per-slot choices (last slot fastest), returning the collapsed
+// sequence's key and the path's log-probability (summed in slot order).
+__device__ __forceinline__ unsigned long long path_key_and_score(const CollapseParams& p, const SlotLists& sl,
+                                                                 int path, double& score) {
+    unsigned rem = (unsigned)path;
+    int digit[CTCSD_MAX_T];
+#pragma unroll
+    for (int t = CTCSD_MAX_T - 1; t >= 0; --t) {
+        if (t < p.T) {
+            const unsigned q = __umulhi(rem, p.k_magic);     // rem / k for rem < 2^16, k <= 8
+            digit[t] = (int)(rem - q * (unsigned)p.k);
+            rem = q;
+        } else {
+            digit[t] = 0;
+        }
+    }
+    double s = 0.0;
+    unsigned long long key = 0ull;
+    int prev = -1;
+#pragma unroll
+    for (int t = 0; t < CTCSD_MAX_T; ++t) {
+        if (t < p.T) {
+            const int e = t * p.k + digit[t];
+            s += sl.lp[e];
+            const int m = sl.lid[e];
+            if (m != prev && m != kBlankMark) key = key_append(key, m);
+            prev = m;
+        }
+    }
+    score = s;
+    return key;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -194,7 +366,9 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     unsigned long long* fsum = reinterpret_cast<unsigned long long*>(best + p.cap);    // [cap] fixed-point sum
     unsigned short* path_slot = reinterpret_cast<unsigned short*>(fsum + p.cap);       // [npaths]
     __shared__ SlotLists sl;
-    __shared__ int s_count;
+    __shared__ SelectScratch S;
+    __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
+    __shared__ int s_count, s_has_empty;
 
     const int b = blockIdx.x, tid = threadIdx.x;
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -205,30 +379,13 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     load_slot_lists(p, row, sl);
     const long long neg_inf_sortable = dbl_sortable(-INFINITY);
     for (int i = tid; i < p.cap; i += kThreads) { keys[i] = kEmpty; best[i] = neg_inf_sortable; fsum[i] = 0ull; }
-    if (tid == 0) s_count = 0;
+    if (tid == 0) { s_count = 0; s_has_empty = 0; }
     __syncthreads();
 
     // pass 1: collapse every path, claim a table slot, track the best alignment
     for (int path = tid; path < p.npaths; path += kThreads) {
-        int rem = path;
-        int digit[CTCSD_MAX_T];
-#pragma unroll
-        for (int t = CTCSD_MAX_T - 1; t >= 0; --t) {
-            if (t < p.T) { digit[t] = rem % p.k; rem /= p.k; } else digit[t] = 0;
-        }
-        double s = 0.0;
-        unsigned long long key = 0ull;
-        int prev = -1;
-#pragma unroll
-        for (int t = 0; t < CTCSD_MAX_T; ++t) {
-            if (t < p.T) {
-                int e = t * p.k + digit[t];
-                s += sl.lp[e];
-                int m = sl.lid[e];
-                if (m != prev && m != kBlankMark) key = key_append(key, m);
-                prev = m;
-            }
-        }
+        double s;
+        const unsigned long long key = path_key_and_score(p, sl, path, s);
         int slot = table_insert(keys, p.cap, key);
         if (slot < 0) { report_error(p.status, CTCSD_ERR_INTERNAL, 1); slot = 0; }
         path_slot[path] = (unsigned short)slot;
@@ -236,37 +393,33 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     }
     __syncthreads();
 
-    // pass 2: sum exp(s - best) per candidate in fixed point (order independent)
+    // pass 2: sum exp(s - best) per candidate in fixed point (order independent).  The best
+    // alignment itself contributes exp(0) = 1 exactly, so it needs no call to exp.
     if (p.score_mode == CTCSD_SCORE_SUM) {
         for (int path = tid; path < p.npaths; path += kThreads) {
-            int rem = path;
-            double s = 0.0;
-            int digit[CTCSD_MAX_T];
-#pragma unroll
-            for (int t = CTCSD_MAX_T - 1; t >= 0; --t) {
-                if (t < p.T) { digit[t] = rem % p.k; rem /= p.k; } else digit[t] = 0;
-            }
-#pragma unroll
-            for (int t = 0; t < CTCSD_MAX_T; ++t)
-                if (t < p.T) s += sl.lp[t * p.k + digit[t]];
-            int slot = path_slot[path];
-            double mx = sortable_dbl(best[slot]);
-            double term = exp(s - mx) * kFix;
-            atomicAdd(&fsum[slot], __double2ull_rn(term));
+            double s;
+            path_key_and_score(p, sl, path, s);
+            const int slot = path_slot[path];
+            const long long bs = best[slot];
+            unsigned long long term = 1ull << 50;
+            if (dbl_sortable(s) != bs) term = __double2ull_rn(exp(s - sortable_dbl(bs)) * kFix);
+            atomicAdd(&fsum[slot], term);
         }
     }
     __syncthreads();
     double* score = reinterpret_cast<double*>(best);
     for (int i = tid; i < p.cap; i += kThreads) {
         if (keys[i] == kEmpty) continue;
-        double mx = sortable_dbl(best[i]);
+        const double mx = sortable_dbl(best[i]);
         double sc = mx;
-        if (p.score_mode == CTCSD_SCORE_SUM) sc = mx + log((double)fsum[i] * (1.0 / kFix));
+        // a single alignment sums to exactly 1: log(1) = 0
+        if (p.score_mode == CTCSD_SCORE_SUM && fsum[i] != (1ull << 50)) sc = mx + log((double)fsum[i] * (1.0 / kFix));
         score[i] = sc;
     }
     __syncthreads();
 
-    // compact the distinct candidates into the (now free) sum array and sort them best first
+    // compact the distinct candidates into the (now free) sum array, pick the best topN (+1
+    // because the empty sequence may be among them) and write them out
     double* c_sc = reinterpret_cast<double*>(fsum);                     // [cap/2]
     unsigned long long* c_ky = fsum + (p.cap >> 1);                     // [cap/2]
     for (int i = tid; i < p.cap; i += kThreads) {
@@ -274,16 +427,14 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
         if (ki == kEmpty) continue;
         const double si = score[i];
         const int at = atomicAdd(&s_count, 1);
+        if (ki == 0ull) s_has_empty = 1;
         c_sc[at] = si;
         c_ky[at] = ki;
     }
     __syncthreads();
     const int count = s_count;
-    const int n2 = next_pow2(count);
-    for (int i = count + tid; i < n2; i += kThreads) { c_sc[i] = -INFINITY; c_ky[i] = kEmpty; }
-    __syncthreads();
-    bitonic_sort_best_first(c_sc, c_ky, nullptr, n2);
-    emit_candidates(p, b, sl, c_sc, c_ky, count);
+    const int nsel = block_select_top(c_sc, c_ky, nullptr, count, p.topN + 1, s_sel, S);
+    emit_candidates(p, b, sl, c_sc, c_ky, s_sel, nsel, count - s_has_empty);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -302,6 +453,8 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     __shared__ double bm_pb[CTCSD_MAX_BEAM], bm_pnb[CTCSD_MAX_BEAM], bm_tot[CTCSD_MAX_BEAM];
     __shared__ int s_nbeam, s_next;
     __shared__ SlotLists sl;
+    __shared__ SelectScratch S;
+    __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
     const int b = blockIdx.x, tid = threadIdx.x;
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -362,23 +515,23 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         }
         __syncthreads();
         const int count = s_next;
-        const int n2 = next_pow2(count);
-        for (int i = count + tid; i < n2; i += kThreads) { c_sc[i] = -INFINITY; c_ky[i] = kEmpty; c_ix[i] = 0; }
-        __syncthreads();
-        bitonic_sort_best_first(c_sc, c_ky, c_ix, n2);
-        const int keep = count < p.beam ? count : p.beam;
+        const int keep = block_select_top(c_sc, c_ky, c_ix, count, p.beam, s_sel, S);
         for (int r = tid; r < keep; r += kThreads) {
-            const int slot = c_ix[r];
-            bm_key[r] = c_ky[r];
+            const int i = s_sel[r];
+            const int slot = c_ix[i];
+            bm_key[r] = c_ky[i];
             bm_pb[r] = t_pb[slot];
             bm_pnb[r] = t_stay[slot];
-            bm_tot[r] = c_sc[r];
+            bm_tot[r] = c_sc[i];
         }
         if (tid == 0) s_nbeam = keep;
         __syncthreads();
     }
     // the beam is already ranked best first by total mass
-    emit_candidates(p, b, sl, bm_tot, bm_key, s_nbeam);
+    const int nbeam = s_nbeam;
+    for (int r = tid; r < nbeam; r += kThreads) s_sel[r] = r;
+    __syncthreads();
+    emit_candidates(p, b, sl, bm_tot, bm_key, s_sel, nbeam, -1);
 }
 
 }  // namespace
@@ -403,6 +556,7 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     p.sel_row = sel_row;
     p.M = M; p.T = c.T; p.k = c.k; p.V = c.V; p.topN = c.topN; p.beam = c.beam; p.score_mode = c.score_mode;
     p.npaths = 0; p.cap = 0;
+    p.k_magic = (unsigned)((1ull << 32) / (unsigned)c.k) + 1u;
     p.out_cand_tok = out_cand_tok;
     p.out_cand_len = out_cand_len;
     p.out_cand_score = out_cand_score;
