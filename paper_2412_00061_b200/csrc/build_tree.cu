@@ -1,15 +1,19 @@
 // ctcsd_build_tree: ranked candidates -> prefix trie with ancestor bit-masks.
 //
-// One CTA per sequence, one thread per (candidate c, prefix length l).  A prefix creates a
-// node iff no better-ranked candidate starts with the same l tokens; node ids are the
-// 1-based positions of the creating prefixes in (c, l) order, which is the order of first
-// appearance, so the node budget is applied by dropping ids >= max_nodes.
+// One warp per sequence; lane c (and c + 32 when more than 32 candidates are kept) owns
+// candidate c and keeps its tokens in registers.  The trie is grown level by level: the
+// prefix of length l of candidate c is identified by (owner of its length l-1 prefix, token
+// l), and its owner - the best-ranked candidate with the same prefix - is found with one
+// warp match instruction.  A prefix creates a node iff its owner is the candidate itself;
+// since a candidate's new prefixes are always its longest ones, node ids follow from an
+// exclusive scan of the per-candidate counts, which reproduces the order of first
+// appearance (candidates by rank, each left to right).  Ids >= max_nodes are dropped.
 #include "common.cuh"
 
 namespace ctcsd {
 namespace {
 
-constexpr int kThreads = 512;   // >= CTCSD_MAX_TOPN * CTCSD_MAX_T
+constexpr int kT = CTCSD_MAX_T;
 
 struct TreeParams {
     const int* base_tok; const int* kv_len;
@@ -19,96 +23,135 @@ struct TreeParams {
     unsigned long long* mask; int* retrieve; int* n_nodes;
 };
 
-__global__ void __launch_bounds__(kThreads) build_tree_kernel(TreeParams p) {
-    __shared__ int s_tok[CTCSD_MAX_TOPN * CTCSD_MAX_T];
-    __shared__ int s_len[CTCSD_MAX_TOPN];
-    __shared__ int s_node[CTCSD_MAX_TOPN * CTCSD_MAX_T];     // node id of each (c,l), -1 if none
-    __shared__ int s_newid[CTCSD_MAX_TOPN * CTCSD_MAX_T];    // id given to a creating prefix
-    __shared__ int s_parent[CTCSD_MAX_NODES];
-    __shared__ int s_warp_total[kThreads / 32];
-    __shared__ int s_total;
+__device__ __forceinline__ int warp_excl_scan(int v, int lane, int& total) {
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    total = __shfl_sync(0xffffffffu, inc, 31);
+    return inc - v;
+}
 
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+__global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
+    const int b = blockIdx.x, lane = threadIdx.x;
     const int T = p.T, N = p.topN, n_max = p.max_nodes;
     int nc = p.n_cand[b];
     nc = nc < 0 ? 0 : (nc > N ? N : nc);
-    const int* ctok = p.cand_tok + (size_t)b * N * T;
-    if (tid < N * T) s_tok[tid] = ctok[tid];
-    if (tid < N) {
-        int l = tid < nc ? p.cand_len[(size_t)b * N + tid] : 0;
-        s_len[tid] = l < 0 ? 0 : (l > T ? T : l);
-    }
-    __syncthreads();
+    const int L = p.kv_len[b];
+    const int halves = nc > 32 ? 2 : 1;
+    const int W = (n_max + 63) / 64;
 
-    // does this thread's prefix exist, and is it the first candidate to contain it?
-    const int c = tid / T, l = tid - c * T + 1;          // prefix = first l tokens of candidate c
-    const bool live = tid < N * T && c < nc && l <= s_len[c];
-    int owner = c;
-    if (live) {
-        for (int c2 = 0; c2 < c; ++c2) {
-            if (s_len[c2] < l) continue;
-            bool same = true;
-            for (int q = 0; q < l; ++q) same = same && (s_tok[c2 * T + q] == s_tok[c * T + q]);
-            if (same) { owner = c2; break; }
+    int tok[2][kT], len[2], shared_lv[2], base[2];
+    int own[2][kT];                      // owner candidate of each prefix (valid for l < len)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        int l = 0;
+        if (c < nc) { l = p.cand_len[(size_t)b * N + c]; l = l < 0 ? 0 : (l > T ? T : l); }
+        len[h] = l;
+#pragma unroll
+        for (int q = 0; q < kT; ++q) tok[h][q] = (q < l) ? p.cand_tok[((size_t)b * N + c) * T + q] : -1;
+    }
+
+    // ---- owners, level by level ----
+    int prev[2] = {0, 0};                // owner of the previous level's prefix (all start at the root)
+#pragma unroll
+    for (int l = 0; l < kT; ++l) {
+        if (l < T) {
+            unsigned long long key[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const bool active = len[h] > l;
+                // inactive lanes get a key nobody else has
+                key[h] = active ? (((unsigned long long)(unsigned)prev[h] << 32) | (unsigned)tok[h][l])
+                                : (0xffffffff00000000ull | (unsigned)(lane + 32 * h));
+            }
+            unsigned m0 = __match_any_sync(0xffffffffu, key[0]);
+            own[0][l] = __ffs(m0) - 1;
+            own[1][l] = -1;
+            if (halves == 2) {
+                unsigned m1 = __match_any_sync(0xffffffffu, key[1]);
+                int o = 32 + __ffs(m1) - 1;
+                for (int j = 31; j >= 0; --j) {              // a match among candidates 0..31 ranks first
+                    unsigned long long kj = __shfl_sync(0xffffffffu, key[0], j);
+                    if (kj == key[1]) o = j;
+                }
+                own[1][l] = o;
+            }
+            prev[0] = own[0][l];
+            prev[1] = own[1][l];
         }
     }
-    const bool creates = live && owner == c;
-    unsigned bal = __ballot_sync(0xffffffffu, creates);
-    if (lane == 0) s_warp_total[warp] = __popc(bal);
-    __syncthreads();
-    int before = __popc(bal & ((1u << lane) - 1u));
-    for (int w = 0; w < warp; ++w) before += s_warp_total[w];
-    if (tid == 0) {
-        int tot = 0;
-        for (int w = 0; w < kThreads / 32; ++w) tot += s_warp_total[w];
-        s_total = tot;
-    }
-    if (tid < N * T) s_newid[tid] = creates ? 1 + before : -1;
-    __syncthreads();
-    int node = -1;
-    if (live) {
-        int id = s_newid[owner * T + (l - 1)];
-        node = id < n_max ? id : -1;
-    }
-    if (tid < N * T) s_node[tid] = node;
-    __syncthreads();
 
-    const int n = (1 + s_total) < n_max ? (1 + s_total) : n_max;
+    // ---- node ids: a candidate's shared prefixes come first, its own (new) ones after ----
+    int total[2] = {0, 0};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        int sh = 0;
+#pragma unroll
+        for (int l = 0; l < kT; ++l) sh += (l < len[h] && own[h][l] != lane + 32 * h) ? 1 : 0;
+        shared_lv[h] = sh;
+        base[h] = warp_excl_scan(len[h] - sh, lane, total[h]);
+    }
+    base[0] += 1;
+    base[1] += 1 + total[0];
+    const int n_all = 1 + total[0] + total[1];
+    const int n = n_all < n_max ? n_all : n_max;
+
     int* o_tok = p.node_tok + (size_t)b * n_max;
     int* o_par = p.parent + (size_t)b * n_max;
     int* o_dep = p.depth + (size_t)b * n_max;
     int* o_pos = p.pos + (size_t)b * n_max;
-    const int L = p.kv_len[b];
-    if (tid < N * T) p.retrieve[(size_t)b * N * T + tid] = node;
-    if (creates && node >= 0) {
-        int par = (l == 1) ? 0 : s_node[c * T + (l - 2)];
-        o_tok[node] = s_tok[c * T + (l - 1)];
-        o_par[node] = par;
-        o_dep[node] = l;
-        o_pos[node] = L + l;
-        s_parent[node] = par;
-    }
-    if (tid == 0) {
-        o_tok[0] = p.base_tok[b]; o_par[0] = -1; o_dep[0] = 0; o_pos[0] = L;
-        s_parent[0] = -1;
-        p.n_nodes[b] = n;
-    }
-    if (tid >= n && tid < n_max) { o_tok[tid] = -1; o_par[tid] = -1; o_dep[tid] = 0; o_pos[tid] = 0; }
-    __syncthreads();
+    unsigned long long* o_mask = p.mask + (size_t)b * n_max * W;
 
-    const int W = (n_max + 63) / 64;
-    if (tid < n_max) {
-        unsigned long long m0 = 0ull, m1 = 0ull;
-        if (tid < n) {
-            int j = tid;
-            for (int hop = 0; hop <= CTCSD_MAX_T && j >= 0; ++hop) {
-                if (j < 64) m0 |= 1ull << j; else m1 |= 1ull << (j - 64);
-                j = s_parent[j];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        unsigned long long m0 = 1ull, m1 = 0ull;       // the root is everybody's ancestor
+        int parent_node = 0;
+#pragma unroll
+        for (int l = 0; l < kT; ++l) {
+            if (l < T) {
+                // owner's numbering data (all lanes take part in the shuffles)
+                const int o = (l < len[h]) ? own[h][l] : 0;
+                const int ob0 = __shfl_sync(0xffffffffu, base[0], o & 31);
+                const int ob1 = __shfl_sync(0xffffffffu, base[1], o & 31);
+                const int os0 = __shfl_sync(0xffffffffu, shared_lv[0], o & 31);
+                const int os1 = __shfl_sync(0xffffffffu, shared_lv[1], o & 31);
+                int node = -1;
+                if (l < len[h] && parent_node >= 0) {
+                    const int ob = o >= 32 ? ob1 : ob0, os = o >= 32 ? os1 : os0;
+                    node = ob + (l - os);
+                    if (node >= n_max) node = -1;
+                }
+                if (c < N) p.retrieve[((size_t)b * N + c) * T + l] = node;
+                if (node >= 0) {
+                    if (node < 64) m0 |= 1ull << node; else m1 |= 1ull << (node - 64);
+                    if (o == c) {                          // this candidate creates the node
+                        o_tok[node] = tok[h][l];
+                        o_par[node] = parent_node;
+                        o_dep[node] = l + 1;
+                        o_pos[node] = L + l + 1;
+                        o_mask[(size_t)node * W] = m0;
+                        if (W > 1) o_mask[(size_t)node * W + 1] = m1;
+                    }
+                }
+                parent_node = node;
             }
         }
-        unsigned long long* row = p.mask + ((size_t)b * n_max + tid) * W;
-        row[0] = m0;
-        if (W > 1) row[1] = m1;
+    }
+    if (lane == 0) {
+        o_tok[0] = p.base_tok[b]; o_par[0] = -1; o_dep[0] = 0; o_pos[0] = L;
+        o_mask[0] = 1ull;
+        if (W > 1) o_mask[1] = 0ull;
+        p.n_nodes[b] = n;
+    }
+    for (int i = n + lane; i < n_max; i += 32) {
+        o_tok[i] = -1; o_par[i] = -1; o_dep[i] = 0; o_pos[i] = 0;
+        o_mask[(size_t)i * W] = 0ull;
+        if (W > 1) o_mask[(size_t)i * W + 1] = 0ull;
     }
 }
 
@@ -132,7 +175,7 @@ extern "C" int ctcsd_build_tree(ctcsd_handle* hh, void* stream, const int* base_
     p.T = c.T; p.topN = c.topN; p.max_nodes = c.max_nodes;
     p.node_tok = out_node_tok; p.parent = out_parent; p.depth = out_depth; p.pos = out_pos;
     p.mask = out_mask; p.retrieve = out_retrieve; p.n_nodes = out_n_nodes;
-    build_tree_kernel<<<c.B, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    build_tree_kernel<<<c.B, 32, 0, static_cast<cudaStream_t>(stream)>>>(p);
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
