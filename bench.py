@@ -12,6 +12,7 @@ Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import subprocess
@@ -24,6 +25,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 import numpy as np  # noqa: E402
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the draft-head kernel, from the
+# ncu capture summarised in profiles/gemv_stream_kernel_c2.md (None once the kernel has changed
+# since that capture).
+NCU_TRAFFIC_BYTES = {"c2": 1310.863e6 + 3.704e6}
 
 METRIC = "draft+verify steps/s at 7B shape (batch 1, 64-node tree)"
 UNIT = "steps/s"
@@ -49,21 +55,31 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run.
+    It is started before the warm-up (nvidia-smi needs a moment to come up); only samples whose
+    timestamp falls inside a window opened with begin() and closed with end() are kept."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_ms: int = 50):
+        self.windows = []
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", str(period_ms)],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
 
+    def begin(self):
+        self._t0 = datetime.datetime.now()
+
+    def end(self):
+        self.windows.append((self._t0, datetime.datetime.now()))
+
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
         self.p.terminate()
@@ -77,14 +93,18 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             parts = [s.strip() for s in line.split(",")]
-            if len(parts) < 6:
+            if len(parts) < 7:
                 continue
             try:
-                clocks.append(float(parts[0]))
-                mx = float(parts[1])
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                clk, cmx = float(parts[1]), float(parts[2])
             except ValueError:
                 continue
-            for nme, v in zip(names, parts[2:6]):
+            if not any(a <= ts <= b for a, b in self.windows):
+                continue
+            clocks.append(clk)
+            mx = cmx
+            for nme, v in zip(names, parts[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(nme)
         self.f.close()
@@ -219,6 +239,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     K, Wm = args.steps, max(3, args.warmup)
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(Wm):
         step.run()
     step.check_status()
@@ -228,9 +249,10 @@ def run_ours(args):
     t_beg, t_end = ev(), ev()
     d_beg = [ev() for _ in range(K)]
     d_end = [ev() for _ in range(K)]
-    sampler = ClockSampler(local) if rank == 0 else None
     launches0 = step.h.launch_count
     barrier()
+    if sampler:
+        sampler.begin()
     t_beg.record()
     for i in range(K):
         d_beg[i].record()
@@ -242,8 +264,9 @@ def run_ours(args):
         step.verify()
     t_end.record()
     barrier()
+    if sampler:
+        sampler.end()
     launches = step.h.launch_count - launches0
-    clocks = sampler.stop() if sampler else None
     step.check_status()
     ms = t_beg.elapsed_time(t_end)
     draft_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(d_beg, d_end)]))
@@ -267,12 +290,17 @@ def run_ours(args):
     for _ in range(3):
         e2e_step()
     barrier()
+    if sampler:
+        sampler.begin()
     e_beg, e_end = ev(), ev()
     e_beg.record()
     for _ in range(K):
         e2e_step()
     e_end.record()
     barrier()
+    if sampler:
+        sampler.end()
+    clocks = sampler.stop() if sampler else None
     e2e_ms = e_beg.elapsed_time(e_end)
 
     if world > 1:
@@ -305,10 +333,10 @@ def run_ours(args):
             "gpu_launches": launches,
             "roofline": {"kernel": "gemv_stream_kernel (draft head)", "bound": "hbm", "achieved": achieved,
                          "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": args.traffic},
+                         "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
         }
         if world == 1 and not args.no_cpu_baseline:
-            n_or = 5
+            n_or = 10
             sec = time_oracle(cfg, inp, n_or, 1)
             line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                     "sample": "%d full steps of the fp64 oracle on the same inputs" % n_or}
@@ -320,13 +348,11 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per launch of the dominant kernel from an ncu capture (recorded in profiles/)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
