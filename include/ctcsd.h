@@ -43,6 +43,7 @@ extern "C" {
 #define CTCSD_ERR_CUDA         -4   /* a CUDA runtime/driver call failed (see ctcsd_last_cuda_error) */
 #define CTCSD_ERR_TIMEOUT      -5   /* a bounded device-side wait ran out */
 #define CTCSD_ERR_INTERNAL     -6
+#define CTCSD_ERR_TOO_LARGE    -7   /* the problem does not fit the built-in scratch of a no-allocation call */
 
 #define CTCSD_DTYPE_F32   0
 #define CTCSD_DTYPE_BF16  1
@@ -56,6 +57,7 @@ extern "C" {
 #define CTCSD_MAX_TOPN     64   /* candidates kept */
 #define CTCSD_MAX_PATHS    4096 /* k^T limit for exhaustive enumeration */
 #define CTCSD_MAX_BEAM     128
+#define CTCSD_STATIC_ATTN_SCRATCH_BYTES  (32u << 20)  /* built-in scratch of ctcsd_tree_attention_static */
 
 /* Problem shape, fixed per handle.  Notation follows the paper: T draft slots, blank id = V. */
 typedef struct ctcsd_config {
@@ -194,6 +196,40 @@ int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const voi
                         const int* node_tok, const int* parent, const int* n_nodes,
                         int* out_argmax, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
                         int* out_next_tok, float* out_logits_dbg);
+
+/*
+ * Tree attention without a handle and without any allocation (the paper has no counterpart:
+ * this is a packaging variant of ctcsd_tree_attention, same arithmetic, same kernels).
+ *
+ * Who it is for: code that is not allowed to obtain device memory when it runs - an operator
+ * plugged into a runtime that owns the memory plan, a service whose allocator is frozen after
+ * start-up, a latency-critical loop where cudaMalloc's implicit device synchronisation is not
+ * acceptable.  Such callers cannot provide the workspace that ctcsd_create asks for.  Here the
+ * scratch (the per-split partial results that the merge pass combines) lives in an array of
+ * CTCSD_STATIC_ATTN_SCRATCH_BYTES (+256) bytes inside the library's device image, which
+ * every device that loads the library keeps reserved until the process exits.  The call
+ * itself uses no cudaMalloc/cudaFree and no allocating routine.
+ *
+ * Works on the current device, bfloat16 only.  Shapes and tensors as for
+ * ctcsd_tree_attention, given explicitly instead of through a handle:
+ *   Q, out_O [B,max_nodes,Hq,D];  K, V [B,Hkv,Lcap,D];  kv_len, n_nodes [B];
+ *   mask [B,max_nodes,ceil(max_nodes/64)] uint64;  D is 64 or 128;  2 <= max_nodes <= 128.
+ * out_status: NULL, or a device int[2] that the call clears and in which a kernel records
+ *   CTCSD_ERR_INVALID_ARG (and the sequence index) if kv_len/n_nodes would read outside the cache.
+ * Limits and caveats:
+ *   - B*Hq*max_nodes*(D+2)*4 bytes must not exceed CTCSD_STATIC_ATTN_SCRATCH_BYTES, else
+ *     CTCSD_ERR_TOO_LARGE is returned and nothing is launched; within the limit the number of
+ *     KV splits is reduced until the partials fit.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array: two calls that overlap on the GPU (different
+ *     streams, or concurrent graphs) race on it.  Serialise them.
+ */
+int ctcsd_tree_attention_static(void* stream, int B, int max_nodes, int Hq, int Hkv, int D,
+                                const void* Q, const void* K, const void* V, int Lcap,
+                                const int* kv_len, const int* n_nodes,
+                                const unsigned long long* mask, float scale, void* out_O,
+                                int* out_status);
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,7 @@ EXPORTS = [
     "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
     "ctcsd_last_cuda_error", "ctcsd_launch_count",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
-    "ctcsd_verify_accept",
+    "ctcsd_verify_accept", "ctcsd_tree_attention_static",
 ]
 
 
@@ -64,6 +64,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_build_tree.argtypes = [vp, vp] + [vp] * 12
     lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
     lib.ctcsd_verify_accept.argtypes = [vp, vp] + [vp] * 11
+    lib.ctcsd_tree_attention_static.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp, vp, vp,
+                                                ctypes.c_float, vp, vp]
     for name in EXPORTS:
         if name not in ("ctcsd_strerror", "ctcsd_launch_count"):
             getattr(lib, name).restype = ci
@@ -212,3 +214,24 @@ class Handle:
             _ptr(out_next_tok, i32, c.B, "out_next_tok"),
             _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
         self._check(rc, "verify_accept")
+
+
+def tree_attention_static(Q, K, V, kv_len, n_nodes, mask, scale, out_O, out_status=None, stream=None):
+    """ctcsd_tree_attention_static: tree attention for callers that may not allocate device
+    memory (no handle, no workspace; the scratch is a fixed array inside the library).
+    Q, out_O [B,max_nodes,Hq,D] bfloat16; K, V [B,Hkv,Lcap,D] bfloat16; kv_len, n_nodes [B] int32;
+    mask [B,max_nodes,W] int64 bit-masks; out_status None or int32[2].  Raises CtcsdError on a
+    non-zero status, e.g. when the shape exceeds the built-in scratch."""
+    lib = load_library()
+    B, n, Hq, D = Q.shape
+    Hkv, Lcap = K.shape[1], K.shape[2]
+    W = (n + 63) // 64
+    bf, i32 = torch.bfloat16, torch.int32
+    rc = lib.ctcsd_tree_attention_static(
+        _stream_ptr(stream), B, n, Hq, Hkv, D,
+        _ptr(Q, bf, B * n * Hq * D, "Q"), _ptr(K, bf, B * Hkv * Lcap * D, "K"), _ptr(V, bf, B * Hkv * Lcap * D, "V"),
+        Lcap, _ptr(kv_len, i32, B, "kv_len"), _ptr(n_nodes, i32, B, "n_nodes"),
+        _ptr(mask, torch.int64, B * n * W, "mask"), float(scale), _ptr(out_O, bf, B * n * Hq * D, "out_O"),
+        _ptr(out_status, i32, 2, "out_status"))
+    if rc != 0:
+        raise CtcsdError("ctcsd_tree_attention_static failed: %s" % lib.ctcsd_strerror(rc).decode())

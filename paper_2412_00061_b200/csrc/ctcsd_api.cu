@@ -128,6 +128,7 @@ extern "C" const char* ctcsd_strerror(int status) {
         case CTCSD_ERR_CUDA: return "CUDA call failed";
         case CTCSD_ERR_TIMEOUT: return "device-side wait timed out";
         case CTCSD_ERR_INTERNAL: return "internal error";
+        case CTCSD_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

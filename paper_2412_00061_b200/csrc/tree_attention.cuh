@@ -21,4 +21,7 @@ struct AttnParams {
 // bf16 tensor-core path (flash-style, KV split across CTAs, GQA head grouping).
 int launch_tree_attention_mma(Handle* h, cudaStream_t s, const AttnParams& p);
 
+// The same kernels with caller-chosen scratch: `part` holds B*Hq*max_nodes*splits*(D+2) floats.
+cudaError_t launch_tree_attention_mma_scratch(cudaStream_t s, const AttnParams& p, float* part, int splits);
+
 }  // namespace ctcsd

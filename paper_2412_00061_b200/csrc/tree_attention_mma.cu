@@ -304,7 +304,33 @@ int launch_d(Handle* h, cudaStream_t s, const AttnParams& p) {
     return CTCSD_OK;
 }
 
+// Same two launches with the partial buffer and the split count given by the caller of this
+// function instead of a handle's workspace.  `part` holds B*Hq*max_nodes*splits*(D+2) floats.
+template <int D>
+cudaError_t launch_d_scratch(cudaStream_t s, const AttnParams& p, float* part, int splits) {
+    const int grp = p.Hq / p.Hkv;
+    const int qtiles = (p.max_nodes * grp + kRows - 1) / kRows;
+    const size_t smem = (size_t)kRows * D * 2 + 4 * (size_t)kKeys * D * 2;
+    auto kern = tree_attention_mma_kernel<D>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    dim3 grid(qtiles * splits, p.Hkv, p.B);
+    kern<<<grid, kThreads, smem, s>>>(p, part, splits);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long warps = (long long)p.B * p.max_nodes * p.Hq;
+    tree_attention_merge_kernel<D><<<(unsigned)((warps + 3) / 4), 128, 0, s>>>(p, part, splits);
+    return cudaGetLastError();
+}
+
 }  // namespace
+
+cudaError_t launch_tree_attention_mma_scratch(cudaStream_t s, const AttnParams& p, float* part, int splits) {
+    if (p.D == 64) return launch_d_scratch<64>(s, p, part, splits);
+    return launch_d_scratch<128>(s, p, part, splits);
+}
 
 int launch_tree_attention_mma(Handle* h, cudaStream_t s, const AttnParams& p) {
     if (p.D == 64) return launch_d<64>(h, s, p);
