@@ -35,11 +35,12 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
     size_t off = 0;
     l.status_off = off;      off = align_up(off + 16 * sizeof(int), 256);
     l.counter_off = off;     off = align_up(off + kCounters * sizeof(unsigned), 256);
+    l.lm_key_count = (c.B * c.max_nodes + 127) / 128 * 128;
+    l.lm_key_off = off;      off = align_up(off + sizeof(unsigned long long) * (size_t)l.lm_key_count, 256);
+    l.zeroed_bytes = off;
     l.gemv_grid_max = num_sms * 8 > 64 ? num_sms * 8 : 64;
     l.draft_part_off = off;  off = align_up(off + sizeof(DraftPartial) * 4 * (size_t)l.gemv_grid_max * 2, 256);
     l.part_slot_off = off;   off = align_up(off + sizeof(int) * (size_t)l.gemv_grid_max * 2, 256);
-    l.lm_tiles_max = (c.V + 15) / 16 + 8;
-    l.lm_part_off = off;     off = align_up(off + sizeof(ArgmaxPartial) * (size_t)l.lm_tiles_max * c.B * c.max_nodes, 256);
     int units = c.B * c.Hkv;
     int splits = (2 * num_sms + units - 1) / units;
     if (splits < 1) splits = 1;
@@ -89,8 +90,8 @@ extern "C" int ctcsd_create(ctcsd_handle** out_handle, const ctcsd_config* cfg, 
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, h->device);
     if (e == cudaSuccess && major != 10) { delete hh; return CTCSD_ERR_UNSUPPORTED; }
     if (e == cudaSuccess && h->num_sms > kLayoutSms) { delete hh; return CTCSD_ERR_UNSUPPORTED; }
-    // status word and ticket counters start at zero
-    if (e == cudaSuccess) e = cudaMemset(workspace, 0, lay.draft_part_off);
+    // status word, ticket counters and running maxima start at zero
+    if (e == cudaSuccess) e = cudaMemset(workspace, 0, lay.zeroed_bytes);
     if (e != cudaSuccess) { delete hh; return CTCSD_ERR_CUDA; }
     *out_handle = hh;
     return CTCSD_OK;
@@ -110,9 +111,8 @@ extern "C" int ctcsd_poll_status(ctcsd_handle* hh, void* stream, int* out_status
     CTCSD_CUDA_CHECK(h, cudaMemcpyAsync(st, status_ptr(h), sizeof(st), cudaMemcpyDeviceToHost, s));
     CTCSD_CUDA_CHECK(h, cudaStreamSynchronize(s));
     if (st[0] != 0) {
-        CTCSD_CUDA_CHECK(h, cudaMemsetAsync(status_ptr(h), 0, 16 * sizeof(int), s));
-        // a kernel that gave up may have left its ticket counters mid-count
-        CTCSD_CUDA_CHECK(h, cudaMemsetAsync(counter_ptr(h), 0, kCounters * sizeof(unsigned), s));
+        // a kernel that gave up may have left its ticket counters and running maxima mid-way
+        CTCSD_CUDA_CHECK(h, cudaMemsetAsync(h->ws, 0, h->lay.zeroed_bytes, s));
         CTCSD_CUDA_CHECK(h, cudaStreamSynchronize(s));
     }
     *out_status = st[0];

@@ -8,8 +8,10 @@
 // fetched from HBM once; the kernel is a weight stream whose math hides behind the loads.
 // Warp 0 issues TMA loads into a ring of shared-memory stages, warp 1 issues the MMAs,
 // warps 2..5 read the accumulator back (each warp its own 32 TMEM lanes) and keep the
-// running arg-max of their row.  Per-unit winners go to the workspace; the last CTA to
-// finish reduces them over the vocabulary tiles (ties -> lower id).
+// running arg-max of their row.  Each tile's winner is folded into the row's global maximum
+// with one 64-bit atomic max on a packed (logit, complemented id) key, so ties go to the
+// lower id; the CTA that finishes last unpacks the keys, clears them for the next call and
+// runs the greedy acceptance walk.
 #include "lm_head_tc.cuh"
 #include "tc_primitives.cuh"
 
@@ -32,7 +34,8 @@ struct TcParams {
     int n_tiles;      // vocabulary tiles
     int m_tiles;      // row tiles of 128
     int stages;
-    ArgmaxPartial* part;      // [n_tiles][m_tiles*128]
+    unsigned long long* keys; // [m_tiles*128] packed (logit, id) maxima, zero between calls
+    AcceptParams acc;
     unsigned* counter;
     int* out_argmax;          // [M]
     float* logits_dbg;        // null or [M][V]
@@ -185,10 +188,13 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&sh->tmem_empty);
-            ArgmaxPartial out;
-            out.val = best;
-            out.idx = best_idx;
-            p.part[(size_t)nt * (p.m_tiles * kTileM) + row] = out;
+            // fold this tile's winner into the row's global maximum: larger logit first, equal
+            // logits -> lower id (the id is stored complemented in the low word)
+            if (row < p.M && best_idx != 0x7fffffff) {
+                const unsigned u = __float_as_uint(best);
+                const unsigned sortable = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+                atomicMax(p.keys + row, ((unsigned long long)sortable << 32) | (0xffffffffu - (unsigned)best_idx));
+            }
         }
         if (!ok && lane == 0) {
             if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 3);
@@ -211,20 +217,15 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     if (!sh->is_last) return;
     __threadfence();
-    if (sh->abort_flag == 0) {
-        const int mpad = p.m_tiles * kTileM;
-        for (int row = tid; row < p.M; row += kThreads) {
-            float best = -INFINITY;
-            int best_idx = 0x7fffffff;
-            for (int nt = 0; nt < p.n_tiles; ++nt) {
-                const ArgmaxPartial* src = p.part + (size_t)nt * mpad + row;
-                float v = __ldcg(&src->val);
-                int ix = __ldcg(&src->idx);
-                if (v > best || (v == best && ix < best_idx)) { best = v; best_idx = ix; }
-            }
-            p.out_argmax[row] = best_idx;
-        }
+    const bool good = sh->abort_flag == 0;
+    for (int row = tid; row < p.M; row += kThreads) {
+        const unsigned long long key = __ldcg(p.keys + row);
+        if (good) p.out_argmax[row] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
+        p.keys[row] = 0ull;
     }
+    __syncthreads();
+    if (good)
+        for (int b = warp; b < p.acc.B; b += kThreads / 32) greedy_accept_warp(p.acc, b, lane);
     if (tid == 0) *p.counter = 0u;
 }
 
@@ -266,7 +267,7 @@ bool lm_head_tc_supported(const Handle* h) {
 }
 
 int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, const void* Wl,
-                      int* out_argmax, float* out_logits_dbg) {
+                      int* out_argmax, float* out_logits_dbg, const AcceptParams& acc) {
     const ctcsd_config& c = h->cfg;
     if (!lm_head_tc_supported(h)) return CTCSD_ERR_UNSUPPORTED;
 
@@ -282,13 +283,14 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     int g_per_tile = (per_sm + rounds - 1) / rounds;
     p.Nt = 16 * g_per_tile;
     p.n_tiles = (c.V + p.Nt - 1) / p.Nt;
-    if (p.n_tiles > h->lay.lm_tiles_max) return CTCSD_ERR_WORKSPACE;
+    if (p.m_tiles * kTileM > h->lay.lm_key_count) return CTCSD_ERR_WORKSPACE;
     const int stage_bytes = kABytes + p.Nt * 128;
     int stages = (int)((220 * 1024 - (int)sizeof(TcShared) - 1024) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return CTCSD_ERR_UNSUPPORTED;
     p.stages = stages;
-    p.part = reinterpret_cast<ArgmaxPartial*>(h->ws + h->lay.lm_part_off);
+    p.keys = reinterpret_cast<unsigned long long*>(h->ws + h->lay.lm_key_off);
+    p.acc = acc;
     p.counter = counter_ptr(h) + 1;
     p.out_argmax = out_argmax;
     p.logits_dbg = out_logits_dbg;

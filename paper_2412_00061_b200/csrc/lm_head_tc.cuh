@@ -2,6 +2,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "accept.cuh"
 
 namespace ctcsd {
 
@@ -9,8 +10,9 @@ namespace ctcsd {
 bool lm_head_tc_supported(const Handle* h);
 
 // y = hn . Wl^T on the 5th-generation tensor cores with the row arg-max folded into the
-// epilogue.  Returns CTCSD_ERR_UNSUPPORTED when the shape is not covered.
+// epilogue; the CTA that finishes last decodes the arg-max and runs the greedy acceptance walk
+// `acc` over it.  Returns CTCSD_ERR_UNSUPPORTED when the shape is not covered.
 int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, const void* Wl,
-                      int* out_argmax, float* out_logits_dbg);
+                      int* out_argmax, float* out_logits_dbg, const AcceptParams& acc);
 
 }  // namespace ctcsd
