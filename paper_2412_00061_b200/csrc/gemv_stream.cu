@@ -1,5 +1,6 @@
 // Weight-streaming matrix-vector kernel (see gemv_stream.cuh).
 #include "gemv_stream.cuh"
+#include "tc_primitives.cuh"
 
 #include <limits.h>
 #include <math.h>
@@ -8,9 +9,9 @@ namespace ctcsd {
 
 namespace {
 
-constexpr int kRW = 4;            // weight rows a warp carries through one sweep over H
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
+constexpr int kWarps = 8;                     // consumer warps
+constexpr int kThreads = (kWarps + 1) * 32;   // plus one producer warp
+constexpr int kMaxSlots = 32;                 // ring slots
 
 template <typename T> struct Elem;
 
@@ -119,16 +120,42 @@ __device__ __forceinline__ void warp_combine(RunState& st) {
     for (int q = 0; q < kTopSlots; ++q) { st.val[q] = ov[q]; st.id[q] = oi[q]; }
 }
 
+// Shared-memory bookkeeping of the weight ring.
+struct __align__(8) RingShared {
+    uint64_t full[kMaxSlots];     // the slot's weight rows have landed
+    uint64_t empty[kMaxSlots];    // every consumer warp of the slot has read its row
+    int abort_flag;
+    int never_set;                // stays zero: lets a drain wait run to its time limit after an abort
+    int is_last;
+};
+
+// One CTA per SM.  Warp 8 is the producer: it walks the CTA's contiguous range of weight rows
+// and copies `G` rows (about 32 KB) per ring slot with the bulk-copy engine, as far ahead as
+// the ring allows (about 190 KB in flight per SM).  Warps 0..7 are consumers: they form 8/G
+// groups that take the slots in turn; within a group each warp owns one row of the slot,
+// multiplies it with the activation rows held in shared memory, frees the slot and folds the
+// logit into its lanes' running (max, sum of exp, best-8) states.
 template <typename T, int MROWS>
-__global__ void __launch_bounds__(kThreads) gemv_stream_kernel(GemvParams p) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint4* xs = reinterpret_cast<uint4*>(smem_raw);                 // [MROWS][nch]
-    __shared__ DraftPartial s_part[kWarps][MROWS];
-    __shared__ int s_last;
+__global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, int nslots, int G) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int row_bytes = p.H * (int)sizeof(T);
+    const int nch = row_bytes / 16;                                  // 16-byte chunks per row
+    const int slot_bytes = G * row_bytes;
+    uint4* xs = reinterpret_cast<uint4*>(smem_raw);                  // [MROWS][nch]
+    unsigned char* ring = smem_raw + (size_t)MROWS * row_bytes;      // [nslots][G][row_bytes]
+    RingShared* sh = reinterpret_cast<RingShared*>(ring + (size_t)nslots * slot_bytes);
+    __shared__ DraftPartial s_part[2][kWarps][MROWS];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nch = p.H * (int)sizeof(T) / 16;                      // 16-byte chunks per row
+    volatile int* abort_flag = &sh->abort_flag;
 
+    if (tid == 0) {
+        for (int s = 0; s < nslots; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], G); }
+        sh->abort_flag = 0;
+        sh->never_set = 0;
+        sh->is_last = 0;
+        tc::fence_barrier_init();
+    }
     for (int i = tid; i < MROWS * nch; i += kThreads) {
         int m = i / nch, ch = i - m * nch;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -146,84 +173,124 @@ __global__ void __launch_bounds__(kThreads) gemv_stream_kernel(GemvParams p) {
     const long long R = rps * p.slots;
     const long long r0 = R * blockIdx.x / gridDim.x;
     const long long r1 = R * (blockIdx.x + 1) / gridDim.x;
+    const int ntotal = (int)(r1 - r0);                               // rows of this CTA
+    const int nfill = (ntotal + G - 1) / G;                          // ring fills of this CTA
     const int slot0 = (int)(r0 / rps);
-    const uint4* Wbase = reinterpret_cast<const uint4*>(p.W);
-    const uint64_t policy = l2_policy_evict_first();
+    const long long seg_end = (long long)(slot0 + 1) * rps;          // first row of the next slot
+    const int n_seg0 = (int)((r1 < seg_end ? r1 : seg_end) - r0);    // rows that belong to slot0
+    const unsigned char* Wbase = reinterpret_cast<const unsigned char*>(p.W);
 
-    for (int seg = 0; seg < 2; ++seg) {
-        const int slot = slot0 + seg;
-        long long a = seg == 0 ? r0 : (long long)(slot0 + 1) * rps;
-        long long b = seg == 0 ? (r1 < (long long)(slot0 + 1) * rps ? r1 : (long long)(slot0 + 1) * rps) : r1;
-        const int nrows = b > a ? (int)(b - a) : 0;
-        const int v0 = (int)(a - (long long)slot * rps);            // first class id of the segment
-
-        RunState st;
-        st.init();
-        const int ngroups = (nrows + kRW - 1) / kRW;
-        for (int g = warp; g < ngroups; g += kWarps) {
-            const uint4* wp[kRW];
-#pragma unroll
-            for (int r = 0; r < kRW; ++r) {
-                int lr = g * kRW + r;
-                if (lr >= nrows) lr = nrows - 1;                     // clamp: loaded again, result unused
-                wp[r] = Wbase + (size_t)(a + lr) * nch;
-            }
-            float acc[kRW][MROWS];
-#pragma unroll
-            for (int r = 0; r < kRW; ++r)
-#pragma unroll
-                for (int m = 0; m < MROWS; ++m) acc[r][m] = 0.f;
-
-#pragma unroll 2
-            for (int ch = lane; ch < nch; ch += 32) {
-                uint4 w[kRW];
-#pragma unroll
-                for (int r = 0; r < kRW; ++r) w[r] = ld_stream16(wp[r] + ch, policy);
-#pragma unroll
-                for (int m = 0; m < MROWS; ++m) {
-                    uint4 xv = xs[m * nch + ch];
-#pragma unroll
-                    for (int r = 0; r < kRW; ++r) acc[r][m] = Elem<T>::dot(w[r], xv, acc[r][m]);
+    if (warp == kWarps) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            const uint64_t policy = tc::policy_evict_first();
+            bool ok = true;
+            int j = 0;
+            for (; j < nfill; ++j) {
+                const int s = j % nslots;
+                const uint32_t ph = (uint32_t)(j / nslots) & 1u;
+                if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                const int rows = (ntotal - j * G < G) ? ntotal - j * G : G;
+                const uint32_t bytes = (uint32_t)rows * (uint32_t)row_bytes;
+                // never hand the copy engine a range outside the weights or the ring
+                const long long first = r0 + (long long)j * G;
+                if (rows < 1 || first < 0 || first + rows > R || (bytes & 15u) != 0 || bytes > (uint32_t)slot_bytes ||
+                    s >= nslots) {
+                    report_error(p.status, CTCSD_ERR_INTERNAL, 12);
+                    ok = false;
+                    break;
                 }
+                tc::mbar_arrive_expect_tx(&sh->full[s], bytes);
+                tc::bulk_load_1d(ring + (size_t)s * slot_bytes, Wbase + (size_t)first * row_bytes, bytes,
+                                 &sh->full[s], policy);
             }
-#pragma unroll
-            for (int r = 0; r < kRW; ++r)
-#pragma unroll
-                for (int m = 0; m < MROWS; ++m) acc[r][m] = warp_sum(acc[r][m]);
-
-#pragma unroll
-            for (int r = 0; r < kRW; ++r) {
-                int lr = g * kRW + r;
-                if (lr < nrows) {
-                    float z = 0.f;
-#pragma unroll
-                    for (int m = 0; m < MROWS; ++m) if (lane == m) z = acc[r][m];
-                    if (lane < p.mcount) {
-                        int v = v0 + lr;
-                        if (v == (int)rps - 1) z += bias;
-                        if (p.logits_dbg)
-                            p.logits_dbg[((size_t)(p.m0 + lane) * p.slots + slot) * rps + v] = z;
-                        st.push(z, v);
-                    }
+            if (!ok) {
+                if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 10);
+                *abort_flag = 1;
+            }
+            if (*abort_flag != 0) {
+                // let copies that are still in flight land before the CTA gives its memory back
+                for (int back = 1; back <= nslots && back <= j; ++back) {
+                    const int q = j - back;
+                    tc::mbar_wait(&sh->full[q % nslots], (uint32_t)(q / nslots) & 1u, &sh->never_set, 1ll << 24);
                 }
             }
         }
+    } else {
+        // ---------------- consumers ----------------
+        RunState st;
+        st.init();
+        int cur_seg = 0;
+        bool ok = true;
+        const int groups = kWarps / G;
+        const int rin = warp % G;                       // this warp's row within a slot
+        for (int j = warp / G; j < nfill; j += groups) {
+            const int s = j % nslots;
+            const uint32_t ph = (uint32_t)(j / nslots) & 1u;
+            if (!tc::mbar_wait(&sh->full[s], ph, abort_flag)) { ok = false; break; }
+            const int i = j * G + rin;                  // row of the CTA's range
+            float acc[MROWS];
+#pragma unroll
+            for (int m = 0; m < MROWS; ++m) acc[m] = 0.f;
+            if (i < ntotal) {
+                const uint4* wrow = reinterpret_cast<const uint4*>(ring + (size_t)s * slot_bytes + (size_t)rin * row_bytes);
+#pragma unroll 4
+                for (int ch = lane; ch < nch; ch += 32) {
+                    const uint4 w = wrow[ch];
+#pragma unroll
+                    for (int m = 0; m < MROWS; ++m) acc[m] = Elem<T>::dot(w, xs[m * nch + ch], acc[m]);
+                }
+            }
+            // the accumulators depend on every load of the row: the slot can be refilled
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+            if (i >= ntotal) continue;
+            const int seg = i >= n_seg0 ? 1 : 0;
+            if (seg != cur_seg) {                       // this warp's rows now belong to the next slot
+                if (lane < MROWS) st.store(&s_part[0][warp][lane]);
+                st.init();
+                cur_seg = 1;
+            }
+#pragma unroll
+            for (int m = 0; m < MROWS; ++m) acc[m] = warp_sum(acc[m]);
+            float z = 0.f;
+#pragma unroll
+            for (int m = 0; m < MROWS; ++m) if (lane == m) z = acc[m];
+            if (lane < p.mcount) {
+                const int slot = slot0 + seg;
+                const int v = (int)(r0 + i - (long long)slot * rps);
+                if (v == (int)rps - 1) z += bias;
+                if (p.logits_dbg) p.logits_dbg[((size_t)(p.m0 + lane) * p.slots + slot) * rps + v] = z;
+                st.push(z, v);
+            }
+        }
+        if (!ok && lane == 0) {
+            if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 11);
+            *abort_flag = 1;
+        }
+        if (lane < MROWS) {
+            if (cur_seg == 0) {
+                st.store(&s_part[0][warp][lane]);
+                st.init();
+            }
+            st.store(&s_part[1][warp][lane]);
+        }
+    }
+    __syncthreads();
 
-        // fold the 8 warps' states: warp m merges row m's states, one per lane
-        if (lane < MROWS) st.store(&s_part[warp][lane]);
-        __syncthreads();
+    // fold the 8 warps' states per segment: warp m merges activation row m's states, one per lane
+    for (int seg = 0; seg < 2; ++seg) {
         if (warp < MROWS) {
             RunState ms;
             ms.init();
-            if (lane < kWarps) ms.absorb(s_part[lane][warp]);
+            if (lane < kWarps) ms.absorb(s_part[seg][lane][warp]);
             warp_combine(ms);
-            if (lane == 0) {
-                DraftPartial* dst = p.part + ((size_t)warp * p.grid + blockIdx.x) * 2 + seg;
-                ms.store(dst);
-            }
+            if (lane == 0) ms.store(p.part + ((size_t)warp * p.grid + blockIdx.x) * 2 + seg);
         }
-        if (tid == 0) p.part_slot[blockIdx.x * 2 + seg] = (nrows > 0 && slot < p.slots) ? slot : -1;
-        __syncthreads();
+        if (tid == 0) {
+            const int nrows = seg == 0 ? n_seg0 : ntotal - n_seg0;
+            p.part_slot[blockIdx.x * 2 + seg] = (nrows > 0 && slot0 + seg < p.slots) ? slot0 + seg : -1;
+        }
     }
 
     // the last CTA to arrive merges every CTA's partials into the final outputs
@@ -231,14 +298,14 @@ __global__ void __launch_bounds__(kThreads) gemv_stream_kernel(GemvParams p) {
     __syncthreads();
     if (tid == 0) {
         unsigned t = atomicAdd(p.counter, 1u);
-        s_last = (t == gridDim.x - 1);
+        sh->is_last = (t == gridDim.x - 1);
     }
     __syncthreads();
-    if (!s_last) return;
+    if (!sh->is_last) return;
     __threadfence();
 
     const int ntask = p.mcount * p.slots;
-    for (int task = warp; task < ntask; task += kWarps) {
+    for (int task = warp; task < ntask; task += kThreads / 32) {
         const int m = task / p.slots, slot = task - m * p.slots;
         RunState fs;
         fs.init();
@@ -273,20 +340,25 @@ __global__ void __launch_bounds__(kThreads) gemv_stream_kernel(GemvParams p) {
 template <typename T, int MROWS>
 int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     auto kern = gemv_stream_kernel<T, MROWS>;
-    size_t smem = (size_t)MROWS * p.H * sizeof(T);
-    if (smem > 200 * 1024) return CTCSD_ERR_UNSUPPORTED;
-    if (smem > 48 * 1024)
-        CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int occ = 0;
-    CTCSD_CUDA_CHECK(h, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, smem));
-    if (occ < 1) return CTCSD_ERR_UNSUPPORTED;
-    if (occ > 8) occ = 8;
+    const size_t row_bytes = (size_t)p.H * sizeof(T);
+    const size_t budget = 200 * 1024;                          // dynamic shared memory per CTA
+    const size_t fixed = (size_t)MROWS * row_bytes + sizeof(RingShared);
+    // rows per ring slot: a power of two that divides the 8 consumer warps, about 32 KB per copy
+    int G = 1;
+    while (G < kWarps && (size_t)(2 * G) * row_bytes <= 32 * 1024) G *= 2;
+    while (G > 1 && fixed + 3 * (size_t)G * row_bytes > budget) G /= 2;
+    const size_t slot_bytes = (size_t)G * row_bytes;
+    if (fixed + 2 * slot_bytes > budget) return CTCSD_ERR_UNSUPPORTED;
+    long long nslots = (long long)((budget - fixed) / slot_bytes);
+    if (nslots > kMaxSlots) nslots = kMaxSlots;
+    const size_t smem = fixed + (size_t)nslots * slot_bytes;
+    CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     long long R = (long long)p.slots * p.rows_per_slot;
-    long long grid = (long long)h->num_sms * occ;
+    long long grid = h->num_sms;
     if (grid > R) grid = R;
     if (grid < p.slots) grid = p.slots;         // a CTA's range then touches at most two slots
     p.grid = (int)grid;
-    kern<<<(unsigned)grid, kThreads, smem, stream>>>(p);
+    kern<<<(unsigned)grid, kThreads, smem, stream>>>(p, (int)nslots, G);
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
@@ -311,6 +383,7 @@ int launch_gemv_stream(Handle* h, cudaStream_t stream, int dtype, int M, GemvPar
     p.part = reinterpret_cast<DraftPartial*>(h->ws + h->lay.draft_part_off);
     p.part_slot = reinterpret_cast<int*>(h->ws + h->lay.part_slot_off);
     p.counter = counter_ptr(h);
+    p.status = status_ptr(h);
     if (dtype == CTCSD_DTYPE_BF16) return launch_typed<__nv_bfloat16>(h, stream, M, p);
     return launch_typed<float>(h, stream, M, p);
 }

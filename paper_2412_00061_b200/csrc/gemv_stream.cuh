@@ -1,8 +1,8 @@
 // Weight-streaming matrix-vector kernel for small row counts (CUDA cores).
 //
 // Used where the projection is bound by HBM bandwidth: every weight row is read exactly
-// once with 128-bit streaming loads and multiplied with up to four activation rows that
-// sit in shared memory.  The logits are never written out (unless the caller asks for the
+// once, by a bulk copy into a deep shared-memory ring, and multiplied with up to four
+// activation rows that sit in shared memory.  The logits are never written out (unless the caller asks for the
 // debug dump); each CTA folds them into a running (max, sum of exp, best-8) state per
 // (activation row, slot), and the last CTA to finish merges all partial states into the
 // per-slot log-sum-exp and top-k (draft head) or the arg-max (LM head).
@@ -33,6 +33,7 @@ struct GemvParams {
     float* out_lse;           // mode 0: [M,slots]
     int* out_argmax;          // mode 1: [M]
     float* logits_dbg;        // null or [M,slots,rows_per_slot]
+    int* status;              // device status word
 };
 
 int launch_gemv_stream(Handle* h, cudaStream_t stream, int dtype, int M, GemvParams p);
