@@ -31,7 +31,7 @@ struct Layout {
     size_t status_off;        // int[16]: [0] status word, [1] detail
     size_t counter_off;       // unsigned[kCounters]: "chunks finished" tickets, zero between calls
     size_t zeroed_bytes;      // everything below this offset is cleared when the handle is created
-    size_t draft_part_off;    // DraftPartial[4][gemv_grid_max][2]  (weight-streaming GEMV partials)
+    size_t draft_part_off;    // DraftPartial[8][gemv_grid_max][2]  (weight-streaming GEMV partials)
     size_t part_slot_off;     // int[gemv_grid_max][2]
     size_t lm_key_off;        // uint64[lm_key_count]: packed (logit, id) row maxima of the tensor-core LM head, zero between calls
     size_t attn_part_off;     // float[B][Hq][max_nodes][kv_splits][D+2]

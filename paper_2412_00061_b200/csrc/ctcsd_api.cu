@@ -39,7 +39,7 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
     l.lm_key_off = off;      off = align_up(off + sizeof(unsigned long long) * (size_t)l.lm_key_count, 256);
     l.zeroed_bytes = off;
     l.gemv_grid_max = num_sms * 8 > 64 ? num_sms * 8 : 64;
-    l.draft_part_off = off;  off = align_up(off + sizeof(DraftPartial) * 4 * (size_t)l.gemv_grid_max * 2, 256);
+    l.draft_part_off = off;  off = align_up(off + sizeof(DraftPartial) * 8 * (size_t)l.gemv_grid_max * 2, 256);
     l.part_slot_off = off;   off = align_up(off + sizeof(int) * (size_t)l.gemv_grid_max * 2, 256);
     int units = c.B * c.Hkv;
     int splits = (2 * num_sms + units - 1) / units;

@@ -10,8 +10,11 @@ namespace ctcsd {
 namespace {
 
 constexpr int kWarps = 8;                     // consumer warps
-constexpr int kThreads = (kWarps + 1) * 32;   // plus one producer warp
+constexpr int kEpiWarps = 4;                  // warps that fold logits into the running states (bf16 path)
+constexpr int kThreads = (kWarps + 1 + kEpiWarps) * 32;   // consumers, one producer warp, epilogue warps
+constexpr int kCDepth = 4;                    // partial-sum buffers between consumers and epilogue
 constexpr int kMaxSlots = 32;                 // ring slots
+constexpr int kRowsPerWarp = 2;               // a slot holds at most kWarps * kRowsPerWarp weight rows
 
 template <typename T> struct Elem;
 
@@ -123,34 +126,60 @@ __device__ __forceinline__ void warp_combine(RunState& st) {
 // Shared-memory bookkeeping of the weight ring.
 struct __align__(8) RingShared {
     uint64_t full[kMaxSlots];     // the slot's weight rows have landed
-    uint64_t empty[kMaxSlots];    // every consumer warp of the slot has read its row
+    uint64_t empty[kMaxSlots];    // every consumer warp has read its part of the slot
+    uint64_t cfull[kCDepth];      // every consumer warp has written its partial sums of a fill
+    uint64_t cempty[kCDepth];     // every epilogue warp has read them
     int abort_flag;
     int never_set;                // stays zero: lets a drain wait run to its time limit after an abort
     int is_last;
 };
 
+constexpr int kStateRows = 16;    // running states per activation row inside a CTA (merged at the end)
+
+// D[16x8] += A[16x16] * B[16x8], bf16 operands, fp32 accumulators (warp-wide).
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // One CTA per SM.  Warp 8 is the producer: it walks the CTA's contiguous range of weight rows
-// and copies `G` rows (about 32 KB) per ring slot with the bulk-copy engine, as far ahead as
-// the ring allows (about 190 KB in flight per SM).  Warps 0..7 are consumers: they form 8/G
-// groups that take the slots in turn; within a group each warp owns one row of the slot,
-// multiplies it with the activation rows held in shared memory, frees the slot and folds the
-// logit into its lanes' running (max, sum of exp, best-8) states.
+// and copies G rows (about 64 KB: the copy engine's cost per copy is high) per ring slot with
+// the bulk-copy engine, as far ahead as the ring allows.  Warps 0..7 consume the slots in
+// order.
+//   bfloat16: the warps split the hidden axis.  Each warp multiplies its share of all G rows
+//   with the activation rows on the tensor cores (mma.m16n8k16: the 16 "M" rows are weight
+//   rows, the 8 "N" columns are activation rows, so up to 8 activation rows cost the same as
+//   one); the per-warp partial sums go to a small ring in shared memory, from which warps
+//   9..12 (the epilogue) add them up and fold the logits into the running states, off the
+//   consumers' critical path.
+//   float32: each warp owns whole rows of the slot, uses fused multiply-adds and folds its own
+//   logits.
+// The running (max, sum of exp, best-8) states are held by the threads that own a (weight row
+// of the slot, activation row) pair; they are merged per CTA at the end and per grid by the CTA
+// that finishes last.
 template <typename T, int MROWS>
 __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, int nslots, int G) {
+    constexpr bool kMma = sizeof(T) == 2;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int row_bytes = p.H * (int)sizeof(T);
     const int nch = row_bytes / 16;                                  // 16-byte chunks per row
     const int slot_bytes = G * row_bytes;
-    uint4* xs = reinterpret_cast<uint4*>(smem_raw);                  // [MROWS][nch]
-    unsigned char* ring = smem_raw + (size_t)MROWS * row_bytes;      // [nslots][G][row_bytes]
+    // activation rows are padded by 64 bytes so that neighbouring rows start in different banks
+    const int x_stride = nch + 4;                                    // in 16-byte chunks
+    uint4* xs = reinterpret_cast<uint4*>(smem_raw);                  // [MROWS][x_stride]
+    unsigned char* ring = smem_raw + (size_t)MROWS * x_stride * 16;  // [nslots][G][row_bytes]
     RingShared* sh = reinterpret_cast<RingShared*>(ring + (size_t)nslots * slot_bytes);
-    __shared__ DraftPartial s_part[2][kWarps][MROWS];
+    __shared__ DraftPartial s_part[2][kStateRows][MROWS];
+    __shared__ float s_cpart[kCDepth][kWarps][16][8];                // per-warp partial sums of a fill (bf16 path)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     volatile int* abort_flag = &sh->abort_flag;
 
     if (tid == 0) {
-        for (int s = 0; s < nslots; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], G); }
+        for (int s = 0; s < nslots; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], kWarps); }
+        for (int d = 0; d < kCDepth; ++d) { tc::mbar_init(&sh->cfull[d], kWarps); tc::mbar_init(&sh->cempty[d], kEpiWarps); }
         sh->abort_flag = 0;
         sh->never_set = 0;
         sh->is_last = 0;
@@ -160,12 +189,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
         int m = i / nch, ch = i - m * nch;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (m < p.mcount) v = reinterpret_cast<const uint4*>(p.x)[(size_t)(p.m0 + m) * nch + ch];
-        xs[i] = v;
+        xs[m * x_stride + ch] = v;
     }
-    float bias = 0.f;
-    if (lane < p.mcount && p.blank_bias != nullptr) {
-        int row = p.m0 + lane;
-        bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
+    for (int i = tid; i < 2 * kStateRows * MROWS; i += kThreads) {   // states nobody fills stay empty
+        DraftPartial* d = &s_part[0][0][0] + i;
+        d->mx = -INFINITY;
+        d->sum = 0.f;
+#pragma unroll
+        for (int q = 0; q < kTopSlots; ++q) { d->val[q] = -INFINITY; d->id[q] = INT_MAX; }
     }
     __syncthreads();
 
@@ -194,8 +225,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                 const uint32_t bytes = (uint32_t)rows * (uint32_t)row_bytes;
                 // never hand the copy engine a range outside the weights or the ring
                 const long long first = r0 + (long long)j * G;
-                if (rows < 1 || first < 0 || first + rows > R || (bytes & 15u) != 0 || bytes > (uint32_t)slot_bytes ||
-                    s >= nslots) {
+                if (rows < 1 || first < 0 || first + rows > R || (bytes & 15u) != 0 || bytes > (uint32_t)slot_bytes) {
                     report_error(p.status, CTCSD_ERR_INTERNAL, 12);
                     ok = false;
                     break;
@@ -217,73 +247,158 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
             }
         }
     } else {
-        // ---------------- consumers ----------------
-        RunState st;
-        st.init();
-        int cur_seg = 0;
-        bool ok = true;
-        const int groups = kWarps / G;
-        const int rin = warp % G;                       // this warp's row within a slot
-        for (int j = warp / G; j < nfill; j += groups) {
-            const int s = j % nslots;
-            const uint32_t ph = (uint32_t)(j / nslots) & 1u;
-            if (!tc::mbar_wait(&sh->full[s], ph, abort_flag)) { ok = false; break; }
-            const int i = j * G + rin;                  // row of the CTA's range
-            float acc[MROWS];
-#pragma unroll
-            for (int m = 0; m < MROWS; ++m) acc[m] = 0.f;
-            if (i < ntotal) {
-                const uint4* wrow = reinterpret_cast<const uint4*>(ring + (size_t)s * slot_bytes + (size_t)rin * row_bytes);
-#pragma unroll 4
-                for (int ch = lane; ch < nch; ch += 32) {
-                    const uint4 w = wrow[ch];
-#pragma unroll
-                    for (int m = 0; m < MROWS; ++m) acc[m] = Elem<T>::dot(w, xs[m * nch + ch], acc[m]);
+        // ---------------- consumers (warps 0..7) and epilogue (warps 9..12) ----------------
+        // Every warp visits every fill in order and arrives on the barriers it takes part in, so
+        // no warp is ever more than one phase away from a barrier it waits on (a parity wait
+        // means nothing to a waiter that is further behind).
+        const bool is_epi = warp > kWarps;
+        if (kMma ? true : !is_epi) {
+            RunState st;
+            st.init();
+            int cur_seg = 0;
+            // the (row of the slot, activation row) pair whose state this thread keeps
+            const int epi_idx = (warp - kWarps - 1) * 32 + lane;
+            const int own_r = kMma ? (epi_idx >> 3) : warp;
+            const int own_m = kMma ? (epi_idx & 7) : lane;
+            const bool owner = kMma ? (is_epi && own_m < p.mcount) : (lane < p.mcount);
+            float bias = 0.f;
+            if (owner && p.blank_bias != nullptr) {
+                const int row = p.m0 + own_m;
+                bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
+            }
+            auto push_logit = [&](float z, int i) {          // i: row of the CTA's range
+                const int seg = i >= n_seg0 ? 1 : 0;
+                if (seg != cur_seg) {                         // this thread's rows now belong to the next slot
+                    st.store(&s_part[0][own_r][own_m]);
+                    st.init();
+                    cur_seg = 1;
                 }
-            }
-            // the accumulators depend on every load of the row: the slot can be refilled
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
-            if (i >= ntotal) continue;
-            const int seg = i >= n_seg0 ? 1 : 0;
-            if (seg != cur_seg) {                       // this warp's rows now belong to the next slot
-                if (lane < MROWS) st.store(&s_part[0][warp][lane]);
-                st.init();
-                cur_seg = 1;
-            }
-#pragma unroll
-            for (int m = 0; m < MROWS; ++m) acc[m] = warp_sum(acc[m]);
-            float z = 0.f;
-#pragma unroll
-            for (int m = 0; m < MROWS; ++m) if (lane == m) z = acc[m];
-            if (lane < p.mcount) {
                 const int slot = slot0 + seg;
                 const int v = (int)(r0 + i - (long long)slot * rps);
                 if (v == (int)rps - 1) z += bias;
-                if (p.logits_dbg) p.logits_dbg[((size_t)(p.m0 + lane) * p.slots + slot) * rps + v] = z;
+                if (p.logits_dbg) p.logits_dbg[((size_t)(p.m0 + own_m) * p.slots + slot) * rps + v] = z;
                 st.push(z, v);
+            };
+
+            bool failed = false;
+            for (int j = 0; j < nfill; ++j) {
+                const int rows = (ntotal - j * G < G) ? ntotal - j * G : G;
+                const int d = j % kCDepth;
+                const uint32_t dph = (uint32_t)(j / kCDepth) & 1u;
+                if (kMma && is_epi) {
+                    // ---- epilogue: add the eight partial sums, fold the logit into the state ----
+                    if (!tc::mbar_wait(&sh->cfull[d], dph, abort_flag)) { failed = true; break; }
+                    if (owner && own_r < rows) {
+                        float z = 0.f;
+#pragma unroll
+                        for (int w = 0; w < kWarps; ++w) z += s_cpart[d][w][own_r][own_m];
+                        push_logit(z, j * G + own_r);
+                    }
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&sh->cempty[d]);
+                    continue;
+                }
+                const int s = j % nslots;
+                const uint32_t ph = (uint32_t)(j / nslots) & 1u;
+                if (!tc::mbar_wait(&sh->full[s], ph, abort_flag)) { failed = true; break; }
+                const unsigned char* slot_base = ring + (size_t)s * slot_bytes;
+                if constexpr (kMma) {
+                    const int g = lane >> 2, t = lane & 3;
+                    const uint4* rowA = reinterpret_cast<const uint4*>(slot_base + (size_t)g * row_bytes);
+                    const uint4* rowB = reinterpret_cast<const uint4*>(slot_base + (size_t)(g + 8) * row_bytes);
+                    const bool hasA = g < rows, hasB = g + 8 < rows, hasX = g < MROWS;
+                    const uint4* xrow = xs + (hasX ? g : 0) * x_stride;
+                    // A block of 32 hidden elements = four 16-byte chunks, one per thread of a quad;
+                    // the k index inside a block is permuted the same way for weights and activations.
+                    // Four blocks are in flight at a time, each with its own accumulators, so that
+                    // neither the loads nor the dependent tensor-core instructions serialise.
+                    constexpr int kU = 4;
+                    float cc[kU][4];
+#pragma unroll
+                    for (int u = 0; u < kU; ++u) { cc[u][0] = cc[u][1] = cc[u][2] = cc[u][3] = 0.f; }
+                    for (int kb0 = warp; kb0 * 4 < nch; kb0 += kWarps * kU) {      // the same trip count for all lanes
+                        uint4 P[kU], Q[kU], X[kU];
+#pragma unroll
+                        for (int u = 0; u < kU; ++u) {
+                            const int ch = (kb0 + u * kWarps) * 4 + t;
+                            const bool in = ch < nch;
+                            const uint4 z4 = make_uint4(0, 0, 0, 0);
+                            P[u] = (hasA && in) ? rowA[ch] : z4;
+                            Q[u] = (hasB && in) ? rowB[ch] : z4;
+                            X[u] = (hasX && in) ? xrow[ch] : z4;
+                        }
+#pragma unroll
+                        for (int u = 0; u < kU; ++u) {
+                            mma_16816(cc[u], P[u].x, Q[u].x, P[u].y, Q[u].y, X[u].x, X[u].y);
+                            mma_16816(cc[u], P[u].z, Q[u].z, P[u].w, Q[u].w, X[u].z, X[u].w);
+                        }
+                    }
+                    // the accumulators depend on every load of the slot: it can be refilled
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+                    // c0,c1: weight row g x activation rows 2t,2t+1;  c2,c3: weight row g+8
+                    if (!tc::mbar_wait(&sh->cempty[d], dph ^ 1u, abort_flag)) { failed = true; break; }
+                    float* cp = &s_cpart[d][warp][0][0];
+                    *reinterpret_cast<float2*>(cp + g * 8 + 2 * t) =
+                        make_float2((cc[0][0] + cc[1][0]) + (cc[2][0] + cc[3][0]), (cc[0][1] + cc[1][1]) + (cc[2][1] + cc[3][1]));
+                    *reinterpret_cast<float2*>(cp + (g + 8) * 8 + 2 * t) =
+                        make_float2((cc[0][2] + cc[1][2]) + (cc[2][2] + cc[3][2]), (cc[0][3] + cc[1][3]) + (cc[2][3] + cc[3][3]));
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&sh->cfull[d]);
+                } else {
+                    float zrow[kRowsPerWarp];
+                    int nmine = 0;
+#pragma unroll
+                    for (int q = 0; q < kRowsPerWarp; ++q) {
+                        const int rin = warp + q * kWarps;          // row within the slot
+                        zrow[q] = 0.f;
+                        if (rin < rows) {
+                            const uint4* wrow = reinterpret_cast<const uint4*>(slot_base + (size_t)rin * row_bytes);
+                            float acc[MROWS];
+#pragma unroll
+                            for (int m = 0; m < MROWS; ++m) acc[m] = 0.f;
+#pragma unroll 4
+                            for (int ch = lane; ch < nch; ch += 32) {
+                                const uint4 w = wrow[ch];
+#pragma unroll
+                                for (int m = 0; m < MROWS; ++m) acc[m] = Elem<T>::dot(w, xs[m * x_stride + ch], acc[m]);
+                            }
+#pragma unroll
+                            for (int m = 0; m < MROWS; ++m) {
+                                const float v = warp_sum(acc[m]);
+                                if (lane == m) zrow[q] = v;
+                            }
+                            nmine = q + 1;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+#pragma unroll
+                    for (int q = 0; q < kRowsPerWarp; ++q)
+                        if (q < nmine && owner) push_logit(zrow[q], j * G + warp + q * kWarps);
+                }
             }
-        }
-        if (!ok && lane == 0) {
-            if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 11);
-            *abort_flag = 1;
-        }
-        if (lane < MROWS) {
-            if (cur_seg == 0) {
-                st.store(&s_part[0][warp][lane]);
-                st.init();
+            if (failed && lane == 0) {
+                if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 11);
+                *abort_flag = 1;
             }
-            st.store(&s_part[1][warp][lane]);
+            if (owner) {
+                if (cur_seg == 0) {
+                    st.store(&s_part[0][own_r][own_m]);
+                    st.init();
+                }
+                st.store(&s_part[1][own_r][own_m]);
+            }
         }
     }
     __syncthreads();
 
-    // fold the 8 warps' states per segment: warp m merges activation row m's states, one per lane
+    // fold the CTA's states per segment: warp m merges activation row m's states, one per lane
     for (int seg = 0; seg < 2; ++seg) {
         if (warp < MROWS) {
             RunState ms;
             ms.init();
-            if (lane < kWarps) ms.absorb(s_part[seg][lane][warp]);
+            if (lane < kStateRows) ms.absorb(s_part[seg][lane][warp]);
             warp_combine(ms);
             if (lane == 0) ms.store(p.part + ((size_t)warp * p.grid + blockIdx.x) * 2 + seg);
         }
@@ -341,14 +456,23 @@ template <typename T, int MROWS>
 int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     auto kern = gemv_stream_kernel<T, MROWS>;
     const size_t row_bytes = (size_t)p.H * sizeof(T);
-    const size_t budget = 200 * 1024;                          // dynamic shared memory per CTA
-    const size_t fixed = (size_t)MROWS * row_bytes + sizeof(RingShared);
-    // rows per ring slot: a power of two that divides the 8 consumer warps, about 32 KB per copy
-    int G = 1;
-    while (G < kWarps && (size_t)(2 * G) * row_bytes <= 32 * 1024) G *= 2;
-    while (G > 1 && fixed + 3 * (size_t)G * row_bytes > budget) G /= 2;
+    // dynamic shared memory per CTA: what the device allows minus the kernel's static part
+    cudaFuncAttributes fa;
+    CTCSD_CUDA_CHECK(h, cudaFuncGetAttributes(&fa, kern));
+    int optin = 0;
+    CTCSD_CUDA_CHECK(h, cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
+    if ((size_t)optin < fa.sharedSizeBytes + 32 * 1024) return CTCSD_ERR_UNSUPPORTED;
+    size_t budget = (size_t)optin - fa.sharedSizeBytes - 2048;
+    if (budget > 208 * 1024) budget = 208 * 1024;
+    const size_t fixed = (size_t)MROWS * (row_bytes + 64) + sizeof(RingShared);
+    // rows per ring slot: copies of about 64 KB keep the copy engine busiest (its cost per copy is
+    // large), as long as at least three slots fit
+    int G = (int)((64 * 1024) / row_bytes);
+    if (G < 1) G = 1;
+    if (G > kWarps * kRowsPerWarp) G = kWarps * kRowsPerWarp;
+    while (G > 1 && fixed + 3 * (size_t)G * row_bytes > budget) --G;
     const size_t slot_bytes = (size_t)G * row_bytes;
-    if (fixed + 2 * slot_bytes > budget) return CTCSD_ERR_UNSUPPORTED;
+    if (fixed + slot_bytes > budget) return CTCSD_ERR_UNSUPPORTED;
     long long nslots = (long long)((budget - fixed) / slot_bytes);
     if (nslots > kMaxSlots) nslots = kMaxSlots;
     const size_t smem = fixed + (size_t)nslots * slot_bytes;
@@ -363,15 +487,30 @@ int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     return CTCSD_OK;
 }
 
-template <typename T>
-int launch_typed(Handle* h, cudaStream_t stream, int M, GemvParams& p) {
+// bfloat16 rows go through the tensor-core consumer, up to 8 activation rows per pass over the
+// weights; float32 rows through the fused-multiply-add consumer, up to 4 per pass.
+int launch_typed_bf16(Handle* h, cudaStream_t stream, int M, GemvParams& p) {
+    for (int m0 = 0; m0 < M; m0 += 8) {
+        p.m0 = m0;
+        p.mcount = (M - m0 < 8) ? (M - m0) : 8;
+        int rc;
+        if (p.mcount == 1) rc = launch_one<__nv_bfloat16, 1>(h, stream, p);
+        else if (p.mcount == 2) rc = launch_one<__nv_bfloat16, 2>(h, stream, p);
+        else if (p.mcount <= 4) rc = launch_one<__nv_bfloat16, 4>(h, stream, p);
+        else rc = launch_one<__nv_bfloat16, 8>(h, stream, p);
+        if (rc != CTCSD_OK) return rc;
+    }
+    return CTCSD_OK;
+}
+
+int launch_typed_f32(Handle* h, cudaStream_t stream, int M, GemvParams& p) {
     for (int m0 = 0; m0 < M; m0 += 4) {
         p.m0 = m0;
         p.mcount = (M - m0 < 4) ? (M - m0) : 4;
         int rc;
-        if (p.mcount == 1) rc = launch_one<T, 1>(h, stream, p);
-        else if (p.mcount == 2) rc = launch_one<T, 2>(h, stream, p);
-        else rc = launch_one<T, 4>(h, stream, p);
+        if (p.mcount == 1) rc = launch_one<float, 1>(h, stream, p);
+        else if (p.mcount == 2) rc = launch_one<float, 2>(h, stream, p);
+        else rc = launch_one<float, 4>(h, stream, p);
         if (rc != CTCSD_OK) return rc;
     }
     return CTCSD_OK;
@@ -384,8 +523,8 @@ int launch_gemv_stream(Handle* h, cudaStream_t stream, int dtype, int M, GemvPar
     p.part_slot = reinterpret_cast<int*>(h->ws + h->lay.part_slot_off);
     p.counter = counter_ptr(h);
     p.status = status_ptr(h);
-    if (dtype == CTCSD_DTYPE_BF16) return launch_typed<__nv_bfloat16>(h, stream, M, p);
-    return launch_typed<float>(h, stream, M, p);
+    if (dtype == CTCSD_DTYPE_BF16) return launch_typed_bf16(h, stream, M, p);
+    return launch_typed_f32(h, stream, M, p);
 }
 
 }  // namespace ctcsd

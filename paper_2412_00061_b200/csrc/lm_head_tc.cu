@@ -94,6 +94,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc::prefetch_tensormap(&tmW);
             const uint64_t pol_w = tc::policy_evict_first();
             const uint64_t pol_a = tc::policy_evict_last();
+            const int k_start = (int)(((long long)blockIdx.x * p.num_k) / gridDim.x);
             int it = 0;
             bool ok = true;
             for (int u = u0; u < u1 && ok; ++u) {
@@ -104,8 +105,12 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                     unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
                     tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)stage_bytes);
-                    tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kb * kBlockK, mt * kTileM, pol_a);
-                    tc::tma_load_2d(a_dst + kABytes, &tmW, &sh->full[s], kb * kBlockK, nt * p.Nt, pol_w);
+                    // every CTA walks the K axis from its own starting block (and wraps), so that at
+                    // any moment the CTAs ask L2 for different parts of the shared activations
+                    int kq = kb + k_start;
+                    if (kq >= p.num_k) kq -= p.num_k;
+                    tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kq * kBlockK, mt * kTileM, pol_a);
+                    tc::tma_load_2d(a_dst + kABytes, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
                 }
             }
             if (!ok) {
