@@ -12,6 +12,7 @@
 #include "tree_attention.cuh"
 
 #include <math.h>
+#include <string.h>
 
 namespace ctcsd {
 namespace {
@@ -47,12 +48,47 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// ---- thread-block cluster helpers (distributed shared memory) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in the CTA with rank `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_cluster_v2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
 // byte offset of 16-byte chunk `chunk` of row `row` in a tile with D bf16 per row, swizzled
 template <int D> __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
     return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
 }
 
-template <int D>
+// CLUSTER = false: every CTA writes its partial (max, sum, unnormalised O) rows to `part` and a
+// second kernel merges the KV splits.  CLUSTER = true: the `splits` CTAs of a query tile form a
+// thread-block cluster, leave their partial rows in their own shared memory, and every CTA
+// merges a share of the rows by reading its peers' shared memory; `part` is not used.
+template <int D, bool CLUSTER>
 __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams p, float* part, int splits) {
     constexpr int CH = D / 8;                  // 16-byte chunks per row
     constexpr int KS = D / 16;                 // k-steps of the QK^T product
@@ -76,9 +112,8 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
     }
     const int Ltot = L + n;
     const int nblk = (Ltot + kKeys - 1) / kKeys;
-    const int bps = (nblk + splits - 1) / splits;
-    const int blk0 = split * bps;
-    const int blk1 = (blk0 + bps < nblk) ? blk0 + bps : nblk;
+    const int blk0 = (int)((long long)nblk * split / splits);           // key blocks spread evenly over the splits
+    const int blk1 = (int)((long long)nblk * (split + 1) / splits);
 
     const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q);
     const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(p.K) + ((size_t)b * p.Hkv + g) * (size_t)p.Lcap * D;
@@ -226,24 +261,88 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
     }
     cp_async_wait<0>();
 
-    // per-row partials: [b][hq][node][split][D+2] = (max in log2 units, sum, unnormalised O)
     sumA += __shfl_xor_sync(0xffffffffu, sumA, 1);
     sumA += __shfl_xor_sync(0xffffffffu, sumA, 2);
     sumB += __shfl_xor_sync(0xffffffffu, sumB, 1);
     sumB += __shfl_xor_sync(0xffffffffu, sumB, 2);
+    if constexpr (!CLUSTER) {
+        // per-row partials: [b][hq][node][split][D+2] = (max in log2 units, sum, unnormalised O)
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        const int r = half ? rB : rA;
-        const int i = half ? iB : iA;
-        if (i >= n) continue;                                   // dead rows are zeroed by the merge kernel
-        const int hq = g * grp + (r - i * grp);
-        float* dst = part + ((((size_t)b * p.Hq + hq) * p.max_nodes + i) * splits + split) * (D + 2);
-        if (tig == 0) { dst[0] = half ? mxB : mxA; dst[1] = half ? sumB : sumA; }
+        for (int half = 0; half < 2; ++half) {
+            const int r = half ? rB : rA;
+            const int i = half ? iB : iA;
+            if (i >= n) continue;                                   // dead rows are zeroed by the merge kernel
+            const int hq = g * grp + (r - i * grp);
+            float* dst = part + ((((size_t)b * p.Hq + hq) * p.max_nodes + i) * splits + split) * (D + 2);
+            if (tig == 0) { dst[0] = half ? mxB : mxA; dst[1] = half ? sumB : sumA; }
 #pragma unroll
-        for (int t = 0; t < DT; ++t) {
-            float2 v = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
-            *reinterpret_cast<float2*>(dst + 2 + 8 * t + 2 * tig) = v;
+            for (int t = 0; t < DT; ++t) {
+                float2 v = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
+                *reinterpret_cast<float2*>(dst + 2 + 8 * t + 2 * tig) = v;
+            }
         }
+    } else {
+        // partial rows go to this CTA's shared memory (the K/V tiles are no longer needed):
+        // [row][D+4] floats = unnormalised O, then max (log2 units) and sum
+        constexpr int RS = D + 4;
+        constexpr int PER = D / 32;
+        __syncthreads();
+        float* rowbuf = reinterpret_cast<float*>(Ks);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            float* dst = rowbuf + (warp * 16 + gid + 8 * half) * RS;
+            if (tig == 0) { dst[D] = half ? mxB : mxA; dst[D + 1] = half ? sumB : sumA; }
+#pragma unroll
+            for (int t = 0; t < DT; ++t) {
+                float2 v = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
+                *reinterpret_cast<float2*>(dst + 8 * t + 2 * tig) = v;
+            }
+        }
+        cluster_sync_all();
+        // this CTA (cluster rank = split) merges rows split, split + splits, ...; one warp per row
+        const uint32_t base = smem_u32(rowbuf);
+        for (int rl = split + splits * warp; rl < kRows; rl += splits * (kThreads / 32)) {
+            const int r = qtile * kRows + rl;
+            const int i = r / grp;
+            if (i >= p.max_nodes) continue;                         // padding rows of the last query tile
+            const int hq = g * grp + (r - i * grp);
+            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.O) + (((size_t)b * p.max_nodes + i) * p.Hq + hq) * D;
+            float acc[PER], tot = 0.f;
+#pragma unroll
+            for (int d = 0; d < PER; ++d) acc[d] = 0.f;
+            if (i < n) {
+                float gm = -INFINITY;
+                for (int c = 0; c < splits; ++c)
+                    gm = fmaxf(gm, ld_cluster_f32(map_to_cta(base + (uint32_t)(rl * RS + D) * 4u, (uint32_t)c)));
+                if (gm != -INFINITY) {
+                    for (int c = 0; c < splits; ++c) {
+                        const uint32_t rowaddr = map_to_cta(base + (uint32_t)(rl * RS) * 4u, (uint32_t)c);
+                        const float m = ld_cluster_f32(rowaddr + D * 4u);
+                        if (m == -INFINITY) continue;
+                        const float w = exp2f(m - gm);
+                        tot += w * ld_cluster_f32(rowaddr + (D + 1) * 4u);
+                        if constexpr (PER == 4) {
+                            const float4 v = ld_cluster_v4(rowaddr + (uint32_t)lane * 16u);
+                            acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
+                        } else {
+                            const float2 v = ld_cluster_v2(rowaddr + (uint32_t)lane * 8u);
+                            acc[0] += w * v.x; acc[1] += w * v.y;
+                        }
+                    }
+                }
+            }
+            const float inv = tot > 0.f ? 1.f / tot : 0.f;
+            if constexpr (PER == 4) {
+                uint2 pk;
+                pk.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+                pk.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+                *reinterpret_cast<uint2*>(out + 4 * lane) = pk;
+            } else {
+                *reinterpret_cast<uint32_t*>(out + 2 * lane) = pack_bf16(acc[0] * inv, acc[1] * inv);
+            }
+        }
+        // nobody may leave while a peer can still read its shared memory
+        cluster_sync_all();
     }
 }
 
@@ -285,22 +384,35 @@ __global__ void __launch_bounds__(128) tree_attention_merge_kernel(AttnParams p,
     for (int d = 0; d < PER; ++d) out[lane + 32 * d] = __float2bfloat16_rn(acc[d] * inv);
 }
 
+// The KV splits of a query tile run as one thread-block cluster and merge through distributed
+// shared memory: one launch, no partial results in global memory.
 template <int D>
 int launch_d(Handle* h, cudaStream_t s, const AttnParams& p) {
     const int grp = p.Hq / p.Hkv;
     const int qtiles = (p.max_nodes * grp + kRows - 1) / kRows;
-    const int splits = h->lay.kv_splits;
-    float* part = reinterpret_cast<float*>(h->ws + h->lay.attn_part_off);
+    // enough CTAs for two per SM, as a cluster size that is portable: 1, 2, 4 or 8
+    const long long units = (long long)p.B * p.Hkv * qtiles;
+    int splits = 1;
+    while (splits < 8 && units * splits < 2ll * h->num_sms) splits *= 2;
     const size_t smem = (size_t)kRows * D * 2 + 4 * (size_t)kKeys * D * 2;
-    auto kern = tree_attention_mma_kernel<D>;
-    if (smem > 48 * 1024)
-        CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    dim3 grid(qtiles * splits, p.Hkv, p.B);
-    kern<<<grid, kThreads, smem, s>>>(p, part, splits);
-    CTCSD_LAUNCH_CHECK(h);
-    const long long warps = (long long)p.B * p.max_nodes * p.Hq;
-    tree_attention_merge_kernel<D><<<(unsigned)((warps + 3) / 4), 128, 0, s>>>(p, part, splits);
-    CTCSD_LAUNCH_CHECK(h);
+    auto kern = tree_attention_mma_kernel<D, true>;
+    CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(qtiles * splits, p.Hkv, p.B);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    float* no_part = nullptr;
+    CTCSD_CUDA_CHECK(h, cudaLaunchKernelEx(&cfg, kern, p, no_part, splits));
+    h->launches++;
     return CTCSD_OK;
 }
 
@@ -311,7 +423,7 @@ cudaError_t launch_d_scratch(cudaStream_t s, const AttnParams& p, float* part, i
     const int grp = p.Hq / p.Hkv;
     const int qtiles = (p.max_nodes * grp + kRows - 1) / kRows;
     const size_t smem = (size_t)kRows * D * 2 + 4 * (size_t)kKeys * D * 2;
-    auto kern = tree_attention_mma_kernel<D>;
+    auto kern = tree_attention_mma_kernel<D, false>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
