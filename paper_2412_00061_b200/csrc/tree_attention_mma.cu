@@ -20,6 +20,7 @@ namespace {
 constexpr int kRows = 64;          // query rows per CTA
 constexpr int kKeys = 64;          // keys per tile
 constexpr int kThreads = 128;
+constexpr int kStages = 4;         // K/V tile buffers: three tiles are in flight while one is used
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -87,21 +88,28 @@ template <int D> __device__ __forceinline__ uint32_t tile_off(int row, int chunk
 // CLUSTER = false: every CTA writes its partial (max, sum, unnormalised O) rows to `part` and a
 // second kernel merges the KV splits.  CLUSTER = true: the `splits` CTAs of a query tile form a
 // thread-block cluster, leave their partial rows in their own shared memory, and every CTA
-// merges a share of the rows by reading its peers' shared memory; `part` is not used.
+// merges a share of the rows by reading its peers' shared memory; `part` is not used.  In this
+// mode the CTA has two groups of four warps: each group takes half of the keys of every tile
+// and keeps its own running softmax state, which shortens the dependent instruction chain per
+// tile; the two states are simply two more partials for the merge.
 template <int D, bool CLUSTER>
-__global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams p, float* part, int splits) {
+__global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_mma_kernel(AttnParams p, float* part, int splits) {
+    constexpr int KG = CLUSTER ? 2 : 1;        // key groups (warps 4*kg .. 4*kg+3)
+    constexpr int NT = kThreads * KG;          // threads per CTA
+    constexpr int KPW = kKeys / KG;            // keys of a tile handled by one warp
     constexpr int CH = D / 8;                  // 16-byte chunks per row
     constexpr int KS = D / 16;                 // k-steps of the QK^T product
     constexpr int DT = D / 8;                  // 8-wide output tiles of O
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* Qs = smem;                                  // [64][D]
-    unsigned char* Ks = Qs + kRows * D * 2;                    // [2][64][D]
-    unsigned char* Vs = Ks + 2 * kKeys * D * 2;                // [2][64][D]
+    unsigned char* Ks = Qs + kRows * D * 2;                    // [kStages][64][D]
+    unsigned char* Vs = Ks + kStages * kKeys * D * 2;          // [kStages][64][D]
 
     const int grp = p.Hq / p.Hkv;
     const int qtile = blockIdx.x / splits, split = blockIdx.x - qtile * splits;
     const int g = blockIdx.y, b = blockIdx.z;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, wfull = tid >> 5, lane = tid & 31;
+    const int warp = wfull & 3, kg = wfull >> 2;               // row group, key group
     const int gid = lane >> 2, tig = lane & 3;
 
     int n = p.n_nodes[b];
@@ -133,7 +141,7 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
         const int key0 = blk * kKeys;
         unsigned char* kd = Ks + buf * (kKeys * D * 2);
         unsigned char* vd = Vs + buf * (kKeys * D * 2);
-        for (int c = tid; c < kKeys * CH; c += kThreads) {
+        for (int c = tid; c < kKeys * CH; c += NT) {
             const int row = c / CH, ch = c - row * CH;
             const int key = key0 + row;
             const bool ok = key < Ltot;
@@ -144,7 +152,7 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
     };
 
     // Q tile (rows past the live rows are zero-filled) and the first KV tile
-    for (int c = tid; c < kRows * CH; c += kThreads) {
+    for (int c = tid; c < kRows * CH; c += NT) {
         const int row = c / CH, ch = c - row * CH;
         const int r = qtile * kRows + row;
         const int i = r / grp, hq = g * grp + (r - i * grp);
@@ -152,8 +160,13 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
         const size_t src = (((size_t)b * p.max_nodes + (ok ? i : 0)) * p.Hq + hq) * D + ch * 8;
         cp_async16(Qs + tile_off<D>(row, ch), Qg + src, ok);
     }
-    if (blk0 < blk1) load_kv(blk0, 0);
-    cp_async_commit();
+    // one commit group per tile (possibly empty), so that "all but the newest kStages-1 groups
+    // are complete" always means "the tile about to be used has landed"
+#pragma unroll
+    for (int pre = 0; pre < kStages - 1; ++pre) {
+        if (blk0 + pre < blk1) load_kv(blk0 + pre, pre);
+        cp_async_commit();
+    }
 
     float o[DT][4];
 #pragma unroll
@@ -163,10 +176,10 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
     uint32_t qf[KS][4];
 
     for (int blk = blk0; blk < blk1; ++blk) {
-        const int buf = (blk - blk0) & 1;
-        if (blk + 1 < blk1) load_kv(blk + 1, buf ^ 1);
+        const int buf = (blk - blk0) % kStages;
+        if (blk + kStages - 1 < blk1) load_kv(blk + kStages - 1, (blk - blk0 + kStages - 1) % kStages);
         cp_async_commit();
-        cp_async_wait<1>();
+        cp_async_wait<kStages - 1>();
         __syncthreads();
         if (blk == blk0) {
 #pragma unroll
@@ -178,36 +191,51 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
         const unsigned char* kb = Ks + buf * (kKeys * D * 2);
         const unsigned char* vb = Vs + buf * (kKeys * D * 2);
 
-        // S = Q K^T for 16 rows x 64 keys
-        float s[kKeys / 8][4];
+        // S = Q K^T for 16 rows x this warp's KPW keys of the tile.  The k-steps feed NCH separate
+        // accumulator sets that are added afterwards: a tensor-core instruction has a long
+        // latency, and one accumulator per tile would chain all D/16 of them.
+        constexpr int NCH = CLUSTER ? 4 : 2;
+        float sp[NCH][KPW / 8][4];
 #pragma unroll
-        for (int t = 0; t < kKeys / 8; ++t) { s[t][0] = s[t][1] = s[t][2] = s[t][3] = 0.f; }
+        for (int c = 0; c < NCH; ++c)
+#pragma unroll
+            for (int t = 0; t < KPW / 8; ++t) { sp[c][t][0] = sp[c][t][1] = sp[c][t][2] = sp[c][t][3] = 0.f; }
 #pragma unroll
         for (int kk = 0; kk < KS; ++kk) {
 #pragma unroll
-            for (int pr = 0; pr < kKeys / 16; ++pr) {
+            for (int pr = 0; pr < KPW / 16; ++pr) {
                 uint32_t kf[4];
                 const int mi = lane >> 3, rin = lane & 7;
-                const int key = 16 * pr + (mi >> 1) * 8 + rin, ch = 2 * kk + (mi & 1);
+                const int key = kg * KPW + 16 * pr + (mi >> 1) * 8 + rin, ch = 2 * kk + (mi & 1);
                 ldmatrix_x4(kf, smem_u32(kb + tile_off<D>(key, ch)));
-                mma_bf16(s[2 * pr], qf[kk], kf[0], kf[1]);
-                mma_bf16(s[2 * pr + 1], qf[kk], kf[2], kf[3]);
+                mma_bf16(sp[kk % NCH][2 * pr], qf[kk], kf[0], kf[1]);
+                mma_bf16(sp[kk % NCH][2 * pr + 1], qf[kk], kf[2], kf[3]);
             }
         }
+        float s[KPW / 8][4];
+#pragma unroll
+        for (int t = 0; t < KPW / 8; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float v = sp[0][t][e];
+#pragma unroll
+                for (int c = 1; c < NCH; ++c) v += sp[c][t][e];
+                s[t][e] = v;
+            }
 
         // scale, mask, online softmax
         const int key0 = blk * kKeys;
         const bool need_mask = key0 + kKeys > L;
         float bmA = -INFINITY, bmB = -INFINITY;
 #pragma unroll
-        for (int t = 0; t < kKeys / 8; ++t) {
+        for (int t = 0; t < KPW / 8; ++t) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float v = s[t][e] * sl2;
                 const bool second = e >= 2;                     // c2,c3 belong to row gid+8
                 bool vis = second ? liveB : liveA;
                 if (need_mask) {
-                    const int key = key0 + 8 * t + 2 * tig + (e & 1);
+                    const int key = key0 + kg * KPW + 8 * t + 2 * tig + (e & 1);
                     if (key >= L) {
                         const int tn = key - L;
                         const unsigned long long w0 = second ? mB0 : mA0, w1 = second ? mB1 : mA1;
@@ -229,9 +257,9 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
         const float corrA = exp2f(mxA - refA), corrB = exp2f(mxB - refB);   // exp2(-inf) = 0
         mxA = nmA; mxB = nmB;
         float psA = 0.f, psB = 0.f;
-        uint32_t pf[kKeys / 16][4];
+        uint32_t pf[KPW / 16][4];
 #pragma unroll
-        for (int t = 0; t < kKeys / 8; ++t) {
+        for (int t = 0; t < KPW / 8; ++t) {
             const float p0 = exp2f(s[t][0] - refA), p1 = exp2f(s[t][1] - refA);
             const float p2 = exp2f(s[t][2] - refB), p3 = exp2f(s[t][3] - refB);
             psA += p0 + p1;
@@ -246,12 +274,12 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
 
         // O += P V
 #pragma unroll
-        for (int kk = 0; kk < kKeys / 16; ++kk) {
+        for (int kk = 0; kk < KPW / 16; ++kk) {
 #pragma unroll
             for (int pr = 0; pr < DT / 2; ++pr) {
                 uint32_t vf[4];
                 const int mi = lane >> 3, rin = lane & 7;
-                const int key = 16 * kk + (mi & 1) * 8 + rin, ch = 2 * pr + (mi >> 1);
+                const int key = kg * KPW + 16 * kk + (mi & 1) * 8 + rin, ch = 2 * pr + (mi >> 1);
                 ldmatrix_x4_trans(vf, smem_u32(vb + tile_off<D>(key, ch)));
                 mma_bf16(o[2 * pr], pf[kk], vf[0], vf[1]);
                 mma_bf16(o[2 * pr + 1], pf[kk], vf[2], vf[3]);
@@ -283,14 +311,14 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
         }
     } else {
         // partial rows go to this CTA's shared memory (the K/V tiles are no longer needed):
-        // [row][D+4] floats = unnormalised O, then max (log2 units) and sum
+        // [key group][row][D+4] floats = unnormalised O, then max (log2 units) and sum
         constexpr int RS = D + 4;
         constexpr int PER = D / 32;
         __syncthreads();
         float* rowbuf = reinterpret_cast<float*>(Ks);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-            float* dst = rowbuf + (warp * 16 + gid + 8 * half) * RS;
+            float* dst = rowbuf + (kg * kRows + warp * 16 + gid + 8 * half) * RS;
             if (tig == 0) { dst[D] = half ? mxB : mxA; dst[D + 1] = half ? sumB : sumA; }
 #pragma unroll
             for (int t = 0; t < DT; ++t) {
@@ -301,7 +329,7 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
         cluster_sync_all();
         // this CTA (cluster rank = split) merges rows split, split + splits, ...; one warp per row
         const uint32_t base = smem_u32(rowbuf);
-        for (int rl = split + splits * warp; rl < kRows; rl += splits * (kThreads / 32)) {
+        for (int rl = split + splits * wfull; rl < kRows; rl += splits * (NT / 32)) {
             const int r = qtile * kRows + rl;
             const int i = r / grp;
             if (i >= p.max_nodes) continue;                         // padding rows of the last query tile
@@ -310,17 +338,26 @@ __global__ void __launch_bounds__(kThreads) tree_attention_mma_kernel(AttnParams
             float acc[PER], tot = 0.f;
 #pragma unroll
             for (int d = 0; d < PER; ++d) acc[d] = 0.f;
-            if (i < n) {
-                float gm = -INFINITY;
-                for (int c = 0; c < splits; ++c)
-                    gm = fmaxf(gm, ld_cluster_f32(map_to_cta(base + (uint32_t)(rl * RS + D) * 4u, (uint32_t)c)));
-                if (gm != -INFINITY) {
-                    for (int c = 0; c < splits; ++c) {
-                        const uint32_t rowaddr = map_to_cta(base + (uint32_t)(rl * RS) * 4u, (uint32_t)c);
-                        const float m = ld_cluster_f32(rowaddr + D * 4u);
-                        if (m == -INFINITY) continue;
-                        const float w = exp2f(m - gm);
-                        tot += w * ld_cluster_f32(rowaddr + (D + 1) * 4u);
+            if (i < n) {                                            // uniform over the warp
+                // lane c fetches partial c's (max, sum): partial c = key group c % KG of split c / KG;
+                // the row loads below do not depend on one another
+                float m_l = -INFINITY, l_l = 0.f;
+                if (lane < splits * KG) {
+                    const uint32_t a = map_to_cta(base + (uint32_t)(((lane % KG) * kRows + rl) * RS + D) * 4u,
+                                                  (uint32_t)(lane / KG));
+                    const float2 ml = ld_cluster_v2(a);
+                    m_l = ml.x;
+                    l_l = ml.y;
+                }
+                const float gm = warp_max(m_l);
+                const float w_l = (m_l == -INFINITY) ? 0.f : exp2f(m_l - gm);
+                tot = warp_sum(w_l * l_l);
+#pragma unroll
+                for (int c = 0; c < 8 * KG; ++c) {
+                    if (c < splits * KG) {
+                        const float w = __shfl_sync(0xffffffffu, w_l, c);
+                        const uint32_t rowaddr = map_to_cta(base + (uint32_t)(((c % KG) * kRows + rl) * RS) * 4u,
+                                                            (uint32_t)(c / KG));
                         if constexpr (PER == 4) {
                             const float4 v = ld_cluster_v4(rowaddr + (uint32_t)lane * 16u);
                             acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
@@ -390,17 +427,18 @@ template <int D>
 int launch_d(Handle* h, cudaStream_t s, const AttnParams& p) {
     const int grp = p.Hq / p.Hkv;
     const int qtiles = (p.max_nodes * grp + kRows - 1) / kRows;
-    // enough CTAs for two per SM, as a cluster size that is portable: 1, 2, 4 or 8
+    // as many KV splits as still run in one wave (one CTA per SM), as a cluster size that is
+    // portable: 1, 2, 4 or 8
     const long long units = (long long)p.B * p.Hkv * qtiles;
     int splits = 1;
-    while (splits < 8 && units * splits < 2ll * h->num_sms) splits *= 2;
-    const size_t smem = (size_t)kRows * D * 2 + 4 * (size_t)kKeys * D * 2;
+    while (splits < 8 && units * splits * 2 <= (long long)h->num_sms) splits *= 2;
+    const size_t smem = (size_t)kRows * D * 2 + 2 * kStages * (size_t)kKeys * D * 2;
     auto kern = tree_attention_mma_kernel<D, true>;
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(qtiles * splits, p.Hkv, p.B);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(kThreads * 2, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -422,7 +460,7 @@ template <int D>
 cudaError_t launch_d_scratch(cudaStream_t s, const AttnParams& p, float* part, int splits) {
     const int grp = p.Hq / p.Hkv;
     const int qtiles = (p.max_nodes * grp + kRows - 1) / kRows;
-    const size_t smem = (size_t)kRows * D * 2 + 4 * (size_t)kKeys * D * 2;
+    const size_t smem = (size_t)kRows * D * 2 + 2 * kStages * (size_t)kKeys * D * 2;
     auto kern = tree_attention_mma_kernel<D, false>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
