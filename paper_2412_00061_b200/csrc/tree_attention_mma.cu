@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
     const int rA = row_base + gid, rB = rA + 8;
     const int iA = rA / grp, iB = rB / grp;                     // tree node of each row
     const bool liveA = iA < n, liveB = iB < n;
+    const bool warp_live = row_base / grp < n;                  // rows ascend: if the first is dead, all 16 are
     const int W = (p.max_nodes + 63) / 64;
     unsigned long long mA0 = 0, mA1 = 0, mB0 = 0, mB1 = 0;
     if (liveA) { const unsigned long long* m = p.mask + ((size_t)b * p.max_nodes + iA) * W; mA0 = m[0]; if (W > 1) mA1 = m[1]; }
@@ -190,6 +191,7 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
         }
         const unsigned char* kb = Ks + buf * (kKeys * D * 2);
         const unsigned char* vb = Vs + buf * (kKeys * D * 2);
+        if (warp_live) {                                        // warps whose 16 rows are all beyond the tree skip the math
 
         // S = Q K^T for 16 rows x this warp's KPW keys of the tile.  The k-steps feed NCH separate
         // accumulator sets that are added afterwards: a tensor-core instruction has a long
@@ -285,6 +287,7 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
                 mma_bf16(o[2 * pr + 1], pf[kk], vf[2], vf[3]);
             }
         }
+        }
         __syncthreads();                                        // the other buffer may be overwritten next
     }
     cp_async_wait<0>();
@@ -311,19 +314,43 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
         }
     } else {
         // partial rows go to this CTA's shared memory (the K/V tiles are no longer needed):
-        // [key group][row][D+4] floats = unnormalised O, then max (log2 units) and sum
+        // [row][D+4] floats = unnormalised O, then max (log2 units) and sum.  Key group 1 writes
+        // first; key group 0 folds those values into its own registers and writes the result.
         constexpr int RS = D + 4;
         constexpr int PER = D / 32;
         __syncthreads();
         float* rowbuf = reinterpret_cast<float*>(Ks);
+        if (kg == 1) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            float* dst = rowbuf + (kg * kRows + warp * 16 + gid + 8 * half) * RS;
-            if (tig == 0) { dst[D] = half ? mxB : mxA; dst[D + 1] = half ? sumB : sumA; }
+            for (int half = 0; half < 2; ++half) {
+                float* dst = rowbuf + (warp * 16 + gid + 8 * half) * RS;
+                if (tig == 0) { dst[D] = half ? mxB : mxA; dst[D + 1] = half ? sumB : sumA; }
 #pragma unroll
-            for (int t = 0; t < DT; ++t) {
-                float2 v = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
-                *reinterpret_cast<float2*>(dst + 8 * t + 2 * tig) = v;
+                for (int t = 0; t < DT; ++t) {
+                    float2 v = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
+                    *reinterpret_cast<float2*>(dst + 8 * t + 2 * tig) = v;
+                }
+            }
+        }
+        __syncthreads();
+        if (kg == 0) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float* dst = rowbuf + (warp * 16 + gid + 8 * half) * RS;
+                const float m0 = half ? mxB : mxA, l0 = half ? sumB : sumA;
+                const float m1 = dst[D], l1 = dst[D + 1];
+                const float gm = fmaxf(m0, m1);
+                const float w0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - gm);
+                const float w1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - gm);
+                __syncwarp();                                       // every lane of the quad has read max and sum
+                if (tig == 0) { dst[D] = gm; dst[D + 1] = w0 * l0 + w1 * l1; }
+#pragma unroll
+                for (int t = 0; t < DT; ++t) {
+                    float2* q = reinterpret_cast<float2*>(dst + 8 * t + 2 * tig);
+                    const float2 v1 = *q;
+                    const float2 v0 = half ? make_float2(o[t][2], o[t][3]) : make_float2(o[t][0], o[t][1]);
+                    *q = make_float2(w0 * v0.x + w1 * v1.x, w0 * v0.y + w1 * v1.y);
+                }
             }
         }
         cluster_sync_all();
@@ -339,12 +366,10 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
 #pragma unroll
             for (int d = 0; d < PER; ++d) acc[d] = 0.f;
             if (i < n) {                                            // uniform over the warp
-                // lane c fetches partial c's (max, sum): partial c = key group c % KG of split c / KG;
-                // the row loads below do not depend on one another
+                // lane c fetches split c's (max, sum); the row loads below do not depend on one another
                 float m_l = -INFINITY, l_l = 0.f;
-                if (lane < splits * KG) {
-                    const uint32_t a = map_to_cta(base + (uint32_t)(((lane % KG) * kRows + rl) * RS + D) * 4u,
-                                                  (uint32_t)(lane / KG));
+                if (lane < splits) {
+                    const uint32_t a = map_to_cta(base + (uint32_t)(rl * RS + D) * 4u, (uint32_t)lane);
                     const float2 ml = ld_cluster_v2(a);
                     m_l = ml.x;
                     l_l = ml.y;
@@ -353,11 +378,10 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
                 const float w_l = (m_l == -INFINITY) ? 0.f : exp2f(m_l - gm);
                 tot = warp_sum(w_l * l_l);
 #pragma unroll
-                for (int c = 0; c < 8 * KG; ++c) {
-                    if (c < splits * KG) {
+                for (int c = 0; c < 8; ++c) {
+                    if (c < splits) {
                         const float w = __shfl_sync(0xffffffffu, w_l, c);
-                        const uint32_t rowaddr = map_to_cta(base + (uint32_t)(((c % KG) * kRows + rl) * RS) * 4u,
-                                                            (uint32_t)(c / KG));
+                        const uint32_t rowaddr = map_to_cta(base + (uint32_t)(rl * RS) * 4u, (uint32_t)c);
                         if constexpr (PER == 4) {
                             const float4 v = ld_cluster_v4(rowaddr + (uint32_t)lane * 16u);
                             acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
