@@ -200,7 +200,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2412_00061_b200 import binding, build, synth
+    from paper_2412_00061_b200 import binding, build, replicas, synth
     from paper_2412_00061_b200.step import DraftVerifyStep, to_device
 
     rank = int(os.environ.get("RANK", "0"))
@@ -216,7 +216,7 @@ def run_ours(args):
     binding.load_library()
 
     cfg = synth.CONFIGS[args.config]
-    seed = rank                                    # every rank drafts for its own sequences
+    seed = replicas.rank_seed(0, rank)             # every rank drafts for its own sequences
     inp = host_inputs(cfg, seed)
     step = DraftVerifyStep(cfg, device=str(dev))
     i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
@@ -303,13 +303,8 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     e2e_ms = e_beg.elapsed_time(e_end)
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms, draft_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms, draft_ms = [float(v) for v in t.tolist()]
-        tl = torch.tensor([launches], device=dev, dtype=torch.int64)
-        dist.all_reduce(tl)
-        launches = int(tl.item())
+    ms, e2e_ms, draft_ms = replicas.max_over_ranks([ms, e2e_ms, draft_ms])
+    launches = replicas.sum_over_ranks(launches)
 
     if rank == 0:
         peak, peak_kind = load_peaks()
