@@ -75,6 +75,16 @@ def test_c2_full_size_sampled():
     assert 2 <= r["n_nodes"][0] <= 64
 
 
+@pytest.mark.parametrize("name", ["c3", "c4", "c5"])
+def test_batched_workloads_full_size_sampled(name):
+    """The batched workloads at full size (prefix beam, ragged KV lengths, 128-node trees, GQA):
+    all integer stages are compared in full; the definition-mode oracle checks one draft row,
+    sampled LM-head rows and sampled attention (sequence, head) pairs."""
+    cfg = C[name]
+    r = _run(cfg, seed=0, attention_rows=3, lm_rows=6, draft_rows=[cfg.B - 1])
+    assert all(2 <= n <= cfg.max_nodes for n in r["n_nodes"])
+
+
 def test_invalid_arguments_are_rejected_on_the_host():
     import ctypes
     from paper_2412_00061_b200 import binding
