@@ -37,6 +37,8 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane, int& total) {
 __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     const int b = blockIdx.x, lane = threadIdx.x;
     const int T = p.T, N = p.topN, n_max = p.max_nodes;
+    pdl_wait();                      // the candidates come from the preceding kernel
+    pdl_trigger();
     int nc = p.n_cand[b];
     nc = nc < 0 ? 0 : (nc > N ? N : nc);
     const int L = p.kv_len[b];
@@ -175,7 +177,7 @@ extern "C" int ctcsd_build_tree(ctcsd_handle* hh, void* stream, const int* base_
     p.T = c.T; p.topN = c.topN; p.max_nodes = c.max_nodes;
     p.node_tok = out_node_tok; p.parent = out_parent; p.depth = out_depth; p.pos = out_pos;
     p.mask = out_mask; p.retrieve = out_retrieve; p.n_nodes = out_n_nodes;
-    build_tree_kernel<<<c.B, 32, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    CTCSD_CUDA_CHECK(h, launch_pdl(build_tree_kernel, dim3(c.B), dim3(32), 0, static_cast<cudaStream_t>(stream), 1, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

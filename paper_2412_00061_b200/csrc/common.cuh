@@ -73,6 +73,35 @@ int validate_config(const ctcsd_config& cfg);
         CTCSD_CUDA_CHECK(h, cudaGetLastError());                    \
     } while (0)
 
+#ifdef __CUDACC__
+// Launches `kernel` with the programmatic-dependent-launch attribute (and, if cluster_x > 1, as
+// thread-block clusters of that many CTAs along x).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              int cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+    if (cluster_x > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)cluster_x;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)na;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 inline int* status_ptr(const Handle* h) { return reinterpret_cast<int*>(h->ws + h->lay.status_off); }
 inline unsigned* counter_ptr(const Handle* h) { return reinterpret_cast<unsigned*>(h->ws + h->lay.counter_off); }
 
@@ -131,6 +160,16 @@ __device__ __forceinline__ void topk_insert(float (&val)[kTopSlots], int (&id)[k
         else if (here) { val[s] = v; id[s] = i; }
     }
 }
+
+// Programmatic dependent launch.  Every kernel of the step is launched so that it may start
+// while its predecessor in the stream is still draining: what it does before pdl_wait() (set
+// up shared memory and barriers, prefetch weights, which no kernel ever writes) overlaps with the
+// predecessor's tail.  pdl_wait() returns once the predecessor grid has completed and its
+// writes are visible; nothing that a predecessor produces may be read, and no global memory
+// may be written, before it.  Every kernel calls it, which orders the whole chain.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream begin to launch (it still waits in its own pdl_wait()).
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void report_error(int* status, int code, int detail) {
     if (atomicCAS(status, 0, code) == 0) status[1] = detail;

@@ -185,6 +185,49 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
         sh->is_last = 0;
         tc::fence_barrier_init();
     }
+    __syncthreads();                                                 // the barriers exist
+
+    const long long rps = p.rows_per_slot;
+    const long long R = rps * p.slots;
+    const long long r0 = R * blockIdx.x / gridDim.x;
+    const long long r1 = R * (blockIdx.x + 1) / gridDim.x;
+    const int ntotal = (int)(r1 - r0);                               // rows of this CTA
+    const int nfill = (ntotal + G - 1) / G;                          // ring fills of this CTA
+    const int slot0 = (int)(r0 / rps);
+    const long long seg_end = (long long)(slot0 + 1) * rps;          // first row of the next slot
+    const int n_seg0 = (int)((r1 < seg_end ? r1 : seg_end) - r0);    // rows that belong to slot0
+    const unsigned char* Wbase = reinterpret_cast<const unsigned char*>(p.W);
+
+    // producer state (used by lane 0 of warp 8 only)
+    const uint64_t policy = tc::policy_evict_first();
+    bool prod_ok = true;
+    int prod_j = 0;
+    auto issue_fill = [&](int j) -> bool {
+        const int s = j % nslots;
+        const uint32_t ph = (uint32_t)(j / nslots) & 1u;
+        if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) return false;
+        const int rows = (ntotal - j * G < G) ? ntotal - j * G : G;
+        const uint32_t bytes = (uint32_t)rows * (uint32_t)row_bytes;
+        // never hand the copy engine a range outside the weights or the ring
+        const long long first = r0 + (long long)j * G;
+        if (rows < 1 || first < 0 || first + rows > R || (bytes & 15u) != 0 || bytes > (uint32_t)slot_bytes) {
+            report_error(p.status, CTCSD_ERR_INTERNAL, 12);
+            return false;
+        }
+        tc::mbar_arrive_expect_tx(&sh->full[s], bytes);
+        tc::bulk_load_1d(ring + (size_t)s * slot_bytes, Wbase + (size_t)first * row_bytes, bytes, &sh->full[s], policy);
+        return true;
+    };
+    // The weights are never written by any kernel, so the ring is filled before this kernel waits
+    // for its predecessor in the stream: the copies run while the predecessor drains.
+    if (warp == kWarps && lane == 0) {
+        for (; prod_j < nfill && prod_j < nslots && prod_ok; ++prod_j) prod_ok = issue_fill(prod_j);
+        if (!prod_ok) --prod_j;
+    }
+    // everything above touches only the weights and this CTA's shared memory; the activations
+    // below may come from the kernel that precedes this one in the stream
+    pdl_wait();
+    pdl_trigger();
     for (int i = tid; i < MROWS * nch; i += kThreads) {
         int m = i / nch, ch = i - m * nch;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -200,39 +243,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
     }
     __syncthreads();
 
-    const long long rps = p.rows_per_slot;
-    const long long R = rps * p.slots;
-    const long long r0 = R * blockIdx.x / gridDim.x;
-    const long long r1 = R * (blockIdx.x + 1) / gridDim.x;
-    const int ntotal = (int)(r1 - r0);                               // rows of this CTA
-    const int nfill = (ntotal + G - 1) / G;                          // ring fills of this CTA
-    const int slot0 = (int)(r0 / rps);
-    const long long seg_end = (long long)(slot0 + 1) * rps;          // first row of the next slot
-    const int n_seg0 = (int)((r1 < seg_end ? r1 : seg_end) - r0);    // rows that belong to slot0
-    const unsigned char* Wbase = reinterpret_cast<const unsigned char*>(p.W);
-
     if (warp == kWarps) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            const uint64_t policy = tc::policy_evict_first();
-            bool ok = true;
-            int j = 0;
-            for (; j < nfill; ++j) {
-                const int s = j % nslots;
-                const uint32_t ph = (uint32_t)(j / nslots) & 1u;
-                if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-                const int rows = (ntotal - j * G < G) ? ntotal - j * G : G;
-                const uint32_t bytes = (uint32_t)rows * (uint32_t)row_bytes;
-                // never hand the copy engine a range outside the weights or the ring
-                const long long first = r0 + (long long)j * G;
-                if (rows < 1 || first < 0 || first + rows > R || (bytes & 15u) != 0 || bytes > (uint32_t)slot_bytes) {
-                    report_error(p.status, CTCSD_ERR_INTERNAL, 12);
-                    ok = false;
-                    break;
-                }
-                tc::mbar_arrive_expect_tx(&sh->full[s], bytes);
-                tc::bulk_load_1d(ring + (size_t)s * slot_bytes, Wbase + (size_t)first * row_bytes, bytes,
-                                 &sh->full[s], policy);
+            bool ok = prod_ok;
+            int j = prod_j;
+            for (; j < nfill && ok; ++j) {
+                ok = issue_fill(j);
+                if (!ok) break;
             }
             if (!ok) {
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 10);
@@ -482,7 +500,7 @@ int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     if (grid > R) grid = R;
     if (grid < p.slots) grid = p.slots;         // a CTA's range then touches at most two slots
     p.grid = (int)grid;
-    kern<<<(unsigned)grid, kThreads, smem, stream>>>(p, (int)nslots, G);
+    CTCSD_CUDA_CHECK(h, launch_pdl(kern, dim3((unsigned)grid), dim3(kThreads), smem, stream, 1, p, (int)nslots, G));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

@@ -82,36 +82,54 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
-
     const long long units = (long long)p.n_tiles * p.m_tiles;
     const int u0 = (int)(units * blockIdx.x / gridDim.x);
     const int u1 = (int)(units * (blockIdx.x + 1) / gridDim.x);
 
+    // producer state (lane 0 of warp 0 only).  Stage `it` holds K block it % num_k of unit
+    // u0 + it / num_k; every CTA walks the K axis from its own starting block (and wraps), so that
+    // at any moment the CTAs ask L2 for different parts of the shared activations.
+    const int total_it = (u1 - u0) * p.num_k;
+    const int k_start = (int)(((long long)blockIdx.x * p.num_k) / gridDim.x);
+    const uint64_t pol_w = tc::policy_evict_first();
+    const uint64_t pol_a = tc::policy_evict_last();
+    auto load_stage = [&](int it, bool do_w, bool do_a) {
+        const int u = u0 + it / p.num_k, kb = it - (it / p.num_k) * p.num_k;
+        const int nt = u / p.m_tiles, mt = u - nt * p.m_tiles;
+        const int s = it % p.stages;
+        unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
+        int kq = kb + k_start;
+        if (kq >= p.num_k) kq -= p.num_k;
+        if (do_w) {
+            tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)stage_bytes);
+            tc::tma_load_2d(a_dst + kABytes, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
+        }
+        if (do_a) tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kq * kBlockK, mt * kTileM, pol_a);
+    };
+    // The weights are never written by any kernel: their tiles of the first stages are requested
+    // before this kernel waits for its predecessor in the stream.
+    int pre = 0;
+    if (warp == 0 && lane == 0) {
+        tc::prefetch_tensormap(&tmA);
+        tc::prefetch_tensormap(&tmW);
+        pre = total_it < p.stages ? total_it : p.stages;
+        for (int it = 0; it < pre; ++it) load_stage(it, true, false);
+    }
+    // barriers and tensor memory are set up; the activations may come from the preceding kernel
+    pdl_wait();
+    pdl_trigger();
+
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            tc::prefetch_tensormap(&tmA);
-            tc::prefetch_tensormap(&tmW);
-            const uint64_t pol_w = tc::policy_evict_first();
-            const uint64_t pol_a = tc::policy_evict_last();
-            const int k_start = (int)(((long long)blockIdx.x * p.num_k) / gridDim.x);
-            int it = 0;
+            for (int it = 0; it < pre; ++it) load_stage(it, false, true);
+            int it = pre;
             bool ok = true;
-            for (int u = u0; u < u1 && ok; ++u) {
-                const int nt = u / p.m_tiles, mt = u - nt * p.m_tiles;
-                for (int kb = 0; kb < p.num_k; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-                    if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-                    unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
-                    tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)stage_bytes);
-                    // every CTA walks the K axis from its own starting block (and wraps), so that at
-                    // any moment the CTAs ask L2 for different parts of the shared activations
-                    int kq = kb + k_start;
-                    if (kq >= p.num_k) kq -= p.num_k;
-                    tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kq * kBlockK, mt * kTileM, pol_a);
-                    tc::tma_load_2d(a_dst + kABytes, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
-                }
+            for (; it < total_it; ++it) {
+                const int s = it % p.stages;
+                const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+                if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                load_stage(it, true, true);
             }
             if (!ok) {
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 1);
@@ -309,7 +327,7 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     long long units = (long long)p.n_tiles * p.m_tiles;
     int grid = (int)(units < h->num_sms ? units : h->num_sms);
-    lm_head_tc_kernel<<<grid, kThreads, smem, stream>>>(tmA, tmW, p);
+    CTCSD_CUDA_CHECK(h, launch_pdl(lm_head_tc_kernel, dim3(grid), dim3(kThreads), smem, stream, 1, tmA, tmW, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

@@ -371,6 +371,8 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     __shared__ int s_count, s_has_empty;
 
     const int b = blockIdx.x, tid = threadIdx.x;
+    pdl_wait();                      // the per-slot lists come from the preceding kernel
+    pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
     if (row < 0 || row >= p.M) {
         if (tid == 0) { report_error(p.status, CTCSD_ERR_INVALID_ARG, b); p.out_n_cand[b] = 0; }
@@ -457,6 +459,8 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
     const int b = blockIdx.x, tid = threadIdx.x;
+    pdl_wait();                      // the per-slot lists come from the preceding kernel
+    pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
     if (row < 0 || row >= p.M) {
         if (tid == 0) { report_error(p.status, CTCSD_ERR_INVALID_ARG, b); p.out_n_cand[b] = 0; }
@@ -566,7 +570,7 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     if (c.beam > 0) {
         const size_t smem = (size_t)kBeamCap * 52;
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_beam_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        collapse_beam_kernel<<<c.B, kThreads, smem, s>>>(p);
+        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
         CTCSD_LAUNCH_CHECK(h);
         return CTCSD_OK;
     }
@@ -579,7 +583,7 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     size_t smem = (size_t)cap * 24 + (size_t)npaths * 2;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_enum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    collapse_enum_kernel<<<c.B, kThreads, smem, s>>>(p);
+    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

@@ -112,6 +112,8 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
     const int warp = wfull & 3, kg = wfull >> 2;               // row group, key group
     const int gid = lane >> 2, tig = lane & 3;
 
+    pdl_wait();                      // the tree (node count, mask) comes from the preceding kernel
+    pdl_trigger();
     int n = p.n_nodes[b];
     const int L = p.kv_len[b];
     if (n < 0 || n > p.max_nodes || L < 0 || L + n > p.Lcap) {
@@ -459,21 +461,9 @@ int launch_d(Handle* h, cudaStream_t s, const AttnParams& p) {
     const size_t smem = (size_t)kRows * D * 2 + 2 * kStages * (size_t)kKeys * D * 2;
     auto kern = tree_attention_mma_kernel<D, true>;
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3(qtiles * splits, p.Hkv, p.B);
-    cfg.blockDim = dim3(kThreads * 2, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = splits;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     float* no_part = nullptr;
-    CTCSD_CUDA_CHECK(h, cudaLaunchKernelEx(&cfg, kern, p, no_part, splits));
+    CTCSD_CUDA_CHECK(h, launch_pdl(kern, dim3(qtiles * splits, p.Hkv, p.B), dim3(kThreads * 2), smem, s, splits,
+                                   p, no_part, splits));
     h->launches++;
     return CTCSD_OK;
 }
