@@ -12,8 +12,9 @@ beta^{-1} the collapse map, Y the collapsed candidate.
 Pins (see tests/test_oracle_pins.py): every function below is pinned by something other
 than itself - hand-worked collapse cases, the total-mass closed form, the Graves forward
 recursion (torch's ctc_loss and an independent alpha recursion), library matmul /
-log-softmax / top-k / scaled-dot-product attention in fp64, and brute-force tries and
-acceptance definitions.  The finite-beam prefix search is a heuristic the paper does not
+log-softmax / top-k / scaled-dot-product attention in fp64, brute-force tries and
+acceptance definitions, and - for the history update - the equality of ordinary attention over
+the updated prefix with tree attention over the old cache, plus a hand-worked overlap case.  The finite-beam prefix search is a heuristic the paper does not
 specify ("a group of the most valuable combinations are reserved", Sec. 3.3): with a beam
 that never prunes it is pinned to exact enumeration; with a pruning beam it is pinned only
 by bounds (candidate subset, score <= exact) - beyond that: parity unpinned.
@@ -346,3 +347,31 @@ def greedy_accept(node_tok: np.ndarray, parent: np.ndarray, n_nodes: np.ndarray,
             cur = nxt
         next_tok[b] = int(am[b, cur])
     return acc_len, acc_nodes, acc_tok, next_tok
+
+
+# --------------------------------------------------------------------------------------
+# S12  history update after acceptance (Sec. 3.3: "the decoding history is updated
+#      according to the output"): the accepted path becomes part of the cached prefix
+# --------------------------------------------------------------------------------------
+def commit_accepted(K: np.ndarray, Vc: np.ndarray, kv_len: np.ndarray, acc_len: np.ndarray,
+                    acc_nodes: np.ndarray, max_nodes: int):
+    """K, Vc [B,Hkv,Lcap,D] with tree node j of sequence b at cache row kv_len[b]+j.  The root
+    (row kv_len[b]) stays; the l-th accepted node's key/value row moves to row kv_len[b]+1+l,
+    read from the cache as it was before the call.  Returns (K', V', kv_len' = kv_len+1+acc_len,
+    sel_row [B] = b*max_nodes + last accepted node (the root if nothing was accepted): the tree
+    row whose hidden state the next step drafts from)."""
+    K2, V2 = np.array(K, copy=True), np.array(Vc, copy=True)
+    B = K.shape[0]
+    new_len = np.zeros((B,), dtype=np.int64)
+    sel_row = np.zeros((B,), dtype=np.int64)
+    for b in range(B):
+        L = int(kv_len[b])
+        last = 0
+        for l in range(int(acc_len[b])):
+            node = int(acc_nodes[b, l])
+            K2[b, :, L + 1 + l, :] = K[b, :, L + node, :]
+            V2[b, :, L + 1 + l, :] = Vc[b, :, L + node, :]
+            last = node
+        new_len[b] = L + 1 + int(acc_len[b])
+        sel_row[b] = b * max_nodes + last
+    return K2, V2, new_len, sel_row

@@ -424,3 +424,71 @@ def test_greedy_accept_chain_extremes():
     am[0, 0] = 7                                          # no agreement at the root
     acc_len, acc_nodes, acc_tok, next_tok = orc.greedy_accept(node_tok, parent, n, am, 4)
     assert acc_len[0] == 0 and next_tok[0] == 7
+
+
+# ------------------------------------------------------------------ S12 history update
+def test_commit_accepted_makes_the_accepted_path_the_prefix():
+    """After the update, ordinary attention of the last accepted node over the new prefix must
+    equal tree attention of that node over the old cache (prefix + its ancestors): the same
+    key/value rows in both, so the two (separately pinned) attention results agree to rounding."""
+    rng = np.random.default_rng(5)
+    B, Hkv, Hq, D, n_max, T = 3, 2, 4, 8, 16, 4
+    for trial in range(6):
+        kv_len = rng.integers(1, 9, size=B)
+        Lcap = int(kv_len.max()) + n_max
+        # random tree: parent[i] < i
+        parent = np.full((B, n_max), -1, dtype=np.int64)
+        n_nodes = rng.integers(2, n_max + 1, size=B)
+        mask = np.zeros((B, n_max, 1), dtype=np.uint64)
+        depth = np.zeros((B, n_max), dtype=np.int64)
+        for b in range(B):
+            mask[b, 0, 0] = np.uint64(1)
+            for i in range(1, int(n_nodes[b])):
+                par = int(rng.integers(max(0, i - 3), i))
+                if depth[b, par] >= T:
+                    par = 0
+                parent[b, i] = par
+                depth[b, i] = depth[b, par] + 1
+                mask[b, i, 0] = mask[b, par, 0] | np.uint64(1 << i)
+        # an accepted path: walk down from the root picking children at random
+        acc_len = np.zeros(B, dtype=np.int64)
+        acc_nodes = np.full((B, T), -1, dtype=np.int64)
+        for b in range(B):
+            cur = 0
+            while acc_len[b] < T:
+                kids = [c for c in range(int(n_nodes[b])) if parent[b, c] == cur]
+                if not kids or rng.random() < 0.2:
+                    break
+                cur = int(rng.choice(kids))
+                acc_nodes[b, acc_len[b]] = cur
+                acc_len[b] += 1
+        K = rng.standard_normal((B, Hkv, Lcap, D))
+        V = rng.standard_normal((B, Hkv, Lcap, D))
+        Q = rng.standard_normal((B, n_max, Hq, D))
+        K2, V2, new_len, sel_row = orc.commit_accepted(K, V, kv_len, acc_len, acc_nodes, n_max)
+        O_tree = orc.tree_attention(Q, K, V, kv_len, n_nodes, mask, 0.3)
+        for b in range(B):
+            last = int(acc_nodes[b, acc_len[b] - 1]) if acc_len[b] > 0 else 0
+            assert sel_row[b] == b * n_max + last
+            assert new_len[b] == kv_len[b] + 1 + acc_len[b]
+            # the last accepted node as a one-node "tree" on top of the new prefix
+            q1 = np.zeros((1, n_max, Hq, D))
+            q1[0, 0] = Q[b, last]
+            one = orc.tree_attention(q1, K2[b:b + 1], V2[b:b + 1], np.array([new_len[b] - 1]), np.array([1]),
+                                     np.ones((1, n_max, 1), dtype=np.uint64), 0.3)
+            np.testing.assert_allclose(one[0, 0], O_tree[b, last], rtol=1e-12, atol=1e-12)
+            # nothing below the tree rows changes; a chain 1,2,..,k is already in place
+            assert np.array_equal(K2[b, :, :kv_len[b] + 1], K[b, :, :kv_len[b] + 1])
+            if list(acc_nodes[b, :acc_len[b]]) == list(range(1, int(acc_len[b]) + 1)):
+                assert np.array_equal(K2[b], K[b]) and np.array_equal(V2[b], V[b])
+
+
+def test_commit_accepted_reads_the_cache_as_it_was():
+    # accepted nodes 2 then 3: row L+1 <- row L+2, row L+2 <- row L+3 (the old row L+2 must be read first)
+    K = np.arange(2 * 1 * 8 * 1, dtype=np.float64).reshape(2, 1, 8, 1)
+    V = -K
+    K2, V2, new_len, sel = orc.commit_accepted(K, V, np.array([2, 1]), np.array([2, 0]),
+                                               np.array([[2, 3], [-1, -1]]), 4)
+    assert K2[0, 0, :, 0].tolist() == [0, 1, 2, 4, 5, 5, 6, 7]
+    assert V2[0, 0, :, 0].tolist() == [0, -1, -2, -4, -5, -5, -6, -7]
+    assert np.array_equal(K2[1], K[1]) and new_len.tolist() == [5, 2] and sel.tolist() == [3, 4]
