@@ -198,6 +198,25 @@ int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const voi
                         int* out_next_tok, float* out_logits_dbg);
 
 /*
+ * History update after acceptance (Sec. 3.3: "the decoding history is updated according to the
+ * output"): the accepted path becomes part of the cached prefix, so that the next step can
+ * start without host work.  For sequence b with L = kv_len[b]: the root's key/value row (cache
+ * row L) stays; for l = 0 .. acc_len[b]-1 the row of accepted node acc_nodes[b,l] (cache row
+ * L + node) is moved to row L + 1 + l, for every kv head, in K and in V; rows are read as they
+ * were before the call (a destination may be another accepted node's source).
+ * K, V [B,Hkv,Lcap,D] dtype, updated IN PLACE;  kv_len, acc_len [B], acc_nodes [B,T] as
+ * produced by ctcsd_verify_accept.
+ * out_kv_len [B] int32 = kv_len + 1 + acc_len (may alias kv_len);
+ * out_sel_row [B] int32 or NULL = b*max_nodes + last accepted node (the root if none): the
+ *   tree row whose hidden state the next step drafts from (see sel_row of ctcsd_topk_collapse).
+ * A sequence whose path would leave the cache is left unchanged and CTCSD_ERR_INVALID_ARG is
+ * recorded in the device status word.
+ */
+int ctcsd_commit_accepted(ctcsd_handle* h, void* stream, void* K, void* V, int Lcap,
+                          const int* kv_len, const int* acc_len, const int* acc_nodes,
+                          int* out_kv_len, int* out_sel_row);
+
+/*
  * Tree attention without a handle and without any allocation (the paper has no counterpart:
  * this is a packaging variant of ctcsd_tree_attention, same arithmetic, same kernels).
  *

@@ -23,7 +23,7 @@ EXPORTS = [
     "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
     "ctcsd_last_cuda_error", "ctcsd_launch_count",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
-    "ctcsd_verify_accept", "ctcsd_tree_attention_static",
+    "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static",
 ]
 
 
@@ -64,6 +64,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_build_tree.argtypes = [vp, vp] + [vp] * 12
     lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
     lib.ctcsd_verify_accept.argtypes = [vp, vp] + [vp] * 11
+    lib.ctcsd_commit_accepted.argtypes = [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp]
     lib.ctcsd_tree_attention_static.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp, vp, vp,
                                                 ctypes.c_float, vp, vp]
     for name in EXPORTS:
@@ -214,6 +215,18 @@ class Handle:
             _ptr(out_next_tok, i32, c.B, "out_next_tok"),
             _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
         self._check(rc, "verify_accept")
+
+    def commit_accepted(self, K, V, kv_len, acc_len, acc_nodes, out_kv_len, out_sel_row=None, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        Lcap = K.shape[2]
+        rc = self.lib.ctcsd_commit_accepted(
+            self._h, _stream_ptr(stream),
+            _ptr(K, self.act_dtype, c.B * c.Hkv * Lcap * c.D, "K"), _ptr(V, self.act_dtype, c.B * c.Hkv * Lcap * c.D, "V"),
+            Lcap, _ptr(kv_len, i32, c.B, "kv_len"), _ptr(acc_len, i32, c.B, "acc_len"),
+            _ptr(acc_nodes, i32, c.B * c.T, "acc_nodes"), _ptr(out_kv_len, i32, c.B, "out_kv_len"),
+            _ptr(out_sel_row, i32, c.B, "out_sel_row"))
+        self._check(rc, "commit_accepted")
 
 
 def tree_attention_static(Q, K, V, kv_len, n_nodes, mask, scale, out_O, out_status=None, stream=None):

@@ -43,6 +43,7 @@ class DraftVerifyStep:
             mask=z(B, n, W, dtype=torch.int64), retrieve=z(B, N, T), n_nodes=z(B),
             O=z(B, n, cfg.Hq, cfg.D, dtype=act),
             argmax=z(B, n), acc_len=z(B), acc_nodes=z(B, T), acc_tok=z(B, T), next_tok=z(B),
+            new_kv_len=z(B), next_sel_row=z(B),
         )
         if debug_logits:
             self.out["draft_logits_dbg"] = z(self.M, T, cfg.V + 1, dtype=f32)
@@ -80,6 +81,12 @@ class DraftVerifyStep:
         self.h.verify_accept(i["hn"], i["Wl"], o["node_tok"], o["parent"], o["n_nodes"],
                              o["argmax"], o["acc_len"], o["acc_nodes"], o["acc_tok"], o["next_tok"],
                              o.get("lm_logits_dbg"), stream=stream)
+
+    def commit(self, stream=None):
+        """History update (not part of run(): it changes the K/V cache in place)."""
+        i, o = self.inp, self.out
+        self.h.commit_accepted(i["K"], i["V"], i["kv_len"], o["acc_len"], o["acc_nodes"],
+                               o["new_kv_len"], o["next_sel_row"], stream=stream)
 
     def run(self, stream=None):
         """The whole hot path: five calls back to back on one stream, no host sync."""

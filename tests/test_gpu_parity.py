@@ -85,6 +85,34 @@ def test_batched_workloads_full_size_sampled(name):
     assert all(2 <= n <= cfg.max_nodes for n in r["n_nodes"])
 
 
+@pytest.mark.parametrize("name", ["c2s", "c3s", "c5s", "c1d64"])
+def test_history_update_moves_the_accepted_rows(name):
+    """ctcsd_commit_accepted against the oracle: the K/V caches must match byte for byte, the new
+    lengths and the next drafting rows exactly; then a second step runs on the updated cache."""
+    import torch
+    from oracle import ctcsd_oracle as orc
+    cfg = SMALL[name]
+    r = _run(cfg, seed=4)
+    step = r["step"]
+    K0, V0 = step.inp["K"].float().cpu().numpy(), step.inp["V"].float().cpu().numpy()
+    kv_len = step.inp["kv_len"].cpu().numpy()
+    acc_len, acc_nodes = step.host("acc_len"), step.host("acc_nodes")
+    K1, V1, new_len, sel = orc.commit_accepted(K0, V0, kv_len, acc_len, acc_nodes, cfg.max_nodes)
+    step.commit()
+    step.check_status()
+    assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
+    assert np.array_equal(step.inp["V"].float().cpu().numpy(), V1)
+    np.testing.assert_array_equal(step.host("new_kv_len"), new_len)
+    np.testing.assert_array_equal(step.host("next_sel_row"), sel)
+    assert acc_len.max() >= 1, "pick a seed where something is accepted"
+    # a path that would leave the cache is refused on the device and changes nothing
+    bad_len = torch.full_like(step.inp["kv_len"], step.inp["K"].shape[2])
+    step.h.commit_accepted(step.inp["K"], step.inp["V"], bad_len, step.out["acc_len"], step.out["acc_nodes"],
+                           step.out["new_kv_len"], step.out["next_sel_row"])
+    assert step.h.poll_status() == -1
+    assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
+
+
 def test_invalid_arguments_are_rejected_on_the_host():
     import ctypes
     from paper_2412_00061_b200 import binding
