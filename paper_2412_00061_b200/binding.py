@@ -21,7 +21,7 @@ SCORE_SUM, SCORE_MAX = 0, 1
 
 EXPORTS = [
     "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
-    "ctcsd_last_cuda_error", "ctcsd_launch_count",
+    "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
     "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static",
 ]
@@ -57,6 +57,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_strerror.argtypes = [ci]
     lib.ctcsd_strerror.restype = ctypes.c_char_p
     lib.ctcsd_last_cuda_error.argtypes = [vp]
+    lib.ctcsd_set_l2_prefetch.argtypes = [vp, vp, cs]
     lib.ctcsd_launch_count.argtypes = [vp]
     lib.ctcsd_launch_count.restype = ctypes.c_longlong
     lib.ctcsd_draft_logits.argtypes = [vp, vp, ci] + [vp] * 8
@@ -136,6 +137,15 @@ class Handle:
     @property
     def launch_count(self) -> int:
         return int(self.lib.ctcsd_launch_count(self._h))
+
+    def set_l2_prefetch(self, tensor: Optional[torch.Tensor], nbytes: int = 0):
+        """Hint: after the draft head, prefetch the first `nbytes` of `tensor` (the LM-head weights)
+        into L2; None or 0 turns it off."""
+        if tensor is None or nbytes <= 0:
+            self._check(self.lib.ctcsd_set_l2_prefetch(self._h, None, 0), "set_l2_prefetch")
+            return
+        nbytes = min(int(nbytes), tensor.numel() * tensor.element_size())
+        self._check(self.lib.ctcsd_set_l2_prefetch(self._h, _ptr(tensor, name="prefetch"), nbytes), "set_l2_prefetch")
 
     def poll_status(self, stream=None) -> int:
         st = ctypes.c_int(0)

@@ -51,6 +51,8 @@ struct Handle {
     int num_sms;
     int last_cuda_error;
     long long launches;
+    const void* l2_hint_ptr;     // range that ctcsd_draft_logits asks L2 to fetch when it finishes
+    size_t l2_hint_bytes;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

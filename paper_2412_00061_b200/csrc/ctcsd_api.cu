@@ -119,6 +119,13 @@ extern "C" int ctcsd_poll_status(ctcsd_handle* hh, void* stream, int* out_status
     return CTCSD_OK;
 }
 
+extern "C" int ctcsd_set_l2_prefetch(ctcsd_handle* hh, const void* ptr, size_t bytes) {
+    if (!hh || (bytes != 0 && !ptr) || (reinterpret_cast<uintptr_t>(ptr) & 15)) return CTCSD_ERR_INVALID_ARG;
+    hh->h.l2_hint_ptr = bytes ? ptr : nullptr;
+    hh->h.l2_hint_bytes = bytes;
+    return CTCSD_OK;
+}
+
 extern "C" const char* ctcsd_strerror(int status) {
     switch (status) {
         case CTCSD_OK: return "ok";

@@ -34,5 +34,7 @@ extern "C" int ctcsd_draft_logits(ctcsd_handle* hh, void* stream, int M, const v
     p.out_lse = out_lse;
     p.out_argmax = nullptr;
     p.logits_dbg = out_logits_dbg;
+    p.pf_ptr = h->l2_hint_ptr;
+    p.pf_bytes = h->l2_hint_bytes;
     return launch_gemv_stream(h, static_cast<cudaStream_t>(stream), c.dtype, M, p);
 }

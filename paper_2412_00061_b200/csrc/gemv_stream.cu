@@ -256,6 +256,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 10);
                 *abort_flag = 1;
             }
+            // All of this CTA's weights are requested.  If the caller named a range that the next
+            // heavy kernel will stream, ask L2 for this CTA's share of it now: the fetch runs
+            // while the small kernels that follow leave HBM idle.
+            if (ok && p.pf_bytes != 0) {
+                const unsigned long long chunk = 64 * 1024;
+                const unsigned long long nchunks = (p.pf_bytes + chunk - 1) / chunk;
+                for (unsigned long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
+                    unsigned long long len = p.pf_bytes - c * chunk;
+                    if (len > chunk) len = chunk;
+                    len &= ~15ull;
+                    if (len) tc::bulk_prefetch_l2(static_cast<const unsigned char*>(p.pf_ptr) + c * chunk, (uint32_t)len);
+                }
+            }
             if (*abort_flag != 0) {
                 // let copies that are still in flight land before the CTA gives its memory back
                 for (int back = 1; back <= nslots && back <= j; ++back) {
@@ -541,6 +554,7 @@ int launch_gemv_stream(Handle* h, cudaStream_t stream, int dtype, int M, GemvPar
     p.part_slot = reinterpret_cast<int*>(h->ws + h->lay.part_slot_off);
     p.counter = counter_ptr(h);
     p.status = status_ptr(h);
+    if (p.mode != 0) { p.pf_ptr = nullptr; p.pf_bytes = 0; }
     if (dtype == CTCSD_DTYPE_BF16) return launch_typed_bf16(h, stream, M, p);
     return launch_typed_f32(h, stream, M, p);
 }

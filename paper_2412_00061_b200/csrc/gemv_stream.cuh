@@ -34,6 +34,8 @@ struct GemvParams {
     int* out_argmax;          // mode 1: [M]
     float* logits_dbg;        // null or [M,slots,rows_per_slot]
     int* status;              // device status word
+    const void* pf_ptr;       // optional: range the CTAs ask L2 to fetch once their own stream is issued
+    unsigned long long pf_bytes;
 };
 
 int launch_gemv_stream(Handle* h, cudaStream_t stream, int dtype, int M, GemvParams p);

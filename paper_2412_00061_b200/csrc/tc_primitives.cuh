@@ -88,6 +88,12 @@ __device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_
         : "memory");
 }
 
+// Asks L2 to fetch [src, src + bytes) from HBM (no destination, no completion to wait for).
+// `src` must be 16-byte aligned and `bytes` a multiple of 16.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes) : "memory");
+}
+
 // ---- tensor memory ------------------------------------------------------------------------
 // Executed by one full warp; writes the TMEM base address to *dst_smem.
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {

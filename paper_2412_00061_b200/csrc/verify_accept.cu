@@ -48,6 +48,7 @@ extern "C" int ctcsd_verify_accept(ctcsd_handle* hh, void* stream, const void* h
     g.out_topk_id = nullptr; g.out_topk_lp = nullptr; g.out_lse = nullptr;
     g.out_argmax = out_argmax;
     g.logits_dbg = out_logits_dbg;
+    g.pf_ptr = nullptr; g.pf_bytes = 0;
     int rc = launch_gemv_stream(h, s, c.dtype, M, g);
     if (rc != CTCSD_OK) return rc;
     greedy_accept_kernel<<<c.B, 32, 0, s>>>(a);

@@ -23,6 +23,7 @@ def to_device(a: np.ndarray, dtype: str, device) -> torch.Tensor:
 
 
 class DraftVerifyStep:
+    L2_PREFETCH_BYTES = 48 << 20
     def __init__(self, cfg: StepConfig, device="cuda:0", max_draft_rows: int = 0, debug_logits: bool = False):
         self.cfg = cfg
         self.device = torch.device(device)
@@ -53,6 +54,10 @@ class DraftVerifyStep:
     def set_inputs(self, **tensors):
         """x, Wd, blank_bias, row_seq, sel_row, base_tok, kv_len, Q, K, V, hn, Wl (device tensors)."""
         self.inp.update(tensors)
+        if "Wl" in tensors and self.cfg.dtype == "bf16":
+            # while the small kernels between draft head and LM head run, HBM is idle: let L2
+            # fetch the head of the LM-head weights then
+            self.h.set_l2_prefetch(tensors["Wl"], self.L2_PREFETCH_BYTES)
 
     # individual stages ----------------------------------------------------------------
     def draft(self, stream=None):
