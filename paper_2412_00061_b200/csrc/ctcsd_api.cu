@@ -41,6 +41,18 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
     l.gemv_grid_max = num_sms * 8 > 64 ? num_sms * 8 : 64;
     l.draft_part_off = off;  off = align_up(off + sizeof(DraftPartial) * 8 * (size_t)l.gemv_grid_max * 2, 256);
     l.part_slot_off = off;   off = align_up(off + sizeof(int) * (size_t)l.gemv_grid_max * 2, 256);
+    {
+        const int rows = c.max_draft_rows > 0 ? c.max_draft_rows : c.B;
+        l.tc_part_off = off;
+        l.tc_part_bytes = 0;
+        if (rows > 8 && c.dtype == CTCSD_DTYPE_BF16) {
+            const int classes = c.V + 1;
+            const int nt = classes >= 224 ? 224 : (classes + 15) / 16 * 16;
+            const size_t tiles = (size_t)c.T * ((classes + nt - 1) / nt);
+            l.tc_part_bytes = sizeof(DraftPartial) * tiles * (size_t)((rows + 127) / 128 * 128);
+            off = align_up(off + l.tc_part_bytes, 256);
+        }
+    }
     int units = c.B * c.Hkv;
     int splits = (2 * num_sms + units - 1) / units;
     if (splits < 1) splits = 1;

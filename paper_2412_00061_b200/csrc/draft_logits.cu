@@ -1,5 +1,6 @@
 // ctcsd_draft_logits: draft-head projection, per-slot log-softmax and per-slot top-k.
 #include "gemv_stream.cuh"
+#include "lm_head_tc.cuh"
 
 using namespace ctcsd;
 
@@ -13,6 +14,12 @@ extern "C" int ctcsd_draft_logits(ctcsd_handle* hh, void* stream, int M, const v
     if (!row_seq && blank_bias && M > c.B) return CTCSD_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(Wd)) & 15) return CTCSD_ERR_INVALID_ARG;
 
+    // more than 8 rows: the tensor-core weight stream reads the weights once for up to 128 rows
+    if (draft_head_tc_supported(h, M)) {
+        int rc = launch_draft_head_tc(h, static_cast<cudaStream_t>(stream), M, x, Wd, row_seq, blank_bias,
+                                      out_topk_id, out_topk_lp, out_lse, out_logits_dbg);
+        if (rc != CTCSD_ERR_UNSUPPORTED) return rc;
+    }
     GemvParams p;
     p.x = x;
     p.W = Wd;

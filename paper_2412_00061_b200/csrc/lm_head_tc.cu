@@ -14,8 +14,10 @@
 // runs the greedy acceptance walk.
 #include "lm_head_tc.cuh"
 #include "tc_primitives.cuh"
+#include "run_state.cuh"
 
 #include <math.h>
+#include <string.h>
 
 namespace ctcsd {
 namespace {
@@ -38,8 +40,14 @@ struct TcParams {
     AcceptParams acc;
     unsigned* counter;
     int* out_argmax;          // [M]
-    float* logits_dbg;        // null or [M][V]
+    float* logits_dbg;        // null or [M][V]  (draft mode: [M][slots][V])
     int* status;
+    // draft mode: W is [slots][V][H]; n_tiles = slots * tiles_per_slot
+    int slots;
+    int tiles_per_slot;
+    DraftPartial* part;       // [n_tiles][m_tiles*128] per-tile states
+    const int* row_seq;       // [M] or null
+    const float* blank_bias;  // [B] or null; added to class V-1 of every slot
 };
 
 struct __align__(8) TcShared {
@@ -53,6 +61,11 @@ struct __align__(8) TcShared {
     int never_set;      // stays zero: lets a drain wait run to its time limit after an abort
 };
 
+// MODE 0: LM head (row arg-max + acceptance).  MODE 1: draft head (W is a 3-D tensor
+// [slots][V][H]; a vocabulary tile never crosses a slot; every epilogue thread folds its
+// row's logits of the tile into an online (max, sum of exp, best-8) state and stores one
+// state per (tile, row); a second kernel merges the tiles of every slot).
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TcParams p) {
     extern __shared__ unsigned char dyn_raw[];
@@ -102,7 +115,12 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (kq >= p.num_k) kq -= p.num_k;
         if (do_w) {
             tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)stage_bytes);
-            tc::tma_load_2d(a_dst + kABytes, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
+            if constexpr (MODE == 0) {
+                tc::tma_load_2d(a_dst + kABytes, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
+            } else {
+                const int t = nt / p.tiles_per_slot, ntl = nt - t * p.tiles_per_slot;
+                tc::tma_load_3d(a_dst + kABytes, &tmW, &sh->full[s], kq * kBlockK, ntl * p.Nt, t, pol_w);
+            }
         }
         if (do_a) tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kq * kBlockK, mt * kTileM, pol_a);
     };
@@ -173,7 +191,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
         }
     } else {
-        // ---------------- epilogue: arg-max of each accumulator row ----------------
+        // ---------------- epilogue ----------------
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int row_in_tile = q * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -181,12 +199,18 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         for (int u = u0; u < u1 && ok; ++u, ++ucount) {
             const int nt = u / p.m_tiles, mt = u - nt * p.m_tiles;
-            const int n0 = nt * p.Nt;
             const int row = mt * kTileM + row_in_tile;
+            // draft mode: tile nt is tile ntl of slot t
+            const int t = MODE == 1 ? nt / p.tiles_per_slot : 0;
+            const int n0 = (MODE == 1 ? nt - t * p.tiles_per_slot : nt) * p.Nt;
+            float bias = 0.f;
+            if (MODE == 1 && p.blank_bias != nullptr && row < p.M) bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
             if (!tc::mbar_wait(&sh->tmem_full, (uint32_t)ucount & 1u, abort_flag)) { ok = false; break; }
             tc::tc_fence_after_sync();
             float best = -INFINITY;
             int best_idx = 0x7fffffff;
+            RunState st;
+            if constexpr (MODE == 1) st.init();
             for (int c0 = 0; c0 < p.Nt; c0 += 32) {
                 uint32_t r[32];
                 if (c0 + 32 <= p.Nt) {
@@ -200,23 +224,34 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const float v = __uint_as_float(r[j]);
+                    float v = __uint_as_float(r[j]);
                     const int col = n0 + c0 + j;
                     if (col < p.V && c0 + j < p.Nt) {
-                        if (v > best) { best = v; best_idx = col; }
-                        if (p.logits_dbg != nullptr && row < p.M) p.logits_dbg[(size_t)row * p.V + col] = v;
+                        if constexpr (MODE == 0) {
+                            if (v > best) { best = v; best_idx = col; }
+                            if (p.logits_dbg != nullptr && row < p.M) p.logits_dbg[(size_t)row * p.V + col] = v;
+                        } else {
+                            if (col == p.V - 1) v += bias;
+                            if (p.logits_dbg != nullptr && row < p.M)
+                                p.logits_dbg[((size_t)row * p.slots + t) * p.V + col] = v;
+                            st.push(v, col);
+                        }
                     }
                 }
             }
             tc::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&sh->tmem_empty);
+            if constexpr (MODE == 1) {
+                st.store(p.part + (size_t)nt * (p.m_tiles * kTileM) + row);
+            } else {
             // fold this tile's winner into the row's global maximum: larger logit first, equal
             // logits -> lower id (the id is stored complemented in the low word)
             if (row < p.M && best_idx != 0x7fffffff) {
                 const unsigned u = __float_as_uint(best);
                 const unsigned sortable = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
                 atomicMax(p.keys + row, ((unsigned long long)sortable << 32) | (0xffffffffu - (unsigned)best_idx));
+            }
             }
         }
         if (!ok && lane == 0) {
@@ -233,6 +268,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tc::tc_fence_after_sync();
         tc::tmem_dealloc(tmem_base, 256);
     }
+    if constexpr (MODE == 1) return;                 // the tiles are merged by draft_tc_merge_kernel
     if (tid == 0) {
         unsigned t = atomicAdd(p.counter, 1u);
         sh->is_last = (t == gridDim.x - 1) ? 1 : 0;
@@ -282,7 +318,114 @@ bool make_map(CUtensorMap* map, const void* base, long long rows, long long cols
     return r == CUDA_SUCCESS;
 }
 
+// 3-D bf16 tensor [slots][rows][cols] (cols contiguous), box = [1][box_rows][64 cols], 128-byte
+// swizzle; rows past the end of a slot read as zero.
+bool make_map3(CUtensorMap* map, const void* base, long long slots, long long rows, long long cols, int box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)slots};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)rows};
+    cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+struct DraftMergeParams {
+    const DraftPartial* part;     // [slots * tiles_per_slot][mpad]
+    int M, mpad, slots, tiles_per_slot, k;
+    int* out_topk_id; float* out_topk_lp; float* out_lse;
+};
+
+// One warp per (activation row, slot): merges the per-tile states of the slot into the
+// log-sum-exp and the top-k of the row.
+__global__ void __launch_bounds__(128) draft_tc_merge_kernel(DraftMergeParams p) {
+    const int lane = threadIdx.x & 31;
+    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    pdl_wait();
+    pdl_trigger();
+    if (wid >= (long long)p.M * p.slots) return;
+    const int m = (int)(wid / p.slots), t = (int)(wid - (long long)m * p.slots);
+    RunState fs;
+    fs.init();
+    for (int e = lane; e < p.tiles_per_slot; e += 32)
+        fs.absorb(load_partial_cg(p.part + ((size_t)t * p.tiles_per_slot + e) * p.mpad + m));
+    warp_combine(fs);
+    if (lane == 0) {
+        const float lse = fs.mx + logf(fs.sum);
+        p.out_lse[(size_t)m * p.slots + t] = lse;
+#pragma unroll
+        for (int j = 0; j < kTopSlots; ++j) {
+            if (j < p.k) {
+                const size_t o = ((size_t)m * p.slots + t) * p.k + j;
+                p.out_topk_id[o] = fs.id[j];
+                p.out_topk_lp[o] = fs.val[j] - lse;
+            }
+        }
+    }
+}
+
 }  // namespace
+
+int draft_tc_tile_rows(int classes) {
+    if (classes >= 224) return 224;
+    return (classes + 15) / 16 * 16;
+}
+
+bool draft_head_tc_supported(const Handle* h, int M) {
+    const ctcsd_config& c = h->cfg;
+    return c.dtype == CTCSD_DTYPE_BF16 && c.H >= 64 && c.V + 1 >= 16 && M > 8 && h->lay.tc_part_bytes > 0;
+}
+
+int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, const void* Wd, const int* row_seq,
+                         const float* blank_bias, int* out_topk_id, float* out_topk_lp, float* out_lse,
+                         float* out_logits_dbg) {
+    const ctcsd_config& c = h->cfg;
+    if (!draft_head_tc_supported(h, M)) return CTCSD_ERR_UNSUPPORTED;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = M;
+    p.V = c.V + 1;                                   // classes per slot, blank included
+    p.num_k = (c.H + kBlockK - 1) / kBlockK;
+    p.m_tiles = (M + kTileM - 1) / kTileM;
+    p.Nt = draft_tc_tile_rows(p.V);
+    p.slots = c.T;
+    p.tiles_per_slot = (p.V + p.Nt - 1) / p.Nt;
+    p.n_tiles = p.slots * p.tiles_per_slot;
+    const size_t need = sizeof(DraftPartial) * (size_t)p.n_tiles * p.m_tiles * kTileM;
+    if (need > h->lay.tc_part_bytes) return CTCSD_ERR_WORKSPACE;
+    const int stage_bytes = kABytes + p.Nt * 128;
+    int stages = (int)((220 * 1024 - (int)sizeof(TcShared) - 1024) / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return CTCSD_ERR_UNSUPPORTED;
+    p.stages = stages;
+    p.part = reinterpret_cast<DraftPartial*>(h->ws + h->lay.tc_part_off);
+    p.row_seq = row_seq;
+    p.blank_bias = blank_bias;
+    p.logits_dbg = out_logits_dbg;
+    p.status = status_ptr(h);
+
+    CUtensorMap tmA, tmW;
+    if (!make_map(&tmA, x, M, c.H, kTileM)) return CTCSD_ERR_CUDA;
+    if (!make_map3(&tmW, Wd, p.slots, p.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
+    const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
+    CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    long long units = (long long)p.n_tiles * p.m_tiles;
+    int grid = (int)(units < h->num_sms ? units : h->num_sms);
+    CTCSD_CUDA_CHECK(h, launch_pdl(lm_head_tc_kernel<1>, dim3(grid), dim3(kThreads), smem, stream, 1, tmA, tmW, p));
+    CTCSD_LAUNCH_CHECK(h);
+
+    DraftMergeParams mp;
+    mp.part = p.part;
+    mp.M = M; mp.mpad = p.m_tiles * kTileM; mp.slots = p.slots; mp.tiles_per_slot = p.tiles_per_slot; mp.k = c.k;
+    mp.out_topk_id = out_topk_id; mp.out_topk_lp = out_topk_lp; mp.out_lse = out_lse;
+    const long long warps = (long long)M * p.slots;
+    CTCSD_CUDA_CHECK(h, launch_pdl(draft_tc_merge_kernel, dim3((unsigned)((warps + 3) / 4)), dim3(128), 0, stream, 1, mp));
+    CTCSD_LAUNCH_CHECK(h);
+    return CTCSD_OK;
+}
 
 bool lm_head_tc_supported(const Handle* h) {
     const ctcsd_config& c = h->cfg;
@@ -295,6 +438,7 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     if (!lm_head_tc_supported(h)) return CTCSD_ERR_UNSUPPORTED;
 
     TcParams p;
+    memset(&p, 0, sizeof(p));
     p.M = M;
     p.V = c.V;
     p.num_k = (c.H + kBlockK - 1) / kBlockK;
@@ -324,10 +468,10 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     if (!make_map(&tmW, Wl, c.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
 
     const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
-    CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     long long units = (long long)p.n_tiles * p.m_tiles;
     int grid = (int)(units < h->num_sms ? units : h->num_sms);
-    CTCSD_CUDA_CHECK(h, launch_pdl(lm_head_tc_kernel, dim3(grid), dim3(kThreads), smem, stream, 1, tmA, tmW, p));
+    CTCSD_CUDA_CHECK(h, launch_pdl(lm_head_tc_kernel<0>, dim3(grid), dim3(kThreads), smem, stream, 1, tmA, tmW, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

@@ -15,4 +15,13 @@ bool lm_head_tc_supported(const Handle* h);
 int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, const void* Wl,
                       int* out_argmax, float* out_logits_dbg, const AcceptParams& acc);
 
+// Draft head on the tensor cores for more than 8 activation rows: the same weight-stream kernel
+// with a per-row online (max, sum of exp, best-8) epilogue per vocabulary tile and a merge
+// kernel over the tiles of every slot.
+bool draft_head_tc_supported(const Handle* h, int M);
+int draft_tc_tile_rows(int classes);
+int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, const void* Wd, const int* row_seq,
+                         const float* blank_bias, int* out_topk_id, float* out_topk_lp, float* out_lse,
+                         float* out_logits_dbg);
+
 }  // namespace ctcsd
