@@ -52,6 +52,16 @@ def test_many_draft_rows_with_row_and_sel_maps():
     _run(cfg, seed=2, M=11, row_seq=row_seq, sel_row=sel_row)
 
 
+def test_draft_head_on_every_tree_row_uses_several_row_tiles():
+    # the "draft head on all tree rows" variant: 5 sequences x 64 tree rows = 320 draft rows (three
+    # 128-row tiles of the tensor-core path), each sequence drafting from one of its own rows
+    cfg = SMALL["c5s"]
+    M = cfg.B * cfg.max_nodes
+    row_seq = (np.arange(M) // cfg.max_nodes).astype(np.int32)
+    sel_row = np.array([b * cfg.max_nodes + (7 * b + 3) % cfg.max_nodes for b in range(cfg.B)], dtype=np.int32)
+    _run(cfg, seed=1, M=M, row_seq=row_seq, sel_row=sel_row, draft_rows=[0, 127, 128, 200, 319])
+
+
 def test_enumeration_limits_and_max_score_mode():
     # 4096 paths (T=6, k=4) enumerated exhaustively; best-alignment scoring variant
     _run(C["c1"].replace(name="enum4096", T=6, k=4, topN=64, max_nodes=128), seed=0)
