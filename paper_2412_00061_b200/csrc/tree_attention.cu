@@ -116,6 +116,9 @@ extern "C" int ctcsd_tree_attention(ctcsd_handle* hh, void* stream, const void* 
     p.scale = scale;
     p.status = status_ptr(h);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (c.dtype == CTCSD_DTYPE_BF16) return launch_tree_attention_mma(h, s, p);
+    if (c.dtype == CTCSD_DTYPE_BF16) {
+        if (tree_attention_tc_supported(p)) return launch_tree_attention_tc(h, s, p);
+        return launch_tree_attention_mma(h, s, p);
+    }
     return launch_simple<float>(h, s, p);
 }

@@ -18,7 +18,11 @@ struct AttnParams {
     int* status;
 };
 
-// bf16 tensor-core path (flash-style, KV split across CTAs, GQA head grouping).
+// bf16 on tcgen05 / tensor memory (128-row query tiles; needs Hq/Hkv to divide 128).
+bool tree_attention_tc_supported(const AttnParams& p);
+int launch_tree_attention_tc(Handle* h, cudaStream_t s, const AttnParams& p);
+
+// bf16 on the warp-level tensor-core instructions (64-row query tiles; any head grouping).
 int launch_tree_attention_mma(Handle* h, cudaStream_t s, const AttnParams& p);
 
 // The same kernels with caller-chosen scratch: `part` holds B*Hq*max_nodes*splits*(D+2) floats.

@@ -1,0 +1,485 @@
+// Tree attention for bf16 on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// Work decomposition: CTA = (128 query rows, one KV split, kv head g, sequence b).  Query row
+// r of kv head g is (node i = r / grp, query head g*grp + r % grp), so all query heads that
+// share a kv head use the same K/V tiles (GQA grouping).  Per tile of 128 keys:
+//   S[128 x 128] = Q K^T        tcgen05.mma, both operands K-major from shared memory (TMA,
+//                               128-byte swizzle), accumulator in tensor memory;
+//   softmax                     four warps, one thread per query row: the row is read from
+//                               tensor memory twice (max, then exp2 and sum), the ancestor mask
+//                               is applied to the columns that are tree nodes, P goes to shared
+//                               memory as bf16 in the K-major swizzled layout;
+//   O_tile[128 x D] = P V       tcgen05.mma with V as an MN-major operand (V is [key][d]);
+//   O = O * corr + O_tile       in the row's registers.
+// Warp 0 issues the TMA loads (Q once, K/V tiles into a two-stage ring), warp 1 issues the
+// MMAs, warps 2..5 are the softmax warps.  The KV splits of a query tile form a thread-block
+// cluster and merge their (max, sum, O) rows through distributed shared memory.
+#include "tree_attention.cuh"
+#include "tc_primitives.cuh"
+
+#include <math.h>
+#include <string.h>
+
+namespace ctcsd {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kRows = 128;         // query rows per CTA
+constexpr int kKeys = 128;         // keys per tile
+constexpr int kStages = 2;         // K/V tile buffers
+
+struct __align__(8) AttnShared {
+    uint64_t q_full;
+    uint64_t full[kStages];        // K and V tile landed
+    uint64_t empty[kStages];       // both MMAs of the tile have read it
+    uint64_t s_full;               // S is in tensor memory
+    uint64_t p_full;               // P is in shared memory (and S has been read)
+    uint64_t o_full;               // O_tile is in tensor memory
+    uint32_t tmem_base;
+    int abort_flag;
+    int never_set;
+};
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float2 ld_cluster_v2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                         const __grid_constant__ CUtensorMap tmV, AttnParams p, int splits) {
+    constexpr int DH = D / 64;                     // 64-column halves of a row of D elements
+    constexpr int kQBytes = kRows * D * 2;
+    constexpr int kTileBytes = kKeys * D * 2;      // one K or V tile
+    constexpr int kPBytes = kRows * kKeys * 2;
+    constexpr int RS = D + 4;                      // floats per row of the merge buffer
+    constexpr int PER = D / 32;
+    extern __shared__ unsigned char dyn_raw[];
+    const uint32_t raw_addr = tc::smem_u32(dyn_raw);
+    unsigned char* dyn = dyn_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+    unsigned char* Qs = dyn;                                           // [DH][128 rows][128 B]
+    unsigned char* KV = Qs + kQBytes;                                  // [kStages][K tile | V tile]
+    unsigned char* Ps = KV + kStages * 2 * kTileBytes;                 // [2][128 rows][128 B]
+    AttnShared* sh = reinterpret_cast<AttnShared*>(Ps + kPBytes);
+
+    const int grp = p.Hq / p.Hkv;
+    const int qtile = blockIdx.x / splits, split = blockIdx.x - qtile * splits;
+    const int g = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int* abort_flag = &sh->abort_flag;
+
+    if (tid == 0) {
+        tc::mbar_init(&sh->q_full, 1);
+        for (int s = 0; s < kStages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
+        tc::mbar_init(&sh->s_full, 1);
+        tc::mbar_init(&sh->p_full, 4);
+        tc::mbar_init(&sh->o_full, 1);
+        sh->abort_flag = 0;
+        sh->never_set = 0;
+        tc::fence_barrier_init();
+    }
+    if (warp == 1) {
+        tc::tmem_alloc(&sh->tmem_base, 256);
+        tc::tmem_relinquish();
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_s = sh->tmem_base;               // S: columns 0..127
+    const uint32_t tmem_o = sh->tmem_base + 128;         // O_tile: columns 128..128+D-1
+
+    pdl_wait();                      // the tree (node count, mask) and Q/K/V come from preceding kernels
+    pdl_trigger();
+    int n = p.n_nodes[b];
+    const int L = p.kv_len[b];
+    if (n < 0 || n > p.max_nodes || L < 0 || L + n > p.Lcap) {
+        if (tid == 0) report_error(p.status, CTCSD_ERR_INVALID_ARG, b);
+        n = 0;
+    }
+    const int Ltot = L + n;
+    const int nblk = (Ltot + kKeys - 1) / kKeys;
+    const int blk0 = (int)((long long)nblk * split / splits);           // key tiles spread evenly over the splits
+    const int blk1 = (int)((long long)nblk * (split + 1) / splits);
+    const int ntile = blk1 - blk0;
+
+    // softmax state of the row owned by this thread (softmax warps only)
+    float acc[D];
+    float mx = -INFINITY, sum = 0.f;
+    bool failed = false;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && ntile > 0) {
+            tc::prefetch_tensormap(&tmQ);
+            tc::prefetch_tensormap(&tmK);
+            tc::prefetch_tensormap(&tmV);
+            const uint64_t pol = tc::policy_evict_last();
+            tc::mbar_arrive_expect_tx(&sh->q_full, (uint32_t)kQBytes);
+            for (int hh = 0; hh < DH; ++hh)
+                tc::tma_load_5d(Qs + hh * (kRows * 128), &tmQ, &sh->q_full, hh * 64, 0, g, qtile * (kRows / grp), b, pol);
+            int it = 0;
+            for (int blk = blk0; blk < blk1; ++blk, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { failed = true; break; }
+                unsigned char* kd = KV + (size_t)s * 2 * kTileBytes;
+                tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)(2 * kTileBytes));
+                for (int hh = 0; hh < DH; ++hh) {
+                    tc::tma_load_4d(kd + hh * (kKeys * 128), &tmK, &sh->full[s], hh * 64, blk * kKeys, g, b, pol);
+                    tc::tma_load_4d(kd + kTileBytes + hh * (kKeys * 128), &tmV, &sh->full[s], hh * 64, blk * kKeys, g, b, pol);
+                }
+            }
+            if (failed) {
+                if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 21);
+                *abort_flag = 1;
+                for (int back = 1; back <= kStages && back <= it; ++back) {
+                    const int j = it - back;
+                    tc::mbar_wait(&sh->full[j % kStages], (uint32_t)(j / kStages) & 1u, &sh->never_set, 1ll << 24);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && ntile > 0) {
+            const uint32_t idesc_s = tc::idesc_bf16_f32(kRows, kKeys);
+            const uint32_t idesc_o = tc::idesc_bf16_f32_b_mn(kRows, D);
+            bool ok = tc::mbar_wait(&sh->q_full, 0u, abort_flag);
+            for (int it = 0; it < ntile && ok; ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                if (!tc::mbar_wait(&sh->full[s], ph, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after_sync();
+                const uint32_t k_addr = tc::smem_u32(KV + (size_t)s * 2 * kTileBytes);
+                const uint32_t v_addr = k_addr + kTileBytes;
+                // S = Q K^T: D/16 steps of 16 elements along the head dimension
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t adesc = tc::smem_desc_k_sw128(tc::smem_u32(Qs) + (kk / 4) * (kRows * 128)) + 2 * (kk % 4);
+                    const uint64_t bdesc = tc::smem_desc_k_sw128(k_addr + (kk / 4) * (kKeys * 128)) + 2 * (kk % 4);
+                    tc::mma_bf16_ss(tmem_s, adesc, bdesc, idesc_s, kk != 0 ? 1u : 0u);
+                }
+                tc::mma_commit(&sh->s_full);
+                // O_tile = P V once the softmax warps have written P (they have then also read S)
+                if (!tc::mbar_wait(&sh->p_full, (uint32_t)it & 1u, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < kKeys / 16; ++kk) {
+                    const uint64_t adesc = tc::smem_desc_k_sw128(tc::smem_u32(Ps) + (kk / 4) * (kRows * 128)) + 2 * (kk % 4);
+                    // 16 keys further along K = 16 rows of 128 bytes
+                    const uint64_t bdesc = tc::smem_desc_mn_sw128(v_addr + kk * (16 * 128), kKeys * 128);
+                    tc::mma_bf16_ss(tmem_o, adesc, bdesc, idesc_o, kk != 0 ? 1u : 0u);
+                }
+                tc::mma_commit(&sh->o_full);
+                tc::mma_commit(&sh->empty[s]);
+            }
+            if (!ok) {
+                if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 22);
+                *abort_flag = 1;
+            }
+        }
+    } else {
+        // ---------------- softmax warps: thread = query row ----------------
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int rl = q * 32 + lane;                 // row of the tile
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        const int r = qtile * kRows + rl;
+        const int i = r / grp;                        // tree node of the row
+        const bool live = i < n;
+        const int W = (p.max_nodes + 63) / 64;
+        unsigned long long m0 = 0, m1 = 0;
+        if (live) {
+            const unsigned long long* m = p.mask + ((size_t)b * p.max_nodes + i) * W;
+            m0 = m[0];
+            if (W > 1) m1 = m[1];
+        }
+#pragma unroll
+        for (int d = 0; d < D; ++d) acc[d] = 0.f;
+        const float sl2 = p.scale * 1.4426950408889634f;          // scores are kept in log2 units
+        for (int it = 0; it < ntile; ++it) {
+            const int key0 = (blk0 + it) * kKeys;
+            const int s = it % kStages;
+            if (!tc::mbar_wait(&sh->s_full, (uint32_t)it & 1u, abort_flag)) { failed = true; break; }
+            tc::tc_fence_after_sync();
+            const bool tail = key0 + kKeys > L;       // the tile holds tree nodes or keys past the end
+            // V rows past the last key may hold anything (the cache is only written up to there):
+            // clear them, a zero weight does not cancel a NaN
+            if (key0 + rl >= Ltot) {
+                unsigned char* vrow = KV + (size_t)s * 2 * kTileBytes + kTileBytes + rl * 128;
+#pragma unroll
+                for (int hh = 0; hh < DH; ++hh)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4*>(vrow + hh * (kKeys * 128) + c * 16) = make_uint4(0, 0, 0, 0);
+            }
+            auto visible = [&](int key) -> bool {
+                if (key < L) return live;
+                const int tn = key - L;
+                const unsigned long long w = tn < 64 ? m0 : m1;
+                return live && key < Ltot && ((w >> (tn & 63)) & 1ull);
+            };
+            // pass 1: row maximum
+            float bm = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kKeys; c0 += 32) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
+                tc::tmem_ld_wait();
+                if (!tail) {
+                    if (live) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) bm = fmaxf(bm, __uint_as_float(v[j]));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (visible(key0 + c0 + j)) bm = fmaxf(bm, __uint_as_float(v[j]));
+                }
+            }
+            bm *= sl2;                                 // scale > 0: the maximum commutes with it
+            const float nm = fmaxf(mx, bm);
+            const float ref = nm == -INFINITY ? 0.f : nm;
+            const float corr = exp2f(mx - ref);        // exp2(-inf) = 0
+            mx = nm;
+            // pass 2: P = exp2(S - max), row sum, P to shared memory as bf16 (K-major, 128-byte swizzle)
+            float ps = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kKeys; c0 += 32) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
+                tc::tmem_ld_wait();
+                float pv[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const bool vis = tail ? visible(key0 + c0 + j) : live;
+                    const float e = exp2f(fmaf(__uint_as_float(v[j]), sl2, -ref));
+                    pv[j] = vis ? e : 0.f;
+                    ps += pv[j];
+                }
+                unsigned char* prow = Ps + (c0 / 64) * (kRows * 128) + rl * 128;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint4 w;
+                    w.x = pack_bf16(pv[8 * c + 0], pv[8 * c + 1]);
+                    w.y = pack_bf16(pv[8 * c + 2], pv[8 * c + 3]);
+                    w.z = pack_bf16(pv[8 * c + 4], pv[8 * c + 5]);
+                    w.w = pack_bf16(pv[8 * c + 6], pv[8 * c + 7]);
+                    const int chunk = (c0 % 64) / 8 + c;
+                    *reinterpret_cast<uint4*>(prow + ((chunk ^ (rl & 7)) << 4)) = w;
+                }
+            }
+            sum = sum * corr + ps;
+            // make P (and the cleared V rows) visible to the tensor core, then hand over
+            tc::fence_proxy_async();
+            tc::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&sh->p_full);
+            // O = O * corr + O_tile
+            if (!tc::mbar_wait(&sh->o_full, (uint32_t)it & 1u, abort_flag)) { failed = true; break; }
+            tc::tc_fence_after_sync();
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_o + lane_off + (uint32_t)c0, v);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[c0 + j] = fmaf(acc[c0 + j], corr, __uint_as_float(v[j]));
+            }
+            tc::tc_fence_before_sync();
+        }
+        if (failed && lane == 0) {
+            if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 23);
+            *abort_flag = 1;
+        }
+    }
+
+    // ---------------- output ----------------
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc::tc_fence_after_sync();
+        tc::tmem_dealloc(sh->tmem_base, 256);
+    }
+    const bool good = sh->abort_flag == 0;
+    if (splits == 1) {
+        if (warp >= 2 && good) {
+            const int rl = (warp & 3) * 32 + lane;
+            const int r = qtile * kRows + rl;
+            const int i = r / grp;
+            if (i < p.max_nodes) {
+                const int hq = g * grp + (r - i * grp);
+                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.O) + (((size_t)b * p.max_nodes + i) * p.Hq + hq) * D;
+                const float inv = (i < n && sum > 0.f) ? 1.f / sum : 0.f;
+#pragma unroll
+                for (int c = 0; c < D / 8; ++c) {
+                    uint4 w;
+                    w.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
+                    w.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
+                    w.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
+                    w.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
+                    reinterpret_cast<uint4*>(out)[c] = w;
+                }
+            }
+        }
+        return;
+    }
+    // several KV splits: every CTA leaves its rows (unnormalised O, max, sum) in its shared memory
+    // (the K/V tiles are no longer needed) and merges rows split, split + splits, ... of all CTAs
+    float* rowbuf = reinterpret_cast<float*>(KV);
+    if (warp >= 2) {
+        const int rl = (warp & 3) * 32 + lane;
+        float* dst = rowbuf + rl * RS;
+#pragma unroll
+        for (int c = 0; c < D / 4; ++c)
+            *reinterpret_cast<float4*>(dst + 4 * c) = make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+        dst[D] = mx;
+        dst[D + 1] = sum;
+    }
+    cluster_sync_all();
+    const uint32_t base = tc::smem_u32(rowbuf);
+    for (int rl = split + splits * warp; rl < kRows && good; rl += splits * (kThreads / 32)) {
+        const int r = qtile * kRows + rl;
+        const int i = r / grp;
+        if (i >= p.max_nodes) continue;                         // padding rows of the last query tile
+        const int hq = g * grp + (r - i * grp);
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.O) + (((size_t)b * p.max_nodes + i) * p.Hq + hq) * D;
+        float o[PER], tot = 0.f;
+#pragma unroll
+        for (int d = 0; d < PER; ++d) o[d] = 0.f;
+        if (i < n) {                                            // uniform over the warp
+            // lane c fetches split c's (max, sum); the row loads below do not depend on one another
+            float m_l = -INFINITY, l_l = 0.f;
+            if (lane < splits) {
+                const float2 ml = ld_cluster_v2(map_to_cta(base + (uint32_t)(rl * RS + D) * 4u, (uint32_t)lane));
+                m_l = ml.x;
+                l_l = ml.y;
+            }
+            const float gm = warp_max(m_l);
+            const float w_l = (m_l == -INFINITY) ? 0.f : exp2f(m_l - gm);
+            tot = warp_sum(w_l * l_l);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                if (c < splits) {
+                    const float w = __shfl_sync(0xffffffffu, w_l, c);
+                    const uint32_t rowaddr = map_to_cta(base + (uint32_t)(rl * RS) * 4u, (uint32_t)c);
+                    if constexpr (PER == 4) {
+                        const float4 v = ld_cluster_v4(rowaddr + (uint32_t)lane * 16u);
+                        o[0] += w * v.x; o[1] += w * v.y; o[2] += w * v.z; o[3] += w * v.w;
+                    } else {
+                        const float2 v = ld_cluster_v2(rowaddr + (uint32_t)lane * 8u);
+                        o[0] += w * v.x; o[1] += w * v.y;
+                    }
+                }
+            }
+        }
+        const float inv = tot > 0.f ? 1.f / tot : 0.f;
+        if constexpr (PER == 4) {
+            uint2 pk;
+            pk.x = pack_bf16(o[0] * inv, o[1] * inv);
+            pk.y = pack_bf16(o[2] * inv, o[3] * inv);
+            *reinterpret_cast<uint2*>(out + 4 * lane) = pk;
+        } else {
+            *reinterpret_cast<uint32_t*>(out + 2 * lane) = pack_bf16(o[0] * inv, o[1] * inv);
+        }
+    }
+    // nobody may leave while a peer can still read its shared memory
+    cluster_sync_all();
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+    if (qres != cudaDriverEntryPointSuccess) return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(sym);
+    return fn;
+}
+
+// bf16 tensor of rank `rank`: dims[0] is the contiguous axis, strides[] in bytes for dims 1..;
+// box[0] = 64 elements (one 128-byte swizzle row); out-of-range elements read as zero.
+bool make_map_nd(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
+                 const cuuint32_t* box) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <int D>
+int launch_tc(Handle* h, cudaStream_t s, const AttnParams& p) {
+    const int grp = p.Hq / p.Hkv;
+    const int rows_total = p.max_nodes * grp;
+    const int qtiles = (rows_total + kRows - 1) / kRows;
+    // KV splits as a portable cluster size, all CTAs in one wave (clusters of 8 schedule badly here)
+    const long long units = (long long)p.B * p.Hkv * qtiles;
+    int splits = 1;
+    while (splits < 4 && units * splits * 2 <= (long long)h->num_sms) splits *= 2;
+
+    CUtensorMap tmQ, tmK, tmV;
+    {   // Q [B][max_nodes][Hkv][grp][D]: box = 64 columns x grp heads x 1 kv head x 128/grp nodes x 1 sequence
+        cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)grp, (cuuint64_t)p.Hkv, (cuuint64_t)p.max_nodes, (cuuint64_t)p.B};
+        cuuint64_t str[4] = {(cuuint64_t)D * 2, (cuuint64_t)grp * D * 2, (cuuint64_t)p.Hq * D * 2,
+                             (cuuint64_t)p.max_nodes * p.Hq * D * 2};
+        cuuint32_t box[5] = {64, (cuuint32_t)grp, 1, (cuuint32_t)(kRows / grp), 1};
+        if (!make_map_nd(&tmQ, p.Q, 5, dims, str, box)) return CTCSD_ERR_CUDA;
+    }
+    {   // K, V [B][Hkv][Lcap][D]: box = 64 columns x 128 keys
+        cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)p.Lcap, (cuuint64_t)p.Hkv, (cuuint64_t)p.B};
+        cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)p.Lcap * D * 2, (cuuint64_t)p.Hkv * p.Lcap * D * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)kKeys, 1, 1};
+        if (!make_map_nd(&tmK, p.K, 4, dims, str, box)) return CTCSD_ERR_CUDA;
+        if (!make_map_nd(&tmV, p.V, 4, dims, str, box)) return CTCSD_ERR_CUDA;
+    }
+    const size_t smem = (size_t)kRows * D * 2 + (size_t)kStages * 2 * kKeys * D * 2 + (size_t)kRows * kKeys * 2 +
+                        sizeof(AttnShared) + 1024;
+    auto kern = tree_attention_tc_kernel<D>;
+    CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    CTCSD_CUDA_CHECK(h, launch_pdl(kern, dim3(qtiles * splits, p.Hkv, p.B), dim3(kThreads), smem, s, splits,
+                                   tmQ, tmK, tmV, p, splits));
+    h->launches++;
+    return CTCSD_OK;
+}
+
+}  // namespace
+
+bool tree_attention_tc_supported(const AttnParams& p) {
+    const int grp = p.Hq / p.Hkv;
+    if (grp < 1 || grp > kRows || (kRows % grp) != 0) return false;      // a query tile holds whole nodes
+    if ((reinterpret_cast<uintptr_t>(p.Q) | reinterpret_cast<uintptr_t>(p.K) | reinterpret_cast<uintptr_t>(p.V)) & 15) return false;
+    return p.D == 64 || p.D == 128;
+}
+
+int launch_tree_attention_tc(Handle* h, cudaStream_t s, const AttnParams& p) {
+    if (!tree_attention_tc_supported(p)) return CTCSD_ERR_UNSUPPORTED;
+    if (p.D == 64) return launch_tc<64>(h, s, p);
+    return launch_tc<128>(h, s, p);
+}
+
+}  // namespace ctcsd
