@@ -230,11 +230,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                     for (int c = 0; c < 8; ++c)
                         *reinterpret_cast<uint4*>(vrow + hh * (kKeys * 128) + c * 16) = make_uint4(0, 0, 0, 0);
             }
-            auto visible = [&](int key) -> bool {
-                if (key < L) return live;
-                const int tn = key - L;
-                const unsigned long long w = tn < 64 ? m0 : m1;
-                return live && key < Ltot && ((w >> (tn & 63)) & 1ull);
+            // visibility of the 32 keys key0 + c0 .. + 31 for this row as a bit mask: cached keys are
+            // visible to every live row, tree node t only if the row's ancestor mask has bit t (bits
+            // of nodes past the tree are never set, so keys past the end come out invisible)
+            auto visible32 = [&](int c0) -> uint32_t {
+                if (!live) return 0u;
+                if (!tail) return 0xffffffffu;
+                const int t0 = key0 + c0 - L;                   // tree index of the chunk's first key
+                if (t0 <= -32) return 0xffffffffu;
+                if (t0 < 0) return (uint32_t)((m0 << (-t0)) | ((1ull << (-t0)) - 1ull));
+                if (t0 < 64) return (uint32_t)((m0 >> t0) | (t0 ? (m1 << (64 - t0)) : 0ull));
+                if (t0 < 128) return (uint32_t)(m1 >> (t0 - 64));
+                return 0u;
             };
             // pass 1: row maximum
             float bm = -INFINITY;
@@ -242,17 +249,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             for (int c0 = 0; c0 < kKeys; c0 += 32) {
                 uint32_t v[32];
                 tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
+                const uint32_t vm = visible32(c0);
                 tc::tmem_ld_wait();
-                if (!tail) {
-                    if (live) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) bm = fmaxf(bm, __uint_as_float(v[j]));
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (visible(key0 + c0 + j)) bm = fmaxf(bm, __uint_as_float(v[j]));
-                }
+                for (int j = 0; j < 32; ++j)
+                    if ((vm >> j) & 1u) bm = fmaxf(bm, __uint_as_float(v[j]));
             }
             bm *= sl2;                                 // scale > 0: the maximum commutes with it
             const float nm = fmaxf(mx, bm);
@@ -266,12 +267,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 uint32_t v[32];
                 tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
                 tc::tmem_ld_wait();
+                const uint32_t vm = visible32(c0);
                 float pv[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const bool vis = tail ? visible(key0 + c0 + j) : live;
                     const float e = exp2f(fmaf(__uint_as_float(v[j]), sl2, -ref));
-                    pv[j] = vis ? e : 0.f;
+                    pv[j] = ((vm >> j) & 1u) ? e : 0.f;
                     ps += pv[j];
                 }
                 unsigned char* prow = Ps + (c0 / 64) * (kRows * 128) + rl * 128;
