@@ -58,6 +58,12 @@ __device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr) {
     asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
 }
+// 2^x for x <= 0 (the softmax exponent is never positive): the hardware approximation, no range fix-up
+__device__ __forceinline__ float exp2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -244,7 +250,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 return 0u;
             };
             // pass 1: row maximum
-            float bm = -INFINITY;
+            float bm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four chains instead of one
 #pragma unroll 1
             for (int c0 = 0; c0 < kKeys; c0 += 32) {
                 uint32_t v[32];
@@ -253,15 +259,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                    if ((vm >> j) & 1u) bm = fmaxf(bm, __uint_as_float(v[j]));
+                    if ((vm >> j) & 1u) bm4[j & 3] = fmaxf(bm4[j & 3], __uint_as_float(v[j]));
             }
+            float bm = fmaxf(fmaxf(bm4[0], bm4[1]), fmaxf(bm4[2], bm4[3]));
             bm *= sl2;                                 // scale > 0: the maximum commutes with it
             const float nm = fmaxf(mx, bm);
             const float ref = nm == -INFINITY ? 0.f : nm;
-            const float corr = exp2f(mx - ref);        // exp2(-inf) = 0
+            const float corr = exp2_fast(mx - ref);    // exp2(-inf) = 0
             mx = nm;
             // pass 2: P = exp2(S - max), row sum, P to shared memory as bf16 (K-major, 128-byte swizzle)
-            float ps = 0.f;
+            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
             for (int c0 = 0; c0 < kKeys; c0 += 32) {
                 uint32_t v[32];
@@ -271,9 +278,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 float pv[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const float e = exp2f(fmaf(__uint_as_float(v[j]), sl2, -ref));
+                    const float e = exp2_fast(fmaf(__uint_as_float(v[j]), sl2, -ref));
                     pv[j] = ((vm >> j) & 1u) ? e : 0.f;
-                    ps += pv[j];
+                    ps4[j & 3] += pv[j];
                 }
                 unsigned char* prow = Ps + (c0 / 64) * (kRows * 128) + rl * 128;
 #pragma unroll
@@ -287,7 +294,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                     *reinterpret_cast<uint4*>(prow + ((chunk ^ (rl & 7)) << 4)) = w;
                 }
             }
-            sum = sum * corr + ps;
+            sum = sum * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
             // make P (and the cleared V rows) visible to the tensor core, then hand over
             tc::fence_proxy_async();
             tc::tc_fence_before_sync();
@@ -440,8 +447,20 @@ int launch_tc(Handle* h, cudaStream_t s, const AttnParams& p) {
     const int qtiles = (rows_total + kRows - 1) / kRows;
     // KV splits as a portable cluster size, all CTAs in one wave (clusters of 8 schedule badly here)
     const long long units = (long long)p.B * p.Hkv * qtiles;
+    // (1, 2 or 4: clusters of 8 schedule badly here).  The CTAs run in waves of one per SM; pick
+    // the smallest split count whose waves are within 10 % of the shortest total.
     int splits = 1;
-    while (splits < 4 && units * splits * 2 <= (long long)h->num_sms) splits *= 2;
+    {
+        double best = 1e30;
+        double cost[3];
+        for (int e = 0; e < 3; ++e) {
+            const long long ctas = units << e;
+            cost[e] = (double)((ctas + h->num_sms - 1) / h->num_sms) / (double)(1 << e) + 0.15 * e;   // a split costs a cluster merge
+            if (cost[e] < best) best = cost[e];
+        }
+        for (int e = 0; e < 3; ++e)
+            if (cost[e] <= best * 1.10) { splits = 1 << e; break; }
+    }
 
     CUtensorMap tmQ, tmK, tmV;
     {   // Q [B][max_nodes][Hkv][grp][D]: box = 64 columns x grp heads x 1 kv head x 128/grp nodes x 1 sequence
