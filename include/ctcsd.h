@@ -95,6 +95,12 @@ int ctcsd_destroy(ctcsd_handle* h);
  * receives CTCSD_OK or the first error a kernel recorded. */
 int ctcsd_poll_status(ctcsd_handle* h, void* stream, int* out_status);
 
+/* Self-test of the failure path: enqueues a kernel that waits, with the bounded wait all
+ * streaming kernels use, on a barrier nothing ever signals.  The wait gives up after about a
+ * millisecond and records CTCSD_ERR_TIMEOUT in the device status word (ctcsd_poll_status then
+ * returns it and clears it); the context stays usable. */
+int ctcsd_selftest_timeout(ctcsd_handle* h, void* stream);
+
 /* Text for a status code; never NULL.  The string is static. */
 const char* ctcsd_strerror(int status);
 

@@ -21,7 +21,7 @@ SCORE_SUM, SCORE_MAX = 0, 1
 
 EXPORTS = [
     "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
-    "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch",
+    "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
     "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static",
 ]
@@ -58,6 +58,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_strerror.restype = ctypes.c_char_p
     lib.ctcsd_last_cuda_error.argtypes = [vp]
     lib.ctcsd_set_l2_prefetch.argtypes = [vp, vp, cs]
+    lib.ctcsd_selftest_timeout.argtypes = [vp, vp]
     lib.ctcsd_launch_count.argtypes = [vp]
     lib.ctcsd_launch_count.restype = ctypes.c_longlong
     lib.ctcsd_draft_logits.argtypes = [vp, vp, ci] + [vp] * 8
@@ -146,6 +147,9 @@ class Handle:
             return
         nbytes = min(int(nbytes), tensor.numel() * tensor.element_size())
         self._check(self.lib.ctcsd_set_l2_prefetch(self._h, _ptr(tensor, name="prefetch"), nbytes), "set_l2_prefetch")
+
+    def selftest_timeout(self, stream=None):
+        self._check(self.lib.ctcsd_selftest_timeout(self._h, _stream_ptr(stream)), "selftest_timeout")
 
     def poll_status(self, stream=None) -> int:
         st = ctypes.c_int(0)

@@ -155,3 +155,40 @@ extern "C" const char* ctcsd_strerror(int status) {
 extern "C" int ctcsd_last_cuda_error(const ctcsd_handle* h) { return h ? h->h.last_cuda_error : 0; }
 
 extern "C" long long ctcsd_launch_count(const ctcsd_handle* h) { return h ? h->h.launches : 0; }
+
+// ---------------------------------------------------------------------------------------
+// Self-test of the bounded-wait machinery
+// ---------------------------------------------------------------------------------------
+#include "tc_primitives.cuh"
+
+namespace ctcsd {
+namespace {
+
+// Waits on an mbarrier that nothing ever arrives on, with the same bounded wait the streaming
+// kernels use but a short limit, and records the outcome the way they do.
+__global__ void __launch_bounds__(32) selftest_timeout_kernel(int* status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int never_set;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        never_set = 0;
+        tc::fence_barrier_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        const bool done = tc::mbar_wait(&bar, 0u, &never_set, limit_cycles);
+        if (!done) report_error(status, CTCSD_ERR_TIMEOUT, 99);
+    }
+}
+
+}  // namespace
+}  // namespace ctcsd
+
+extern "C" int ctcsd_selftest_timeout(ctcsd_handle* hh, void* stream) {
+    if (!hh) return CTCSD_ERR_INVALID_ARG;
+    Handle* h = &hh->h;
+    // about a millisecond at 2 GHz: long enough to be a real wait, short enough for a test
+    selftest_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status_ptr(h), 2000000ll);
+    CTCSD_LAUNCH_CHECK(h);
+    return CTCSD_OK;
+}

@@ -123,6 +123,22 @@ def test_history_update_moves_the_accepted_rows(name):
     assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
 
 
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
+    """Failure detection without a fault: a bounded device-side wait on a barrier that nothing
+    signals gives up, the status word says CTCSD_ERR_TIMEOUT, polling clears it, and the same
+    handle then runs a full step that matches the oracle."""
+    r = _run(C["c1"], seed=1)
+    step = r["step"]
+    before = {k: step.host(k).copy() for k in ("cand_tok", "node_tok", "argmax", "acc_len")}
+    step.h.selftest_timeout()
+    assert step.h.poll_status() == -5
+    assert step.h.poll_status() == 0
+    step.run()
+    step.check_status()
+    for k, v in before.items():
+        np.testing.assert_array_equal(step.host(k), v)
+
+
 def test_invalid_arguments_are_rejected_on_the_host():
     import ctypes
     from paper_2412_00061_b200 import binding
