@@ -417,11 +417,11 @@ int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     if (budget > 208 * 1024) budget = 208 * 1024;
     const size_t fixed = (size_t)MROWS * (row_bytes + 64) + sizeof(RingShared);
     // rows per ring slot: copies of about 64 KB keep the copy engine busiest (its cost per copy is
-    // large), as long as at least three slots fit
+    // large), as long as at least two slots fit (two 64 KB slots stream as fast as three)
     int G = (int)((64 * 1024) / row_bytes);
     if (G < 1) G = 1;
     if (G > kWarps * kRowsPerWarp) G = kWarps * kRowsPerWarp;
-    while (G > 1 && fixed + 3 * (size_t)G * row_bytes > budget) --G;
+    while (G > 1 && fixed + 2 * (size_t)G * row_bytes > budget) --G;
     const size_t slot_bytes = (size_t)G * row_bytes;
     if (fixed + slot_bytes > budget) return CTCSD_ERR_UNSUPPORTED;
     long long nslots = (long long)((budget - fixed) / slot_bytes);
