@@ -301,12 +301,12 @@ def run_ours(args):
     draft_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(d_beg, d_end)]))
 
     # ---- end to end: per-step inputs come from pinned host memory, results go back ------
-    act = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
-    pin = lambda t: t.cpu().pin_memory()
-    h_in = {k: pin(step.inp[k]) for k in ("x", "base_tok", "kv_len", "Q", "hn")}
-    h_out = {k: torch.empty_like(step.out[k], device="cpu").pin_memory() for k in ("acc_len", "acc_tok", "next_tok")}
-    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
-    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+    # the per-step inputs (x, base token, cache length, tree queries, tree-node hidden states) sit in
+    # one device buffer and the results in another: one copy each way per step
+    h_in = step.pack_step_inputs()
+    h_out = torch.empty_like(step.result, device="cpu").pin_memory()
+    h2d = h_in.numel() * h_in.element_size()
+    d2h = h_out.numel() * h_out.element_size()
 
     graph1 = None
     if use_graph:
@@ -318,14 +318,12 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def e2e_step():
-        for k, t in h_in.items():
-            step.inp[k].copy_(t, non_blocking=True)
+        step.upload(h_in)
         if graph1 is not None:
             graph1.replay()
         else:
             step.run()
-        for k, t in h_out.items():
-            t.copy_(step.out[k], non_blocking=True)
+        step.download(h_out)
         torch.cuda.synchronize()
 
     for _ in range(3):

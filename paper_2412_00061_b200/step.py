@@ -43,9 +43,18 @@ class DraftVerifyStep:
             node_tok=z(B, n), parent=z(B, n), depth=z(B, n), pos=z(B, n),
             mask=z(B, n, W, dtype=torch.int64), retrieve=z(B, N, T), n_nodes=z(B),
             O=z(B, n, cfg.Hq, cfg.D, dtype=act),
-            argmax=z(B, n), acc_len=z(B), acc_nodes=z(B, T), acc_tok=z(B, T), next_tok=z(B),
-            new_kv_len=z(B), next_sel_row=z(B),
+            argmax=z(B, n),
         )
+        # the step's results share one buffer, so that reading them back is a single copy
+        names = [("acc_len", (B,)), ("acc_nodes", (B, T)), ("acc_tok", (B, T)), ("next_tok", (B,)),
+                 ("new_kv_len", (B,)), ("next_sel_row", (B,))]
+        self.result = z(sum(int(np.prod(sh)) for _, sh in names))
+        off = 0
+        for nm, sh in names:
+            cnt = int(np.prod(sh))
+            self.out[nm] = self.result[off:off + cnt].view(*sh)
+            off += cnt
+        self.input_arena = None
         if debug_logits:
             self.out["draft_logits_dbg"] = z(self.M, T, cfg.V + 1, dtype=f32)
             self.out["lm_logits_dbg"] = z(B * n, cfg.V, dtype=f32)
@@ -58,6 +67,34 @@ class DraftVerifyStep:
             # while the small kernels between draft head and LM head run, HBM is idle: let L2
             # fetch the head of the LM-head weights then
             self.h.set_l2_prefetch(tensors["Wl"], self.L2_PREFETCH_BYTES)
+
+    PER_STEP_INPUTS = ("x", "base_tok", "kv_len", "Q", "hn")
+
+    def pack_step_inputs(self):
+        """Moves the tensors that change every step (hidden state, base token, cache length, tree
+        queries, tree-node hidden states) into one device buffer, 256-byte aligned each, so that a
+        step's host-to-device traffic is a single copy.  Returns a pinned host mirror of that
+        buffer holding the current values; upload() copies a mirror to the device."""
+        sizes = []
+        for k in self.PER_STEP_INPUTS:
+            t = self.inp[k]
+            sizes.append((k, t, (t.numel() * t.element_size() + 255) // 256 * 256))
+        self.input_arena = torch.empty(sum(sz for _, _, sz in sizes), dtype=torch.uint8, device=self.device)
+        off = 0
+        for k, t, sz in sizes:
+            nbytes = t.numel() * t.element_size()
+            view = self.input_arena[off:off + nbytes].view(t.dtype).view(t.shape)
+            view.copy_(t)
+            self.inp[k] = view
+            off += sz
+        torch.cuda.synchronize(self.device)
+        return self.input_arena.cpu().pin_memory()
+
+    def upload(self, host_arena: torch.Tensor):
+        self.input_arena.copy_(host_arena, non_blocking=True)
+
+    def download(self, host_result: torch.Tensor):
+        host_result.copy_(self.result, non_blocking=True)
 
     # individual stages ----------------------------------------------------------------
     def draft(self, stream=None):
