@@ -375,3 +375,110 @@ def commit_accepted(K: np.ndarray, Vc: np.ndarray, kv_len: np.ndarray, acc_len: 
         new_len[b] = L + 1 + int(acc_len[b])
         sel_row[b] = b * max_nodes + last
     return K2, V2, new_len, sel_row
+
+
+# --------------------------------------------------------------------------------------
+# The paper's own verification layout (Sec. 3.1 "CTC Transform Module", Sec. 3.3): the raw,
+# fixed-length slot paths stay in the token tree; the tokens that the CTC transform removes
+# (blanks, and repeats of the previous slot's symbol) are masked out of the attention map
+# instead of being dropped from the tree.
+# --------------------------------------------------------------------------------------
+def select_raw_paths(topk_id: np.ndarray, topk_lp: np.ndarray, N: int):
+    """The N most probable slot paths of one sequence ("a group of the most valuable combinations
+    are reserved as the raw candidate sequences", Sec. 3.3): path probability = product over the
+    slots (Eq. 6); equal scores go to the path that is first when the per-slot ranks are read as
+    a number (slot 1 most significant).  topk_id/topk_lp [T,k] -> (raw_tok [n,T], score [n])."""
+    T, k = topk_id.shape
+    paths = []
+    for idx, a in enumerate(itertools.product(range(k), repeat=T)):
+        s = 0.0
+        for t in range(T):
+            s += float(topk_lp[t, a[t]])
+        paths.append((-s, idx, a))
+    paths.sort(key=lambda e: (e[0], e[1]))
+    keep = paths[:N]
+    raw = np.array([[int(topk_id[t, a[t]]) for t in range(T)] for _, _, a in keep], dtype=np.int64).reshape(len(keep), T)
+    score = np.array([-ns for ns, _, _ in keep], dtype=np.float64)
+    return raw, score
+
+
+def build_raw_tree(base_tok: np.ndarray, kv_len: np.ndarray, raw_tok: np.ndarray, n_raw: np.ndarray,
+                   blank: int, n_max: int):
+    """Token tree over the raw paths raw_tok [B,N,T] (symbols include the blank).  The trie is
+    the one build_tree makes; on top of it:
+      kept[i]   - node i survives the CTC transform: its symbol is not the blank and differs from
+                  its parent's symbol (the root, which holds the base token, is not part of the
+                  alignment: a first-slot symbol is kept iff it is not the blank; the root is kept);
+      mask[i]   - bit j set iff j is the root or a kept ancestor of i, or j == i and i is kept
+                  (the removed tokens' positions are masked in the attention map);
+      pos[i]    - kv_len + number of kept non-root nodes on the path root..i;
+      nka[i]    - nearest kept proper ancestor of i (-1 for the root)."""
+    B, N, T = raw_tok.shape
+    raw_len = np.full((B, N), T, dtype=np.int64)
+    node_tok, parent, depth, _, anc, retrieve, n_nodes = build_tree(base_tok, kv_len, raw_tok, raw_len, n_raw, n_max)
+    W = (n_max + 63) // 64
+    kept = np.zeros((B, n_max), dtype=np.int64)
+    nka = np.full((B, n_max), -1, dtype=np.int64)
+    pos = np.zeros((B, n_max), dtype=np.int64)
+    mask = np.zeros((B, n_max, W), dtype=np.uint64)
+    for b in range(B):
+        for i in range(int(n_nodes[b])):
+            if i == 0:
+                kept[b, 0] = 1
+            else:
+                par = int(parent[b, i])
+                s = int(node_tok[b, i])
+                prev = None if par == 0 else int(node_tok[b, par])
+                kept[b, i] = 1 if (s != blank and s != prev) else 0
+            path = []
+            j = i
+            while j >= 0:
+                path.append(j)
+                j = int(parent[b, j])
+            count = 0
+            for j in path:
+                if j == 0 or kept[b, j]:
+                    mask[b, i, j // 64] |= np.uint64(1) << np.uint64(j % 64)
+                    if j != 0:
+                        count += 1
+            pos[b, i] = int(kv_len[b]) + count
+            for j in path[1:]:
+                if j == 0 or kept[b, j]:
+                    nka[b, i] = j
+                    break
+    return node_tok, parent, depth, pos, mask, retrieve, n_nodes, kept, nka
+
+
+def raw_accept(node_tok: np.ndarray, kept: np.ndarray, nka: np.ndarray, n_nodes: np.ndarray,
+               am: np.ndarray, T: int):
+    """Greedy acceptance on the raw tree (Sec. 3.3: "the longest sequence that satisfies the
+    criterion").  am[b,i] is the base model's greedy token after kept node i.  A kept node d
+    follows kept node p when p is d's nearest kept ancestor (removed nodes in between are
+    transparent).  best[p] = longest chain p -> d1 -> d2 ... with node_tok[d] == am[previous];
+    among equally long continuations the lowest node id wins.
+    Returns acc_len [B], acc_nodes [B,T] (kept node ids, pad -1), acc_tok [B,T], next_tok [B]."""
+    B = node_tok.shape[0]
+    acc_len = np.zeros((B,), dtype=np.int64)
+    acc_nodes = np.full((B, T), -1, dtype=np.int64)
+    acc_tok = np.full((B, T), -1, dtype=np.int64)
+    next_tok = np.zeros((B,), dtype=np.int64)
+    for b in range(B):
+        n = int(n_nodes[b])
+        best = [0] * n
+        succ = [-1] * n
+        for p in range(n - 1, -1, -1):                # children have larger ids than their ancestors
+            if not kept[b, p]:
+                continue
+            for d in range(p + 1, n):
+                if kept[b, d] and int(nka[b, d]) == p and int(node_tok[b, d]) == int(am[b, p]):
+                    if 1 + best[d] > best[p]:
+                        best[p] = 1 + best[d]
+                        succ[p] = d
+        cur = 0
+        while succ[cur] >= 0 and acc_len[b] < T:
+            cur = succ[cur]
+            acc_nodes[b, acc_len[b]] = cur
+            acc_tok[b, acc_len[b]] = int(node_tok[b, cur])
+            acc_len[b] += 1
+        next_tok[b] = int(am[b, cur])
+    return acc_len, acc_nodes, acc_tok, next_tok

@@ -492,3 +492,94 @@ def test_commit_accepted_reads_the_cache_as_it_was():
     assert K2[0, 0, :, 0].tolist() == [0, 1, 2, 4, 5, 5, 6, 7]
     assert V2[0, 0, :, 0].tolist() == [0, -1, -2, -4, -5, -5, -6, -7]
     assert np.array_equal(K2[1], K[1]) and new_len.tolist() == [5, 2] and sel.tolist() == [3, 4]
+
+
+# ------------------------------------------------------------------ the paper's raw-tree layout
+def test_raw_paths_are_the_most_probable_alignments():
+    rng = np.random.default_rng(11)
+    ids, lps = _rand_topk(rng, 4, 3, 7)
+    raw, score = orc.select_raw_paths(ids, lps, 10)
+    # brute force with a different mechanism: score every alignment with numpy, stable argsort
+    idx = np.array(list(itertools.product(range(3), repeat=4)))
+    tot = lps[np.arange(4)[None, :], idx].sum(axis=1)
+    order = np.argsort(-tot, kind="stable")[:10]
+    np.testing.assert_array_equal(raw, ids[np.arange(4)[None, :], idx[order]])
+    np.testing.assert_allclose(score, tot[order], rtol=0, atol=1e-12)
+    assert np.all(np.diff(score) <= 1e-15)
+
+
+def test_raw_tree_masks_exactly_the_tokens_the_ctc_transform_removes():
+    """Along every root-to-node path of the raw tree, the kept nodes spell the CTC collapse of the
+    raw prefix (the pinned collapse function), the attention mask holds the root plus those kept
+    nodes, and the position counts them."""
+    rng = np.random.default_rng(12)
+    V = 5
+    for trial in range(8):
+        T, k, N = 5, 3, 12
+        ids, lps = _rand_topk(rng, T, k, V, blank_rate=0.7, repeat_rate=0.8)
+        raw, _ = orc.select_raw_paths(ids, lps, N)
+        raw_tok = raw[None]
+        out = orc.build_raw_tree(np.array([3]), np.array([10]), raw_tok, np.array([N]), V, 64)
+        node_tok, parent, depth, pos, mask, retrieve, n_nodes, kept, nka = out
+        n = int(n_nodes[0])
+        for c in range(N):
+            for l in range(1, T + 1):
+                i = int(retrieve[0, c, l - 1])
+                want = orc.ctc_collapse(raw[c, :l].tolist(), V)
+                path = []
+                j = i
+                while j > 0:
+                    path.append(j)
+                    j = int(parent[0, j])
+                path.reverse()
+                got = tuple(int(node_tok[0, j]) for j in path if kept[0, j])
+                assert got == want
+                bits = {j for j in range(n) if (int(mask[0, i, 0]) >> j) & 1}
+                assert bits == {0} | {j for j in path if kept[0, j]}
+                assert pos[0, i] == 10 + len(want)
+                kept_anc = [j for j in [0] + path[:-1] if j == 0 or kept[0, j]]
+                assert nka[0, i] == kept_anc[-1]
+        assert kept[0, 0] == 1 and nka[0, 0] == -1
+
+
+def test_raw_accept_is_the_longest_collapsed_candidate_that_agrees():
+    """Brute force over the raw paths: collapse each one, count how many of its tokens agree with
+    the base model's greedy choice after the (collapsed) prefix, take the longest."""
+    rng = np.random.default_rng(13)
+    V = 4
+    for trial in range(30):
+        T, k, N = 5, 3, 14
+        ids, lps = _rand_topk(rng, T, k, V, blank_rate=0.7, repeat_rate=0.8)
+        raw, _ = orc.select_raw_paths(ids, lps, N)
+        out = orc.build_raw_tree(np.array([1]), np.array([0]), raw[None], np.array([N]), V, 64)
+        node_tok, parent, depth, pos, mask, retrieve, n_nodes, kept, nka = out
+        n = int(n_nodes[0])
+        # the base model's greedy token is a function of the collapsed prefix only
+        table = {}
+        def nxt(prefix):
+            if prefix not in table:
+                table[prefix] = int(rng.integers(0, V))
+            return table[prefix]
+        am = np.zeros((1, 64), dtype=np.int64)
+        for i in range(n):
+            path = []
+            j = i
+            while j > 0:
+                path.append(j)
+                j = int(parent[0, j])
+            path.reverse()
+            am[0, i] = nxt(tuple(int(node_tok[0, j]) for j in path if kept[0, j]))
+        acc_len, acc_nodes, acc_tok, next_tok = orc.raw_accept(node_tok, kept, nka, n_nodes, am, T)
+        best = ()
+        for c in range(N):
+            y = orc.ctc_collapse(raw[c].tolist(), V)
+            l = 0
+            while l < len(y) and y[l] == nxt(y[:l]):
+                l += 1
+            if l > len(best):
+                best = y[:l]
+        assert acc_len[0] == len(best)
+        # greedy agreement determines the tokens uniquely: every agreeing prefix is the same sequence
+        assert tuple(int(v) for v in acc_tok[0, :acc_len[0]]) == best
+        assert next_tok[0] == nxt(best)
+        assert all(kept[0, int(i)] for i in acc_nodes[0, :acc_len[0]])
