@@ -233,6 +233,52 @@ int ctcsd_commit_accepted(ctcsd_handle* h, void* stream, void* K, void* V, int L
                           int* out_kv_len, int* out_sel_row);
 
 /*
+ * The paper's own verification layout (Sec. 3.3): instead of collapsing the slot paths before
+ * the tree is built, the most probable RAW paths - blanks and repeats still in place - form the
+ * token tree, and the CTC transform acts through the attention map: a position whose symbol the
+ * transform removes is masked for every query row, so that the base model scores exactly the
+ * collapsed sequences.  Three calls replace ctcsd_topk_collapse / ctcsd_build_tree /
+ * ctcsd_verify_accept; ctcsd_draft_logits, ctcsd_tree_attention and ctcsd_commit_accepted are
+ * used unchanged (the latter moves kept nodes only, since only those are ever accepted).
+ *
+ * ctcsd_select_raw_paths: the topN most probable of the k^T slot paths of each sequence.  Path
+ *   score = sum over the slots of the per-slot log-probability (Eq. 6), accumulated in slot
+ *   order in float64; equal scores are ordered by path index (slot 1 most significant, the
+ *   per-slot rank as the digit).  Requires k^T <= CTCSD_MAX_PATHS (else CTCSD_ERR_UNSUPPORTED);
+ *   the handle's beam setting plays no part.
+ *   topk_id, topk_lp [M,T,k], sel_row [B] or NULL: as for ctcsd_topk_collapse.
+ *   out_raw_tok [B,topN,T] int32 (the blank is id V; unused rows -1);
+ *   out_raw_score [B,topN] float32 (unused -inf);  out_n_raw [B] int32 = min(topN, k^T).
+ *
+ * ctcsd_build_raw_tree: the prefix trie of the raw paths, numbered like ctcsd_build_tree (the
+ *   blank is a symbol like any other; every path has T symbols), plus the transform:
+ *   out_kept [B,max_nodes] int32: 1 iff the node survives - its symbol is not the blank and
+ *     differs from its parent's symbol; the root (the base token, not part of the alignment)
+ *     is kept and does not count as a preceding symbol;  0 for removed and unused nodes;
+ *   out_nka [B,max_nodes] int32: nearest kept proper ancestor (-1 for the root and unused nodes);
+ *   out_mask: bit j of row i set iff j is the root, a kept proper ancestor of i, or i itself
+ *     when i is kept;  out_pos = kv_len + number of kept non-root nodes on the path root..i;
+ *   the remaining outputs as for ctcsd_build_tree.  Nodes beyond max_nodes are dropped.
+ *
+ * ctcsd_verify_accept_raw: LM head and arg-max exactly as ctcsd_verify_accept, then acceptance
+ *   over the kept nodes: kept node d follows kept node p when nka[d] == p; the accepted path is
+ *   the longest chain root -> d1 -> d2 ... in which every node's token equals the arg-max at
+ *   its predecessor; among equally long continuations the lowest node id wins (at every level).
+ *   out_acc_nodes holds kept node ids.  max_nodes <= 128.
+ */
+int ctcsd_select_raw_paths(ctcsd_handle* h, void* stream, int M, const int* topk_id, const float* topk_lp,
+                           const int* sel_row, int* out_raw_tok, float* out_raw_score, int* out_n_raw);
+int ctcsd_build_raw_tree(ctcsd_handle* h, void* stream, const int* base_tok, const int* kv_len,
+                         const int* raw_tok, const int* n_raw,
+                         int* out_node_tok, int* out_parent, int* out_depth, int* out_pos,
+                         unsigned long long* out_mask, int* out_retrieve, int* out_n_nodes,
+                         int* out_kept, int* out_nka);
+int ctcsd_verify_accept_raw(ctcsd_handle* h, void* stream, const void* hn, const void* Wl,
+                            const int* node_tok, const int* kept, const int* nka, const int* n_nodes,
+                            int* out_argmax, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
+                            int* out_next_tok, float* out_logits_dbg);
+
+/*
  * Tree attention without a handle and without any allocation (the paper has no counterpart:
  * this is a packaging variant of ctcsd_tree_attention, same arithmetic, same kernels).
  *

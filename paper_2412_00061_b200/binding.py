@@ -24,6 +24,7 @@ EXPORTS = [
     "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
     "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static",
+    "ctcsd_select_raw_paths", "ctcsd_build_raw_tree", "ctcsd_verify_accept_raw",
 ]
 
 
@@ -67,6 +68,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
     lib.ctcsd_verify_accept.argtypes = [vp, vp] + [vp] * 11
     lib.ctcsd_commit_accepted.argtypes = [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp]
+    lib.ctcsd_select_raw_paths.argtypes = [vp, vp, ci] + [vp] * 6
+    lib.ctcsd_build_raw_tree.argtypes = [vp, vp] + [vp] * 13
+    lib.ctcsd_verify_accept_raw.argtypes = [vp, vp] + [vp] * 12
     lib.ctcsd_tree_attention_static.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp, vp, vp,
                                                 ctypes.c_float, vp, vp]
     for name in EXPORTS:
@@ -229,6 +233,52 @@ class Handle:
             _ptr(out_next_tok, i32, c.B, "out_next_tok"),
             _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
         self._check(rc, "verify_accept")
+
+    # ---- the paper's raw-tree layout (Sec. 3.3) ----
+    def select_raw_paths(self, topk_id, topk_lp, sel_row, out_raw_tok, out_raw_score, out_n_raw, stream=None):
+        c = self.cfg
+        M = topk_id.shape[0]
+        i32, f32 = torch.int32, torch.float32
+        rc = self.lib.ctcsd_select_raw_paths(
+            self._h, _stream_ptr(stream), M,
+            _ptr(topk_id, i32, M * c.T * c.k, "topk_id"), _ptr(topk_lp, f32, M * c.T * c.k, "topk_lp"),
+            _ptr(sel_row, i32, c.B, "sel_row"),
+            _ptr(out_raw_tok, i32, c.B * c.topN * c.T, "out_raw_tok"),
+            _ptr(out_raw_score, f32, c.B * c.topN, "out_raw_score"), _ptr(out_n_raw, i32, c.B, "out_n_raw"))
+        self._check(rc, "select_raw_paths")
+
+    def build_raw_tree(self, base_tok, kv_len, raw_tok, n_raw, out_node_tok, out_parent, out_depth, out_pos,
+                       out_mask, out_retrieve, out_n_nodes, out_kept, out_nka, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        W = (c.max_nodes + 63) // 64
+        nn = c.B * c.max_nodes
+        rc = self.lib.ctcsd_build_raw_tree(
+            self._h, _stream_ptr(stream),
+            _ptr(base_tok, i32, c.B, "base_tok"), _ptr(kv_len, i32, c.B, "kv_len"),
+            _ptr(raw_tok, i32, c.B * c.topN * c.T, "raw_tok"), _ptr(n_raw, i32, c.B, "n_raw"),
+            _ptr(out_node_tok, i32, nn, "out_node_tok"), _ptr(out_parent, i32, nn, "out_parent"),
+            _ptr(out_depth, i32, nn, "out_depth"), _ptr(out_pos, i32, nn, "out_pos"),
+            _ptr(out_mask, torch.int64, nn * W, "out_mask"),
+            _ptr(out_retrieve, i32, c.B * c.topN * c.T, "out_retrieve"), _ptr(out_n_nodes, i32, c.B, "out_n_nodes"),
+            _ptr(out_kept, i32, nn, "out_kept"), _ptr(out_nka, i32, nn, "out_nka"))
+        self._check(rc, "build_raw_tree")
+
+    def verify_accept_raw(self, hn, Wl, node_tok, kept, nka, n_nodes, out_argmax, out_acc_len, out_acc_nodes,
+                          out_acc_tok, out_next_tok, out_logits_dbg=None, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        nn = c.B * c.max_nodes
+        rc = self.lib.ctcsd_verify_accept_raw(
+            self._h, _stream_ptr(stream),
+            _ptr(hn, self.act_dtype, nn * c.H, "hn"), _ptr(Wl, self.act_dtype, c.V * c.H, "Wl"),
+            _ptr(node_tok, i32, nn, "node_tok"), _ptr(kept, i32, nn, "kept"), _ptr(nka, i32, nn, "nka"),
+            _ptr(n_nodes, i32, c.B, "n_nodes"),
+            _ptr(out_argmax, i32, nn, "out_argmax"), _ptr(out_acc_len, i32, c.B, "out_acc_len"),
+            _ptr(out_acc_nodes, i32, c.B * c.T, "out_acc_nodes"), _ptr(out_acc_tok, i32, c.B * c.T, "out_acc_tok"),
+            _ptr(out_next_tok, i32, c.B, "out_next_tok"),
+            _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
+        self._check(rc, "verify_accept_raw")
 
     def commit_accepted(self, K, V, kv_len, acc_len, acc_nodes, out_kv_len, out_sel_row=None, stream=None):
         c = self.cfg

@@ -21,6 +21,9 @@ struct TreeParams {
     int T, topN, max_nodes;
     int* node_tok; int* parent; int* depth; int* pos;
     unsigned long long* mask; int* retrieve; int* n_nodes;
+    // raw layout (Sec. 3.3): candidates are full-length slot paths (cand_len null), the blank is
+    // a symbol like any other in the trie, and kept/nka/mask/pos describe the CTC transform
+    int* kept; int* nka; int blank;
 };
 
 __device__ __forceinline__ int warp_excl_scan(int v, int lane, int& total) {
@@ -51,7 +54,7 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     for (int h = 0; h < 2; ++h) {
         const int c = lane + 32 * h;
         int l = 0;
-        if (c < nc) { l = p.cand_len[(size_t)b * N + c]; l = l < 0 ? 0 : (l > T ? T : l); }
+        if (c < nc) { l = p.cand_len ? p.cand_len[(size_t)b * N + c] : T; l = l < 0 ? 0 : (l > T ? T : l); }
         len[h] = l;
 #pragma unroll
         for (int q = 0; q < kT; ++q) tok[h][q] = (q < l) ? p.cand_tok[((size_t)b * N + c) * T + q] : -1;
@@ -155,6 +158,39 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
         o_mask[(size_t)i * W] = 0ull;
         if (W > 1) o_mask[(size_t)i * W + 1] = 0ull;
     }
+    if (p.kept == nullptr) return;
+
+    // ---- raw layout: which nodes survive the CTC transform, and what each node may attend to ----
+    // A node is kept iff its symbol is not the blank and differs from its parent's symbol (the
+    // root holds the base token and is not part of the alignment).  Removed nodes are masked out
+    // of every row, their own included; positions count kept nodes only.
+    __syncwarp();                                   // the warp's own writes above are now visible to it
+    int* o_kept = p.kept + (size_t)b * n_max;
+    int* o_nka = p.nka + (size_t)b * n_max;
+    for (int i = lane; i < n_max; i += 32) {
+        if (i >= n) { o_kept[i] = 0; o_nka[i] = -1; continue; }
+        unsigned long long m0 = 1ull, m1 = 0ull;
+        int count = 0, near = -1, self_kept = 1;
+        int j = i;
+        for (int step = 0; step <= kT && j > 0; ++step) {
+            const int par = o_par[j];
+            const int sym = o_tok[j];
+            const bool kj = sym != p.blank && (par == 0 || sym != o_tok[par]);
+            if (j == i) self_kept = kj ? 1 : 0;
+            if (kj) {
+                if (j < 64) m0 |= 1ull << j; else m1 |= 1ull << (j - 64);
+                ++count;
+                if (j != i && near < 0) near = j;
+            }
+            j = par;
+        }
+        if (i > 0 && near < 0) near = 0;
+        o_kept[i] = self_kept;
+        o_nka[i] = near;
+        o_pos[i] = L + count;
+        o_mask[(size_t)i * W] = m0;
+        if (W > 1) o_mask[(size_t)i * W + 1] = m1;
+    }
 }
 
 }  // namespace
@@ -177,6 +213,29 @@ extern "C" int ctcsd_build_tree(ctcsd_handle* hh, void* stream, const int* base_
     p.T = c.T; p.topN = c.topN; p.max_nodes = c.max_nodes;
     p.node_tok = out_node_tok; p.parent = out_parent; p.depth = out_depth; p.pos = out_pos;
     p.mask = out_mask; p.retrieve = out_retrieve; p.n_nodes = out_n_nodes;
+    p.kept = nullptr; p.nka = nullptr; p.blank = c.V;
+    CTCSD_CUDA_CHECK(h, launch_pdl(build_tree_kernel, dim3(c.B), dim3(32), 0, static_cast<cudaStream_t>(stream), 1, p));
+    CTCSD_LAUNCH_CHECK(h);
+    return CTCSD_OK;
+}
+
+extern "C" int ctcsd_build_raw_tree(ctcsd_handle* hh, void* stream, const int* base_tok, const int* kv_len,
+                                    const int* raw_tok, const int* n_raw,
+                                    int* out_node_tok, int* out_parent, int* out_depth, int* out_pos,
+                                    unsigned long long* out_mask, int* out_retrieve, int* out_n_nodes,
+                                    int* out_kept, int* out_nka) {
+    if (!hh || !base_tok || !kv_len || !raw_tok || !n_raw || !out_node_tok || !out_parent || !out_depth ||
+        !out_pos || !out_mask || !out_retrieve || !out_n_nodes || !out_kept || !out_nka)
+        return CTCSD_ERR_INVALID_ARG;
+    Handle* h = &hh->h;
+    const ctcsd_config& c = h->cfg;
+    TreeParams p;
+    p.base_tok = base_tok; p.kv_len = kv_len;
+    p.cand_tok = raw_tok; p.cand_len = nullptr; p.n_cand = n_raw;
+    p.T = c.T; p.topN = c.topN; p.max_nodes = c.max_nodes;
+    p.node_tok = out_node_tok; p.parent = out_parent; p.depth = out_depth; p.pos = out_pos;
+    p.mask = out_mask; p.retrieve = out_retrieve; p.n_nodes = out_n_nodes;
+    p.kept = out_kept; p.nka = out_nka; p.blank = c.V;
     CTCSD_CUDA_CHECK(h, launch_pdl(build_tree_kernel, dim3(c.B), dim3(32), 0, static_cast<cudaStream_t>(stream), 1, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;

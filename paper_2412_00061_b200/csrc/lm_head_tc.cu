@@ -284,7 +284,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     __syncthreads();
     if (good)
-        for (int b = warp; b < p.acc.B; b += kThreads / 32) greedy_accept_warp(p.acc, b, lane);
+        for (int b = warp; b < p.acc.B; b += kThreads / 32) accept_warp(p.acc, b, lane);
     if (tid == 0) *p.counter = 0u;
 }
 

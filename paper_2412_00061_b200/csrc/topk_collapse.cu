@@ -538,10 +538,72 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     emit_candidates(p, b, sl, bm_tot, bm_key, s_sel, nbeam, -1);
 }
 
+// ---------------------------------------------------------------------------------------
+// Raw-path selection (Sec. 3.3, the paper's own verification layout): the topN most probable
+// slot paths, blanks and repeats left in place.  Path probability = product over the slots
+// (Eq. 6), summed in slot order in float64; equal scores go to the lower path index (slot 1
+// most significant, per-slot rank as the digit).
+// ---------------------------------------------------------------------------------------
+struct RawParams {
+    CollapseParams c;
+    int* out_raw_tok;        // [B,topN,T]
+    float* out_raw_score;    // [B,topN]
+    int* out_n_raw;          // [B]
+};
+
+__global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    const CollapseParams& p = rp.c;
+    double* sc = reinterpret_cast<double*>(dyn);                                   // [cap]
+    unsigned long long* ky = reinterpret_cast<unsigned long long*>(sc + p.cap);    // [cap]
+    __shared__ SlotLists sl;
+    __shared__ SelectScratch S;
+    __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
+
+    const int b = blockIdx.x, tid = threadIdx.x;
+    pdl_wait();                      // the per-slot lists come from the preceding kernel
+    pdl_trigger();
+    const int row = p.sel_row ? p.sel_row[b] : b;
+    int* rtok = rp.out_raw_tok + (size_t)b * p.topN * p.T;
+    float* rscore = rp.out_raw_score + (size_t)b * p.topN;
+    if (row < 0 || row >= p.M) {
+        if (tid == 0) { report_error(p.status, CTCSD_ERR_INVALID_ARG, b); rp.out_n_raw[b] = 0; }
+        return;
+    }
+    load_slot_lists(p, row, sl);
+    for (int path = tid; path < p.npaths; path += kThreads) {
+        double s;
+        path_key_and_score(p, sl, path, s);
+        sc[path] = s;
+        ky[path] = (unsigned long long)path;
+    }
+    for (int i = tid; i < p.topN * p.T; i += kThreads) rtok[i] = -1;
+    for (int i = tid; i < p.topN; i += kThreads) rscore[i] = -INFINITY;
+    __syncthreads();
+    const int nsel = block_select_top(sc, ky, nullptr, p.npaths, p.topN, s_sel, S);
+    for (int e = tid; e < nsel; e += kThreads) {
+        const int at = s_sel[e];
+        unsigned rem = (unsigned)ky[at];
+        rscore[e] = (float)sc[at];
+        for (int t = p.T - 1; t >= 0; --t) {
+            const unsigned q = rem / (unsigned)p.k;
+            rtok[e * p.T + t] = sl.tok[t * p.k + (int)(rem - q * (unsigned)p.k)];
+            rem = q;
+        }
+    }
+    if (tid == 0) rp.out_n_raw[b] = nsel;
+}
+
 }  // namespace
 }  // namespace ctcsd
 
 using namespace ctcsd;
+
+static int next_pow2_host(int v) {
+    int n = 2;
+    while (n < v) n <<= 1;
+    return n;
+}
 
 extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const int* topk_id, const float* topk_lp,
                                    const int* sel_row,
@@ -584,6 +646,38 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_enum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
+    CTCSD_LAUNCH_CHECK(h);
+    return CTCSD_OK;
+}
+
+extern "C" int ctcsd_select_raw_paths(ctcsd_handle* hh, void* stream, int M, const int* topk_id, const float* topk_lp,
+                                      const int* sel_row, int* out_raw_tok, float* out_raw_score, int* out_n_raw) {
+    if (!hh || !topk_id || !topk_lp || !out_raw_tok || !out_raw_score || !out_n_raw) return CTCSD_ERR_INVALID_ARG;
+    Handle* h = &hh->h;
+    const ctcsd_config& c = h->cfg;
+    if (M < 1) return CTCSD_ERR_INVALID_ARG;
+    if (!sel_row && M < c.B) return CTCSD_ERR_INVALID_ARG;
+    long long npaths = 1;
+    for (int t = 0; t < c.T; ++t) {
+        npaths *= c.k;
+        if (npaths > CTCSD_MAX_PATHS) return CTCSD_ERR_UNSUPPORTED;
+    }
+    RawParams rp;
+    CollapseParams& p = rp.c;
+    p.topk_id = topk_id;
+    p.topk_lp = topk_lp;
+    p.sel_row = sel_row;
+    p.M = M; p.T = c.T; p.k = c.k; p.V = c.V; p.topN = c.topN; p.beam = 0; p.score_mode = CTCSD_SCORE_MAX;
+    p.npaths = (int)npaths;
+    p.cap = next_pow2_host((int)npaths);
+    p.k_magic = (unsigned)((1ull << 32) / (unsigned)c.k) + 1u;
+    p.out_cand_tok = nullptr; p.out_cand_len = nullptr; p.out_cand_score = nullptr; p.out_n_cand = nullptr;
+    p.status = status_ptr(h);
+    rp.out_raw_tok = out_raw_tok; rp.out_raw_score = out_raw_score; rp.out_n_raw = out_n_raw;
+    const size_t smem = (size_t)p.cap * 16;
+    if (smem > 48 * 1024)
+        CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(raw_paths_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B), dim3(kThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

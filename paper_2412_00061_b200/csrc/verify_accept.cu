@@ -9,7 +9,7 @@ namespace {
 
 // One warp per sequence (used when the arg-max comes from the CUDA-core path).
 __global__ void __launch_bounds__(32) greedy_accept_kernel(AcceptParams p) {
-    greedy_accept_warp(p, blockIdx.x, threadIdx.x);
+    accept_warp(p, blockIdx.x, threadIdx.x);
 }
 
 }  // namespace
@@ -17,13 +17,10 @@ __global__ void __launch_bounds__(32) greedy_accept_kernel(AcceptParams p) {
 
 using namespace ctcsd;
 
-extern "C" int ctcsd_verify_accept(ctcsd_handle* hh, void* stream, const void* hn, const void* Wl,
-                                   const int* node_tok, const int* parent, const int* n_nodes,
-                                   int* out_argmax, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
-                                   int* out_next_tok, float* out_logits_dbg) {
-    if (!hh || !hn || !Wl || !node_tok || !parent || !n_nodes || !out_argmax || !out_acc_len || !out_acc_nodes ||
-        !out_acc_tok || !out_next_tok)
-        return CTCSD_ERR_INVALID_ARG;
+static int verify_accept_common(ctcsd_handle* hh, void* stream, const void* hn, const void* Wl,
+                                const int* node_tok, const int* parent, const int* kept, const int* nka,
+                                const int* n_nodes, int* out_argmax, int* out_acc_len, int* out_acc_nodes,
+                                int* out_acc_tok, int* out_next_tok, float* out_logits_dbg) {
     Handle* h = &hh->h;
     const ctcsd_config& c = h->cfg;
     if ((reinterpret_cast<uintptr_t>(hn) | reinterpret_cast<uintptr_t>(Wl)) & 15) return CTCSD_ERR_INVALID_ARG;
@@ -34,6 +31,7 @@ extern "C" int ctcsd_verify_accept(ctcsd_handle* hh, void* stream, const void* h
     a.node_tok = node_tok; a.parent = parent; a.n_nodes = n_nodes; a.argmax = out_argmax;
     a.B = c.B; a.T = c.T; a.max_nodes = c.max_nodes;
     a.acc_len = out_acc_len; a.acc_nodes = out_acc_nodes; a.acc_tok = out_acc_tok; a.next_tok = out_next_tok;
+    a.kept = kept; a.nka = nka;
 
     // tensor-core path: the acceptance walk runs in the tail of the LM-head kernel
     if (lm_head_tc_supported(h)) {
@@ -54,4 +52,27 @@ extern "C" int ctcsd_verify_accept(ctcsd_handle* hh, void* stream, const void* h
     greedy_accept_kernel<<<c.B, 32, 0, s>>>(a);
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
+}
+
+extern "C" int ctcsd_verify_accept(ctcsd_handle* hh, void* stream, const void* hn, const void* Wl,
+                                   const int* node_tok, const int* parent, const int* n_nodes,
+                                   int* out_argmax, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
+                                   int* out_next_tok, float* out_logits_dbg) {
+    if (!hh || !hn || !Wl || !node_tok || !parent || !n_nodes || !out_argmax || !out_acc_len || !out_acc_nodes ||
+        !out_acc_tok || !out_next_tok)
+        return CTCSD_ERR_INVALID_ARG;
+    return verify_accept_common(hh, stream, hn, Wl, node_tok, parent, nullptr, nullptr, n_nodes, out_argmax,
+                                out_acc_len, out_acc_nodes, out_acc_tok, out_next_tok, out_logits_dbg);
+}
+
+extern "C" int ctcsd_verify_accept_raw(ctcsd_handle* hh, void* stream, const void* hn, const void* Wl,
+                                       const int* node_tok, const int* kept, const int* nka, const int* n_nodes,
+                                       int* out_argmax, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
+                                       int* out_next_tok, float* out_logits_dbg) {
+    if (!hh || !hn || !Wl || !node_tok || !kept || !nka || !n_nodes || !out_argmax || !out_acc_len || !out_acc_nodes ||
+        !out_acc_tok || !out_next_tok)
+        return CTCSD_ERR_INVALID_ARG;
+    if (hh->h.cfg.max_nodes > 128) return CTCSD_ERR_UNSUPPORTED;
+    return verify_accept_common(hh, stream, hn, Wl, node_tok, nullptr, kept, nka, n_nodes, out_argmax,
+                                out_acc_len, out_acc_nodes, out_acc_tok, out_next_tok, out_logits_dbg);
 }

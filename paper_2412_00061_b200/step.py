@@ -24,7 +24,14 @@ def to_device(a: np.ndarray, dtype: str, device) -> torch.Tensor:
 
 class DraftVerifyStep:
     L2_PREFETCH_BYTES = 48 << 20
-    def __init__(self, cfg: StepConfig, device="cuda:0", max_draft_rows: int = 0, debug_logits: bool = False):
+    def __init__(self, cfg: StepConfig, device="cuda:0", max_draft_rows: int = 0, debug_logits: bool = False,
+                 layout: str = "packed"):
+        """layout "packed": collapse first, tree over the collapsed candidates (the default);
+        "raw": the paper's own layout (Sec. 3.3) - tree over the most probable raw slot paths,
+        removed symbols masked in the attention map."""
+        if layout not in ("packed", "raw"):
+            raise ValueError("layout must be 'packed' or 'raw'")
+        self.layout = layout
         self.cfg = cfg
         self.device = torch.device(device)
         self.h = binding.Handle(cfg.B, cfg.H, cfg.V, cfg.T, cfg.k, cfg.beam, cfg.topN, cfg.max_nodes,
@@ -45,6 +52,8 @@ class DraftVerifyStep:
             O=z(B, n, cfg.Hq, cfg.D, dtype=act),
             argmax=z(B, n),
         )
+        if layout == "raw":
+            self.out.update(kept=z(B, n), nka=z(B, n))
         # the step's results share one buffer, so that reading them back is a single copy
         names = [("acc_len", (B,)), ("acc_nodes", (B, T)), ("acc_tok", (B, T)), ("next_tok", (B,)),
                  ("new_kv_len", (B,)), ("next_sel_row", (B,))]
@@ -104,11 +113,20 @@ class DraftVerifyStep:
 
     def collapse(self, stream=None):
         i, o = self.inp, self.out
+        if self.layout == "raw":      # cand_tok / cand_score / n_cand then hold the raw paths
+            self.h.select_raw_paths(o["topk_id"], o["topk_lp"], i.get("sel_row"),
+                                    o["cand_tok"], o["cand_score"], o["n_cand"], stream=stream)
+            return
         self.h.topk_collapse(o["topk_id"], o["topk_lp"], i.get("sel_row"),
                              o["cand_tok"], o["cand_len"], o["cand_score"], o["n_cand"], stream=stream)
 
     def tree(self, stream=None):
         i, o = self.inp, self.out
+        if self.layout == "raw":
+            self.h.build_raw_tree(i["base_tok"], i["kv_len"], o["cand_tok"], o["n_cand"],
+                                  o["node_tok"], o["parent"], o["depth"], o["pos"], o["mask"], o["retrieve"],
+                                  o["n_nodes"], o["kept"], o["nka"], stream=stream)
+            return
         self.h.build_tree(i["base_tok"], i["kv_len"], o["cand_tok"], o["cand_len"], o["n_cand"],
                           o["node_tok"], o["parent"], o["depth"], o["pos"], o["mask"], o["retrieve"], o["n_nodes"],
                           stream=stream)
@@ -120,6 +138,11 @@ class DraftVerifyStep:
 
     def verify(self, stream=None):
         i, o = self.inp, self.out
+        if self.layout == "raw":
+            self.h.verify_accept_raw(i["hn"], i["Wl"], o["node_tok"], o["kept"], o["nka"], o["n_nodes"],
+                                     o["argmax"], o["acc_len"], o["acc_nodes"], o["acc_tok"], o["next_tok"],
+                                     o.get("lm_logits_dbg"), stream=stream)
+            return
         self.h.verify_accept(i["hn"], i["Wl"], o["node_tok"], o["parent"], o["n_nodes"],
                              o["argmax"], o["acc_len"], o["acc_nodes"], o["acc_tok"], o["next_tok"],
                              o.get("lm_logits_dbg"), stream=stream)

@@ -183,3 +183,102 @@ def run_parity(cfg, seed=0, M=None, force_repeats=False, row_seq=None, sel_row=N
     for k, v in before.items():
         np.testing.assert_array_equal(step.host(k), v, err_msg="rerun " + k)
     return dict(certified=certified, acc_len=acc[0], n_nodes=n_nodes, step=step)
+
+
+def run_parity_raw(cfg, seed=0, force_repeats=False, device="cuda:0", attention_rows: Optional[int] = None,
+                   lm_rows: Optional[int] = None):
+    """The paper's raw-tree layout (Sec. 3.3) through the C ABI against the oracle: raw-path
+    selection, raw tree with the transform's mask, attention under that mask, acceptance over
+    the kept nodes.  Integer outputs are compared bit for bit (the oracle is fed the CUDA path's
+    previous-stage output); path scores are float64 sums of the same float32 terms in the same
+    order on both sides, so even the order of equal scores must agree."""
+    logit_tol, rel = tolerances(cfg.dtype)
+    inp = make_inputs(cfg, seed, None, force_repeats, None, None)
+    step = DraftVerifyStep(cfg, device=device, debug_logits=True, layout="raw")
+    dev = step.device
+    i32 = lambda a: None if a is None else torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    step.set_inputs(
+        x=to_device(inp["x"], cfg.dtype, dev), Wd=to_device(inp["Wd"], cfg.dtype, dev),
+        blank_bias=torch.from_numpy(inp["blank_bias"]).to(dev), row_seq=None, sel_row=None,
+        base_tok=i32(inp["base_tok"]), kv_len=i32(inp["kv_len"]),
+        Q=to_device(inp["Q"], cfg.dtype, dev), K=to_device(inp["K"], cfg.dtype, dev),
+        V=to_device(inp["V"], cfg.dtype, dev), Wl=to_device(inp["Wl"], cfg.dtype, dev))
+    step.draft()
+    step.check_status()
+    check_topk(step.host("draft_logits_dbg"), step.host("topk_id"), step.host("topk_lp"), step.host("lse"), cfg.k, rel)
+
+    # ---- raw-path selection -----------------------------------------------------------------
+    step.collapse()
+    step.check_status()
+    tid, tlp = step.host("topk_id").astype(np.int64), step.host("topk_lp").astype(np.float64)
+    raw_tok, raw_score, n_raw = step.host("cand_tok"), step.host("cand_score"), step.host("n_cand")
+    for b in range(cfg.B):
+        want_tok, want_score = orc.select_raw_paths(tid[b], tlp[b], cfg.topN)
+        n = want_tok.shape[0]
+        assert n_raw[b] == n == min(cfg.topN, cfg.k ** cfg.T)
+        np.testing.assert_array_equal(raw_tok[b, :n], want_tok)
+        np.testing.assert_allclose(raw_score[b, :n], want_score, rtol=1e-6, atol=1e-6)
+        assert np.all(raw_tok[b, n:] == -1) and np.all(np.isneginf(raw_score[b, n:]))
+
+    # ---- raw tree ---------------------------------------------------------------------------
+    step.tree()
+    step.check_status()
+    o_tree = orc.build_raw_tree(inp["base_tok"], inp["kv_len"], raw_tok.astype(np.int64), n_raw.astype(np.int64),
+                                cfg.V, cfg.max_nodes)
+    names = ["node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes", "kept", "nka"]
+    for name, want in zip(names, o_tree):
+        have = step.host(name)
+        if name == "mask":
+            have = have.view(np.uint64)
+        np.testing.assert_array_equal(have, want, err_msg=name)
+    node_tok, parent, depth, pos, mask, retrieve, n_nodes, kept, nka = o_tree
+
+    # ---- attention under the transform's mask -------------------------------------------------
+    step.attention()
+    step.check_status()
+    O_gpu = step.host("O")
+    if attention_rows is None:
+        O_def = orc.tree_attention(inp["Q"], inp["K"], inp["V"], inp["kv_len"], n_nodes, mask, 1.0 / math.sqrt(cfg.D))
+        assert np.max(np.abs(O_gpu - O_def)) <= logit_tol
+    else:
+        rng = np.random.default_rng(seed + 77)
+        for _ in range(attention_rows):
+            b = int(rng.integers(0, cfg.B))
+            h = int(rng.integers(0, cfg.Hq))
+            g = h // (cfg.Hq // cfg.Hkv)
+            one = orc.tree_attention(inp["Q"][b:b + 1, :, h:h + 1], inp["K"][b:b + 1, g:g + 1],
+                                     inp["V"][b:b + 1, g:g + 1], inp["kv_len"][b:b + 1], n_nodes[b:b + 1],
+                                     mask[b:b + 1], 1.0 / math.sqrt(cfg.D))
+            assert np.max(np.abs(O_gpu[b, :, h] - one[0, :, 0])) <= logit_tol
+
+    # ---- LM head + acceptance over the kept nodes -----------------------------------------------
+    follows = np.where(kept != 0, nka, -1)          # who a node may follow; removed nodes follow nobody
+    hn, target = synth.gen_node_hidden(cfg, seed, inp["Wl"], node_tok, follows, n_nodes)
+    step.set_inputs(hn=to_device(hn, cfg.dtype, dev))
+    step.verify()
+    step.check_status()
+    y_gpu = step.host("lm_logits_dbg")
+    live = [b * cfg.max_nodes + i for b in range(cfg.B) for i in range(int(n_nodes[b]))]
+    rows = live
+    if lm_rows is not None and len(live) > lm_rows:
+        rows = [live[j] for j in np.random.default_rng(seed + 5).choice(len(live), lm_rows, replace=False)]
+    y_def, am_def = orc.lm_head_argmax(hn[rows], inp["Wl"])
+    assert np.max(np.abs(y_gpu[rows] - y_def)) <= logit_tol
+    am_gpu = step.host("argmax")
+    np.testing.assert_array_equal(am_gpu.reshape(-1), orc.argmax_rows(y_gpu))
+    np.testing.assert_array_equal(am_gpu.reshape(-1)[live], target.reshape(-1)[live])
+    acc = orc.raw_accept(node_tok, kept, nka, n_nodes, am_gpu.astype(np.int64), cfg.T)
+    for name, want in zip(["acc_len", "acc_nodes", "acc_tok", "next_tok"], acc):
+        np.testing.assert_array_equal(step.host(name), want, err_msg=name)
+    # accepted nodes are kept, their positions are consecutive after the root's
+    for b in range(cfg.B):
+        for l in range(int(acc[0][b])):
+            d = int(acc[1][b, l])
+            assert kept[b, d] == 1 and pos[b, d] == inp["kv_len"][b] + l + 1
+
+    before = {k: step.host(k).copy() for k in ["cand_tok", "node_tok", "mask", "kept", "nka", "argmax", "acc_len", "acc_tok", "next_tok"]}
+    step.run()
+    step.check_status()
+    for k, v in before.items():
+        np.testing.assert_array_equal(step.host(k), v, err_msg="rerun " + k)
+    return dict(acc_len=acc[0], n_nodes=n_nodes, kept=kept, step=step)

@@ -123,6 +123,49 @@ def test_history_update_moves_the_accepted_rows(name):
     assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
 
 
+RAW = {
+    # the raw trie of N paths of T symbols has up to 1 + N*T nodes
+    "c2raw": C["c2"].replace(name="c2raw", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200, max_nodes=96),
+    "c3raw": C["c3"].replace(name="c3raw", B=3, H=512, V=1777, Hq=4, Hkv=4, kv_lo=70, kv_hi=300, beam=0,
+                             T=4, k=4, topN=24, max_nodes=128),
+    "c5raw_cut": C["c5"].replace(name="c5raw_cut", B=5, H=1024, V=1200, Hq=8, Hkv=2, kv_lo=100, kv_hi=500,
+                                 beam=0, T=5, k=3, topN=32, max_nodes=64),      # node budget cuts the trie
+    "c1raw": C["c1"].replace(name="c1raw", B=2, H=264, V=777, kv_lo=1, kv_hi=90),   # fp32 path
+}
+
+
+@pytest.mark.parametrize("name", sorted(RAW))
+@pytest.mark.parametrize("seed", [3, 5])
+def test_raw_tree_layout(name, seed):
+    """The paper's own verification layout (Sec. 3.3): raw paths, removed symbols masked."""
+    from tests.parity_util import run_parity_raw
+    cfg = RAW[name]
+    r = run_parity_raw(cfg, seed=seed, force_repeats=(seed == 5))
+    live = sum(int(n) for n in r["n_nodes"])
+    removed = live - int(r["kept"].sum())
+    assert removed > 0, "the inputs must exercise the transform (blanks or repeats in the raw paths)"
+
+
+def test_raw_tree_layout_c2_full_size_and_history_update():
+    """Headline shape, raw layout, sampled attention / LM-head rows; then the history update
+    moves the accepted (kept) nodes' rows exactly as the oracle does."""
+    from oracle import ctcsd_oracle as orc
+    from tests.parity_util import run_parity_raw
+    cfg = C["c2"].replace(name="c2rawfull", max_nodes=96)
+    r = run_parity_raw(cfg, seed=1, attention_rows=4, lm_rows=24)
+    step = r["step"]
+    K0, V0 = step.inp["K"].float().cpu().numpy(), step.inp["V"].float().cpu().numpy()
+    kv_len = step.inp["kv_len"].cpu().numpy()
+    acc_len, acc_nodes = step.host("acc_len"), step.host("acc_nodes")
+    K1, V1, new_len, sel = orc.commit_accepted(K0, V0, kv_len, acc_len, acc_nodes, cfg.max_nodes)
+    step.commit()
+    step.check_status()
+    assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
+    assert np.array_equal(step.inp["V"].float().cpu().numpy(), V1)
+    np.testing.assert_array_equal(step.host("new_kv_len"), new_len)
+    np.testing.assert_array_equal(step.host("next_sel_row"), sel)
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
     """Failure detection without a fault: a bounded device-side wait on a barrier that nothing
     signals gives up, the status word says CTCSD_ERR_TIMEOUT, polling clears it, and the same
