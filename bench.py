@@ -118,7 +118,7 @@ class ClockSampler:
         return out
 
 
-def oracle_step(cfg, inp, sample_slots=None):
+def oracle_step(cfg, inp, sample_slots=None, layout="packed"):
     """One pass of the CPU oracle over the step (definition mode, fp64).  Returns nothing:
     it is only timed."""
     import math
@@ -127,6 +127,17 @@ def oracle_step(cfg, inp, sample_slots=None):
     from paper_2412_00061_b200 import synth
     z = orc.draft_logits(inp["x"], inp["Wd"], inp["blank_bias"])
     ids, lps = orc.topk_slots(z, cfg.k)
+    if layout == "raw":
+        raw = [orc.select_raw_paths(ids[b], lps[b], cfg.topN)[0] for b in range(cfg.B)]
+        n_raw = np.array([r.shape[0] for r in raw])
+        tree = orc.build_raw_tree(inp["base_tok"], inp["kv_len"], np.stack(raw), n_raw, cfg.V, cfg.max_nodes)
+        node_tok, parent, depth, pos, mask, retrieve, n_nodes, kept, nka = tree
+        orc.tree_attention(inp["Q"], inp["K"], inp["V"], inp["kv_len"], n_nodes, mask, 1.0 / math.sqrt(cfg.D))
+        if "hn" not in inp:
+            inp["hn"], _ = synth.gen_node_hidden(cfg, 0, inp["Wl"], node_tok, np.where(kept != 0, nka, -1), n_nodes)
+        _, am = orc.lm_head_argmax(inp["hn"], inp["Wl"])
+        orc.raw_accept(node_tok, kept, nka, n_nodes, am.reshape(cfg.B, cfg.max_nodes), cfg.T)
+        return
     ctok, clen, cscore, nc = orc.topk_collapse(ids, lps, cfg.V, cfg.T, cfg.topN, cfg.beam, cfg.score_mode)
     tree = orc.build_tree(inp["base_tok"], inp["kv_len"], ctok, clen, nc, cfg.max_nodes)
     node_tok, parent, depth, pos, mask, retrieve, n_nodes = tree
@@ -155,12 +166,12 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(cfg, inp, steps, warmup):
+def time_oracle(cfg, inp, steps, warmup, layout="packed"):
     for _ in range(warmup):
-        oracle_step(cfg, inp)
+        oracle_step(cfg, inp, layout=layout)
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle_step(cfg, inp)
+        oracle_step(cfg, inp, layout=layout)
     return (time.perf_counter() - t0) / steps
 
 
@@ -175,14 +186,14 @@ def run_reference(args):
     inp = host_inputs(cfg, 0)
     steps = max(1, min(args.steps, 20))
     warmup = max(1, min(args.warmup, 2))
-    sec = time_oracle(cfg, inp, steps, warmup)
+    sec = time_oracle(cfg, inp, steps, warmup, args.layout)
     val = 1.0 / sec
     cores = blas_threads()
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "sample": "whole step, all stages"},
+        "config": {"workload": workload_name(cfg), "layout": args.layout, "sample": "whole step, all stages"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "%d full steps of the fp64 oracle (numpy, BLAS threads = cores)" % steps},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -219,7 +230,7 @@ def run_ours(args):
     cfg = synth.CONFIGS[args.config]
     seed = replicas.rank_seed(0, rank)             # every rank drafts for its own sequences
     inp = host_inputs(cfg, seed)
-    step = DraftVerifyStep(cfg, device=str(dev))
+    step = DraftVerifyStep(cfg, device=str(dev), layout=args.layout)
     i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
     step.set_inputs(x=to_device(inp["x"], cfg.dtype, dev), Wd=to_device(inp["Wd"], cfg.dtype, dev),
                     blank_bias=torch.from_numpy(inp["blank_bias"]).to(dev),
@@ -230,6 +241,8 @@ def run_ours(args):
     step.draft(); step.collapse(); step.tree()
     step.check_status()
     node_tok, parent, n_nodes = step.host("node_tok"), step.host("parent"), step.host("n_nodes")
+    if args.layout == "raw":      # a kept node follows its nearest kept ancestor; removed nodes follow nobody
+        parent = np.where(step.host("kept") != 0, step.host("nka"), -1)
     hn, _ = synth.gen_node_hidden(cfg, seed, inp["Wl"], node_tok, parent, n_nodes)
     inp["hn"] = hn
     step.set_inputs(hn=to_device(hn, cfg.dtype, dev))
@@ -357,7 +370,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (weights %.0f MB)" % (
+            "config": {"workload": workload_name(cfg), "layout": args.layout, "l2": "inputs larger than L2 (weights %.0f MB)" % (
                 (draft_b + lm_b) / 1e6), "parallelism": "replicas x%d" % world,
                 "launch": ("CUDA graph of %d steps, replayed" % S) if use_graph else "direct launches",
                 "tree_nodes": n_live, "step_bytes": step_bytes,
@@ -372,7 +385,7 @@ def run_ours(args):
         }
         if world == 1 and not args.no_cpu_baseline:
             n_or = 10
-            sec = time_oracle(cfg, inp, n_or, 1)
+            sec = time_oracle(cfg, inp, n_or, 1, args.layout)
             line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                     "sample": "%d full steps of the fp64 oracle on the same inputs" % n_or}
         print(json.dumps(line), flush=True)
@@ -387,6 +400,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--layout", default="packed", choices=["packed", "raw"],
+                    help="packed: collapse, then tree (headline); raw: the paper's raw-path tree with masked removed symbols")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every call directly instead of replaying a CUDA graph")
     args = ap.parse_args()
