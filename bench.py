@@ -399,7 +399,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c6"])
     ap.add_argument("--layout", default="packed", choices=["packed", "raw"],
                     help="packed: collapse, then tree (headline); raw: the paper's raw-path tree with masked removed symbols")
     ap.add_argument("--no-cpu-baseline", action="store_true")

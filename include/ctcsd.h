@@ -53,7 +53,7 @@ extern "C" {
 
 #define CTCSD_MAX_T        8    /* draft slots */
 #define CTCSD_MAX_K        8    /* symbols kept per slot */
-#define CTCSD_MAX_NODES    128  /* tree nodes per sequence, root included */
+#define CTCSD_MAX_NODES    256  /* tree nodes per sequence, root included */
 #define CTCSD_MAX_TOPN     64   /* candidates kept */
 #define CTCSD_MAX_PATHS    4096 /* k^T limit for exhaustive enumeration */
 #define CTCSD_MAX_BEAM     128
@@ -264,7 +264,7 @@ int ctcsd_commit_accepted(ctcsd_handle* h, void* stream, void* K, void* V, int L
  *   over the kept nodes: kept node d follows kept node p when nka[d] == p; the accepted path is
  *   the longest chain root -> d1 -> d2 ... in which every node's token equals the arg-max at
  *   its predecessor; among equally long continuations the lowest node id wins (at every level).
- *   out_acc_nodes holds kept node ids.  max_nodes <= 128.
+ *   out_acc_nodes holds kept node ids.
  */
 int ctcsd_select_raw_paths(ctcsd_handle* h, void* stream, int M, const int* topk_id, const float* topk_lp,
                            const int* sel_row, int* out_raw_tok, float* out_raw_score, int* out_n_raw);

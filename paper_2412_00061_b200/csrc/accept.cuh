@@ -54,18 +54,19 @@ __device__ __forceinline__ void greedy_accept_warp(const AcceptParams& p, int b,
     }
 }
 
-// Acceptance on the raw tree, executed by one full warp for sequence b (at most 128 nodes).  A
+// Acceptance on the raw tree, executed by one full warp for sequence b (at most 256 nodes).  A
 // kept node d follows kept node p when nka[d] == p; best[p] = longest chain p -> d1 -> d2 ... in
 // which every node's token equals the arg-max at its predecessor; among equally long
-// continuations the lowest node id wins.  Lane l holds nodes l, l+32, l+64, l+96.
+// continuations the lowest node id wins.  Lane l holds nodes l, l+32, ..., l+224.
 __device__ __forceinline__ void raw_accept_warp(const AcceptParams& p, int b, int lane) {
     const int n_max = p.max_nodes;
     int n = p.n_nodes[b];
     n = n < 1 ? 1 : (n > n_max ? n_max : n);
     const int* am = p.argmax + (size_t)b * n_max;
-    int tok[4], kp[4], na[4], best[4], succ[4];
+    constexpr int kQ = 8;                              // nodes per lane
+    int tok[kQ], kp[kQ], na[kQ], best[kQ], succ[kQ];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < kQ; ++q) {
         const int d = lane + 32 * q;
         const bool in = d < n;
         tok[q] = in ? p.node_tok[(size_t)b * n_max + d] : -1;
@@ -78,14 +79,14 @@ __device__ __forceinline__ void raw_accept_warp(const AcceptParams& p, int b, in
         const int owner = pn & 31, oq = pn >> 5;
         int pk = 0;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) pk = (q == oq) ? kp[q] : pk;
+        for (int q = 0; q < kQ; ++q) pk = (q == oq) ? kp[q] : pk;
         pk = __shfl_sync(0xffffffffu, pk, owner);
         if (!pk) continue;                                      // uniform
         const int want = am[pn];
         // this lane's best follower: longer chain first, then lower id
         int val = 0, who = 0x7fffffff;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < kQ; ++q) {
             const int d = lane + 32 * q;
             if (d > pn && kp[q] && na[q] == pn && tok[q] == want) {
                 const int v = 1 + best[q];
@@ -100,7 +101,7 @@ __device__ __forceinline__ void raw_accept_warp(const AcceptParams& p, int b, in
         }
         if (lane == owner) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+            for (int q = 0; q < kQ; ++q)
                 if (q == oq) { best[q] = val; succ[q] = val > 0 ? who : -1; }
         }
     }
@@ -108,13 +109,13 @@ __device__ __forceinline__ void raw_accept_warp(const AcceptParams& p, int b, in
     while (len < p.T) {
         int sc = -1;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) sc = (q == (cur >> 5)) ? succ[q] : sc;
+        for (int q = 0; q < kQ; ++q) sc = (q == (cur >> 5)) ? succ[q] : sc;
         sc = __shfl_sync(0xffffffffu, sc, cur & 31);
         if (sc < 0) break;
         cur = sc;
         int tk = -1;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) tk = (q == (cur >> 5)) ? tok[q] : tk;
+        for (int q = 0; q < kQ; ++q) tk = (q == (cur >> 5)) ? tok[q] : tk;
         tk = __shfl_sync(0xffffffffu, tk, cur & 31);
         if (lane == 0) {
             p.acc_nodes[(size_t)b * p.T + len] = cur;

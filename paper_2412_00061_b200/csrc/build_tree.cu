@@ -37,6 +37,27 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane, int& total) {
     return inc - v;
 }
 
+// Ancestor set of one node: bit j of word j/64.
+struct NodeSet {
+    unsigned long long w[4];
+    __device__ __forceinline__ void clear() { w[0] = w[1] = w[2] = w[3] = 0ull; }
+    __device__ __forceinline__ void add(int j) {
+        const unsigned long long bit = 1ull << (j & 63);
+        const int q = j >> 6;
+        w[0] |= q == 0 ? bit : 0ull;
+        w[1] |= q == 1 ? bit : 0ull;
+        w[2] |= q == 2 ? bit : 0ull;
+        w[3] |= q == 3 ? bit : 0ull;
+    }
+    __device__ __forceinline__ void store(unsigned long long* dst, int W) const {
+        dst[0] = w[0];
+        if (W > 1) dst[1] = w[1];
+        if (W > 2) dst[2] = w[2];
+        if (W > 3) dst[3] = w[3];
+    }
+};
+static_assert(CTCSD_MAX_NODES <= 256, "NodeSet holds four 64-bit words");
+
 __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     const int b = blockIdx.x, lane = threadIdx.x;
     const int T = p.T, N = p.topN, n_max = p.max_nodes;
@@ -114,7 +135,9 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int c = lane + 32 * h;
-        unsigned long long m0 = 1ull, m1 = 0ull;       // the root is everybody's ancestor
+        NodeSet anc;
+        anc.clear();
+        anc.add(0);                                    // the root is everybody's ancestor
         int parent_node = 0;
 #pragma unroll
         for (int l = 0; l < kT; ++l) {
@@ -133,14 +156,13 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
                 }
                 if (c < N) p.retrieve[((size_t)b * N + c) * T + l] = node;
                 if (node >= 0) {
-                    if (node < 64) m0 |= 1ull << node; else m1 |= 1ull << (node - 64);
+                    anc.add(node);
                     if (o == c) {                          // this candidate creates the node
                         o_tok[node] = tok[h][l];
                         o_par[node] = parent_node;
                         o_dep[node] = l + 1;
                         o_pos[node] = L + l + 1;
-                        o_mask[(size_t)node * W] = m0;
-                        if (W > 1) o_mask[(size_t)node * W + 1] = m1;
+                        anc.store(o_mask + (size_t)node * W, W);
                     }
                 }
                 parent_node = node;
@@ -150,13 +172,12 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     if (lane == 0) {
         o_tok[0] = p.base_tok[b]; o_par[0] = -1; o_dep[0] = 0; o_pos[0] = L;
         o_mask[0] = 1ull;
-        if (W > 1) o_mask[1] = 0ull;
+        for (int w = 1; w < W; ++w) o_mask[w] = 0ull;
         p.n_nodes[b] = n;
     }
     for (int i = n + lane; i < n_max; i += 32) {
         o_tok[i] = -1; o_par[i] = -1; o_dep[i] = 0; o_pos[i] = 0;
-        o_mask[(size_t)i * W] = 0ull;
-        if (W > 1) o_mask[(size_t)i * W + 1] = 0ull;
+        for (int w = 0; w < W; ++w) o_mask[(size_t)i * W + w] = 0ull;
     }
     if (p.kept == nullptr) return;
 
@@ -169,7 +190,9 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     int* o_nka = p.nka + (size_t)b * n_max;
     for (int i = lane; i < n_max; i += 32) {
         if (i >= n) { o_kept[i] = 0; o_nka[i] = -1; continue; }
-        unsigned long long m0 = 1ull, m1 = 0ull;
+        NodeSet vis;
+        vis.clear();
+        vis.add(0);
         int count = 0, near = -1, self_kept = 1;
         int j = i;
         for (int step = 0; step <= kT && j > 0; ++step) {
@@ -178,7 +201,7 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
             const bool kj = sym != p.blank && (par == 0 || sym != o_tok[par]);
             if (j == i) self_kept = kj ? 1 : 0;
             if (kj) {
-                if (j < 64) m0 |= 1ull << j; else m1 |= 1ull << (j - 64);
+                vis.add(j);
                 ++count;
                 if (j != i && near < 0) near = j;
             }
@@ -188,8 +211,7 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
         o_kept[i] = self_kept;
         o_nka[i] = near;
         o_pos[i] = L + count;
-        o_mask[(size_t)i * W] = m0;
-        if (W > 1) o_mask[(size_t)i * W + 1] = m1;
+        vis.store(o_mask + (size_t)i * W, W);
     }
 }
 

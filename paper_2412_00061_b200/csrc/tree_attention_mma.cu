@@ -243,7 +243,9 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
                     if (key >= L) {
                         const int tn = key - L;
                         const unsigned long long w0 = second ? mB0 : mA0, w1 = second ? mB1 : mA1;
-                        const unsigned long long w = tn < 64 ? w0 : w1;
+                        unsigned long long w = tn < 64 ? w0 : w1;
+                        if (tn >= 128)                          // words past the two kept in registers
+                            w = (vis && key < Ltot) ? p.mask[((size_t)b * p.max_nodes + (second ? iB : iA)) * W + (tn >> 6)] : 0ull;
                         vis = vis && key < Ltot && ((w >> (tn & 63)) & 1ull);
                     }
                 }

@@ -65,7 +65,7 @@ extern "C" int ctcsd_tree_attention_static(void* stream, int B, int max_nodes, i
                                            const unsigned long long* mask, float scale, void* out_O,
                                            int* out_status) {
     if (!Q || !K || !V || !kv_len || !n_nodes || !mask || !out_O) return CTCSD_ERR_INVALID_ARG;
-    if (B < 1 || max_nodes < 2 || max_nodes > CTCSD_MAX_NODES) return CTCSD_ERR_INVALID_ARG;
+    if (B < 1 || max_nodes < 2 || max_nodes > 128) return CTCSD_ERR_INVALID_ARG;
     if (Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || (D != 64 && D != 128)) return CTCSD_ERR_INVALID_ARG;
     if (Lcap < max_nodes || (long long)B * max_nodes > (1 << 20)) return CTCSD_ERR_INVALID_ARG;
 

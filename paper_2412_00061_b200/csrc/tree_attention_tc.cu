@@ -211,12 +211,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         const int i = r / grp;                        // tree node of the row
         const bool live = i < n;
         const int W = (p.max_nodes + 63) / 64;
+        // the first two mask words live in registers; trees above 128 nodes read the others
+        // from memory where a chunk of keys needs them
         unsigned long long m0 = 0, m1 = 0;
+        const unsigned long long* mrow = p.mask + ((size_t)b * p.max_nodes + (live ? i : 0)) * W;
         if (live) {
-            const unsigned long long* m = p.mask + ((size_t)b * p.max_nodes + i) * W;
-            m0 = m[0];
-            if (W > 1) m1 = m[1];
+            m0 = mrow[0];
+            if (W > 1) m1 = mrow[1];
         }
+        auto mask_word = [&](int w) -> unsigned long long {
+            return w == 0 ? m0 : (w == 1 ? m1 : (w < W ? mrow[w] : 0ull));
+        };
 #pragma unroll
         for (int d = 0; d < D; ++d) acc[d] = 0.f;
         const float sl2 = p.scale * 1.4426950408889634f;          // scores are kept in log2 units
@@ -245,9 +250,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 const int t0 = key0 + c0 - L;                   // tree index of the chunk's first key
                 if (t0 <= -32) return 0xffffffffu;
                 if (t0 < 0) return (uint32_t)((m0 << (-t0)) | ((1ull << (-t0)) - 1ull));
-                if (t0 < 64) return (uint32_t)((m0 >> t0) | (t0 ? (m1 << (64 - t0)) : 0ull));
-                if (t0 < 128) return (uint32_t)(m1 >> (t0 - 64));
-                return 0u;
+                const int w = t0 >> 6, sft = t0 & 63;
+                unsigned long long bits = mask_word(w) >> sft;
+                if (sft > 32) bits |= mask_word(w + 1) << (64 - sft);
+                return (uint32_t)bits;
             };
             // pass 1: row maximum
             float bm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four chains instead of one

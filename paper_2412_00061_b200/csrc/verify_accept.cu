@@ -72,7 +72,6 @@ extern "C" int ctcsd_verify_accept_raw(ctcsd_handle* hh, void* stream, const voi
     if (!hh || !hn || !Wl || !node_tok || !kept || !nka || !n_nodes || !out_argmax || !out_acc_len || !out_acc_nodes ||
         !out_acc_tok || !out_next_tok)
         return CTCSD_ERR_INVALID_ARG;
-    if (hh->h.cfg.max_nodes > 128) return CTCSD_ERR_UNSUPPORTED;
     return verify_accept_common(hh, stream, hn, Wl, node_tok, nullptr, kept, nka, n_nodes, out_argmax,
                                 out_acc_len, out_acc_nodes, out_acc_tok, out_next_tok, out_logits_dbg);
 }

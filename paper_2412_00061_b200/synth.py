@@ -78,6 +78,9 @@ CONFIGS: Dict[str, StepConfig] = {
     # GQA 70B-shaped stress step
     "c5": StepConfig("c5", B=32, H=8192, V=32000, T=6, k=4, beam=64, topN=16, max_nodes=64,
                      Hq=64, Hkv=8, D=128, kv_lo=1024, kv_hi=4096, dtype="bf16", agree_p=0.6),
+    # the 7B shape with a large tree: 64 candidates of up to 6 tokens, 256 nodes
+    "c6": StepConfig("c6", B=1, H=4096, V=32000, T=6, k=4, beam=0, topN=64, max_nodes=256,
+                     Hq=32, Hkv=32, D=128, kv_lo=1024, kv_hi=1024, dtype="bf16", agree_p=0.6),
 }
 
 

@@ -85,7 +85,7 @@ def test_c2_full_size_sampled():
     assert 2 <= r["n_nodes"][0] <= 64
 
 
-@pytest.mark.parametrize("name", ["c3", "c4", "c5"])
+@pytest.mark.parametrize("name", ["c3", "c4", "c5", "c6"])
 def test_batched_workloads_full_size_sampled(name):
     """The batched workloads at full size (prefix beam, ragged KV lengths, 128-node trees, GQA):
     all integer stages are compared in full; the definition-mode oracle checks one draft row,
@@ -121,6 +121,41 @@ def test_history_update_moves_the_accepted_rows(name):
                            step.out["new_kv_len"], step.out["next_sel_row"])
     assert step.h.poll_status() == -1
     assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
+
+
+BIG = {
+    # trees above 128 nodes: three and four mask words, two LM-head row tiles per sequence
+    "big_enum": C["c2"].replace(name="big_enum", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200,
+                                T=6, k=4, topN=64, max_nodes=256),
+    "big_beam_gqa": C["c5"].replace(name="big_beam_gqa", B=3, H=512, V=1500, Hq=8, Hkv=2, kv_lo=90, kv_hi=400,
+                                    T=8, k=5, beam=128, topN=64, max_nodes=200),
+    "big_fp32": C["c1"].replace(name="big_fp32", B=2, H=264, V=777, kv_lo=1, kv_hi=90, T=6, k=4, topN=64,
+                                max_nodes=200),
+}
+
+
+def test_attention_fallback_when_heads_per_kv_head_do_not_divide_the_row_tile():
+    """Three query heads per kv head: the tensor-core kernel's 128-row tile cannot hold whole
+    nodes, so the warp-level kernel runs; once with a small tree, once above 128 nodes."""
+    small = C["c5"].replace(name="gqa3", B=2, H=512, V=1500, Hq=6, Hkv=2, kv_lo=60, kv_hi=300, beam=16)
+    _run(small, seed=1)
+    big = BIG["big_beam_gqa"].replace(name="gqa3_big", Hq=6, Hkv=2, D=64)
+    r = _run(big, seed=2)
+    assert max(r["n_nodes"]) > 128
+
+
+@pytest.mark.parametrize("name", sorted(BIG))
+def test_trees_above_128_nodes(name):
+    cfg = BIG[name]
+    r = _run(cfg, seed=2)
+    assert max(r["n_nodes"]) > 128, "the tree must reach past the first two mask words"
+
+
+@pytest.mark.parametrize("name", ["big_enum", "big_fp32"])
+def test_raw_layout_on_a_tree_above_128_nodes(name):
+    from tests.parity_util import run_parity_raw
+    r = run_parity_raw(BIG[name], seed=2)
+    assert max(r["n_nodes"]) > 128
 
 
 RAW = {

@@ -265,12 +265,15 @@ def test_tree_hand_example_and_truncation():
 
 def test_tree_invariants_against_bruteforce_trie():
     rng = np.random.default_rng(9)
-    for trial in range(40):
+    for trial in range(46):
         N, T = int(rng.integers(1, 9)), int(rng.integers(1, 6))
         n_max = int(rng.integers(2, 70))
+        alphabet = 3
+        if trial >= 40:                                   # large trees: masks of three and four words
+            N, T, n_max, alphabet = int(rng.integers(40, 65)), 8, int(rng.integers(130, 257)), 4
         seen, cands = set(), []
         for _ in range(N):
-            y = tuple(rng.integers(0, 3, size=int(rng.integers(1, T + 1))).tolist())
+            y = tuple(rng.integers(0, alphabet, size=int(rng.integers(1, T + 1))).tolist())
             if y not in seen:
                 seen.add(y)
                 cands.append(y)
@@ -356,6 +359,15 @@ def test_attention_against_sdpa_and_special_cases():
     O = orc.tree_attention(Q, K, V, kv_len, n_nodes, mask, scale)
     np.testing.assert_allclose(O, _sdpa_ref(Q, K, V, kv_len, n_nodes, mask, scale), atol=1e-12)
     assert np.all(O[1, 9:] == 0)
+    # a tree above 128 nodes: four mask words
+    nb = 256
+    Qb = rng.normal(size=(1, nb, Hq, D))
+    Kb = rng.normal(size=(1, Hkv, 300, D))
+    Vb = rng.normal(size=(1, Hkv, 300, D))
+    mb = np.zeros((1, nb, 4), dtype=np.uint64)
+    _, mb[0] = _random_tree(rng, 231, nb)
+    Ob = orc.tree_attention(Qb, Kb, Vb, np.array([41]), np.array([231]), mb, scale)
+    np.testing.assert_allclose(Ob, _sdpa_ref(Qb, Kb, Vb, np.array([41]), np.array([231]), mb, scale), atol=1e-12)
     # GQA == MHA with the kv heads repeated
     O2 = orc.tree_attention(Q, np.repeat(K, 2, axis=1), np.repeat(V, 2, axis=1), kv_len, n_nodes, mask, scale)
     np.testing.assert_allclose(O, O2, atol=1e-13)
