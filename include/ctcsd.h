@@ -200,7 +200,9 @@ int ctcsd_tree_attention(ctcsd_handle* h, void* stream, const void* Q, const voi
  * argmax of the LM head's distribution; Sec. 2.2: a draft is accepted only where it matches
  * the base model's greedy output; Sec. 3.3: the longest such candidate is the step's output).
  *   y[m,v] = sum_h hn[m,h] * Wl[v,h];  am[m] = argmax_v y[m,v], ties to the lower id.
- *   Walk: cur = root; while some child c of cur has node_tok[c] == am[cur]: accept c.
+ *   Walk: cur = root; while some child c of cur has node_tok[c] == am[cur]: accept c.  Siblings
+ *   carry distinct tokens in a tree from ctcsd_build_tree, so at most one child qualifies; in a
+ *   hand-made tree with equal siblings the longest agreeing path is taken, lowest id on ties.
  * hn [B*max_nodes,H] dtype (row b*max_nodes+i is node i of sequence b; rows of unused nodes
  *   are computed but ignored);  Wl [V,H] dtype;  node_tok, parent [B,max_nodes], n_nodes [B].
  * out_argmax [B,max_nodes] int32;  out_acc_len [B] int32 (accepted draft tokens, root and

@@ -1,5 +1,5 @@
-// Greedy acceptance walk over the token tree (paper Sec. 2.2 / Sec. 3.3: a drafted token is
-// kept only where it equals the base model's greedy choice; the longest such path wins).
+// Greedy acceptance over the token tree (paper Sec. 2.2 / Sec. 3.3: a drafted token is kept
+// only where it equals the base model's greedy choice; the longest such path wins).
 #pragma once
 
 #include "common.cuh"
@@ -17,110 +17,93 @@ struct AcceptParams {
 };
 
 #ifdef __CUDACC__
-// Executed by one full warp for sequence b: starting at the root, move to the child whose
-// token equals the arg-max at the current node; stop when no child matches.
-__device__ __forceinline__ void greedy_accept_warp(const AcceptParams& p, int b, int lane) {
-    const int n_max = p.max_nodes;
-    int n = p.n_nodes[b];
-    n = n < 1 ? 1 : (n > n_max ? n_max : n);
-    const int* tok = p.node_tok + (size_t)b * n_max;
-    const int* par = p.parent + (size_t)b * n_max;
-    const int* am = p.argmax + (size_t)b * n_max;
-    int cur = 0, len = 0;
-    while (len < p.T) {
-        const int want = am[cur];
-        int found = -1;
-        for (int base = 0; base < n && found < 0; base += 32) {
-            int c = base + lane;
-            bool hit = c >= 1 && c < n && par[c] == cur && tok[c] == want;
-            unsigned bal = __ballot_sync(0xffffffffu, hit);
-            if (bal) found = base + __ffs(bal) - 1;
-        }
-        if (found < 0) break;
-        if (lane == 0) {
-            p.acc_nodes[(size_t)b * p.T + len] = found;
-            p.acc_tok[(size_t)b * p.T + len] = want;
-        }
-        cur = found;
-        ++len;
-    }
-    for (int l = len + lane; l < p.T; l += 32) {
-        p.acc_nodes[(size_t)b * p.T + l] = -1;
-        p.acc_tok[(size_t)b * p.T + l] = -1;
-    }
-    if (lane == 0) {
-        p.acc_len[b] = len;
-        p.next_tok[b] = am[cur];
-    }
-}
+constexpr int kAcceptScratchInts = 3 * CTCSD_MAX_NODES;     // shared-memory ints one warp needs
 
-// Acceptance on the raw tree, executed by one full warp for sequence b (at most 256 nodes).  A
-// kept node d follows kept node p when nka[d] == p; best[p] = longest chain p -> d1 -> d2 ... in
-// which every node's token equals the arg-max at its predecessor; among equally long
-// continuations the lowest node id wins.  Lane l holds nodes l, l+32, ..., l+224.
-__device__ __forceinline__ void raw_accept_warp(const AcceptParams& p, int b, int lane) {
+// Acceptance for sequence b, executed by one full warp; `scratch` is kAcceptScratchInts ints of
+// shared memory owned by this warp.
+//
+// Node d follows node a(d): its parent in the packed tree, its nearest kept ancestor in the raw
+// tree (removed nodes follow nobody).  d agrees when its token equals the arg-max at a(d).  The
+// accepted path is the longest chain root -> d1 -> d2 ... of agreeing nodes; among equally long
+// continuations the lowest node id wins at every level.  (In the packed tree siblings carry
+// distinct tokens, so at most one child agrees and this is the plain greedy walk.)
+//
+// Three passes, each over all nodes at once (lane l holds nodes l, l+32, ...), so the cost does
+// not grow with the tree: (1) level[d] = length of the agreeing chain that reaches d, found
+// level by level; (2) from the deepest level up, every reached node offers 1 + its own best
+// continuation to the node it follows (a shared-memory maximum over (length, lowest id));
+// (3) the walk from the root along the recorded best followers.
+__device__ __forceinline__ void accept_warp(const AcceptParams& p, int b, int lane, int* scratch) {
+    constexpr int kQ = CTCSD_MAX_NODES / 32;                // nodes per lane
     const int n_max = p.max_nodes;
     int n = p.n_nodes[b];
     n = n < 1 ? 1 : (n > n_max ? n_max : n);
-    const int* am = p.argmax + (size_t)b * n_max;
-    constexpr int kQ = 8;                              // nodes per lane
-    int tok[kQ], kp[kQ], na[kQ], best[kQ], succ[kQ];
+    int* s_am = scratch;                                    // arg-max at each node
+    int* s_level = scratch + CTCSD_MAX_NODES;               // -1: not reached
+    unsigned* s_best = reinterpret_cast<unsigned*>(scratch + 2 * CTCSD_MAX_NODES);   // (length << 16) | (0xffff - follower)
+    const bool raw = p.kept != nullptr;
+    const int* follows = (raw ? p.nka : p.parent) + (size_t)b * n_max;
+
+    int tok[kQ], fo[kQ], level[kQ];
 #pragma unroll
     for (int q = 0; q < kQ; ++q) {
         const int d = lane + 32 * q;
-        const bool in = d < n;
+        const bool in = d >= 1 && d < n;
         tok[q] = in ? p.node_tok[(size_t)b * n_max + d] : -1;
-        kp[q] = in ? p.kept[(size_t)b * n_max + d] : 0;
-        na[q] = in ? p.nka[(size_t)b * n_max + d] : -2;
-        best[q] = 0;
-        succ[q] = -1;
+        int f = in ? follows[d] : -1;
+        if (raw && in && p.kept[(size_t)b * n_max + d] == 0) f = -1;
+        fo[q] = (f >= 0 && f < n) ? f : -1;
+        level[q] = -1;
+        if (d < CTCSD_MAX_NODES) {
+            s_am[d] = d < n ? p.argmax[(size_t)b * n_max + d] : -1;
+            s_level[d] = d == 0 ? 0 : -1;
+            s_best[d] = 0u;
+        }
     }
-    for (int pn = n - 1; pn >= 0; --pn) {
-        const int owner = pn & 31, oq = pn >> 5;
-        int pk = 0;
+    __syncwarp();
+    bool agrees[kQ];
 #pragma unroll
-        for (int q = 0; q < kQ; ++q) pk = (q == oq) ? kp[q] : pk;
-        pk = __shfl_sync(0xffffffffu, pk, owner);
-        if (!pk) continue;                                      // uniform
-        const int want = am[pn];
-        // this lane's best follower: longer chain first, then lower id
-        int val = 0, who = 0x7fffffff;
+    for (int q = 0; q < kQ; ++q) agrees[q] = fo[q] >= 0 && tok[q] == s_am[fo[q]];
+
+    // (1) levels
+    int deepest = 0;
+    for (int r = 1; r <= p.T; ++r) {
+        bool any = false;
 #pragma unroll
         for (int q = 0; q < kQ; ++q) {
-            const int d = lane + 32 * q;
-            if (d > pn && kp[q] && na[q] == pn && tok[q] == want) {
-                const int v = 1 + best[q];
-                if (v > val || (v == val && d < who)) { val = v; who = d; }
+            if (agrees[q] && level[q] < 0 && s_level[fo[q]] == r - 1) { level[q] = r; any = true; }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < kQ; ++q)
+            if (level[q] == r) s_level[lane + 32 * q] = r;
+        __syncwarp();
+        if (!__any_sync(0xffffffffu, any)) break;
+        deepest = r;
+    }
+    // (2) best continuation, deepest level first
+    for (int r = deepest; r >= 1; --r) {
+#pragma unroll
+        for (int q = 0; q < kQ; ++q) {
+            if (level[q] == r) {
+                const int d = lane + 32 * q;
+                const unsigned len = 1u + (s_best[d] >> 16);
+                atomicMax(&s_best[fo[q]], (len << 16) | (0xffffu - (unsigned)d));
             }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const int v2 = __shfl_xor_sync(0xffffffffu, val, o);
-            const int w2 = __shfl_xor_sync(0xffffffffu, who, o);
-            if (v2 > val || (v2 == val && w2 < who)) { val = v2; who = w2; }
-        }
-        if (lane == owner) {
-#pragma unroll
-            for (int q = 0; q < kQ; ++q)
-                if (q == oq) { best[q] = val; succ[q] = val > 0 ? who : -1; }
-        }
+        __syncwarp();
     }
+    // (3) the walk
     int cur = 0, len = 0;
     while (len < p.T) {
-        int sc = -1;
-#pragma unroll
-        for (int q = 0; q < kQ; ++q) sc = (q == (cur >> 5)) ? succ[q] : sc;
-        sc = __shfl_sync(0xffffffffu, sc, cur & 31);
-        if (sc < 0) break;
-        cur = sc;
-        int tk = -1;
-#pragma unroll
-        for (int q = 0; q < kQ; ++q) tk = (q == (cur >> 5)) ? tok[q] : tk;
-        tk = __shfl_sync(0xffffffffu, tk, cur & 31);
+        const unsigned e = s_best[cur];
+        if ((e >> 16) == 0u) break;
+        const int nxt = (int)(0xffffu - (e & 0xffffu));
         if (lane == 0) {
-            p.acc_nodes[(size_t)b * p.T + len] = cur;
-            p.acc_tok[(size_t)b * p.T + len] = tk;
+            p.acc_nodes[(size_t)b * p.T + len] = nxt;
+            p.acc_tok[(size_t)b * p.T + len] = s_am[cur];      // an agreeing node's token is the arg-max before it
         }
+        cur = nxt;
         ++len;
     }
     for (int l = len + lane; l < p.T; l += 32) {
@@ -129,14 +112,9 @@ __device__ __forceinline__ void raw_accept_warp(const AcceptParams& p, int b, in
     }
     if (lane == 0) {
         p.acc_len[b] = len;
-        p.next_tok[b] = am[cur];
+        p.next_tok[b] = s_am[cur];
     }
-}
-
-// Dispatch on the layout.
-__device__ __forceinline__ void accept_warp(const AcceptParams& p, int b, int lane) {
-    if (p.kept != nullptr) raw_accept_warp(p, b, lane);
-    else greedy_accept_warp(p, b, lane);
+    __syncwarp();
 }
 #endif
 

@@ -283,8 +283,10 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         p.keys[row] = 0ull;
     }
     __syncthreads();
+    // the pipeline stages are idle now: their shared memory serves as the acceptance scratch
     if (good)
-        for (int b = warp; b < p.acc.B; b += kThreads / 32) accept_warp(p.acc, b, lane);
+        for (int b = warp; b < p.acc.B; b += kThreads / 32)
+            accept_warp(p.acc, b, lane, reinterpret_cast<int*>(dyn) + warp * kAcceptScratchInts);
     if (tid == 0) *p.counter = 0u;
 }
 

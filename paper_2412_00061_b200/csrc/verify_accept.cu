@@ -9,7 +9,8 @@ namespace {
 
 // One warp per sequence (used when the arg-max comes from the CUDA-core path).
 __global__ void __launch_bounds__(32) greedy_accept_kernel(AcceptParams p) {
-    accept_warp(p, blockIdx.x, threadIdx.x);
+    __shared__ int scratch[kAcceptScratchInts];
+    accept_warp(p, blockIdx.x, threadIdx.x, scratch);
 }
 
 }  // namespace
