@@ -1,5 +1,6 @@
 // Handle management, configuration checks and workspace layout for the ctcsd C ABI.
 #include "common.cuh"
+#include "lm_head_tc.cuh"
 
 #include <stdlib.h>
 #include <string.h>
@@ -49,7 +50,7 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
             const int classes = c.V + 1;
             const int nt = classes >= 224 ? 224 : (classes + 15) / 16 * 16;
             const size_t tiles = (size_t)c.T * ((classes + nt - 1) / nt);
-            l.tc_part_bytes = sizeof(DraftPartial) * tiles * (size_t)((rows + 127) / 128 * 128);
+            l.tc_part_bytes = sizeof(DraftPartial) * tiles * kDraftColSplit * (size_t)((rows + 127) / 128 * 128);
             off = align_up(off + l.tc_part_bytes, 256);
         }
     }

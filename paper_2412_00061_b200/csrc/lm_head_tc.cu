@@ -22,11 +22,15 @@
 namespace ctcsd {
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kColSplit = kDraftColSplit;   // epilogue warps per TMEM lane quarter: each takes every 4th 32-column chunk
+constexpr int kEpiWarps = 4 * kColSplit;
+constexpr int kThreads = 64 + 32 * kEpiWarps;   // TMA warp, MMA warp, epilogue warps
 constexpr int kBlockK = 64;                 // bf16 elements per 128-byte swizzle row
 constexpr int kTileM = 128;
 constexpr int kABytes = kTileM * 128;       // 16 KB
 constexpr int kMaxStages = 8;
+constexpr int kAccCols = 256;               // TMEM columns per accumulator (tiles are at most 256 wide)
+constexpr int kTmemCols = 2 * kAccCols;
 
 struct TcParams {
     int M;            // activation rows
@@ -46,7 +50,7 @@ struct TcParams {
     // draft mode: W is [slots][V][H]; n_tiles = slots * tiles_per_slot
     int slots;
     int tiles_per_slot;
-    DraftPartial* part;       // [n_tiles][m_tiles*128] per-tile states
+    DraftPartial* part;       // [n_tiles][kColSplit][m_tiles*128] per-tile, per-column-share states
     const int* row_seq;       // [M] or null
     const float* blank_bias;  // [B] or null; added to class V-1 of every slot
 };
@@ -54,8 +58,8 @@ struct TcParams {
 struct __align__(8) TcShared {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t tmem_full;
-    uint64_t tmem_empty;
+    uint64_t tmem_full[2];      // two accumulators: the epilogue of one tile runs under the next tile's MMAs
+    uint64_t tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
     int is_last;
@@ -81,15 +85,14 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
-        tc::mbar_init(&sh->tmem_full, 1);
-        tc::mbar_init(&sh->tmem_empty, 4);
+        for (int a = 0; a < 2; ++a) { tc::mbar_init(&sh->tmem_full[a], 1); tc::mbar_init(&sh->tmem_empty[a], kEpiWarps); }
         sh->abort_flag = 0;
         sh->is_last = 0;
         sh->never_set = 0;
         tc::fence_barrier_init();
     }
     if (warp == 1) {
-        tc::tmem_alloc(&sh->tmem_base, 256);
+        tc::tmem_alloc(&sh->tmem_base, kTmemCols);
         tc::tmem_relinquish();
     }
     tc::tc_fence_before_sync();
@@ -177,7 +180,9 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int it = 0, ucount = 0;
             bool ok = true;
             for (int u = u0; u < u1 && ok; ++u, ++ucount) {
-                if (!tc::mbar_wait(&sh->tmem_empty, ((uint32_t)ucount & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                const int acc = ucount & 1;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
+                if (!tc::mbar_wait(&sh->tmem_empty[acc], ((uint32_t)(ucount >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after_sync();
                 for (int kb = 0; kb < p.num_k; ++kb, ++it) {
                     const int s = it % p.stages;
@@ -190,11 +195,11 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k) {
                         // advancing 16 bf16 along K = 32 bytes = 2 descriptor address units
-                        tc::mma_bf16_ss(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc::mma_bf16_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     tc::mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
                 }
-                if (ok) tc::mma_commit(&sh->tmem_full);
+                if (ok) tc::mma_commit(&sh->tmem_full[acc]);
             }
             if (!ok) {
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 2);
@@ -204,8 +209,9 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     } else {
         // ---------------- epilogue ----------------
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int cs = (warp - 2) >> 2;               // which share of the tile's columns
         const int row_in_tile = q * 32 + lane;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         int ucount = 0;
         bool ok = true;
         for (int u = u0; u < u1 && ok; ++u, ++ucount) {
@@ -216,7 +222,9 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int n0 = (MODE == 1 ? nt - t * p.tiles_per_slot : nt) * p.Nt;
             float bias = 0.f;
             if (MODE == 1 && p.blank_bias != nullptr && row < p.M) bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
-            if (!tc::mbar_wait(&sh->tmem_full, (uint32_t)ucount & 1u, abort_flag)) { ok = false; break; }
+            const int acc = ucount & 1;
+            const uint32_t lane_addr = lane_base + (uint32_t)(acc * kAccCols);
+            if (!tc::mbar_wait(&sh->tmem_full[acc], (uint32_t)(ucount >> 1) & 1u, abort_flag)) { ok = false; break; }
             tc::tc_fence_after_sync();
             float best = -INFINITY;
             int best_idx = 0x7fffffff;
@@ -224,7 +232,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if constexpr (MODE == 1) st.init();
             // a warp whose 32 rows lie past the last activation row has nothing to read
             const int c_end = (mt * kTileM + q * 32 < p.M) ? p.Nt : 0;
-            for (int c0 = 0; c0 < c_end; c0 += 32) {
+            for (int c0 = cs * 32; c0 < c_end; c0 += 32 * kColSplit) {
                 uint32_t r[32];
                 if (c0 + 32 <= p.Nt) {
                     tc::tmem_ld32(lane_addr + (uint32_t)c0, r);
@@ -254,9 +262,9 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
             tc::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&sh->tmem_empty);
+            if (lane == 0) tc::mbar_arrive(&sh->tmem_empty[acc]);
             if constexpr (MODE == 1) {
-                st.store(p.part + (size_t)nt * (p.m_tiles * kTileM) + row);
+                st.store(p.part + ((size_t)nt * kColSplit + cs) * (p.m_tiles * kTileM) + row);
             } else {
             // fold this tile's winner into the row's global maximum: larger logit first, equal
             // logits -> lower id (the id is stored complemented in the low word)
@@ -279,7 +287,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     if (warp == 1) {
         tc::tc_fence_after_sync();
-        tc::tmem_dealloc(tmem_base, 256);
+        tc::tmem_dealloc(tmem_base, kTmemCols);
     }
     if constexpr (MODE == 1) return;                 // the tiles are merged by draft_tc_merge_kernel
     if (tid == 0) {
@@ -298,8 +306,13 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     // the pipeline stages are idle now: their shared memory serves as the acceptance scratch
     if (good)
-        for (int b = warp; b < p.acc.B; b += kThreads / 32)
-            accept_warp(p.acc, b, lane, reinterpret_cast<int*>(dyn) + warp * kAcceptScratchInts);
+    {
+        int aw = (int)(((size_t)p.stages * stage_bytes) / (kAcceptScratchInts * sizeof(int)));
+        aw = aw < kThreads / 32 ? aw : kThreads / 32;          // warps the stage memory can serve (>= 1)
+        if (warp < aw)
+            for (int b = warp; b < p.acc.B; b += aw)
+                accept_warp(p.acc, b, lane, reinterpret_cast<int*>(dyn) + warp * kAcceptScratchInts);
+    }
     if (tid == 0) *p.counter = 0u;
 }
 
@@ -349,7 +362,7 @@ bool make_map3(CUtensorMap* map, const void* base, long long slots, long long ro
 }
 
 struct DraftMergeParams {
-    const DraftPartial* part;     // [slots * tiles_per_slot][mpad]
+    const DraftPartial* part;     // [slots * tiles_per_slot * kColSplit][mpad]
     int M, mpad, slots, tiles_per_slot, k;
     int* out_topk_id; float* out_topk_lp; float* out_lse;
 };
@@ -365,8 +378,9 @@ __global__ void __launch_bounds__(128) draft_tc_merge_kernel(DraftMergeParams p)
     const int m = (int)(wid / p.slots), t = (int)(wid - (long long)m * p.slots);
     RunState fs;
     fs.init();
-    for (int e = lane; e < p.tiles_per_slot; e += 32)
-        fs.absorb(load_partial_cg(p.part + ((size_t)t * p.tiles_per_slot + e) * p.mpad + m));
+    const int entries = p.tiles_per_slot * kColSplit;          // per tile: one state per column share
+    for (int e = lane; e < entries; e += 32)
+        fs.absorb(load_partial_cg(p.part + ((size_t)t * entries + e) * p.mpad + m));
     warp_combine(fs);
     if (lane == 0) {
         const float lse = fs.mx + logf(fs.sum);
@@ -409,7 +423,7 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     p.slots = c.T;
     p.tiles_per_slot = (p.V + p.Nt - 1) / p.Nt;
     p.n_tiles = p.slots * p.tiles_per_slot;
-    const size_t need = sizeof(DraftPartial) * (size_t)p.n_tiles * p.m_tiles * kTileM;
+    const size_t need = sizeof(DraftPartial) * (size_t)p.n_tiles * kColSplit * p.m_tiles * kTileM;
     if (need > h->lay.tc_part_bytes) return CTCSD_ERR_WORKSPACE;
     p.a_bytes = kABytes;
     const int stage_bytes = p.a_bytes + p.Nt * 128;

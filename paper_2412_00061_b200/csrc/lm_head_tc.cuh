@@ -20,6 +20,9 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
 // kernel over the tiles of every slot.
 bool draft_head_tc_supported(const Handle* h, int M);
 int draft_tc_tile_rows(int classes);
+// Each vocabulary tile of the tensor-core draft head leaves this many partial states per row
+// (its epilogue warps split the tile's columns).
+constexpr int kDraftColSplit = 4;
 int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, const void* Wd, const int* row_seq,
                          const float* blank_bias, int* out_topk_id, float* out_topk_lp, float* out_lse,
                          float* out_logits_dbg);
