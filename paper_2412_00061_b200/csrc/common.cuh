@@ -165,6 +165,23 @@ __device__ __forceinline__ void topk_insert(float (&val)[kTopSlots], int (&id)[k
     }
 }
 
+// The same with only the first KS entries of the list in use (the others stay at their initial
+// "nothing" value): a caller that needs at most KS winners pays for KS slots.
+template <int KS>
+__device__ __forceinline__ void topk_insert_n(float (&val)[kTopSlots], int (&id)[kTopSlots], float v, int i) {
+    static_assert(KS >= 1 && KS <= kTopSlots, "slot count");
+    if (!ranks_before(v, i, val[KS - 1], id[KS - 1])) return;
+#pragma unroll
+    for (int s = KS - 1; s >= 0; --s) {
+        bool shift = (s > 0) && ranks_before(v, i, val[s - 1], id[s - 1]);
+        bool here = !shift && ranks_before(v, i, val[s], id[s]);
+        float pv = (s > 0) ? val[s - 1] : 0.f;
+        int pi = (s > 0) ? id[s - 1] : 0;
+        if (shift) { val[s] = pv; id[s] = pi; }
+        else if (here) { val[s] = v; id[s] = i; }
+    }
+}
+
 // Programmatic dependent launch.  Every kernel of the step is launched so that it may start
 // while its predecessor in the stream is still draining: what it does before pdl_wait() (set
 // up shared memory and barriers, prefetch weights, which no kernel ever writes) overlaps with the

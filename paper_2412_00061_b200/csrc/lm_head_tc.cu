@@ -50,6 +50,7 @@ struct TcParams {
     // draft mode: W is [slots][V][H]; n_tiles = slots * tiles_per_slot
     int slots;
     int tiles_per_slot;
+    int topk;                 // k: symbols kept per slot
     DraftPartial* part;       // [n_tiles][kColSplit][m_tiles*128] per-tile, per-column-share states
     const int* row_seq;       // [M] or null
     const float* blank_bias;  // [B] or null; added to class V-1 of every slot
@@ -210,6 +211,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // ---------------- epilogue ----------------
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int cs = (warp - 2) >> 2;               // which share of the tile's columns
+        const bool few = MODE == 1 && p.topk <= 4;    // draft mode: a four-entry list is enough
         const int row_in_tile = q * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         int ucount = 0;
@@ -224,7 +226,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (MODE == 1 && p.blank_bias != nullptr && row < p.M) bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
             const int acc = ucount & 1;
             const uint32_t lane_addr = lane_base + (uint32_t)(acc * kAccCols);
-            if (!tc::mbar_wait(&sh->tmem_full[acc], (uint32_t)(ucount >> 1) & 1u, abort_flag)) { ok = false; break; }
+            if (!tc::mbar_wait_idle(&sh->tmem_full[acc], (uint32_t)(ucount >> 1) & 1u, abort_flag)) { ok = false; break; }
             tc::tc_fence_after_sync();
             float best = -INFINITY;
             int best_idx = 0x7fffffff;
@@ -255,7 +257,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                             if (col == p.V - 1) v += bias;
                             if (p.logits_dbg != nullptr && row < p.M)
                                 p.logits_dbg[((size_t)row * p.slots + t) * p.V + col] = v;
-                            st.push(v, col);
+                            if (few) st.push_n<4>(v, col); else st.push(v, col);
                         }
                     }
                 }
@@ -421,6 +423,7 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     p.m_tiles = (M + kTileM - 1) / kTileM;
     p.Nt = draft_tc_tile_rows(p.V);
     p.slots = c.T;
+    p.topk = c.k;
     p.tiles_per_slot = (p.V + p.Nt - 1) / p.Nt;
     p.n_tiles = p.slots * p.tiles_per_slot;
     const size_t need = sizeof(DraftPartial) * (size_t)p.n_tiles * kColSplit * p.m_tiles * kTileM;

@@ -29,6 +29,17 @@ struct RunState {
         }
         topk_insert(val, id, z, v);
     }
+    // push() keeping only the best KS logits
+    template <int KS>
+    __device__ __forceinline__ void push_n(float z, int v) {
+        if (z > mx) {
+            sum = sum * __expf(mx - z) + 1.f;
+            mx = z;
+        } else {
+            sum += __expf(z - mx);
+        }
+        topk_insert_n<KS>(val, id, z, v);
+    }
     __device__ __forceinline__ void absorb(const DraftPartial& q) {
         if (q.mx == -INFINITY) return;
         float nm = fmaxf(mx, q.mx);

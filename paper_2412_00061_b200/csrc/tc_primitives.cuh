@@ -54,6 +54,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
+// The same wait for warps that expect to wait long (an epilogue waiting for a whole tile): the
+// warp sleeps between polls, so that a dozen waiting warps do not take issue slots and shared-
+// memory bandwidth from the warps that feed the tensor core.
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               unsigned sleep_ns = 400u, long long limit_cycles = (1ll << 31)) {
+    if (mbar_test(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (true) {
+        __nanosleep(sleep_ns);
+        if (mbar_test(bar, parity)) return true;
+        if (((++spins) & 15) == 0) {
+            if (*abort_flag != 0) return false;
+            if (clock64() - t0 > limit_cycles) return false;
+        }
+    }
+}
+
 // ---- TMA ----------------------------------------------------------------------------------
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
