@@ -40,6 +40,10 @@ struct TcParams {
     int n_tiles;      // vocabulary tiles
     int m_tiles;      // row tiles of 128
     int stages;
+    int pair;         // 1: a stage holds two activation row tiles that share its weight tile
+                      //    (both accumulators in use, one per row tile); 0: one row tile per stage,
+                      //    the accumulators alternate between consecutive tiles
+    int m_units;      // row tiles (pair = 0) or pairs of row tiles (pair = 1)
     int a_bytes;      // bytes of the activation tile a stage holds: 128 rows, or 64 when M <= 64
     unsigned long long* keys; // [m_tiles*128] packed (logit, id) maxima, zero between calls
     AcceptParams acc;
@@ -78,7 +82,8 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
     const uint32_t raw_addr = tc::smem_u32(dyn_raw);
     unsigned char* dyn = dyn_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-    const int stage_bytes = p.a_bytes + p.Nt * 128;
+    const int a_all = p.a_bytes * (1 + p.pair);             // activation bytes of a stage
+    const int stage_bytes = a_all + p.Nt * 128;
     TcShared* sh = reinterpret_cast<TcShared*>(dyn + (size_t)p.stages * stage_bytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -100,7 +105,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
-    const long long units = (long long)p.n_tiles * p.m_tiles;
+    const long long units = (long long)p.n_tiles * p.m_units;
     const int u0 = (int)(units * blockIdx.x / gridDim.x);
     const int u1 = (int)(units * (blockIdx.x + 1) / gridDim.x);
 
@@ -113,7 +118,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint64_t pol_a = tc::policy_evict_last();
     auto load_stage = [&](int it, bool do_w, bool do_a) {
         const int u = u0 + it / p.num_k, kb = it - (it / p.num_k) * p.num_k;
-        const int nt = u / p.m_tiles, mt = u - nt * p.m_tiles;
+        const int nt = u / p.m_units, mu = u - nt * p.m_units;
         const int s = it % p.stages;
         unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
         int kq = kb + k_start;
@@ -121,13 +126,18 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (do_w) {
             tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)stage_bytes);
             if constexpr (MODE == 0) {
-                tc::tma_load_2d(a_dst + p.a_bytes, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
+                tc::tma_load_2d(a_dst + a_all, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
             } else {
                 const int t = nt / p.tiles_per_slot, ntl = nt - t * p.tiles_per_slot;
-                tc::tma_load_3d(a_dst + p.a_bytes, &tmW, &sh->full[s], kq * kBlockK, ntl * p.Nt, t, pol_w);
+                tc::tma_load_3d(a_dst + a_all, &tmW, &sh->full[s], kq * kBlockK, ntl * p.Nt, t, pol_w);
             }
         }
-        if (do_a) tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kq * kBlockK, mt * kTileM, pol_a);
+        if (do_a) {
+            // a row tile past the last one (odd tile count in pair mode) reads as zeros
+            for (int h = 0; h <= p.pair; ++h)
+                tc::tma_load_2d(a_dst + h * p.a_bytes, &tmA, &sh->full[s], kq * kBlockK,
+                                ((p.pair ? 2 * mu : mu) + h) * kTileM, pol_a);
+        }
     };
     // The weights are never written by any kernel: their tiles of the first stages are requested
     // before this kernel waits for its predecessor in the stream.
@@ -181,9 +191,10 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int it = 0, ucount = 0;
             bool ok = true;
             for (int u = u0; u < u1 && ok; ++u, ++ucount) {
-                const int acc = ucount & 1;
+                const int acc = p.pair ? 0 : (ucount & 1);            // barrier pair that guards this unit
+                const uint32_t acc_ph = (uint32_t)(p.pair ? ucount : (ucount >> 1)) & 1u;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
-                if (!tc::mbar_wait(&sh->tmem_empty[acc], ((uint32_t)(ucount >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                if (!tc::mbar_wait(&sh->tmem_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after_sync();
                 for (int kb = 0; kb < p.num_k; ++kb, ++it) {
                     const int s = it % p.stages;
@@ -192,11 +203,17 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     tc::tc_fence_after_sync();
                     const uint32_t a_addr = tc::smem_u32(dyn + (size_t)s * stage_bytes);
                     const uint64_t adesc = tc::smem_desc_k_sw128(a_addr);
-                    const uint64_t bdesc = tc::smem_desc_k_sw128(a_addr + p.a_bytes);
+                    const uint64_t bdesc = tc::smem_desc_k_sw128(a_addr + a_all);
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k) {
                         // advancing 16 bf16 along K = 32 bytes = 2 descriptor address units
                         tc::mma_bf16_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    if (p.pair) {                            // the second row tile against the same weights
+                        const uint64_t adesc1 = tc::smem_desc_k_sw128(a_addr + p.a_bytes);
+#pragma unroll
+                        for (int k = 0; k < kBlockK / 16; ++k)
+                            tc::mma_bf16_ss(d_tmem + kAccCols, adesc1 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     tc::mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
                 }
@@ -217,17 +234,20 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int ucount = 0;
         bool ok = true;
         for (int u = u0; u < u1 && ok; ++u, ++ucount) {
-            const int nt = u / p.m_tiles, mt = u - nt * p.m_tiles;
-            const int row = mt * kTileM + row_in_tile;
+            const int nt = u / p.m_units, mu = u - nt * p.m_units;
             // draft mode: tile nt is tile ntl of slot t
             const int t = MODE == 1 ? nt / p.tiles_per_slot : 0;
             const int n0 = (MODE == 1 ? nt - t * p.tiles_per_slot : nt) * p.Nt;
+            const int acc = p.pair ? 0 : (ucount & 1);
+            const uint32_t acc_ph = (uint32_t)(p.pair ? ucount : (ucount >> 1)) & 1u;
+            if (!tc::mbar_wait_idle(&sh->tmem_full[acc], acc_ph, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after_sync();
+            for (int h = 0; h <= p.pair; ++h) {               // pair mode: accumulator h holds row tile 2*mu + h
+            const int mt = p.pair ? 2 * mu + h : mu;
+            const int row = mt * kTileM + row_in_tile;
             float bias = 0.f;
             if (MODE == 1 && p.blank_bias != nullptr && row < p.M) bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
-            const int acc = ucount & 1;
-            const uint32_t lane_addr = lane_base + (uint32_t)(acc * kAccCols);
-            if (!tc::mbar_wait_idle(&sh->tmem_full[acc], (uint32_t)(ucount >> 1) & 1u, abort_flag)) { ok = false; break; }
-            tc::tc_fence_after_sync();
+            const uint32_t lane_addr = lane_base + (uint32_t)((p.pair ? h : acc) * kAccCols);
             float best = -INFINITY;
             int best_idx = 0x7fffffff;
             RunState st;
@@ -262,9 +282,11 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     }
                 }
             }
-            tc::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&sh->tmem_empty[acc]);
+            if (h == p.pair) {                                // the last accumulator of the unit has been read
+                tc::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&sh->tmem_empty[acc]);
+            }
             if constexpr (MODE == 1) {
                 st.store(p.part + ((size_t)nt * kColSplit + cs) * (p.m_tiles * kTileM) + row);
             } else {
@@ -274,6 +296,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 const unsigned u = __float_as_uint(best);
                 const unsigned sortable = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
                 atomicMax(p.keys + row, ((unsigned long long)sortable << 32) | (0xffffffffu - (unsigned)best_idx));
+            }
             }
             }
         }
@@ -429,6 +452,8 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     const size_t need = sizeof(DraftPartial) * (size_t)p.n_tiles * kColSplit * p.m_tiles * kTileM;
     if (need > h->lay.tc_part_bytes) return CTCSD_ERR_WORKSPACE;
     p.a_bytes = kABytes;
+    p.pair = 0;                                      // the heavy epilogue needs the other accumulator for overlap
+    p.m_units = p.m_tiles;
     const int stage_bytes = p.a_bytes + p.Nt * 128;
     int stages = (int)((220 * 1024 - (int)sizeof(TcShared) - 1024) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
@@ -490,7 +515,11 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     // belong to no activation row and are never looked at.
     const bool half_a = M <= 64 && p.Nt * 128 >= kABytes / 2;
     p.a_bytes = half_a ? kABytes / 2 : kABytes;
-    const int stage_bytes = p.a_bytes + p.Nt * 128;
+    // Two or more row tiles: a weight stage feeds two of them, which halves the shared-memory fill
+    // per flop (with one row tile per 28 KB weight stage the tensor core waits for L2).
+    p.pair = p.m_tiles >= 2 ? 1 : 0;
+    p.m_units = p.pair ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    const int stage_bytes = p.a_bytes * (1 + p.pair) + p.Nt * 128;
     int stages = (int)((220 * 1024 - (int)sizeof(TcShared) - 1024) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return CTCSD_ERR_UNSUPPORTED;
@@ -508,7 +537,7 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
 
     const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    long long units = (long long)p.n_tiles * p.m_tiles;
+    long long units = (long long)p.n_tiles * p.m_units;
     int grid = (int)(units < h->num_sms ? units : h->num_sms);
     CTCSD_CUDA_CHECK(h, launch_pdl(lm_head_tc_kernel<0>, dim3(grid), dim3(kThreads), smem, stream, 1, tmA, tmW, p));
     CTCSD_LAUNCH_CHECK(h);
