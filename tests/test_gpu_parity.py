@@ -158,6 +158,19 @@ def test_raw_layout_on_a_tree_above_128_nodes(name):
     assert max(r["n_nodes"]) > 128
 
 
+def test_empty_prefix_and_every_limit_at_once():
+    """kv_len = 0 (the tree attends to nothing but itself) on both attention kernels' dtypes, and a
+    configuration that sits on every documented maximum at once: T = 8 slots, k = 8 symbols per
+    slot (T*k = 64), beam 128, 64 candidates, 256 tree nodes."""
+    for base in ("c2s", "c1d64"):
+        _run(SMALL[base].replace(name=base + "_kv0", kv_lo=0, kv_hi=0), seed=2)
+    _run(C["c1"].replace(name="c1_kv0", kv_lo=0, kv_hi=0), seed=2)
+    top = C["c4"].replace(name="limits", B=2, H=512, V=1500, Hq=8, Hkv=4, kv_lo=50, kv_hi=700,
+                          T=8, k=8, beam=128, topN=64, max_nodes=256)
+    r = _run(top, seed=1)
+    assert max(r["n_nodes"]) > 128
+
+
 RAW = {
     # the raw trie of N paths of T symbols has up to 1 + N*T nodes
     "c2raw": C["c2"].replace(name="c2raw", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200, max_nodes=96),
