@@ -118,7 +118,7 @@ class ClockSampler:
         return out
 
 
-def oracle_step(cfg, inp, sample_slots=None, layout="packed"):
+def oracle_step(cfg, inp, layout="packed"):
     """One pass of the CPU oracle over the step (definition mode, fp64).  Returns nothing:
     it is only timed."""
     import math

@@ -6,12 +6,15 @@
 //   D = fp32 accumulator in tensor memory: lane = hn row, column = vocabulary row.
 // Each CTA owns a contiguous range of (vocabulary tile, row tile) units, so every weight is
 // fetched from HBM once; the kernel is a weight stream whose math hides behind the loads.
-// Warp 0 issues TMA loads into a ring of shared-memory stages, warp 1 issues the MMAs,
-// warps 2..5 read the accumulator back (each warp its own 32 TMEM lanes) and keep the
-// running arg-max of their row.  Each tile's winner is folded into the row's global maximum
-// with one 64-bit atomic max on a packed (logit, complemented id) key, so ties go to the
-// lower id; the CTA that finishes last unpacks the keys, clears them for the next call and
-// runs the greedy acceptance walk.
+// Warp 0 issues TMA loads into a ring of shared-memory stages, warp 1 issues the MMAs, warps
+// 2..17 read the accumulator back: four warps per quarter of the TMEM lanes (a warp may only
+// read its own 32 lanes), each taking every fourth 32-column chunk of the tile, and keep the
+// running arg-max of their row.  There are two accumulators.  With one row tile they alternate
+// between consecutive units, so a unit's read-back runs under the next unit's MMAs; with more
+// rows a stage carries two row tiles against one weight tile and each gets an accumulator.
+// Each tile's winner is folded into the row's global maximum with one 64-bit atomic max on a
+// packed (logit, complemented id) key, so ties go to the lower id; the CTA that finishes last
+// unpacks the keys, clears them for the next call and runs the acceptance passes.
 #include "lm_head_tc.cuh"
 #include "tc_primitives.cuh"
 #include "run_state.cuh"
