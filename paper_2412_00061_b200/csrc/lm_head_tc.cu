@@ -395,20 +395,27 @@ struct DraftMergeParams {
     int* out_topk_id; float* out_topk_lp; float* out_lse;
 };
 
-// One warp per (activation row, slot): merges the per-tile states of the slot into the
-// log-sum-exp and the top-k of the row.
+// One CTA of four warps per (activation row, slot): every thread folds its share of the slot's
+// per-tile states, the warps combine theirs, and the first warp combines the four results into
+// the log-sum-exp and the top-k of the row.
 __global__ void __launch_bounds__(128) draft_tc_merge_kernel(DraftMergeParams p) {
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    __shared__ DraftPartial s_warp[4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long pair = blockIdx.x;
     pdl_wait();
     pdl_trigger();
-    if (wid >= (long long)p.M * p.slots) return;
-    const int m = (int)(wid / p.slots), t = (int)(wid - (long long)m * p.slots);
+    const int m = (int)(pair / p.slots), t = (int)(pair - (long long)m * p.slots);
     RunState fs;
     fs.init();
     const int entries = p.tiles_per_slot * kColSplit;          // per tile: one state per column share
-    for (int e = lane; e < entries; e += 32)
+    for (int e = threadIdx.x; e < entries; e += 128)
         fs.absorb(load_partial_cg(p.part + ((size_t)t * entries + e) * p.mpad + m));
+    warp_combine(fs);
+    if (lane == 0) fs.store(&s_warp[warp]);
+    __syncthreads();
+    if (warp != 0) return;
+    fs.init();
+    if (lane < 4) fs.absorb(s_warp[lane]);
     warp_combine(fs);
     if (lane == 0) {
         const float lse = fs.mx + logf(fs.sum);
@@ -482,8 +489,8 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     mp.part = p.part;
     mp.M = M; mp.mpad = p.m_tiles * kTileM; mp.slots = p.slots; mp.tiles_per_slot = p.tiles_per_slot; mp.k = c.k;
     mp.out_topk_id = out_topk_id; mp.out_topk_lp = out_topk_lp; mp.out_lse = out_lse;
-    const long long warps = (long long)M * p.slots;
-    CTCSD_CUDA_CHECK(h, launch_pdl(draft_tc_merge_kernel, dim3((unsigned)((warps + 3) / 4)), dim3(128), 0, stream, 1, mp));
+    const long long pairs = (long long)M * p.slots;           // one CTA each
+    CTCSD_CUDA_CHECK(h, launch_pdl(draft_tc_merge_kernel, dim3((unsigned)pairs), dim3(128), 0, stream, 1, mp));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
