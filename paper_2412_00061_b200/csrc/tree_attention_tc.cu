@@ -5,14 +5,15 @@
 // share a kv head use the same K/V tiles (GQA grouping).  Per tile of 128 keys:
 //   S[128 x 128] = Q K^T        tcgen05.mma, both operands K-major from shared memory (TMA,
 //                               128-byte swizzle), accumulator in tensor memory;
-//   softmax                     four warps, one thread per query row: the row is read from
+//   softmax                     eight warps, two threads per query row: the row is read from
 //                               tensor memory twice (max, then exp2 and sum), the ancestor mask
 //                               is applied to the columns that are tree nodes, P goes to shared
 //                               memory as bf16 in the K-major swizzled layout;
 //   O_tile[128 x D] = P V       tcgen05.mma with V as an MN-major operand (V is [key][d]);
 //   O = O * corr + O_tile       in the row's registers.
 // Warp 0 issues the TMA loads (Q once, K/V tiles into a two-stage ring), warp 1 issues the
-// MMAs, warps 2..5 are the softmax warps.  The KV splits of a query tile form a thread-block
+// MMAs, warps 2..9 are the softmax warps (two threads per query row: each takes half of a tile's keys
+// and half of O's columns).  The KV splits of a query tile form a thread-block
 // cluster and merge their (max, sum, O) rows through distributed shared memory.
 #include "tree_attention.cuh"
 #include "tc_primitives.cuh"
@@ -23,7 +24,8 @@
 namespace ctcsd {
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kSoftmaxWarps = 8;     // two per quarter of the TMEM lanes
+constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
 constexpr int kRows = 128;         // query rows per CTA
 constexpr int kKeys = 128;         // keys per tile
 constexpr int kStages = 2;         // K/V tile buffers
@@ -38,7 +40,13 @@ struct __align__(8) AttnShared {
     uint32_t tmem_base;
     int abort_flag;
     int never_set;
+    float xch[3][2][kRows];        // row maxima (two tile parities) and row sums exchanged between a row's two threads
 };
+
+// The two softmax warps that share a quarter of the TMEM lanes (64 threads) meet here.
+__device__ __forceinline__ void pair_barrier(int q) {
+    asm volatile("bar.sync %0, 64;" ::"r"(q + 1) : "memory");
+}
 
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -79,6 +87,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     constexpr int kPBytes = kRows * kKeys * 2;
     constexpr int RS = D + 4;                      // floats per row of the merge buffer
     constexpr int PER = D / 32;
+    constexpr int DO = D / 2;                      // O columns per softmax thread
     extern __shared__ unsigned char dyn_raw[];
     const uint32_t raw_addr = tc::smem_u32(dyn_raw);
     unsigned char* dyn = dyn_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
@@ -97,7 +106,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         tc::mbar_init(&sh->q_full, 1);
         for (int s = 0; s < kStages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
         tc::mbar_init(&sh->s_full, 1);
-        tc::mbar_init(&sh->p_full, 4);
+        tc::mbar_init(&sh->p_full, kSoftmaxWarps);
         tc::mbar_init(&sh->o_full, 1);
         sh->abort_flag = 0;
         sh->never_set = 0;
@@ -128,7 +137,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     const int ntile = blk1 - blk0;
 
     // softmax state of the row owned by this thread (softmax warps only)
-    float acc[D];
+    float acc[DO];
     float mx = -INFINITY, sum = 0.f;
     bool failed = false;
 
@@ -203,8 +212,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             }
         }
     } else {
-        // ---------------- softmax warps: thread = query row ----------------
+        // ---------------- softmax warps: two threads per query row ----------------
+        // Warps 2..5 take the first 64 keys of a tile and the first D/2 columns of O, warps 6..9
+        // the other halves; the two threads of a row meet at a 64-thread named barrier to agree on
+        // the tile's maximum.  Every softmax thread executes every one of those barriers, also
+        // after a wait has failed, so a failure cannot leave a partner waiting.
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;             // which half of the keys / of O's columns
+        const int kc0 = half * (kKeys / 2);           // first key column of this thread
+        const int oc0 = half * DO;                    // first O column of this thread
         const int rl = q * 32 + lane;                 // row of the tile
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const int r = qtile * kRows + rl;
@@ -223,17 +239,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             return w == 0 ? m0 : (w == 1 ? m1 : (w < W ? mrow[w] : 0ull));
         };
 #pragma unroll
-        for (int d = 0; d < D; ++d) acc[d] = 0.f;
+        for (int d = 0; d < DO; ++d) acc[d] = 0.f;
         const float sl2 = p.scale * 1.4426950408889634f;          // scores are kept in log2 units
         for (int it = 0; it < ntile; ++it) {
             const int key0 = (blk0 + it) * kKeys;
             const int s = it % kStages;
-            if (!tc::mbar_wait(&sh->s_full, (uint32_t)it & 1u, abort_flag)) { failed = true; break; }
+            if (!failed && !tc::mbar_wait(&sh->s_full, (uint32_t)it & 1u, abort_flag)) failed = true;
+            failed = __any_sync(0xffffffffu, failed);
             tc::tc_fence_after_sync();
             const bool tail = key0 + kKeys > L;       // the tile holds tree nodes or keys past the end
             // V rows past the last key may hold anything (the cache is only written up to there):
             // clear them, a zero weight does not cancel a NaN
-            if (key0 + rl >= Ltot) {
+            if (half == 0 && key0 + rl >= Ltot) {
                 unsigned char* vrow = KV + (size_t)s * 2 * kTileBytes + kTileBytes + rl * 128;
 #pragma unroll
                 for (int hh = 0; hh < DH; ++hh)
@@ -255,28 +272,34 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 if (sft > 32) bits |= mask_word(w + 1) << (64 - sft);
                 return (uint32_t)bits;
             };
-            // pass 1: row maximum
+            // pass 1: maximum over this thread's 64 keys, then over the row
             float bm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four chains instead of one
+            if (!failed) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < kKeys; c0 += 32) {
-                uint32_t v[32];
-                tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
-                const uint32_t vm = visible32(c0);
-                tc::tmem_ld_wait();
+                for (int c0 = kc0; c0 < kc0 + kKeys / 2; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
+                    const uint32_t vm = visible32(c0);
+                    tc::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if ((vm >> j) & 1u) bm4[j & 3] = fmaxf(bm4[j & 3], __uint_as_float(v[j]));
+                    for (int j = 0; j < 32; ++j)
+                        if ((vm >> j) & 1u) bm4[j & 3] = fmaxf(bm4[j & 3], __uint_as_float(v[j]));
+                }
             }
             float bm = fmaxf(fmaxf(bm4[0], bm4[1]), fmaxf(bm4[2], bm4[3]));
+            sh->xch[it & 1][half][rl] = bm;
+            pair_barrier(q);
+            bm = fmaxf(bm, sh->xch[it & 1][half ^ 1][rl]);
             bm *= sl2;                                 // scale > 0: the maximum commutes with it
             const float nm = fmaxf(mx, bm);
             const float ref = nm == -INFINITY ? 0.f : nm;
             const float corr = exp2_fast(mx - ref);    // exp2(-inf) = 0
             mx = nm;
-            // pass 2: P = exp2(S - max), row sum, P to shared memory as bf16 (K-major, 128-byte swizzle)
+            if (failed) continue;
+            // pass 2: P = exp2(S - max), partial row sum, P to shared memory as bf16 (K-major, 128-byte swizzle)
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-            for (int c0 = 0; c0 < kKeys; c0 += 32) {
+            for (int c0 = kc0; c0 < kc0 + kKeys / 2; c0 += 32) {
                 uint32_t v[32];
                 tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
                 tc::tmem_ld_wait();
@@ -306,19 +329,25 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             tc::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&sh->p_full);
-            // O = O * corr + O_tile
-            if (!tc::mbar_wait(&sh->o_full, (uint32_t)it & 1u, abort_flag)) { failed = true; break; }
+            // O = O * corr + O_tile, this thread's half of the columns
+            if (!tc::mbar_wait(&sh->o_full, (uint32_t)it & 1u, abort_flag)) failed = true;
+            failed = __any_sync(0xffffffffu, failed);
+            if (failed) continue;
             tc::tc_fence_after_sync();
 #pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
+            for (int c0 = 0; c0 < DO; c0 += 32) {
                 uint32_t v[32];
-                tc::tmem_ld32(tmem_o + lane_off + (uint32_t)c0, v);
+                tc::tmem_ld32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) acc[c0 + j] = fmaf(acc[c0 + j], corr, __uint_as_float(v[j]));
             }
             tc::tc_fence_before_sync();
         }
+        // the row's sum is the two halves' sums (both were kept against the same running maximum)
+        sh->xch[2][half][rl] = sum;
+        pair_barrier(q);
+        sum += sh->xch[2][half ^ 1][rl];
         if (failed && lane == 0) {
             if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 23);
             *abort_flag = 1;
@@ -336,14 +365,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     if (splits == 1) {
         if (warp >= 2 && good) {
             const int rl = (warp & 3) * 32 + lane;
+            const int half = (warp - 2) >> 2;
             const int r = qtile * kRows + rl;
             const int i = r / grp;
             if (i < p.max_nodes) {
                 const int hq = g * grp + (r - i * grp);
-                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.O) + (((size_t)b * p.max_nodes + i) * p.Hq + hq) * D;
+                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.O) +
+                                     (((size_t)b * p.max_nodes + i) * p.Hq + hq) * D + half * DO;
                 const float inv = (i < n && sum > 0.f) ? 1.f / sum : 0.f;
 #pragma unroll
-                for (int c = 0; c < D / 8; ++c) {
+                for (int c = 0; c < DO / 8; ++c) {
                     uint4 w;
                     w.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
                     w.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
@@ -360,12 +391,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     float* rowbuf = reinterpret_cast<float*>(KV);
     if (warp >= 2) {
         const int rl = (warp & 3) * 32 + lane;
+        const int half = (warp - 2) >> 2;
         float* dst = rowbuf + rl * RS;
 #pragma unroll
-        for (int c = 0; c < D / 4; ++c)
-            *reinterpret_cast<float4*>(dst + 4 * c) = make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
-        dst[D] = mx;
-        dst[D + 1] = sum;
+        for (int c = 0; c < DO / 4; ++c)
+            *reinterpret_cast<float4*>(dst + half * DO + 4 * c) =
+                make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+        if (half == 0) {
+            dst[D] = mx;
+            dst[D + 1] = sum;                      // already the whole row's sum
+        }
     }
     cluster_sync_all();
     const uint32_t base = tc::smem_u32(rowbuf);
