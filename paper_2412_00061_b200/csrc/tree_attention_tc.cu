@@ -34,7 +34,7 @@ struct __align__(8) AttnShared {
     uint64_t q_full;
     uint64_t full[kStages];        // K and V tile landed
     uint64_t empty[kStages];       // both MMAs of the tile have read it
-    uint64_t s_full;               // S is in tensor memory
+    uint64_t s_full[2];            // S of an even / odd tile is in tensor memory
     uint64_t p_full;               // P is in shared memory (and S has been read)
     uint64_t o_full;               // O_tile is in tensor memory
     uint32_t tmem_base;
@@ -105,7 +105,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     if (tid == 0) {
         tc::mbar_init(&sh->q_full, 1);
         for (int s = 0; s < kStages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
-        tc::mbar_init(&sh->s_full, 1);
+        tc::mbar_init(&sh->s_full[0], 1);
+        tc::mbar_init(&sh->s_full[1], 1);
         tc::mbar_init(&sh->p_full, kSoftmaxWarps);
         tc::mbar_init(&sh->o_full, 1);
         sh->abort_flag = 0;
@@ -113,14 +114,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         tc::fence_barrier_init();
     }
     if (warp == 1) {
-        tc::tmem_alloc(&sh->tmem_base, 256);
+        tc::tmem_alloc(&sh->tmem_base, 512);
         tc::tmem_relinquish();
     }
     tc::tc_fence_before_sync();
     __syncthreads();
     tc::tc_fence_after_sync();
-    const uint32_t tmem_s = sh->tmem_base;               // S: columns 0..127
-    const uint32_t tmem_o = sh->tmem_base + 128;         // O_tile: columns 128..128+D-1
+    const uint32_t tmem_s = sh->tmem_base;               // S of even tiles: columns 0..127, of odd tiles: 128..255
+    const uint32_t tmem_o = sh->tmem_base + 256;         // O_tile: columns 256..256+D-1
 
     pdl_wait();                      // the tree (node count, mask) and Q/K/V come from preceding kernels
     pdl_trigger();
@@ -178,21 +179,28 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             const uint32_t idesc_s = tc::idesc_bf16_f32(kRows, kKeys);
             const uint32_t idesc_o = tc::idesc_bf16_f32_b_mn(kRows, D);
             bool ok = tc::mbar_wait(&sh->q_full, 0u, abort_flag);
-            for (int it = 0; it < ntile && ok; ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-                if (!tc::mbar_wait(&sh->full[s], ph, abort_flag)) { ok = false; break; }
+            // S = Q K^T of tile t into S buffer t & 1: D/16 steps of 16 elements along the head dimension.
+            // It is issued one tile ahead, so that it runs while the softmax warps work on tile t - 1
+            // (they finished reading buffer t & 1 before they released P of tile t - 2).
+            auto issue_s = [&](int t) -> bool {
+                const int s = t % kStages;
+                if (!tc::mbar_wait(&sh->full[s], (uint32_t)(t / kStages) & 1u, abort_flag)) return false;
                 tc::tc_fence_after_sync();
                 const uint32_t k_addr = tc::smem_u32(KV + (size_t)s * 2 * kTileBytes);
-                const uint32_t v_addr = k_addr + kTileBytes;
-                // S = Q K^T: D/16 steps of 16 elements along the head dimension
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t adesc = tc::smem_desc_k_sw128(tc::smem_u32(Qs) + (kk / 4) * (kRows * 128)) + 2 * (kk % 4);
                     const uint64_t bdesc = tc::smem_desc_k_sw128(k_addr + (kk / 4) * (kKeys * 128)) + 2 * (kk % 4);
-                    tc::mma_bf16_ss(tmem_s, adesc, bdesc, idesc_s, kk != 0 ? 1u : 0u);
+                    tc::mma_bf16_ss(tmem_s + (uint32_t)((t & 1) * 128), adesc, bdesc, idesc_s, kk != 0 ? 1u : 0u);
                 }
-                tc::mma_commit(&sh->s_full);
+                tc::mma_commit(&sh->s_full[t & 1]);
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int it = 0; it < ntile && ok; ++it) {
+                const int s = it % kStages;
+                if (it + 1 < ntile && !issue_s(it + 1)) { ok = false; break; }
+                const uint32_t v_addr = tc::smem_u32(KV + (size_t)s * 2 * kTileBytes) + kTileBytes;
                 // O_tile = P V once the softmax warps have written P (they have then also read S)
                 if (!tc::mbar_wait(&sh->p_full, (uint32_t)it & 1u, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after_sync();
@@ -244,7 +252,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         for (int it = 0; it < ntile; ++it) {
             const int key0 = (blk0 + it) * kKeys;
             const int s = it % kStages;
-            if (!failed && !tc::mbar_wait(&sh->s_full, (uint32_t)it & 1u, abort_flag)) failed = true;
+            if (!failed && !tc::mbar_wait(&sh->s_full[it & 1], (uint32_t)(it >> 1) & 1u, abort_flag)) failed = true;
             failed = __any_sync(0xffffffffu, failed);
             tc::tc_fence_after_sync();
             const bool tail = key0 + kKeys > L;       // the tile holds tree nodes or keys past the end
@@ -278,7 +286,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 #pragma unroll 1
                 for (int c0 = kc0; c0 < kc0 + kKeys / 2; c0 += 32) {
                     uint32_t v[32];
-                    tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
+                    tc::tmem_ld32(tmem_s + (uint32_t)((it & 1) * 128) + lane_off + (uint32_t)c0, v);
                     const uint32_t vm = visible32(c0);
                     tc::tmem_ld_wait();
 #pragma unroll
@@ -301,7 +309,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 #pragma unroll 1
             for (int c0 = kc0; c0 < kc0 + kKeys / 2; c0 += 32) {
                 uint32_t v[32];
-                tc::tmem_ld32(tmem_s + lane_off + (uint32_t)c0, v);
+                tc::tmem_ld32(tmem_s + (uint32_t)((it & 1) * 128) + lane_off + (uint32_t)c0, v);
                 tc::tmem_ld_wait();
                 const uint32_t vm = visible32(c0);
                 float pv[32];
@@ -359,7 +367,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     __syncthreads();
     if (warp == 1) {
         tc::tc_fence_after_sync();
-        tc::tmem_dealloc(sh->tmem_base, 256);
+        tc::tmem_dealloc(sh->tmem_base, 512);
     }
     const bool good = sh->abort_flag == 0;
     if (splits == 1) {
