@@ -29,6 +29,7 @@ constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
 constexpr int kRows = 128;         // query rows per CTA
 constexpr int kKeys = 128;         // keys per tile
 constexpr int kStages = 2;         // K/V tile buffers
+constexpr float kSlack = 8.f;      // how far (log2 units) the row maximum may run ahead of the exponent's reference
 
 struct __align__(8) AttnShared {
     uint64_t q_full;
@@ -139,7 +140,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 
     // softmax state of the row owned by this thread (softmax warps only)
     float acc[DO];
-    float mx = -INFINITY, sum = 0.f;
+    float ref = -INFINITY, sum = 0.f;           // exponent reference (log2 units) and row sum of the softmax
     bool failed = false;
 
     if (warp == 0) {
@@ -209,7 +210,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                     const uint64_t adesc = tc::smem_desc_k_sw128(tc::smem_u32(Ps) + (kk / 4) * (kRows * 128)) + 2 * (kk % 4);
                     // 16 keys further along K = 16 rows of 128 bytes
                     const uint64_t bdesc = tc::smem_desc_mn_sw128(v_addr + kk * (16 * 128), kKeys * 128);
-                    tc::mma_bf16_ss(tmem_o, adesc, bdesc, idesc_o, kk != 0 ? 1u : 0u);
+                    tc::mma_bf16_ss(tmem_o, adesc, bdesc, idesc_o, (it | kk) != 0 ? 1u : 0u);   // O accumulates over the tiles
                 }
                 tc::mma_commit(&sh->o_full);
                 tc::mma_commit(&sh->empty[s]);
@@ -299,11 +300,33 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             pair_barrier(q);
             bm = fmaxf(bm, sh->xch[it & 1][half ^ 1][rl]);
             bm *= sl2;                                 // scale > 0: the maximum commutes with it
-            const float nm = fmaxf(mx, bm);
-            const float ref = nm == -INFINITY ? 0.f : nm;
-            const float corr = exp2_fast(mx - ref);    // exp2(-inf) = 0
-            mx = nm;
+            // The exponent's reference follows the running maximum lazily: it moves only when the
+            // maximum has grown by more than kSlack (in log2 units), so P stays below 2^kSlack and
+            // O, which accumulates in tensor memory, rarely needs rescaling.  Both threads of a row
+            // see the same numbers and take the same decision.
+            const bool move = bm > ref + kSlack;       // also the first tile with a visible key (ref = -inf)
+            const float nref = move ? bm : ref;
+            const float corr = move ? exp2_fast(ref - nref) : 1.f;     // exp2(-inf) = 0
+            // P of the previous tile must have been consumed before it is overwritten, and O must be
+            // complete before it is rescaled
+            if (it > 0 && !failed && !tc::mbar_wait(&sh->o_full, (uint32_t)(it - 1) & 1u, abort_flag)) failed = true;
+            failed = __any_sync(0xffffffffu, failed);
             if (failed) continue;
+            if (it > 0 && __any_sync(0xffffffffu, move)) {
+                tc::tc_fence_after_sync();
+#pragma unroll
+                for (int c0 = 0; c0 < DO; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * corr);
+                    tc::tmem_st32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
+                }
+                tc::tmem_st_wait();
+            }
+            sum *= corr;
+            ref = nref;
             // pass 2: P = exp2(S - max), partial row sum, P to shared memory as bf16 (K-major, 128-byte swizzle)
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
@@ -331,16 +354,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                     *reinterpret_cast<uint4*>(prow + ((chunk ^ (rl & 7)) << 4)) = w;
                 }
             }
-            sum = sum * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+            sum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
             // make P (and the cleared V rows) visible to the tensor core, then hand over
             tc::fence_proxy_async();
             tc::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&sh->p_full);
-            // O = O * corr + O_tile, this thread's half of the columns
-            if (!tc::mbar_wait(&sh->o_full, (uint32_t)it & 1u, abort_flag)) failed = true;
-            failed = __any_sync(0xffffffffu, failed);
-            if (failed) continue;
+        }
+        // O is complete once the last P V product has landed: fetch this thread's half of the row
+        if (ntile > 0 && !failed && !tc::mbar_wait(&sh->o_full, (uint32_t)(ntile - 1) & 1u, abort_flag)) failed = true;
+        failed = __any_sync(0xffffffffu, failed);
+        if (ntile > 0 && !failed) {
             tc::tc_fence_after_sync();
 #pragma unroll
             for (int c0 = 0; c0 < DO; c0 += 32) {
@@ -348,7 +372,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 tc::tmem_ld32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
                 tc::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[c0 + j] = fmaf(acc[c0 + j], corr, __uint_as_float(v[j]));
+                for (int j = 0; j < 32; ++j) acc[c0 + j] = __uint_as_float(v[j]);
             }
             tc::tc_fence_before_sync();
         }
@@ -406,7 +430,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             *reinterpret_cast<float4*>(dst + half * DO + 4 * c) =
                 make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
         if (half == 0) {
-            dst[D] = mx;
+            dst[D] = ref;                       // the reference the row is expressed against
             dst[D + 1] = sum;                      // already the whole row's sum
         }
     }

@@ -171,6 +171,34 @@ def test_empty_prefix_and_every_limit_at_once():
     assert max(r["n_nodes"]) > 128
 
 
+@pytest.mark.parametrize("grp", [1, 4])
+def test_attention_when_later_keys_score_far_higher(grp):
+    """Keys whose scores grow from tile to tile by far more than the slack the kernel allows between
+    the row maximum and the exponent's reference: every tile then moves the reference and rescales
+    the output accumulated so far (with uniform random keys that path would never run)."""
+    import math
+    import torch
+    from oracle import ctcsd_oracle as orc
+    from paper_2412_00061_b200.step import DraftVerifyStep, to_device
+    cfg = C["c2"].replace(name="grow", H=256, V=999, Hq=8, Hkv=8 // grp, kv_lo=3000, kv_hi=3000)
+    x, Wd, bb = synth.gen_draft(cfg, 7)
+    base_tok, kv_len = synth.gen_base(cfg, 7)
+    Q, K, V = synth.gen_attention(cfg, 7)
+    ramp = 1.0 + 3.0 * (np.arange(cfg.Lcap) // 128).astype(np.float32)          # tile t: keys x (1 + 3t)
+    K = synth.to_dtype(K * ramp[None, None, :, None], cfg.dtype)
+    step = DraftVerifyStep(cfg, device="cuda:0")
+    dev = step.device
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    step.set_inputs(x=to_device(x, cfg.dtype, dev), Wd=to_device(Wd, cfg.dtype, dev),
+                    blank_bias=torch.from_numpy(bb).to(dev), base_tok=i32(base_tok), kv_len=i32(kv_len),
+                    Q=to_device(Q, cfg.dtype, dev), K=to_device(K, cfg.dtype, dev), V=to_device(V, cfg.dtype, dev))
+    step.draft(); step.collapse(); step.tree(); step.attention()
+    step.check_status()
+    n_nodes, mask = step.host("n_nodes"), step.host("mask").view(np.uint64)
+    want = orc.tree_attention(Q, K, V, kv_len, n_nodes, mask, 1.0 / math.sqrt(cfg.D))
+    assert np.max(np.abs(step.host("O") - want)) <= 2e-2
+
+
 RAW = {
     # the raw trie of N paths of T symbols has up to 1 + N*T nodes
     "c2raw": C["c2"].replace(name="c2raw", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200, max_nodes=96),
