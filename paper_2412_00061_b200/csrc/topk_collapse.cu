@@ -257,34 +257,37 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
             else if (top == thr) S.cand[atomicAdd(&S.ccnt, 1)] = i;
         }
         __syncthreads();
-        // exact ranking among the threshold entries
-        for (int c = tid; c < ncand; c += kThreads) {
+        // exact ranking among the threshold entries: one warp per entry, its lanes share the
+        // comparisons (a rank is the number of entries that precede it)
+        for (int c = tid >> 5; c < ncand; c += kThreads / 32) {
             const int i = S.cand[c];
             const double si = sc[i];
             const unsigned long long ki = ky[i];
             int rank = 0;
-            for (int d = 0; d < ncand; ++d) {
+            for (int d = lane; d < ncand; d += 32) {
                 const int j = S.cand[d];
                 rank += precedes(sc[j], ky[j], si, ki) ? 1 : 0;
             }
-            if (rank < remaining) S.win[atomicAdd(&S.nwin, 1)] = i;
+            rank = __reduce_add_sync(0xffffffffu, rank);
+            if (lane == 0 && rank < remaining) S.win[atomicAdd(&S.nwin, 1)] = i;
         }
         __syncthreads();
     } else {
         for (int i = tid; i < count; i += kThreads) S.win[i] = i;
         __syncthreads();
     }
-    // order the winners
-    for (int w = tid; w < need; w += kThreads) {
+    // order the winners, again one warp per winner
+    for (int w = tid >> 5; w < need; w += kThreads / 32) {
         const int i = S.win[w];
         const double si = sc[i];
         const unsigned long long ki = ky[i];
         int rank = 0;
-        for (int d = 0; d < need; ++d) {
+        for (int d = lane; d < need; d += 32) {
             const int j = S.win[d];
             rank += precedes(sc[j], ky[j], si, ki) ? 1 : 0;
         }
-        sel[rank] = i;
+        rank = __reduce_add_sync(0xffffffffu, rank);
+        if (lane == 0) sel[rank] = i;
     }
     __syncthreads();
     return need;
