@@ -4,8 +4,8 @@
 //   A = 128 rows of hn (rows past M are zero-filled by TMA), K-major, 128-byte swizzle,
 //   B = Nt consecutive rows of Wl, K-major, 128-byte swizzle,
 //   D = fp32 accumulator in tensor memory: lane = hn row, column = vocabulary row.
-// Each CTA owns a contiguous range of (vocabulary tile, row tile) units, so every weight is
-// fetched from HBM once; the kernel is a weight stream whose math hides behind the loads.
+// The (vocabulary tile, row tile) units are dealt to the CTAs round-robin, so every weight is
+// fetched from HBM once (row tiles that share a weight tile run at the same time and meet in L2); the kernel is a weight stream whose math hides behind the loads.
 // Warp 0 issues TMA loads into a ring of shared-memory stages, warp 1 issues the MMAs, warps
 // 2..17 read the accumulator back: four warps per quarter of the TMEM lanes (a warp may only
 // read its own 32 lanes), each taking every fourth 32-column chunk of the tile, and keep the
@@ -109,18 +109,21 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
     const long long units = (long long)p.n_tiles * p.m_units;
-    const int u0 = (int)(units * blockIdx.x / gridDim.x);
-    const int u1 = (int)(units * (blockIdx.x + 1) / gridDim.x);
+    // CTA c takes units c, c + grid, c + 2 grid, ...: at any moment the CTAs then work on
+    // neighbouring units, i.e. on the few row tiles of the same few weight tiles, so a weight tile
+    // that several row tiles need is fetched from HBM once and found in L2 by the others.
+    const int u_first = (int)blockIdx.x, u_step = (int)gridDim.x;
+    const int n_units = units > u_first ? (int)((units - u_first + u_step - 1) / u_step) : 0;
 
     // producer state (lane 0 of warp 0 only).  Stage `it` holds K block it % num_k of unit
-    // u0 + it / num_k; every CTA walks the K axis from its own starting block (and wraps), so that
+    // u_first + (it / num_k) * u_step; every CTA walks the K axis from its own starting block (and wraps), so that
     // at any moment the CTAs ask L2 for different parts of the shared activations.
-    const int total_it = (u1 - u0) * p.num_k;
+    const int total_it = n_units * p.num_k;
     const int k_start = (int)(((long long)blockIdx.x * p.num_k) / gridDim.x);
     const uint64_t pol_w = tc::policy_evict_first();
     const uint64_t pol_a = tc::policy_evict_last();
     auto load_stage = [&](int it, bool do_w, bool do_a) {
-        const int u = u0 + it / p.num_k, kb = it - (it / p.num_k) * p.num_k;
+        const int u = u_first + (it / p.num_k) * u_step, kb = it - (it / p.num_k) * p.num_k;
         const int nt = u / p.m_units, mu = u - nt * p.m_units;
         const int s = it % p.stages;
         unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
@@ -193,7 +196,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const uint32_t idesc = tc::idesc_bf16_f32(kTileM, p.Nt);
             int it = 0, ucount = 0;
             bool ok = true;
-            for (int u = u0; u < u1 && ok; ++u, ++ucount) {
+            for (int u = u_first; ucount < n_units && ok; u += u_step, ++ucount) {
                 const int acc = p.pair ? 0 : (ucount & 1);            // barrier pair that guards this unit
                 const uint32_t acc_ph = (uint32_t)(p.pair ? ucount : (ucount >> 1)) & 1u;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
@@ -236,7 +239,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         int ucount = 0;
         bool ok = true;
-        for (int u = u0; u < u1 && ok; ++u, ++ucount) {
+        for (int u = u_first; ucount < n_units && ok; u += u_step, ++ucount) {
             const int nt = u / p.m_units, mu = u - nt * p.m_units;
             // draft mode: tile nt is tile ntl of slot t
             const int t = MODE == 1 ? nt / p.tiles_per_slot : 0;
