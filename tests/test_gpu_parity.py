@@ -62,6 +62,35 @@ def test_draft_head_on_every_tree_row_uses_several_row_tiles():
     _run(cfg, seed=1, M=M, row_seq=row_seq, sel_row=sel_row, draft_rows=[0, 127, 128, 200, 319])
 
 
+def test_c5_draft_head_on_all_2048_tree_rows_full_size():
+    """The 70B-shaped workload with the draft head run on every tree row (32 sequences x 64 rows =
+    2048 rows, sixteen 128-row tiles of the tensor-core path against 3.1 GB of weights).  The
+    logits of sampled rows are compared with the oracle (definition mode) and their top-k and
+    log-sum-exp with the oracle fed those logits (bit-exact ids)."""
+    import torch
+    from oracle import ctcsd_oracle as orc
+    from paper_2412_00061_b200.step import DraftVerifyStep, to_device
+    from tests.parity_util import check_topk, tolerances
+    cfg = C["c5"]
+    M = cfg.B * cfg.max_nodes
+    x, Wd, bb = synth.gen_draft(cfg, 3, M=M)
+    row_seq = (np.arange(M) // cfg.max_nodes).astype(np.int32)
+    step = DraftVerifyStep(cfg, device="cuda:0", max_draft_rows=M, debug_logits=True)
+    dev = step.device
+    step.set_inputs(x=to_device(x, cfg.dtype, dev), Wd=to_device(Wd, cfg.dtype, dev),
+                    blank_bias=torch.from_numpy(bb).to(dev), row_seq=torch.from_numpy(row_seq).to(dev))
+    step.draft()
+    step.check_status()
+    rows = [0, 127, 128, 1000, 2047]
+    idx = torch.tensor(rows, device=dev)
+    z_gpu = step.out["draft_logits_dbg"][idx].cpu().numpy()
+    logit_tol, rel = tolerances(cfg.dtype)
+    z_def = orc.draft_logits(x[rows], Wd, bb, row_seq[rows])
+    assert np.max(np.abs(z_gpu - z_def)) <= logit_tol
+    check_topk(z_gpu, step.out["topk_id"][idx].cpu().numpy(), step.out["topk_lp"][idx].cpu().numpy(),
+               step.out["lse"][idx].cpu().numpy(), cfg.k, rel)
+
+
 def test_enumeration_limits_and_max_score_mode():
     # 4096 paths (T=6, k=4) enumerated exhaustively; best-alignment scoring variant
     _run(C["c1"].replace(name="enum4096", T=6, k=4, topN=64, max_nodes=128), seed=0)
