@@ -169,13 +169,13 @@ __device__ __forceinline__ int next_pow2(int v) {
 }
 
 // Selects the `need` (<= CTCSD_MAX_BEAM) best of `count` entries and writes their indices,
-// best first, to sel[]; returns how many were selected.  A radix select on the float32 image
+// best first (in any order when `ordered` is false), to sel[]; returns how many were selected.  A radix select on the float32 image
 // of the scores finds the threshold in O(count) work; entries on the threshold are ranked
 // exactly (float64 score, then key).  If more than kSelMax entries sit on the threshold the
 // arrays (padded to a power of two, capacity >= next_pow2(count)) are sorted in place instead
 // and sel[] becomes the identity.
 __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int count, int need, int* sel,
-                                SelectScratch& S) {
+                                SelectScratch& S, bool ordered = true) {
     const int tid = threadIdx.x, lane = tid & 31;
     if (need > count) need = count;
     if (tid == 0) { S.fmax = 0u; S.fmin = 0xffffffffu; S.nwin = 0; S.ncand = 0; S.ccnt = 0; }
@@ -275,6 +275,11 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
     } else {
         for (int i = tid; i < count; i += kThreads) S.win[i] = i;
         __syncthreads();
+    }
+    if (!ordered) {                                   // the caller only needs the set
+        for (int w = tid; w < need; w += kThreads) sel[w] = S.win[w];
+        __syncthreads();
+        return need;
     }
     // order the winners, again one warp per winner
     for (int w = tid >> 5; w < need; w += kThreads / 32) {
@@ -522,7 +527,8 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         }
         __syncthreads();
         const int count = s_next;
-        const int keep = block_select_top(c_sc, c_ky, c_ix, count, p.beam, s_sel, S);
+        // between slots the beam is a set; only the last slot's beam is ranked (the candidates come out of it)
+        const int keep = block_select_top(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1);
         for (int r = tid; r < keep; r += kThreads) {
             const int i = s_sel[r];
             const int slot = c_ix[i];
