@@ -63,9 +63,19 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     const int T = p.T, N = p.topN, n_max = p.max_nodes;
     pdl_wait();                      // the candidates come from the preceding kernel
     pdl_trigger();
+    // every input is requested at once (the candidate arrays are full-sized whatever n_cand and the
+    // lengths say), so the kernel pays one memory latency, not three dependent ones
     int nc = p.n_cand[b];
-    nc = nc < 0 ? 0 : (nc > N ? N : nc);
     const int L = p.kv_len[b];
+    int raw_len[2], raw_tok[2][kT];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        raw_len[h] = (c < N && p.cand_len) ? p.cand_len[(size_t)b * N + c] : T;
+#pragma unroll
+        for (int q = 0; q < kT; ++q) raw_tok[h][q] = (c < N && q < T) ? p.cand_tok[((size_t)b * N + c) * T + q] : -1;
+    }
+    nc = nc < 0 ? 0 : (nc > N ? N : nc);
     const int halves = nc > 32 ? 2 : 1;
     const int W = (n_max + 63) / 64;
 
@@ -75,10 +85,10 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
     for (int h = 0; h < 2; ++h) {
         const int c = lane + 32 * h;
         int l = 0;
-        if (c < nc) { l = p.cand_len ? p.cand_len[(size_t)b * N + c] : T; l = l < 0 ? 0 : (l > T ? T : l); }
+        if (c < nc) { l = raw_len[h]; l = l < 0 ? 0 : (l > T ? T : l); }
         len[h] = l;
 #pragma unroll
-        for (int q = 0; q < kT; ++q) tok[h][q] = (q < l) ? p.cand_tok[((size_t)b * N + c) * T + q] : -1;
+        for (int q = 0; q < kT; ++q) tok[h][q] = (q < l) ? raw_tok[h][q] : -1;
     }
 
     // ---- owners, level by level ----
