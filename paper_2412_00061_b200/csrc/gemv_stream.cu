@@ -375,11 +375,24 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
         const int m = task / p.slots, slot = task - m * p.slots;
         RunState fs;
         fs.init();
-        for (int e = lane; e < 2 * (int)gridDim.x; e += 32) {
-            if (__ldcg(p.part_slot + e) == slot) {
-                DraftPartial q = load_partial_cg(p.part + (size_t)m * p.grid * 2 + e);
-                fs.absorb(q);
-            }
+        // The CTAs whose row range touches this slot are a contiguous interval that follows from
+        // the partition formula, so a lane goes straight to "its" CTA's state: one memory latency
+        // instead of a scan over all CTAs' slot tags (the tag is still checked: a CTA marks a
+        // segment without rows as unused).
+        const long long g = gridDim.x;
+        const long long lo_row = (long long)slot * rps, hi_row = lo_row + rps;     // the slot's rows
+        long long c_lo = lo_row * g / R, c_hi = hi_row * g / R;
+        while (c_lo > 0 && R * c_lo / g > lo_row) --c_lo;                          // first CTA with r1 > lo_row
+        while (c_lo < g - 1 && R * (c_lo + 1) / g <= lo_row) ++c_lo;
+        if (c_hi > g - 1) c_hi = g - 1;
+        while (c_hi > 0 && R * c_hi / g >= hi_row) --c_hi;                         // last CTA with r0 < hi_row
+        for (long long c = c_lo + lane; c <= c_hi; c += 32) {
+            const int seg = slot - (int)((R * c / g) / rps);
+            if (seg < 0 || seg > 1) continue;
+            const int e = (int)(2 * c + seg);
+            const int tag = __ldcg(p.part_slot + e);
+            DraftPartial q = load_partial_cg(p.part + (size_t)m * p.grid * 2 + e);
+            if (tag == slot) fs.absorb(q);
         }
         warp_combine(fs);
         if (lane == 0) {
