@@ -122,8 +122,8 @@ int ctcsd_set_l2_prefetch(ctcsd_handle* h, const void* ptr, size_t bytes);
 
 /*
  * Draft head, per-slot log-softmax and per-slot top-k (Sec. 3.2: one probability
- * distribution per place from the projected hidden state; Sec. 3.3: "the top k tokens are
- * selected in descending order of probability").
+ * distribution per place from the projected hidden state; Sec. 3.3: every place keeps its k most
+ * probable symbols, best first, k fixed in advance).
  *   z[m,t,v]   = sum_h x[m,h] * Wd[t,v,h]  (+ blank_bias[row_seq[m]] when v == V)
  *   lse[m,t]   = log sum_v exp z[m,t,v]
  *   top-k      = the k largest z[m,t,:] over all V+1 classes, descending, ties to the lower id;
@@ -142,7 +142,7 @@ int ctcsd_draft_logits(ctcsd_handle* h, void* stream, int M, const void* x, cons
 
 /*
  * Slot paths -> collapsed, deduplicated, scored candidates -> the topN best (Sec. 3.3: the
- * slot tokens are combined and "the most valuable combinations are reserved"; Sec. 2.3 /
+ * slot tokens are combined and only the most valuable combinations go on; Sec. 2.3 /
  * Sec. 3.1: beta^{-1} merges adjacent repeats, then removes blanks; Eq. 6: a path's
  * probability is the product over slots; Eq. 1 / Eq. 5: a candidate's probability is the sum
  * over the paths that collapse to it).
@@ -216,8 +216,8 @@ int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const voi
                         int* out_next_tok, float* out_logits_dbg);
 
 /*
- * History update after acceptance (Sec. 3.3: "the decoding history is updated according to the
- * output"): the accepted path becomes part of the cached prefix, so that the next step can
+ * History update after acceptance (Sec. 3.3, last paragraph: the step's output joins the decoding
+ * history): the accepted path becomes part of the cached prefix, so that the next step can
  * start without host work.  For sequence b with L = kv_len[b]: the root's key/value row (cache
  * row L) stays; for l = 0 .. acc_len[b]-1 the row of accepted node acc_nodes[b,l] (cache row
  * L + node) is moved to row L + 1 + l, for every kv head, in K and in V; rows are read as they

@@ -13,11 +13,16 @@ Pins (see tests/test_oracle_pins.py): every function below is pinned by somethin
 than itself - hand-worked collapse cases, the total-mass closed form, the Graves forward
 recursion (torch's ctc_loss and an independent alpha recursion), library matmul /
 log-softmax / top-k / scaled-dot-product attention in fp64, brute-force tries and
-acceptance definitions, and - for the history update - the equality of ordinary attention over
-the updated prefix with tree attention over the old cache, plus a hand-worked overlap case.  The finite-beam prefix search is a heuristic the paper does not
-specify ("a group of the most valuable combinations are reserved", Sec. 3.3): with a beam
-that never prunes it is pinned to exact enumeration; with a pruning beam it is pinned only
-by bounds (candidate subset, score <= exact) - beyond that: parity unpinned.
+acceptance definitions, the closed-form mean accepted length on a chain, and - for the
+history update - the equality of ordinary attention over the updated prefix with tree
+attention over the old cache, plus a hand-worked overlap case.  The finite-beam prefix
+search is a heuristic the paper does not specify (Sec. 3.3 only says that the most valuable
+combinations are kept): WHICH pruning rule is used is this build's reading; HOW it executes
+is pinned - with a beam that never prunes to exact enumeration, with a pruning beam to an
+alignment-level brute force of the survivor sets after every slot (masses split by the last
+symbol), to hand-worked cases with the arithmetic written out (tests/golden/), ties at the
+cut included.  The batch wrapper topk_collapse (row mapping, padding, decision margin) is
+pinned against per-sequence enumeration and an independent sort.
 """
 from __future__ import annotations
 
@@ -31,7 +36,7 @@ NEG_INF = float("-inf")
 
 
 # --------------------------------------------------------------------------------------
-# S1  draft head: per-slot logits (Sec. 3.2, "Softmax(LmHead(F_hat))" gives one
+# S1  draft head: per-slot logits (Sec. 3.2: the projected draft features give one
 #     distribution per place; here the projection is a linear head over V+1 classes)
 # --------------------------------------------------------------------------------------
 def draft_logits(x: np.ndarray, Wd: np.ndarray, blank_bias: Optional[np.ndarray] = None,
@@ -63,8 +68,8 @@ def log_softmax_slots(z: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
 
 
 # --------------------------------------------------------------------------------------
-# S3  per-slot top-k (Sec. 3.3: "For every position, the top k tokens are selected in
-#     descending order of probability"); blank is eligible; ties go to the lower id
+# S3  per-slot top-k (Sec. 3.3: each place keeps its k most probable symbols, best first,
+#     k fixed in advance); blank is eligible; ties go to the lower id
 # --------------------------------------------------------------------------------------
 def topk_slots(z: np.ndarray, k: int) -> Tuple[np.ndarray, np.ndarray]:
     """Returns (topk_id [M,T,k] int64, topk_lp [M,T,k] fp64) with lp = z - lse."""
@@ -76,8 +81,8 @@ def topk_slots(z: np.ndarray, k: int) -> Tuple[np.ndarray, np.ndarray]:
 
 
 # --------------------------------------------------------------------------------------
-# S5  CTC collapse beta^{-1} (Sec. 2.3: "merging adjacent, repeated tokens and removing
-#     blanks"; Sec. 3.1: "removes consecutive duplicate tokens and blank character")
+# S5  CTC collapse beta^{-1} (Sec. 2.3 and Sec. 3.1, CTC Transform Module: runs of one
+#     repeated symbol shrink to a single symbol, then every blank is deleted)
 # --------------------------------------------------------------------------------------
 def ctc_collapse(a: Sequence[int], blank: int) -> Tuple[int, ...]:
     out: List[int] = []
@@ -134,8 +139,8 @@ def order_o1(item: Tuple[Tuple[int, ...], float]):
 
 
 # --------------------------------------------------------------------------------------
-# S7  keep the N best non-empty candidates (Sec. 3.3: "a group of the most valuable
-#     combinations are reserved")
+# S7  keep the N best non-empty candidates (Sec. 3.3: only the most valuable of the
+#     combined sequences go on to verification)
 # --------------------------------------------------------------------------------------
 def select_top_n(cands: Dict[Tuple[int, ...], float], N: int) -> List[Tuple[Tuple[int, ...], float]]:
     items = [(y, s) for y, s in cands.items() if len(y) > 0]
@@ -164,6 +169,7 @@ def prefix_beam_candidates(topk_id: np.ndarray, topk_lp: np.ndarray, blank: int,
     T, k = topk_id.shape
     cur: Dict[Tuple[int, ...], Tuple[float, float]] = {(): (0.0, NEG_INF)}   # (log pb, log pnb)
     min_cut_gap = float("inf")
+    beams: List[Dict[Tuple[int, ...], Tuple[float, float]]] = []             # the beam after every slot
     for t in range(T):
         nxt: Dict[Tuple[int, ...], List[float]] = {}
 
@@ -190,8 +196,10 @@ def prefix_beam_candidates(topk_id: np.ndarray, topk_lp: np.ndarray, blank: int,
         if len(ranked) > beam:
             min_cut_gap = min(min_cut_gap, ranked[beam - 1][1] - ranked[beam][1])
         cur = {y: (nxt[y][0], nxt[y][1]) for y, _ in ranked[:beam]}
+        beams.append(dict(cur))
     if stats is not None:
         stats["min_cut_gap"] = min_cut_gap
+        stats["beams"] = beams
     return {y: _logaddexp(pb, pnb) for y, (pb, pnb) in cur.items()}
 
 
@@ -350,8 +358,8 @@ def greedy_accept(node_tok: np.ndarray, parent: np.ndarray, n_nodes: np.ndarray,
 
 
 # --------------------------------------------------------------------------------------
-# S12  history update after acceptance (Sec. 3.3: "the decoding history is updated
-#      according to the output"): the accepted path becomes part of the cached prefix
+# S12  history update after acceptance (Sec. 3.3, last paragraph: the step's output is
+#      appended to the decoding history): the accepted path becomes part of the cached prefix
 # --------------------------------------------------------------------------------------
 def commit_accepted(K: np.ndarray, Vc: np.ndarray, kv_len: np.ndarray, acc_len: np.ndarray,
                     acc_nodes: np.ndarray, max_nodes: int):
@@ -384,8 +392,8 @@ def commit_accepted(K: np.ndarray, Vc: np.ndarray, kv_len: np.ndarray, acc_len: 
 # instead of being dropped from the tree.
 # --------------------------------------------------------------------------------------
 def select_raw_paths(topk_id: np.ndarray, topk_lp: np.ndarray, N: int):
-    """The N most probable slot paths of one sequence ("a group of the most valuable combinations
-    are reserved as the raw candidate sequences", Sec. 3.3): path probability = product over the
+    """The N most probable slot paths of one sequence (Sec. 3.3: the raw candidates are the most
+    valuable combinations of the per-place symbols): path probability = product over the
     slots (Eq. 6); equal scores go to the path that is first when the per-slot ranks are read as
     a number (slot 1 most significant).  topk_id/topk_lp [T,k] -> (raw_tok [n,T], score [n])."""
     T, k = topk_id.shape
@@ -451,8 +459,8 @@ def build_raw_tree(base_tok: np.ndarray, kv_len: np.ndarray, raw_tok: np.ndarray
 
 def raw_accept(node_tok: np.ndarray, kept: np.ndarray, nka: np.ndarray, n_nodes: np.ndarray,
                am: np.ndarray, T: int):
-    """Greedy acceptance on the raw tree (Sec. 3.3: "the longest sequence that satisfies the
-    criterion").  am[b,i] is the base model's greedy token after kept node i.  A kept node d
+    """Greedy acceptance on the raw tree (Sec. 3.3: of the candidates that pass verification the
+    longest one is the output).  am[b,i] is the base model's greedy token after kept node i.  A kept node d
     follows kept node p when p is d's nearest kept ancestor (removed nodes in between are
     transparent).  best[p] = longest chain p -> d1 -> d2 ... with node_tok[d] == am[previous];
     among equally long continuations the lowest node id wins.

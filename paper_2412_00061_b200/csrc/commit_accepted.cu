@@ -1,5 +1,5 @@
 // ctcsd_commit_accepted: after acceptance the accepted path becomes part of the cached prefix
-// (paper Sec. 3.3: the decoding history is updated according to the output).
+// (paper Sec. 3.3, last paragraph: what a step outputs is appended to the history).
 #include "common.cuh"
 
 namespace ctcsd {

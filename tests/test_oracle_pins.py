@@ -200,6 +200,185 @@ def test_prefix_beam_pruned_bounds():
         assert best in beam
 
 
+def _beam_trajectory_brute_force(ids, lps, blank, beam):
+    """The pruned search restated over whole alignments, with no per-prefix recursion: an alignment
+    of the first t slots counts at slot t iff the collapse of each of its shorter heads survived
+    the cut at that slot (only survivors are ever extended).  Its probability is the product over
+    the slots (Eq. 6); a prefix's mass is the sum over its alignments (Eq. 1 / Eq. 5), split by
+    whether the alignment's last symbol is the blank.  Returns the survivor sets S_1..S_T as
+    {prefix: (pb, pnb)} in the probability domain."""
+    T, k = ids.shape
+    alive = [{()}]
+    out = []
+    for t in range(1, T + 1):
+        mass = {}
+        for a in itertools.product(range(k), repeat=t):
+            syms = [int(ids[s, a[s]]) for s in range(t)]
+            if any(orc.ctc_collapse(syms[:s], blank) not in alive[s] for s in range(t)):
+                continue
+            p = math.exp(sum(float(lps[s, a[s]]) for s in range(t)))
+            e = mass.setdefault(orc.ctc_collapse(syms, blank), [0.0, 0.0])
+            e[0 if syms[-1] == blank else 1] += p
+        ranked = sorted(mass, key=lambda y: (-(mass[y][0] + mass[y][1]), len(y), y))[:beam]
+        alive.append(set(ranked))
+        out.append({y: tuple(mass[y]) for y in ranked})
+    return out
+
+
+@pytest.mark.parametrize("T,k,V", [(5, 3, 4), (4, 3, 6), (5, 2, 3), (3, 3, 2)])
+@pytest.mark.parametrize("beam", [1, 2, 3, 5])
+def test_pruned_prefix_beam_follows_the_alignment_level_definition(T, k, V, beam):
+    rng = np.random.default_rng(1000 * T + 10 * k + beam)
+    pruned_somewhere = False
+    for trial in range(6):
+        ids, lps = _rand_topk(rng, T, k, V, blank_rate=0.8, repeat_rate=0.8)
+        st = {}
+        final = orc.prefix_beam_candidates(ids, lps, blank=V, beam=beam, stats=st)
+        want = _beam_trajectory_brute_force(ids, lps, V, beam)
+        assert len(st["beams"]) == T
+        for t in range(T):
+            got = st["beams"][t]
+            assert set(got) == set(want[t]), (t, got, want[t])
+            for y, (pb, pnb) in got.items():
+                assert math.exp(pb) == pytest.approx(want[t][y][0], rel=1e-12, abs=1e-15)
+                assert math.exp(pnb) == pytest.approx(want[t][y][1], rel=1e-12, abs=1e-15)
+        assert set(final) == set(want[-1])
+        for y, s in final.items():
+            assert math.exp(s) == pytest.approx(sum(want[-1][y]), rel=1e-12)
+        exact = orc.enumerate_candidates(ids, lps, blank=V)
+        pruned_somewhere = pruned_somewhere or any(
+            math.exp(final[y]) < math.exp(exact[y]) * (1 - 1e-9) for y in final) or len(final) < len(exact)
+    assert pruned_somewhere
+
+
+def test_pruned_prefix_beam_hand_worked_cases():
+    cases, cur = [], None
+    with open(os.path.join(GOLDEN, "prefix_beam_pruned_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            w = line.split()
+            if w[0] == "case":
+                cur = dict(name=w[1], beam=int(w[3]), slots=[], after={})
+                cases.append(cur)
+            elif w[0] == "slot":
+                cur["slots"].append([(s.split("=")[0], float(s.split("=")[1])) for s in w[1:]])
+            elif w[0] == "after":
+                t = int(w[1])
+                entries = line.split(":", 1)[1].split(";")
+                cur["after"][t] = [e.strip().split("|") for e in entries]
+    assert len(cases) >= 4
+    for c in cases:
+        sym = {"_": BLANK}
+        T, k = len(c["slots"]), len(c["slots"][0])
+        ids = np.zeros((T, k), dtype=np.int64)
+        lps = np.zeros((T, k))
+        for t, row in enumerate(c["slots"]):
+            for j, (s, p) in enumerate(row):
+                ids[t, j] = sym.setdefault(s, len(sym))
+                lps[t, j] = math.log(p)
+        st = {}
+        orc.prefix_beam_candidates(ids, lps, blank=BLANK, beam=c["beam"], stats=st)
+        for t in range(1, T + 1):
+            want = {}
+            for pre, pb, pnb in c["after"][t]:
+                y = () if pre.strip() == "-" else tuple(sym[s] for s in pre.split())
+                want[y] = (float(pb), float(pnb))
+            got = st["beams"][t - 1]
+            assert set(got) == set(want), (c["name"], t)
+            for y in want:
+                assert math.exp(got[y][0]) == pytest.approx(want[y][0], abs=1e-12), (c["name"], t, y)
+                assert math.exp(got[y][1]) == pytest.approx(want[y][1], abs=1e-12), (c["name"], t, y)
+
+
+@pytest.mark.parametrize("beam", [0, 3])
+def test_batch_wrapper_maps_rows_pads_and_reports_its_margin(beam):
+    """topk_collapse: sequence b drafts from row sel_row[b] (B < M, rows permuted), unused entries
+    are padded (-1 / 0 / -inf), and the margin it reports is the smallest gap its decisions relied
+    on - recomputed here from scratch with a plain sort of (score, length, tokens)."""
+    rng = np.random.default_rng(77 + beam)
+    M, B, T, k, V, N = 5, 3, 4, 3, 5, 6
+    ids = np.zeros((M, T, k), dtype=np.int64)
+    lps = np.zeros((M, T, k))
+    for m in range(M):
+        ids[m], lps[m] = _rand_topk(rng, T, k, V, blank_rate=0.8, repeat_rate=0.8)
+    sel_row = np.array([4, 0, 2])
+    st = {}
+    tok, ln, sc, nc = orc.topk_collapse(ids, lps, blank=V, T=T, N=N, beam=beam, sel_row=sel_row, B=B, stats=st)
+    assert tok.shape == (B, N, T) and ln.shape == (B, N) and sc.shape == (B, N) and nc.shape == (B,)
+    few = False
+    for b in range(B):
+        r = int(sel_row[b])
+        if beam == 0:
+            cands = orc.enumerate_candidates(ids[r], lps[r], blank=V)            # pinned above
+            cut_gap = float("inf")
+        else:
+            traj = _beam_trajectory_brute_force(ids[r], lps[r], V, beam)        # independent of the oracle
+            cands = {y: math.log(pb + pnb) for y, (pb, pnb) in traj[-1].items()}
+            cut_gap = float("inf")
+            # the gap at every cut: beam-th against (beam+1)-th total mass among that slot's extensions
+            alive = [{()}]
+            for t in range(1, T + 1):
+                mass = {}
+                for a in itertools.product(range(k), repeat=t):
+                    syms = [int(ids[r, s, a[s]]) for s in range(t)]
+                    if any(orc.ctc_collapse(syms[:s], V) not in alive[s] for s in range(t)):
+                        continue
+                    y = orc.ctc_collapse(syms, V)
+                    mass[y] = mass.get(y, 0.0) + math.exp(sum(float(lps[r, s, a[s]]) for s in range(t)))
+                order = sorted(mass, key=lambda y: (-mass[y], len(y), y))
+                if len(order) > beam:
+                    cut_gap = min(cut_gap, math.log(mass[order[beam - 1]]) - math.log(mass[order[beam]]))
+                alive.append(set(order[:beam]))
+        rows = sorted(((-s, len(y), y) for y, s in cands.items() if len(y) > 0))
+        n = min(N, len(rows))
+        few = few or n < N
+        assert nc[b] == n
+        for c in range(n):
+            y = rows[c][2]
+            assert ln[b, c] == len(y)
+            assert tuple(tok[b, c, :len(y)]) == y and np.all(tok[b, c, len(y):] == -1)
+            assert sc[b, c] == pytest.approx(-rows[c][0], abs=1e-12)
+        assert np.all(tok[b, n:] == -1) and np.all(ln[b, n:] == 0) and np.all(np.isneginf(sc[b, n:]))
+        gaps = [rows[i + 1][0] - rows[i][0] for i in range(min(N, len(rows) - 1))]
+        want_margin = min(gaps + [cut_gap])
+        assert st["margin"][b] == pytest.approx(want_margin, abs=1e-9)
+        assert st["margin"][b] >= 0.0
+    if beam > 0:
+        assert few                                   # a beam of 3 leaves fewer than N candidates: padding is exercised
+    # default mapping: no sel_row, B = M
+    tok2, ln2, sc2, nc2 = orc.topk_collapse(ids, lps, blank=V, T=T, N=N, beam=beam)
+    assert tok2.shape[0] == M
+    np.testing.assert_array_equal(tok2[4], tok[0])
+    np.testing.assert_array_equal(tok2[0], tok[1])
+    np.testing.assert_array_equal(tok2[2], tok[2])
+
+
+def test_a_tie_shows_up_as_a_zero_margin():
+    # two alignments with equal probability that collapse to different sequences of equal length
+    ids = np.array([[1, 2]], dtype=np.int64)
+    lps = np.log(np.array([[0.3, 0.3]]))
+    st = {}
+    orc.topk_collapse(ids[None], lps[None], blank=9, T=1, N=2, stats=st)
+    assert st["margin"][0] == 0.0
+    st = {}
+    orc.topk_collapse(ids[None], lps[None], blank=9, T=1, N=1, beam=1, stats=st)
+    assert st["margin"][0] == 0.0                    # the beam cut itself sits on the tie
+    # the gap between the last kept and the first dropped candidate counts too
+    ids = np.array([[1, 2, 3]], dtype=np.int64)
+    lps = np.log(np.array([[0.5, 0.3, 0.29]]))
+    st = {}
+    orc.topk_collapse(ids[None], lps[None], blank=9, T=1, N=2, stats=st)
+    assert st["margin"][0] == pytest.approx(math.log(0.3 / 0.29), abs=1e-12)
+    st = {}
+    orc.topk_collapse(ids[None], lps[None], blank=9, T=1, N=3, stats=st)      # nothing dropped: kept pairs only
+    assert st["margin"][0] == pytest.approx(math.log(0.3 / 0.29), abs=1e-12)
+    st = {}
+    orc.topk_collapse(ids[None], lps[None], blank=9, T=1, N=1, stats=st)
+    assert st["margin"][0] == pytest.approx(math.log(0.5 / 0.3), abs=1e-12)
+
+
 # ------------------------------------------------------------------ S1-S3
 def test_draft_logits_against_library_and_bias_placement():
     rng = np.random.default_rng(2)
@@ -436,6 +615,36 @@ def test_greedy_accept_chain_extremes():
     am[0, 0] = 7                                          # no agreement at the root
     acc_len, acc_nodes, acc_tok, next_tok = orc.greedy_accept(node_tok, parent, n, am, 4)
     assert acc_len[0] == 0 and next_tok[0] == 7
+
+
+def test_mean_accepted_length_on_a_chain_matches_the_closed_form():
+    """Sec. 3.3 accepts the longest agreeing candidate.  On a chain of depth T whose every node
+    agrees with the base model independently with probability p, depth d is reached with
+    probability p^d, so E[acc_len] = sum_{d=1..T} p^d.  The seeded generator of the node hidden
+    states, the LM-head arg-max and the acceptance walk together must reproduce that mean."""
+    from paper_2412_00061_b200 import synth
+    T, p, n_seeds = 5, 0.6, 2400
+    cfg = synth.CONFIGS["c1"].replace(name="chain", H=64, V=40, T=T, max_nodes=8, agree_p=p)
+    Wl = synth.gen_lm_head(cfg, 123)
+    tok, ln, nc = _pack([(3, 4, 5, 6, 7)], 1, T)
+    node_tok, parent, depth, pos, mask, retrieve, n = orc.build_tree(
+        np.array([2]), np.array([0]), tok, ln, nc, n_max=cfg.max_nodes)
+    assert n[0] == T + 1
+    total, hist = 0, np.zeros(T + 1, dtype=np.int64)
+    for seed in range(n_seeds):
+        hn, target = synth.gen_node_hidden(cfg, seed, Wl, node_tok, parent, n)
+        _, am = orc.lm_head_argmax(hn, Wl)
+        assert np.array_equal(am[:T + 1], target[0, :T + 1])           # the planted token wins the arg-max
+        acc_len, acc_nodes, acc_tok, next_tok = orc.greedy_accept(node_tok, parent, n, am.reshape(1, -1), T)
+        total += int(acc_len[0])
+        hist[int(acc_len[0])] += 1
+    want = sum(p ** d for d in range(1, T + 1))
+    var = sum((2 * d - 1) * p ** d for d in range(1, T + 1)) - want ** 2      # E[L^2] = sum (2d-1) P(L >= d)
+    assert abs(total / n_seeds - want) <= 4.0 * math.sqrt(var / n_seeds)
+    # the whole distribution: P(L = d) = p^d (1 - p) below the leaf, p^T at the leaf
+    for d in range(T + 1):
+        q = p ** d * ((1 - p) if d < T else 1.0)
+        assert abs(hist[d] / n_seeds - q) <= 4.0 * math.sqrt(q * (1 - q) / n_seeds) + 1e-3
 
 
 # ------------------------------------------------------------------ S12 history update
