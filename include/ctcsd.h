@@ -141,6 +141,20 @@ int ctcsd_draft_logits(ctcsd_handle* h, void* stream, int M, const void* x, cons
                        int* out_topk_id, float* out_topk_lp, float* out_lse, float* out_logits_dbg);
 
 /*
+ * ctcsd_draft_logits with a row map: draft row m reads the hidden state x[x_rows[m]], everything
+ * else as above.  This is how decoding steps chain without host work (Sec. 3.3: the draft module
+ * takes the base model's hidden state at the current position): x is the previous step's
+ * [B*max_nodes,H] array of tree-node hidden states and x_rows the out_sel_row that
+ * ctcsd_commit_accepted produced, so the next step drafts from the last accepted node.
+ * x [x_row_count,H] dtype;  x_rows [M] int32 (device), each in 0..x_row_count-1: an entry outside
+ * that range records CTCSD_ERR_INVALID_ARG in the device status word and that row drafts from a
+ * zero vector.  With more than 8 rows the weights are streamed once per 8 rows.
+ */
+int ctcsd_draft_logits_rows(ctcsd_handle* h, void* stream, int M, const void* x, int x_row_count,
+                            const int* x_rows, const void* Wd, const int* row_seq, const float* blank_bias,
+                            int* out_topk_id, float* out_topk_lp, float* out_lse, float* out_logits_dbg);
+
+/*
  * Slot paths -> collapsed, deduplicated, scored candidates -> the topN best (Sec. 3.3: the
  * slot tokens are combined and only the most valuable combinations go on; Sec. 2.3 /
  * Sec. 3.1: beta^{-1} merges adjacent repeats, then removes blanks; Eq. 6: a path's
@@ -224,7 +238,8 @@ int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const voi
  * were before the call (a destination may be another accepted node's source).
  * K, V [B,Hkv,Lcap,D] dtype, updated IN PLACE;  kv_len, acc_len [B], acc_nodes [B,T] as
  * produced by ctcsd_verify_accept.
- * out_kv_len [B] int32 = kv_len + 1 + acc_len (may alias kv_len);
+ * out_kv_len [B] int32 = kv_len + 1 + acc_len; it may be the same array as kv_len (the new
+ *   length of a sequence is written only after every kv head of that sequence has read the old one);
  * out_sel_row [B] int32 or NULL = b*max_nodes + last accepted node (the root if none): the
  *   tree row whose hidden state the next step drafts from (see sel_row of ctcsd_topk_collapse).
  * A sequence whose path would leave the cache is left unchanged and CTCSD_ERR_INVALID_ARG is
@@ -298,7 +313,10 @@ int ctcsd_verify_accept_raw(ctcsd_handle* h, void* stream, const void* hn, const
  *   Q, out_O [B,max_nodes,Hq,D];  K, V [B,Hkv,Lcap,D];  kv_len, n_nodes [B];
  *   mask [B,max_nodes,ceil(max_nodes/64)] uint64;  D is 64 or 128;  2 <= max_nodes <= 128.
  * out_status: NULL, or a device int[2] that the call clears and in which a kernel records
- *   CTCSD_ERR_INVALID_ARG (and the sequence index) if kv_len/n_nodes would read outside the cache.
+ *   CTCSD_ERR_INVALID_ARG (and the sequence index) if kv_len/n_nodes would read outside the cache;
+ *   such a sequence is treated as empty (no key is read, its output rows are zero).  With
+ *   out_status == NULL the record goes to a private block that no call reads back: the zero rows
+ *   are then the only sign, so pass a status array unless the lengths are known to be valid.
  * Limits and caveats:
  *   - B*Hq*max_nodes*(D+2)*4 bytes must not exceed CTCSD_STATIC_ATTN_SCRATCH_BYTES, else
  *     CTCSD_ERR_TOO_LARGE is returned and nothing is launched; within the limit the number of

@@ -490,3 +490,63 @@ def raw_accept(node_tok: np.ndarray, kept: np.ndarray, nka: np.ndarray, n_nodes:
             acc_len[b] += 1
         next_tok[b] = int(am[b, cur])
     return acc_len, acc_nodes, acc_tok, next_tok
+
+
+# --------------------------------------------------------------------------------------
+# Several decoding steps in a row (Sec. 3.3 describes one step and ends with the history
+# update; Eq. 11 counts tokens per step over such a loop).  A plain loop over the functions
+# above, nothing else: step s drafts from the base model's hidden state at the last accepted
+# node of step s-1, its root is the bonus token of step s-1, and it runs on the cache that
+# commit_accepted left.
+# --------------------------------------------------------------------------------------
+def decode_chain(n_steps: int, x0: np.ndarray, base_tok0: np.ndarray, kv_len0: np.ndarray,
+                 Wd: np.ndarray, blank_bias: Optional[np.ndarray], Wl: np.ndarray,
+                 K: np.ndarray, Vc: np.ndarray, q_of_step, kv_of_step, hidden_of_step,
+                 T: int, k: int, N: int, n_max: int, beam: int = 0, score_mode: int = 0,
+                 scale: Optional[float] = None):
+    """x0 [B,H]: hidden states the first step drafts from; base_tok0, kv_len0 [B].
+    K, Vc [B,Hkv,Lcap,D]: the cache (copied, not modified).  The base model's per-step outputs
+    are supplied by the caller:
+      q_of_step(s)            -> Q [B,n_max,Hq,D], the tree nodes' queries;
+      kv_of_step(s)           -> (Kt, Vt) [B,Hkv,n_max,D], the tree nodes' keys/values, which are
+                                 written to cache rows kv_len[b]+j for every j < n_max;
+      hidden_of_step(s, tree) -> hn [B*n_max,H], the tree nodes' final hidden states (tree is the
+                                 tuple build_tree returned, so the caller can plant agreement).
+    Returns (records, K, Vc, kv_len): one dict per step with every intermediate result."""
+    B = x0.shape[0]
+    V = Wl.shape[0]
+    K, Vc = np.array(K, copy=True), np.array(Vc, copy=True)
+    kv_len = np.asarray(kv_len0, dtype=np.int64).copy()
+    base_tok = np.asarray(base_tok0, dtype=np.int64).copy()
+    x = np.asarray(x0)
+    records = []
+    for s in range(n_steps):
+        z = draft_logits(x, Wd, blank_bias)
+        ids, lps = topk_slots(z, k)
+        st: dict = {}
+        ctok, clen, cscore, ncand = topk_collapse(ids, lps, V, T, N, beam, score_mode, stats=st)
+        tree = build_tree(base_tok, kv_len, ctok, clen, ncand, n_max)
+        node_tok, parent, depth, pos, mask, retrieve, n_nodes = tree
+        Kt, Vt = kv_of_step(s)
+        for b in range(B):
+            L = int(kv_len[b])
+            K[b, :, L:L + n_max, :] = Kt[b]
+            Vc[b, :, L:L + n_max, :] = Vt[b]
+        Q = q_of_step(s)
+        D = Q.shape[-1]
+        O = tree_attention(Q, K, Vc, kv_len, n_nodes, mask, (1.0 / math.sqrt(D)) if scale is None else scale)
+        hn = hidden_of_step(s, tree)
+        y, am = lm_head_argmax(hn, Wl)
+        am = am.reshape(B, n_max)
+        acc_len, acc_nodes, acc_tok, next_tok = greedy_accept(node_tok, parent, n_nodes, am, T)
+        rec = dict(x=x, base_tok=base_tok.copy(), kv_len=kv_len.copy(), z=z, topk_id=ids, topk_lp=lps,
+                   cand_tok=ctok, cand_len=clen, cand_score=cscore, n_cand=ncand, margin=st["margin"],
+                   node_tok=node_tok, parent=parent, depth=depth, pos=pos, mask=mask, retrieve=retrieve,
+                   n_nodes=n_nodes, O=O, hn=hn, argmax=am, acc_len=acc_len, acc_nodes=acc_nodes,
+                   acc_tok=acc_tok, next_tok=next_tok)
+        K, Vc, kv_len, sel_row = commit_accepted(K, Vc, kv_len, acc_len, acc_nodes, n_max)
+        rec["new_kv_len"], rec["sel_row"] = kv_len.copy(), sel_row
+        records.append(rec)
+        x = hn[sel_row]                       # the next step drafts from the last accepted node's hidden state
+        base_tok = next_tok.copy()            # and its root is this step's bonus token
+    return records, K, Vc, kv_len

@@ -23,7 +23,7 @@ EXPORTS = [
     "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
     "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
-    "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static",
+    "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static", "ctcsd_draft_logits_rows",
     "ctcsd_select_raw_paths", "ctcsd_build_raw_tree", "ctcsd_verify_accept_raw",
 ]
 
@@ -63,6 +63,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_launch_count.argtypes = [vp]
     lib.ctcsd_launch_count.restype = ctypes.c_longlong
     lib.ctcsd_draft_logits.argtypes = [vp, vp, ci] + [vp] * 8
+    lib.ctcsd_draft_logits_rows.argtypes = [vp, vp, ci, vp, ci] + [vp] * 8
     lib.ctcsd_topk_collapse.argtypes = [vp, vp, ci] + [vp] * 7
     lib.ctcsd_build_tree.argtypes = [vp, vp] + [vp] * 12
     lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
@@ -174,6 +175,23 @@ class Handle:
             _ptr(out_lse, f32, M * c.T, "out_lse"),
             _ptr(out_logits_dbg, f32, M * c.T * (c.V + 1), "out_logits_dbg"))
         self._check(rc, "draft_logits")
+
+    def draft_logits_rows(self, x, x_rows, Wd, row_seq, blank_bias, out_topk_id, out_topk_lp, out_lse,
+                          out_logits_dbg=None, stream=None):
+        """Draft row m reads x[x_rows[m]] (x_rows: int32 device tensor of M entries)."""
+        c = self.cfg
+        M = x_rows.shape[0]
+        R = x.shape[0]
+        i32, f32 = torch.int32, torch.float32
+        rc = self.lib.ctcsd_draft_logits_rows(
+            self._h, _stream_ptr(stream), M,
+            _ptr(x, self.act_dtype, R * c.H, "x"), R, _ptr(x_rows, i32, M, "x_rows"),
+            _ptr(Wd, self.act_dtype, c.T * (c.V + 1) * c.H, "Wd"),
+            _ptr(row_seq, i32, M, "row_seq"), _ptr(blank_bias, f32, c.B, "blank_bias"),
+            _ptr(out_topk_id, i32, M * c.T * c.k, "out_topk_id"), _ptr(out_topk_lp, f32, M * c.T * c.k, "out_topk_lp"),
+            _ptr(out_lse, f32, M * c.T, "out_lse"),
+            _ptr(out_logits_dbg, f32, M * c.T * (c.V + 1), "out_logits_dbg"))
+        self._check(rc, "draft_logits_rows")
 
     def topk_collapse(self, topk_id, topk_lp, sel_row, out_cand_tok, out_cand_len, out_cand_score, out_n_cand,
                       stream=None):

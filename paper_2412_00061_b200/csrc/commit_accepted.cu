@@ -10,6 +10,7 @@ struct CommitParams {
     const int* kv_len; const int* acc_len; const int* acc_nodes;
     int B, Hkv, Lcap, T, max_nodes, row_bytes;
     int* out_kv_len; int* out_sel_row;
+    unsigned* seq_ticket;                // [B], zero between calls
     int* status;
 };
 
@@ -49,9 +50,16 @@ __global__ void __launch_bounds__(256) commit_accepted_kernel(CommitParams p) {
         unsigned char* dst = (which ? Vb : Kb) + (size_t)(L + 1 + l) * p.row_bytes;
         reinterpret_cast<uint4*>(dst)[ch] = reinterpret_cast<const uint4*>(rows)[(which * p.T + l) * chunks + ch];
     }
-    if (g == 0 && tid == 0) {
-        p.out_kv_len[b] = bad ? L : L + 1 + n;
-        if (p.out_sel_row) p.out_sel_row[b] = b * p.max_nodes + (n > 0 ? p.acc_nodes[b * p.T + n - 1] : 0);
+    // out_kv_len may be the very array kv_len: the new length is written by whichever CTA of the
+    // sequence finishes last, when every kv head's CTA has read the old one
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(&p.seq_ticket[b], 1u) == (unsigned)p.Hkv - 1u) {
+            p.seq_ticket[b] = 0u;
+            p.out_kv_len[b] = bad ? L : L + 1 + n;
+            if (p.out_sel_row) p.out_sel_row[b] = b * p.max_nodes + (n > 0 ? p.acc_nodes[b * p.T + n - 1] : 0);
+        }
     }
 }
 
@@ -75,6 +83,7 @@ extern "C" int ctcsd_commit_accepted(ctcsd_handle* hh, void* stream, void* K, vo
     p.row_bytes = c.D * (c.dtype == CTCSD_DTYPE_BF16 ? 2 : 4);
     p.out_kv_len = out_kv_len; p.out_sel_row = out_sel_row;
     p.status = status_ptr(h);
+    p.seq_ticket = reinterpret_cast<unsigned*>(h->ws + h->lay.seq_ticket_off);
     const size_t smem = (size_t)2 * c.T * p.row_bytes;
     CTCSD_CUDA_CHECK(h, launch_pdl(commit_accepted_kernel, dim3(c.Hkv, c.B), dim3(256), smem,
                                    static_cast<cudaStream_t>(stream), 1, p));

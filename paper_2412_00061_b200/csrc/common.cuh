@@ -34,13 +34,12 @@ struct Layout {
     size_t draft_part_off;    // DraftPartial[8][gemv_grid_max][2]  (weight-streaming GEMV partials)
     size_t part_slot_off;     // int[gemv_grid_max][2]
     size_t lm_key_off;        // uint64[lm_key_count]: packed (logit, id) row maxima of the tensor-core LM head, zero between calls
+    size_t seq_ticket_off;    // unsigned[B]: per-sequence "CTAs finished" tickets of the history update, zero between calls
     size_t tc_part_off;       // DraftPartial[T * tiles_per_slot][rows padded to 128]: tensor-core draft head (only if max_draft_rows > 8)
     size_t tc_part_bytes;
-    size_t attn_part_off;     // float[B][Hq][max_nodes][kv_splits][D+2]
     size_t total;
     int gemv_grid_max;        // largest grid the GEMV may use
     int lm_key_count;
-    int kv_splits;            // KV-axis splits in tree attention
 };
 
 constexpr int kCounters = 64;

@@ -38,6 +38,7 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
     l.counter_off = off;     off = align_up(off + kCounters * sizeof(unsigned), 256);
     l.lm_key_count = (c.B * c.max_nodes + 127) / 128 * 128;
     l.lm_key_off = off;      off = align_up(off + sizeof(unsigned long long) * (size_t)l.lm_key_count, 256);
+    l.seq_ticket_off = off;  off = align_up(off + sizeof(unsigned) * (size_t)c.B, 256);
     l.zeroed_bytes = off;
     l.gemv_grid_max = num_sms * 8 > 64 ? num_sms * 8 : 64;
     l.draft_part_off = off;  off = align_up(off + sizeof(DraftPartial) * 8 * (size_t)l.gemv_grid_max * 2, 256);
@@ -54,13 +55,6 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
             off = align_up(off + l.tc_part_bytes, 256);
         }
     }
-    int units = c.B * c.Hkv;
-    int splits = (2 * num_sms + units - 1) / units;
-    if (splits < 1) splits = 1;
-    if (splits > 16) splits = 16;
-    l.kv_splits = splits;
-    l.attn_part_off = off;
-    off = align_up(off + sizeof(float) * (size_t)c.B * c.Hq * c.max_nodes * splits * (c.D + 2), 256);
     l.total = off;
     return l;
 }

@@ -151,7 +151,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
     for (int i = tid; i < MROWS * nch; i += kThreads) {
         int m = i / nch, ch = i - m * nch;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (m < p.mcount) v = reinterpret_cast<const uint4*>(p.x)[(size_t)(p.m0 + m) * nch + ch];
+        if (m < p.mcount) {
+            int src = p.m0 + m;
+            if (p.x_rows != nullptr) {
+                src = p.x_rows[p.m0 + m];
+                if (src < 0 || src >= p.x_row_count) {               // a row map that leaves x: read nothing
+                    if (ch == 0) report_error(p.status, CTCSD_ERR_INVALID_ARG, p.m0 + m);
+                    src = -1;
+                }
+            }
+            if (src >= 0) v = reinterpret_cast<const uint4*>(p.x)[(size_t)src * nch + ch];
+        }
         xs[m * x_stride + ch] = v;
     }
     for (int i = tid; i < 2 * kStateRows * MROWS; i += kThreads) {   // states nobody fills stay empty

@@ -13,7 +13,9 @@
 namespace ctcsd {
 
 struct GemvParams {
-    const void* x;            // [M,H]
+    const void* x;            // [x_row_count,H]
+    const int* x_rows;        // [M] or null: activation row m is x[x_rows[m]] (null: x[m])
+    int x_row_count;          // rows of x (bound for x_rows)
     const void* W;            // [slots, rows_per_slot, H]
     const int* row_seq;       // [M] or null
     const float* blank_bias;  // [B] or null; added to the last row of every slot

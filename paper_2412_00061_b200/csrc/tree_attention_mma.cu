@@ -115,10 +115,12 @@ __global__ void __launch_bounds__(kThreads * (CLUSTER ? 2 : 1)) tree_attention_m
     pdl_wait();                      // the tree (node count, mask) comes from the preceding kernel
     pdl_trigger();
     int n = p.n_nodes[b];
-    const int L = p.kv_len[b];
+    int L = p.kv_len[b];
     if (n < 0 || n > p.max_nodes || L < 0 || L + n > p.Lcap) {
+        // a sequence that would read outside the cache is treated as empty: no key is loaded
         if (tid == 0) report_error(p.status, CTCSD_ERR_INVALID_ARG, b);
         n = 0;
+        L = 0;
     }
     const int Ltot = L + n;
     const int nblk = (Ltot + kKeys - 1) / kKeys;

@@ -127,10 +127,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     pdl_wait();                      // the tree (node count, mask) and Q/K/V come from preceding kernels
     pdl_trigger();
     int n = p.n_nodes[b];
-    const int L = p.kv_len[b];
+    int L = p.kv_len[b];
     if (n < 0 || n > p.max_nodes || L < 0 || L + n > p.Lcap) {
         if (tid == 0) report_error(p.status, CTCSD_ERR_INVALID_ARG, b);
         n = 0;
+        L = 0;
     }
     const int Ltot = L + n;
     const int nblk = (Ltot + kKeys - 1) / kKeys;

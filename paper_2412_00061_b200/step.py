@@ -161,6 +161,103 @@ class DraftVerifyStep:
         self.attention(stream)
         self.verify(stream)
 
+    # chained steps ----------------------------------------------------------------------
+    CHAIN_RECORDED = ("topk_id", "topk_lp", "cand_tok", "cand_len", "cand_score", "n_cand", "node_tok", "parent",
+                      "depth", "pos", "mask", "retrieve", "n_nodes", "O", "argmax", "acc_len", "acc_nodes", "acc_tok",
+                      "next_tok", "new_kv_len", "next_sel_row")
+
+    def setup_chain(self, n_steps: int, x0, base_tok0, kv_len0, Qtab, Ktab, Vtab, hntab, record: bool = True):
+        """Device-side state of n_steps chained steps (history update after every step, no host work
+        in between).  x0 [B,H], base_tok0 [B], kv_len0 [B]: where the chain starts.  The per-step
+        tables stand in for the base model: Qtab [S,B,max_nodes,Hq,D] tree-node queries, Ktab/Vtab
+        [S,B,Hkv,max_nodes,D] tree-node keys/values, hntab [S,B*max_nodes,H] tree-node hidden states.
+        K, V (the cache, updated in place), Wd, Wl, blank_bias come from set_inputs()."""
+        cfg, dev = self.cfg, self.device
+        self.chain = dict(n=n_steps, x0=x0, base_tok0=base_tok0, kv_len0=kv_len0, Qtab=Qtab, Ktab=Ktab, Vtab=Vtab,
+                          hntab=hntab, kv_len=kv_len0.clone(), kv_before=None, rec=None,
+                          node_off=torch.arange(cfg.max_nodes, device=dev, dtype=torch.int64))
+        if record:
+            self.chain["rec"] = {k: torch.zeros((n_steps,) + tuple(self.out[k].shape), dtype=self.out[k].dtype,
+                                                device=dev) for k in self.CHAIN_RECORDED if k in self.out}
+            self.chain["kv_before"] = torch.zeros(n_steps, cfg.B, dtype=torch.int32, device=dev)
+            if self.layout == "raw":
+                for k in ("kept", "nka"):
+                    self.chain["rec"][k] = torch.zeros((n_steps,) + tuple(self.out[k].shape), dtype=torch.int32,
+                                                       device=dev)
+
+    def write_tree_kv(self, s: int):
+        """Stand-in for the base model's key/value projection of step s: node j's key and value go
+        to cache row kv_len[b]+j (device-side indices, no host work)."""
+        c, cfg = self.chain, self.cfg
+        rows = c["kv_len"].to(torch.int64)[:, None] + c["node_off"][None, :]                    # [B,n]
+        idx = rows[:, None, :, None].expand(cfg.B, cfg.Hkv, cfg.max_nodes, cfg.D)
+        self.inp["K"].scatter_(2, idx, c["Ktab"][s])
+        self.inp["V"].scatter_(2, idx, c["Vtab"][s])
+
+    def chain_head(self, s: int):
+        """Step s of the chain up to the token tree: draft head, candidates, tree."""
+        c, i, o = self.chain, self.inp, self.out
+        i["kv_len"] = c["kv_len"]
+        i["sel_row"] = None
+        if s == 0:
+            i["base_tok"] = c["base_tok0"]
+            self.h.draft_logits(c["x0"], i["Wd"], None, i.get("blank_bias"), o["topk_id"], o["topk_lp"], o["lse"])
+        else:
+            i["base_tok"] = o["next_tok"]              # the previous step's bonus token is this step's root
+            self.h.draft_logits_rows(c["hntab"][s - 1], o["next_sel_row"], i["Wd"], None, i.get("blank_bias"),
+                                     o["topk_id"], o["topk_lp"], o["lse"])
+        self.collapse()
+        self.tree()
+
+    def chain_tail(self, s: int):
+        """The rest of step s: the base model's stand-in writes the tree's keys/values, then tree
+        attention, LM head + acceptance, and the history update."""
+        c, i, o = self.chain, self.inp, self.out
+        self.write_tree_kv(s)
+        i["Q"] = c["Qtab"][s]
+        i["hn"] = c["hntab"][s]
+        self.attention()
+        self.verify()
+        if c["kv_before"] is not None:
+            c["kv_before"][s].copy_(c["kv_len"])
+        # the new length overwrites the old one in place; the next step drafts from out["next_sel_row"]
+        self.h.commit_accepted(i["K"], i["V"], c["kv_len"], o["acc_len"], o["acc_nodes"], c["kv_len"],
+                               o["next_sel_row"])
+        if c["rec"] is not None:
+            o["new_kv_len"].copy_(c["kv_len"])
+            for k, buf in c["rec"].items():
+                buf[s].copy_(o[k])
+
+    def run_chain(self):
+        """All steps of the chain back to back on the current stream: per step the five calls and
+        the history update, the next step reading its drafting row, root token and cache length
+        from what the previous one left on the device."""
+        c = self.chain
+        c["kv_len"].copy_(c["kv_len0"])
+        for s in range(c["n"]):
+            self.chain_head(s)
+            self.chain_tail(s)
+
+    def plant_chain_hidden(self, seed: int, Wl_host: np.ndarray):
+        """Fills the chain's table of tree-node hidden states so that the base model agrees with the
+        drafts at the configured rate.  The hidden states of step s depend on the tree of step s,
+        which depends on what earlier steps accepted, so this walks the chain once with a host
+        round trip per step (set-up only; run_chain() then needs none)."""
+        from . import synth
+        c, cfg = self.chain, self.cfg
+        c["kv_len"].copy_(c["kv_len0"])
+        for s in range(c["n"]):
+            self.chain_head(s)
+            self.check_status()
+            parent = self.host("parent")
+            if self.layout == "raw":
+                parent = np.where(self.host("kept") != 0, self.host("nka"), -1)
+            hn, _ = synth.gen_node_hidden(cfg, synth.chain_step_seed(seed, s), Wl_host, self.host("node_tok"),
+                                          parent, self.host("n_nodes"))
+            c["hntab"][s].copy_(to_device(hn, cfg.dtype, self.device))
+            self.chain_tail(s)
+        self.check_status()
+
     def check_status(self):
         st = self.h.poll_status()
         if st != 0:

@@ -197,3 +197,28 @@ def gen_node_hidden(cfg: StepConfig, seed: int, Wl: np.ndarray, node_tok: np.nda
     live = flat >= 0
     hn[live] = Wl[flat[live]] + noise[live]
     return to_dtype(hn, cfg.dtype), target
+
+
+def chain_cache_config(cfg: StepConfig, n_steps: int) -> StepConfig:
+    """The same shape with a cache large enough for n_steps chained steps: every step appends
+    its root and at most T accepted tokens, and the last tree still needs max_nodes rows."""
+    return cfg.replace(kv_hi=cfg.kv_hi + n_steps * (cfg.T + 1))
+
+
+def gen_chain_tables(cfg: StepConfig, seed: int, n_steps: int):
+    """Per-step stand-ins for what the base model produces at the tree nodes of each of n_steps
+    chained steps: queries Qtab [S,B,max_nodes,Hq,D] and keys/values Ktab, Vtab
+    [S,B,Hkv,max_nodes,D], all ~ N(0,1), drawn independently per step."""
+    S = n_steps
+    Qtab = np.stack([_normal(seed * 1009 + 1 + s, "Q", (cfg.B, cfg.max_nodes, cfg.Hq, cfg.D), 1.0, cfg.dtype)
+                     for s in range(S)])
+    Ktab = np.stack([_normal(seed * 1009 + 1 + s, "K", (cfg.B, cfg.Hkv, cfg.max_nodes, cfg.D), 1.0, cfg.dtype)
+                     for s in range(S)])
+    Vtab = np.stack([_normal(seed * 1009 + 1 + s, "V", (cfg.B, cfg.Hkv, cfg.max_nodes, cfg.D), 1.0, cfg.dtype)
+                     for s in range(S)])
+    return Qtab, Ktab, Vtab
+
+
+def chain_step_seed(seed: int, step: int) -> int:
+    """Seed of gen_node_hidden for step `step` of a chain."""
+    return seed * 1009 + 1 + step

@@ -22,6 +22,16 @@ from paper_2412_00061_b200.step import DraftVerifyStep, to_device
 TAU = 1e-9          # score gaps below this make the candidate order a tie (fp64 on both sides)
 
 
+def sample_rng(cfg, seed, what):
+    """Generator for the sampled (sequence, head) pairs / rows of the definition-mode checks: it
+    differs per workload, per test seed and per kind of sample, and CTCSD_SAMPLE_SALT (an integer
+    in the environment) moves every sample at once for a run that wants fresh ones."""
+    import os
+    import zlib
+    salt = int(os.environ.get("CTCSD_SAMPLE_SALT", "0"))
+    return np.random.default_rng([seed, zlib.crc32(cfg.name.encode()), zlib.crc32(what.encode()), salt])
+
+
 def tolerances(dtype: str):
     # max-abs error on logits / attention outputs, relative error on log-probs
     return (2e-2, 1e-4) if dtype == "bf16" else (2e-4, 1e-4)
@@ -141,7 +151,7 @@ def run_parity(cfg, seed=0, M=None, force_repeats=False, row_seq=None, sel_row=N
         O_def = orc.tree_attention(inp["Q"], inp["K"], inp["V"], inp["kv_len"], n_nodes, mask, 1.0 / math.sqrt(cfg.D))
         assert np.max(np.abs(O_gpu - O_def)) <= logit_tol
     else:
-        rng = np.random.default_rng(seed + 77)
+        rng = sample_rng(cfg, seed, "attention")
         for _ in range(attention_rows):                 # sampled (sequence, head) pairs, all nodes each
             b = int(rng.integers(0, cfg.B))
             h = int(rng.integers(0, cfg.Hq))
@@ -163,7 +173,7 @@ def run_parity(cfg, seed=0, M=None, force_repeats=False, row_seq=None, sel_row=N
     live = [b * cfg.max_nodes + i for b in range(cfg.B) for i in range(int(n_nodes[b]))]
     rows = live
     if lm_rows is not None and len(live) > lm_rows:
-        rows = [live[j] for j in np.random.default_rng(seed + 5).choice(len(live), lm_rows, replace=False)]
+        rows = [live[j] for j in sample_rng(cfg, seed, "lm_rows").choice(len(live), lm_rows, replace=False)]
     y_def, am_def = orc.lm_head_argmax(hn[rows], inp["Wl"])
     assert np.max(np.abs(y_gpu[rows] - y_def)) <= logit_tol
     am_gpu = step.host("argmax")
@@ -241,7 +251,7 @@ def run_parity_raw(cfg, seed=0, force_repeats=False, device="cuda:0", attention_
         O_def = orc.tree_attention(inp["Q"], inp["K"], inp["V"], inp["kv_len"], n_nodes, mask, 1.0 / math.sqrt(cfg.D))
         assert np.max(np.abs(O_gpu - O_def)) <= logit_tol
     else:
-        rng = np.random.default_rng(seed + 77)
+        rng = sample_rng(cfg, seed, "attention")
         for _ in range(attention_rows):
             b = int(rng.integers(0, cfg.B))
             h = int(rng.integers(0, cfg.Hq))
@@ -261,7 +271,7 @@ def run_parity_raw(cfg, seed=0, force_repeats=False, device="cuda:0", attention_
     live = [b * cfg.max_nodes + i for b in range(cfg.B) for i in range(int(n_nodes[b]))]
     rows = live
     if lm_rows is not None and len(live) > lm_rows:
-        rows = [live[j] for j in np.random.default_rng(seed + 5).choice(len(live), lm_rows, replace=False)]
+        rows = [live[j] for j in sample_rng(cfg, seed, "lm_rows").choice(len(live), lm_rows, replace=False)]
     y_def, am_def = orc.lm_head_argmax(hn[rows], inp["Wl"])
     assert np.max(np.abs(y_gpu[rows] - y_def)) <= logit_tol
     am_gpu = step.host("argmax")
@@ -282,3 +292,189 @@ def run_parity_raw(cfg, seed=0, force_repeats=False, device="cuda:0", attention_
     for k, v in before.items():
         np.testing.assert_array_equal(step.host(k), v, err_msg="rerun " + k)
     return dict(acc_len=acc[0], n_nodes=n_nodes, kept=kept, step=step)
+
+
+def run_chain_parity(cfg, seed=0, n_steps=4, layout="packed", device="cuda:0", graph=False):
+    """n_steps chained steps on the GPU (run_chain: no host work between steps, the new cache length
+    written over the old one in place) against the oracle.
+
+    Stage-fed, every step: the oracle is handed what the GPU produced one stage earlier - its top-k
+    lists, its candidates, its arg-max, its accepted path - plus the chain state the GPU carried over
+    (root token, cache length, drafting row), and every integer output must match bit for bit; the
+    top-k lists themselves are checked against the oracle's logits of the carried-over hidden state,
+    attention outputs against the oracle's on its own running cache (<= 2e-2).  At the end the K/V
+    cache must equal the oracle's byte for byte.  Packed layout only: the whole chain is also run by
+    orc.decode_chain from the raw inputs, and when none of its decisions was a near-tie the GPU chain
+    must reproduce it exactly.  Returns the number of tokens the chain emitted."""
+    logit_tol, rel = tolerances(cfg.dtype)
+    big = synth.chain_cache_config(cfg, n_steps)
+    x0, Wd, bb = synth.gen_draft(cfg, seed)
+    base_tok0, kv_len0 = synth.gen_base(cfg, seed)
+    _, K0, V0 = synth.gen_attention(big, seed)
+    Wl = synth.gen_lm_head(cfg, seed)
+    Qtab, Ktab, Vtab = synth.gen_chain_tables(cfg, seed, n_steps)
+    B, n_max, T = cfg.B, cfg.max_nodes, cfg.T
+
+    step = DraftVerifyStep(cfg, device=device, layout=layout)
+    dev = step.device
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    step.set_inputs(Wd=to_device(Wd, cfg.dtype, dev), blank_bias=torch.from_numpy(bb).to(dev),
+                    K=to_device(K0, cfg.dtype, dev), V=to_device(V0, cfg.dtype, dev), Wl=to_device(Wl, cfg.dtype, dev))
+    act = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    hntab = torch.zeros(n_steps, B * n_max, cfg.H, dtype=act, device=dev)
+    step.setup_chain(n_steps, to_device(x0, cfg.dtype, dev), i32(base_tok0), i32(kv_len0),
+                     to_device(Qtab, cfg.dtype, dev), to_device(Ktab, cfg.dtype, dev), to_device(Vtab, cfg.dtype, dev), hntab)
+
+    # ---- the tree-node hidden states ------------------------------------------------------------
+    chain_def = None
+    if layout == "packed":
+        hidden = lambda s, tree: synth.gen_node_hidden(cfg, synth.chain_step_seed(seed, s), Wl, tree[0], tree[1], tree[6])[0]
+        chain_def = orc.decode_chain(n_steps, x0, base_tok0, kv_len0, Wd, bb, Wl, K0, V0, lambda s: Qtab[s],
+                                     lambda s: (Ktab[s], Vtab[s]), hidden, T, cfg.k, cfg.topN, n_max, cfg.beam,
+                                     cfg.score_mode)
+        hn_host = np.stack([r["hn"] for r in chain_def[0]])
+        hntab.copy_(to_device(hn_host, cfg.dtype, dev))
+    else:
+        step.plant_chain_hidden(seed, Wl)
+        hn_host = hntab.float().cpu().numpy()
+        step.inp["K"].copy_(to_device(K0, cfg.dtype, dev))
+        step.inp["V"].copy_(to_device(V0, cfg.dtype, dev))
+
+    # ---- the chain on the GPU ---------------------------------------------------------------------
+    if graph:
+        side = torch.cuda.Stream(device=dev)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            step.run_chain()                                  # warm-up outside the capture
+            torch.cuda.synchronize()
+            step.inp["K"].copy_(to_device(K0, cfg.dtype, dev))
+            step.inp["V"].copy_(to_device(V0, cfg.dtype, dev))
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                step.run_chain()
+        g.replay()
+    else:
+        step.run_chain()
+    step.check_status()
+    rec = {k: (v.float() if v.dtype == torch.bfloat16 else v).cpu().numpy() for k, v in step.chain["rec"].items()}
+    kv_before = step.chain["kv_before"].cpu().numpy()
+
+    # ---- stage-fed walk ---------------------------------------------------------------------------
+    Kc, Vc = np.array(K0, copy=True), np.array(V0, copy=True)
+    kv_len = kv_len0.astype(np.int64)
+    base_tok = base_tok0.astype(np.int64)
+    x = x0
+    tokens = 0
+    for s in range(n_steps):
+        np.testing.assert_array_equal(kv_before[s], kv_len, err_msg="kv_len at step %d" % s)
+        # S1-S3 from the carried-over hidden state
+        z = orc.draft_logits(x, Wd, bb)
+        ids_o, lp_o = orc.topk_slots(z, cfg.k)
+        srt = -np.sort(-z, axis=-1)[..., :cfg.k + 1]
+        clear = (srt[..., :-1] - srt[..., 1:]).min() > 4 * logit_tol * 1e-2     # gaps far above the fp32 noise
+        ids_g, lp_g = rec["topk_id"][s], rec["topk_lp"][s]
+        if clear:
+            np.testing.assert_array_equal(ids_g, ids_o, err_msg="topk_id at step %d" % s)
+        lse_o, _ = orc.log_softmax_slots(z)
+        lp_at = np.take_along_axis(z, ids_g.astype(np.int64), axis=-1) - lse_o[..., None]
+        np.testing.assert_allclose(lp_g, lp_at, rtol=rel, atol=logit_tol)
+        # S4-S8 fed the GPU's lists
+        if layout == "packed":
+            got = (rec["cand_tok"][s], rec["cand_len"][s], rec["cand_score"][s], rec["n_cand"][s])
+            check_candidates(cfg, ids_g, lp_g, None, got)
+            tree = orc.build_tree(base_tok, kv_len, got[0].astype(np.int64), got[1].astype(np.int64),
+                                  got[3].astype(np.int64), n_max)
+            names = ["node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes"]
+        else:
+            for b in range(B):
+                want_tok, _ = orc.select_raw_paths(ids_g[b].astype(np.int64), lp_g[b].astype(np.float64), cfg.topN)
+                np.testing.assert_array_equal(rec["cand_tok"][s][b, :want_tok.shape[0]], want_tok)
+            tree = orc.build_raw_tree(base_tok, kv_len, rec["cand_tok"][s].astype(np.int64),
+                                      rec["n_cand"][s].astype(np.int64), cfg.V, n_max)
+            names = ["node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes", "kept", "nka"]
+        for name, want in zip(names, tree):
+            have = rec[name][s]
+            if name == "mask":
+                have = have.view(np.uint64)
+            np.testing.assert_array_equal(have, want, err_msg="%s at step %d" % (name, s))
+        node_tok, parent, mask, n_nodes = tree[0], tree[1], tree[4], tree[6]
+        # S9 on the oracle's own running cache
+        for b in range(B):
+            L = int(kv_len[b])
+            Kc[b, :, L:L + n_max] = Ktab[s][b]
+            Vc[b, :, L:L + n_max] = Vtab[s][b]
+        rng = np.random.default_rng(seed * 31 + s)
+        for _ in range(2):
+            b, h = int(rng.integers(0, B)), int(rng.integers(0, cfg.Hq))
+            g_ = h // (cfg.Hq // cfg.Hkv)
+            one = orc.tree_attention(Qtab[s][b:b + 1, :, h:h + 1], Kc[b:b + 1, g_:g_ + 1], Vc[b:b + 1, g_:g_ + 1],
+                                     kv_len[b:b + 1], n_nodes[b:b + 1], mask[b:b + 1], 1.0 / math.sqrt(cfg.D))
+            assert np.max(np.abs(rec["O"][s][b, :, h] - one[0, :, 0])) <= logit_tol
+        # S10-S11
+        am_g = rec["argmax"][s].astype(np.int64)
+        live = [b * n_max + i for b in range(B) for i in range(int(n_nodes[b]))]
+        _, am_def = orc.lm_head_argmax(hn_host[s][live], Wl)
+        np.testing.assert_array_equal(am_g.reshape(-1)[live], am_def, err_msg="argmax at step %d" % s)
+        if layout == "packed":
+            acc = orc.greedy_accept(node_tok, parent, n_nodes, am_g, T)
+        else:
+            acc = orc.raw_accept(node_tok, tree[7], tree[8], n_nodes, am_g, T)
+        for name, want in zip(["acc_len", "acc_nodes", "acc_tok", "next_tok"], acc):
+            np.testing.assert_array_equal(rec[name][s], want, err_msg="%s at step %d" % (name, s))
+        # S12 and the hand-over
+        Kc, Vc, kv_len, sel = orc.commit_accepted(Kc, Vc, kv_len, acc[0], acc[1], n_max)
+        np.testing.assert_array_equal(rec["new_kv_len"][s], kv_len)
+        np.testing.assert_array_equal(rec["next_sel_row"][s], sel)
+        tokens += int(acc[0].sum()) + B
+        x = hn_host[s][sel]
+        base_tok = acc[3].astype(np.int64)
+    assert np.array_equal(step.inp["K"].float().cpu().numpy(), Kc), "K cache after the chain"
+    assert np.array_equal(step.inp["V"].float().cpu().numpy(), Vc), "V cache after the chain"
+
+    # ---- definition mode: the whole chain from the raw inputs ---------------------------------------
+    certified = None
+    if chain_def is not None:
+        recs_o, K_o, V_o, kv_o = chain_def
+        certified = all(min(r["margin"]) > 1e-5 for r in recs_o)
+        if certified:
+            for s, r in enumerate(recs_o):
+                for name in ("cand_tok", "node_tok", "parent", "n_nodes", "argmax", "acc_len", "acc_nodes", "acc_tok", "next_tok"):
+                    np.testing.assert_array_equal(rec[name][s], r[name], err_msg="definition mode, %s at step %d" % (name, s))
+            np.testing.assert_array_equal(kv_len, kv_o)
+            assert np.array_equal(Kc, K_o) and np.array_equal(Vc, V_o)
+    return dict(tokens=tokens, certified=certified, step=step)
+
+
+def check_benchmark_launch_configuration(checked, steps_per_graph=3, replays=2):
+    """`checked` is what run_parity / run_parity_raw returned: a step whose outputs the oracle has
+    verified (run with the debug dumps on, one call at a time).  The benchmark runs the same step
+    differently - no debug pointers, the L2 prefetch hint on, several steps back to back inside one
+    CUDA graph so that every kernel overlaps its neighbour's tail, shared ticket counters reset by
+    the last CTA of each kernel - and this reruns it that way and demands identical results."""
+    ref = checked["step"]
+    cfg = ref.cfg
+    names = ["topk_id", "topk_lp", "lse", "cand_tok", "cand_len", "cand_score", "n_cand", "node_tok", "parent", "depth",
+             "pos", "mask", "retrieve", "n_nodes", "O", "argmax", "acc_len", "acc_nodes", "acc_tok", "next_tok"]
+    if ref.layout == "raw":
+        names += ["kept", "nka"]
+        names.remove("cand_len")
+    want = {k: ref.out[k].clone() for k in names}
+    step = DraftVerifyStep(cfg, device=str(ref.device), max_draft_rows=ref.M, debug_logits=False, layout=ref.layout)
+    step.set_inputs(**{k: v for k, v in ref.inp.items() if v is not None})      # Wl among them: the L2 hint is on
+    assert "draft_logits_dbg" not in step.out and "lm_logits_dbg" not in step.out
+    side = torch.cuda.Stream(device=step.device)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            step.run()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(steps_per_graph):
+                step.run()
+    for _ in range(replays):
+        for t in step.out.values():
+            t.zero_()                                   # nothing may survive from the replay before
+        g.replay()
+        step.check_status()
+        for k in names:
+            assert torch.equal(step.out[k], want[k]), "benchmark configuration differs in " + k

@@ -107,11 +107,21 @@ def test_only_blank_paths_leave_just_the_root():
 
 
 def test_c2_full_size_sampled():
-    """The headline workload at full size, in the launch configuration the benchmark times.
-    The definition-mode oracle checks one draft row in full, sampled LM-head rows and sampled
-    attention (sequence, head) pairs; all integer stages are compared in full."""
+    """The headline workload at full size.  The definition-mode oracle checks one draft row in
+    full, sampled LM-head rows and sampled attention (sequence, head) pairs; all integer stages are
+    compared in full.  Then the step is rerun the way the benchmark launches it (no debug dumps, L2
+    hint, a CUDA graph of three steps replayed twice) and must give the same results bit for bit."""
+    from tests.parity_util import check_benchmark_launch_configuration
     r = _run(C["c2"], seed=0, require_certified=True, attention_rows=4, lm_rows=8)
     assert 2 <= r["n_nodes"][0] <= 64
+    check_benchmark_launch_configuration(r)
+
+
+def test_c2_raw_layout_and_c3_in_the_benchmark_launch_configuration():
+    from tests.parity_util import check_benchmark_launch_configuration, run_parity_raw
+    check_benchmark_launch_configuration(run_parity_raw(C["c2"], seed=0, attention_rows=2, lm_rows=8))
+    check_benchmark_launch_configuration(_run(C["c3"], seed=1, attention_rows=2, lm_rows=6, draft_rows=[0]))
+    check_benchmark_launch_configuration(_run(SMALL["c5s"], seed=2))
 
 
 @pytest.mark.parametrize("name", ["c3", "c4", "c5", "c6"])
@@ -127,7 +137,7 @@ def test_batched_workloads_full_size_sampled(name):
 @pytest.mark.parametrize("name", ["c2s", "c3s", "c5s", "c1d64"])
 def test_history_update_moves_the_accepted_rows(name):
     """ctcsd_commit_accepted against the oracle: the K/V caches must match byte for byte, the new
-    lengths and the next drafting rows exactly; then a second step runs on the updated cache."""
+    lengths and the next drafting rows exactly (steps that run on the updated cache: the chain tests)."""
     import torch
     from oracle import ctcsd_oracle as orc
     cfg = SMALL[name]
@@ -150,6 +160,61 @@ def test_history_update_moves_the_accepted_rows(name):
                            step.out["new_kv_len"], step.out["next_sel_row"])
     assert step.h.poll_status() == -1
     assert np.array_equal(step.inp["K"].float().cpu().numpy(), K1)
+
+
+def test_history_update_may_write_the_new_length_over_the_old_one():
+    """out_kv_len is the same array as kv_len, on a shape with more (sequence, kv head) CTAs than the
+    GPU holds at once (48 x 32 = 1536): a CTA that starts late must still see the old length."""
+    import torch
+    from oracle import ctcsd_oracle as orc
+    from paper_2412_00061_b200 import binding
+    from paper_2412_00061_b200.step import to_device
+    cfg = C["c3"].replace(name="alias", B=48, H=64, V=100, Hq=32, Hkv=32, D=64, kv_lo=3, kv_hi=60, max_nodes=32, T=6)
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(21)
+    _, K, V = synth.gen_attention(cfg, 21)
+    _, kv_len = synth.gen_base(cfg, 21)
+    acc_len = rng.integers(0, cfg.T + 1, size=cfg.B).astype(np.int32)
+    acc_nodes = np.full((cfg.B, cfg.T), -1, dtype=np.int32)
+    for b in range(cfg.B):                       # strictly increasing node ids, node_l >= l + 1
+        acc_nodes[b, :acc_len[b]] = np.sort(rng.choice(np.arange(1, cfg.max_nodes), size=acc_len[b], replace=False))
+    K1, V1, new_len, sel = orc.commit_accepted(K, V, kv_len, acc_len, acc_nodes, cfg.max_nodes)
+    h = binding.Handle(cfg.B, cfg.H, cfg.V, cfg.T, cfg.k, cfg.beam, cfg.topN, cfg.max_nodes, cfg.Hq, cfg.Hkv, cfg.D,
+                       binding.DTYPE_BF16)
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    Kd, Vd, len_d = to_device(K, "bf16", dev), to_device(V, "bf16", dev), i32(kv_len)
+    sel_d = torch.zeros(cfg.B, dtype=torch.int32, device=dev)
+    h.commit_accepted(Kd, Vd, len_d, i32(acc_len), i32(acc_nodes), len_d, sel_d)
+    assert h.poll_status() == 0
+    assert np.array_equal(Kd.float().cpu().numpy(), K1) and np.array_equal(Vd.float().cpu().numpy(), V1)
+    np.testing.assert_array_equal(len_d.cpu().numpy(), new_len)
+    np.testing.assert_array_equal(sel_d.cpu().numpy(), sel)
+    # and once more on the result (the per-sequence tickets were left at zero)
+    K2, V2, new_len2, _ = orc.commit_accepted(K1, V1, new_len, acc_len, acc_nodes, cfg.max_nodes)
+    h.commit_accepted(Kd, Vd, len_d, i32(acc_len), i32(acc_nodes), len_d, sel_d)
+    assert h.poll_status() == 0
+    assert np.array_equal(Kd.float().cpu().numpy(), K2)
+    np.testing.assert_array_equal(len_d.cpu().numpy(), new_len2)
+    h.close()
+
+
+@pytest.mark.parametrize("name", ["c2s", "c3s", "c5s", "c1d64"])
+def test_chained_steps_without_host_work(name):
+    """Five steps in a row, each followed by the history update, the next one taking its root token,
+    cache length and drafting row from the device: every step's integers against the oracle fed the
+    GPU's previous stage, the final K/V cache byte for byte, and the oracle's own chain from the raw
+    inputs wherever none of its decisions was a near-tie."""
+    from tests.parity_util import run_chain_parity
+    r = run_chain_parity(SMALL[name], seed=4, n_steps=5)
+    assert r["tokens"] > 5 * SMALL[name].B, "pick a seed where draft tokens are accepted"
+
+
+def test_chained_steps_fp32_and_inside_a_cuda_graph():
+    from tests.parity_util import run_chain_parity
+    cfg = C["c1"].replace(name="c1chain", B=2, kv_lo=5, kv_hi=90)
+    run_chain_parity(cfg, seed=1, n_steps=4)
+    r = run_chain_parity(SMALL["c3s"], seed=6, n_steps=4, graph=True)
+    assert r["tokens"] > 4 * SMALL["c3s"].B
 
 
 BIG = {
@@ -249,6 +314,13 @@ def test_raw_tree_layout(name, seed):
     live = sum(int(n) for n in r["n_nodes"])
     removed = live - int(r["kept"].sum())
     assert removed > 0, "the inputs must exercise the transform (blanks or repeats in the raw paths)"
+
+
+@pytest.mark.parametrize("name", ["c2raw", "c5raw_cut"])
+def test_chained_steps_raw_layout(name):
+    from tests.parity_util import run_chain_parity
+    r = run_chain_parity(RAW[name], seed=3, n_steps=4, layout="raw")
+    assert r["tokens"] > 4 * RAW[name].B
 
 
 def test_raw_tree_layout_c2_full_size_and_history_update():

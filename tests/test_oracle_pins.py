@@ -715,6 +715,74 @@ def test_commit_accepted_reads_the_cache_as_it_was():
     assert np.array_equal(K2[1], K[1]) and new_len.tolist() == [5, 2] and sel.tolist() == [3, 4]
 
 
+# ------------------------------------------------------------------ chained steps
+def _chain_case(seed, n_steps, p=0.8):
+    from paper_2412_00061_b200 import synth
+    cfg = synth.CONFIGS["c1"].replace(name="chain", B=2, H=48, V=30, T=3, k=3, topN=6, max_nodes=12, Hq=2, Hkv=1,
+                                      D=8, kv_lo=2, kv_hi=6, agree_p=p)
+    big = synth.chain_cache_config(cfg, n_steps)
+    x0, Wd, bb = synth.gen_draft(cfg, seed)
+    base_tok, kv_len = synth.gen_base(cfg, seed)
+    _, K, V = synth.gen_attention(big, seed)
+    Wl = synth.gen_lm_head(cfg, seed)
+    Qtab, Ktab, Vtab = synth.gen_chain_tables(cfg, seed, n_steps)
+    hidden = lambda s, tree: synth.gen_node_hidden(cfg, synth.chain_step_seed(seed, s), Wl, tree[0], tree[1], tree[6])[0]
+    out = orc.decode_chain(n_steps, x0, base_tok, kv_len, Wd, bb, Wl, K, V, lambda s: Qtab[s],
+                           lambda s: (Ktab[s], Vtab[s]), hidden, cfg.T, cfg.k, cfg.topN, cfg.max_nodes)
+    return cfg, (x0, base_tok, kv_len, K, V, Qtab, Ktab, Vtab), out
+
+
+def test_chained_steps_leave_exactly_the_emitted_tokens_in_the_cache():
+    """What a chain of steps must amount to, stated without the loop: the cache grows by each step's
+    root and accepted nodes, in order, and nothing else moves; every step starts where the previous
+    one stopped (root = previous bonus token, drafting state = hidden state of the last accepted
+    node); and the tree attention an accepted node saw equals ordinary causal attention of its
+    query over the final cache up to its own row (the rows before it are exactly its prefix)."""
+    n_steps, accepted = 5, 0
+    for seed in (0, 1, 2):
+        cfg, (x0, base_tok, kv_len0, K0, V0, Qtab, Ktab, Vtab), (recs, K, V, kv_len) = _chain_case(seed, n_steps)
+        n_max = cfg.max_nodes
+        for b in range(cfg.B):
+            L0 = int(kv_len0[b])
+            rows_k, rows_v, queries = [], [], []
+            for s, r in enumerate(recs):
+                path = [0] + [int(v) for v in r["acc_nodes"][b, :r["acc_len"][b]]]
+                accepted += len(path) - 1
+                for node in path:
+                    rows_k.append(Ktab[s][b, :, node])
+                    rows_v.append(Vtab[s][b, :, node])
+                    queries.append((s, node))
+                assert r["kv_len"][b] == L0 + len(rows_k) - len(path)
+                if s + 1 < n_steps:
+                    assert recs[s + 1]["base_tok"][b] == r["next_tok"][b]
+                    np.testing.assert_array_equal(recs[s + 1]["x"][b], r["hn"][b * n_max + path[-1]])
+            assert kv_len[b] == L0 + len(rows_k) == L0 + sum(int(r["acc_len"][b]) + 1 for r in recs)
+            np.testing.assert_array_equal(K[b, :, :L0], K0[b, :, :L0])
+            np.testing.assert_array_equal(K[b, :, L0:L0 + len(rows_k)], np.stack(rows_k, axis=1))
+            np.testing.assert_array_equal(V[b, :, L0:L0 + len(rows_v)], np.stack(rows_v, axis=1))
+            for i, (s, node) in enumerate(queries):
+                for h in range(cfg.Hq):
+                    q = torch.tensor(Qtab[s][b, node, h], dtype=torch.float64)
+                    kk = torch.tensor(K[b, 0, :L0 + i + 1], dtype=torch.float64)
+                    vv = torch.tensor(V[b, 0, :L0 + i + 1], dtype=torch.float64)
+                    pr = torch.softmax(kk @ q / math.sqrt(cfg.D), 0)
+                    np.testing.assert_allclose(recs[s]["O"][b, node, h], (pr @ vv).numpy(), atol=1e-12)
+    assert accepted >= 10                                  # the chains really accept draft tokens
+
+
+def test_a_chain_of_one_step_is_the_single_step():
+    cfg, (x0, base_tok, kv_len0, K0, V0, Qtab, Ktab, Vtab), (recs, K, V, kv_len) = _chain_case(3, 1)
+    r = recs[0]
+    from paper_2412_00061_b200 import synth
+    x, Wd, bb = synth.gen_draft(cfg, 3)
+    ids, lps = orc.topk_slots(orc.draft_logits(x, Wd, bb), cfg.k)
+    np.testing.assert_array_equal(r["topk_id"], ids)
+    ctok, clen, _, nc = orc.topk_collapse(ids, lps, cfg.V, cfg.T, cfg.topN)
+    tree = orc.build_tree(base_tok, kv_len0, ctok, clen, nc, cfg.max_nodes)
+    for name, want in zip(["node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes"], tree):
+        np.testing.assert_array_equal(r[name], want)
+
+
 # ------------------------------------------------------------------ the paper's raw-tree layout
 def test_raw_paths_are_the_most_probable_alignments():
     rng = np.random.default_rng(11)
