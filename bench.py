@@ -13,6 +13,7 @@ from __future__ import annotations
 
 import argparse
 import datetime
+import hashlib
 import json
 import os
 import subprocess
@@ -26,11 +27,30 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the draft-head kernel, from the
-# ncu capture summarised in profiles/gemv_stream_kernel_c2.md (None once the kernel has changed
-# since that capture).  It includes the 48 MB of LM-head weights that the kernel asks L2 to
-# prefetch for the next heavy kernel.
-NCU_TRAFFIC_BYTES = {"c2": 1356.540e6 + 3.153e6}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """DRAM bytes (read + write) of one launch of `kernel` on `workload`, as counted by ncu and
+    recorded in profiles/traffic.json by paper_2412_00061_b200/ncu_traffic.py, or None when no
+    record exists or a source file of the kernel has changed since the counters were taken (the
+    record carries the files' SHA-256)."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f).get(workload, {}).get(kernel)
+    except (OSError, ValueError):
+        return None
+    if not rec:
+        return None
+    for rel, want in rec.get("source_sha256", {}).items():
+        try:
+            with open(os.path.join(ROOT, rel), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != want:
+                    return None
+        except OSError:
+            return None
+    return rec.get("traffic_bytes")
+
 
 METRIC = "draft+verify steps/s at 7B shape (batch 1, 64-node tree)"
 UNIT = "steps/s"
@@ -63,7 +83,7 @@ class ClockSampler:
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int, period_ms: int = 50):
+    def __init__(self, index: int, period_ms: int = 10):
         self.windows = []
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
@@ -148,9 +168,9 @@ def oracle_step(cfg, inp, layout="packed"):
     orc.greedy_accept(node_tok, parent, n_nodes, am.reshape(cfg.B, cfg.max_nodes), cfg.T)
 
 
-def host_inputs(cfg, seed):
+def host_inputs(cfg, seed, force_repeats=False):
     from paper_2412_00061_b200 import synth
-    x, Wd, bb = synth.gen_draft(cfg, seed)
+    x, Wd, bb = synth.gen_draft(cfg, seed, force_repeats=force_repeats)
     base_tok, kv_len = synth.gen_base(cfg, seed)
     Q, K, V = synth.gen_attention(cfg, seed)
     Wl = synth.gen_lm_head(cfg, seed)
@@ -182,8 +202,8 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2412_00061_b200 import synth
-    cfg = synth.CONFIGS[args.config]
-    inp = host_inputs(cfg, 0)
+    cfg = workload_config(args)
+    inp = host_inputs(cfg, 0, args.force_repeats)
     steps = max(1, min(args.steps, 20))
     warmup = max(1, min(args.warmup, 2))
     sec = time_oracle(cfg, inp, steps, warmup, args.layout)
@@ -208,6 +228,98 @@ def workload_name(cfg):
                cfg.Hq, cfg.Hkv, cfg.D, cfg.kv_lo, cfg.kv_hi, cfg.dtype))
 
 
+def workload_config(args):
+    from paper_2412_00061_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    if args.blank_bias is not None:
+        cfg = cfg.replace(blank_bias=(float(args.blank_bias),))
+    return cfg
+
+
+def stage_times_us(step, torch, repeats=20, replays=10):
+    """Device time of each call of the step on its own: `repeats` back-to-back launches of the
+    call in a CUDA graph, replayed `replays` times (the weights exceed L2, so every launch
+    streams from HBM)."""
+    out = {}
+    side = torch.cuda.Stream(device=step.device)
+    for name, fn in (("draft_logits", step.draft), ("topk_collapse", step.collapse), ("build_tree", step.tree),
+                     ("tree_attention", step.attention), ("verify_accept", step.verify), ("whole_step", step.run)):
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(repeats):
+                    fn()
+            g.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(replays):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) * 1e3 / (repeats * replays)
+    return out
+
+
+def roofline_times_us(cfg, mean_kv, n_live, hbm_gbs, tensor_tflops):
+    """Per heavy call: the slower of (algorithmic bytes / measured copy bandwidth) and
+    (flops / measured bf16 matmul rate); the step's roofline time is their sum."""
+    draft_b, lm_b, kv_b = algorithmic_bytes(cfg, mean_kv, n_live)
+    M_lm = cfg.B * cfg.max_nodes
+    fl = {"draft_logits": 2.0 * cfg.B * cfg.T * (cfg.V + 1) * cfg.H,
+          "verify_accept": 2.0 * M_lm * cfg.V * cfg.H,
+          "tree_attention": 4.0 * cfg.B * cfg.Hq * n_live * (mean_kv + n_live) * cfg.D}
+    by = {"draft_logits": draft_b, "verify_accept": lm_b, "tree_attention": kv_b}
+    out = {k: max(by[k] / (hbm_gbs * 1e9), fl[k] / (tensor_tflops * 1e12)) * 1e6 for k in by}
+    out["whole_step"] = sum(out.values())
+    return out
+
+
+def chain_tokens_per_s(args, cfg, step, inp, seed, torch, to_device, synth):
+    """--chain n: n chained steps (five calls + history update each, the next step starting from
+    what the previous one left on the device) captured in one CUDA graph and replayed; tokens/s =
+    emitted tokens (accepted drafts + one bonus token per step and sequence) over device time."""
+    n, dev = args.chain, step.device
+    big = synth.chain_cache_config(cfg, n)
+    _, K, V = synth.gen_attention(big, seed)
+    Qtab, Ktab, Vtab = synth.gen_chain_tables(cfg, seed, n)
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    K0, V0 = to_device(K, cfg.dtype, dev), to_device(V, cfg.dtype, dev)
+    step.set_inputs(K=K0.clone(), V=V0.clone())
+    act = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    hntab = torch.zeros(n, cfg.B * cfg.max_nodes, cfg.H, dtype=act, device=dev)
+    step.setup_chain(n, to_device(inp["x"], cfg.dtype, dev), i32(inp["base_tok"]), i32(inp["kv_len"]),
+                     to_device(Qtab, cfg.dtype, dev), to_device(Ktab, cfg.dtype, dev), to_device(Vtab, cfg.dtype, dev),
+                     hntab, record=True)
+    step.plant_chain_hidden(seed, inp["Wl"])
+    side = torch.cuda.Stream(device=dev)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step.run_chain()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            step.run_chain()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    reps = max(1, min(50, args.steps // n))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    step.check_status()
+    acc = step.chain["rec"]["acc_len"].cpu().numpy()            # [n, B]
+    tokens = int(acc.sum()) + n * cfg.B
+    sec = e0.elapsed_time(e1) * 1e-3 / reps
+    return {"steps": n, "replays": reps, "tokens_per_s": tokens / sec, "tokens_per_step": tokens / (n * cfg.B),
+            "us_per_step": sec * 1e6 / n, "includes": "torch scatter standing in for the base model's K/V write of the tree rows"}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -227,9 +339,9 @@ def run_ours(args):
     build.build()
     binding.load_library()
 
-    cfg = synth.CONFIGS[args.config]
+    cfg = workload_config(args)
     seed = replicas.rank_seed(0, rank)             # every rank drafts for its own sequences
-    inp = host_inputs(cfg, seed)
+    inp = host_inputs(cfg, seed, args.force_repeats)
     step = DraftVerifyStep(cfg, device=str(dev), layout=args.layout)
     i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
     step.set_inputs(x=to_device(inp["x"], cfg.dtype, dev), Wd=to_device(inp["Wd"], cfg.dtype, dev),
@@ -246,6 +358,9 @@ def run_ours(args):
     hn, _ = synth.gen_node_hidden(cfg, seed, inp["Wl"], node_tok, parent, n_nodes)
     inp["hn"] = hn
     step.set_inputs(hn=to_device(hn, cfg.dtype, dev))
+    # how much the inputs exercise the CTC transform: distinct candidates out of k^T slot paths
+    n_cand = step.host("n_cand")
+    cand_len = step.host("cand_len") if args.layout == "packed" else None
 
     def barrier():
         if world > 1:
@@ -267,8 +382,8 @@ def run_ours(args):
     t_beg, t_end = ev(), ev()
     use_graph = not args.no_graph
     S = 1
-    if use_graph:
-        S = max(d for d in range(1, 21) if K % d == 0)
+    if use_graph:                 # at least two replays per timed region when K allows it
+        S = max(d for d in range(1, 21) if K % d == 0 and (d <= K // 2 or K < 2))
     d_beg = [torch.cuda.Event(enable_timing=True, external=use_graph) for _ in range(S if use_graph else K)]
     d_end = [torch.cuda.Event(enable_timing=True, external=use_graph) for _ in range(S if use_graph else K)]
 
@@ -304,9 +419,19 @@ def run_ours(args):
         for _ in range(2):
             graph.replay()
             graph_plain.replay()
+    # Settling run: untimed replays for about half a second with the clock sampler's window open,
+    # so that the record around a timed region of a few milliseconds is never empty and shows the
+    # clocks the GPU runs this very load at.  The timed region follows without a pause.
     barrier()
     if sampler:
         sampler.begin()
+    if use_graph:
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < 0.5:
+            for _ in range(10):
+                graph_plain.replay()
+            torch.cuda.synchronize()
+    barrier()
     t_beg.record()
     if use_graph:
         for _ in range(K // S - 1):
@@ -316,8 +441,6 @@ def run_ours(args):
         timed_steps(K)
     t_end.record()
     barrier()
-    if sampler:
-        sampler.end()
     launches = launches_per_step * K
     step.check_status()
     ms = t_beg.elapsed_time(t_end)
@@ -355,8 +478,6 @@ def run_ours(args):
     for _ in range(3):
         e2e_step()
     barrier()
-    if sampler:
-        sampler.begin()
     e_beg, e_end = ev(), ev()
     e_beg.record()
     for _ in range(K):
@@ -379,24 +500,45 @@ def run_ours(args):
         achieved = draft_b / (draft_ms * 1e-3) / 1e9
         step_bytes = draft_b + lm_b + kv_b
         value = world * K / (ms * 1e-3)
+        paths = cfg.k ** cfg.T
+        config = {"workload": workload_name(cfg), "layout": args.layout, "l2": "inputs larger than L2 (weights %.0f MB)" % (
+            (draft_b + lm_b) / 1e6), "parallelism": "replicas x%d" % world,
+            "launch": ("CUDA graph of %d steps, replayed %d times; the last replay carries an event pair around "
+                       "each draft-head launch" % (S, K // S)) if use_graph
+            else "direct launches",
+            "tree_nodes": n_live, "step_bytes": step_bytes,
+            "step_hbm_frac_of_%s_peak" % peak_kind: step_bytes / (ms / K * 1e-3) / 1e9 / peak,
+            "inputs": {"force_repeats": bool(args.force_repeats), "blank_bias": [float(v) for v in cfg.blank_bias],
+                       "slot_paths": paths, "candidates_kept": [int(v) for v in n_cand[:8]]}}
+        if cand_len is not None:
+            config["inputs"]["kept_candidates_shorter_than_T"] = int((cand_len[cand_len > 0] < cfg.T).sum())
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": workload_name(cfg), "layout": args.layout, "l2": "inputs larger than L2 (weights %.0f MB)" % (
-                (draft_b + lm_b) / 1e6), "parallelism": "replicas x%d" % world,
-                "launch": ("CUDA graph of %d steps, replayed; the last replay carries an event pair around "
-                           "each draft-head launch" % S) if use_graph else "direct launches",
-                "tree_nodes": n_live, "step_bytes": step_bytes,
-                "step_hbm_frac_of_%s_peak" % peak_kind: step_bytes / (ms / K * 1e-3) / 1e9 / peak},
+            "config": config,
             "clocks": clocks,
             "e2e": {"value": world * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": launches,
             "roofline": {"kernel": "gemv_stream_kernel (draft head)", "bound": "hbm", "achieved": achieved,
                          "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
+                         "traffic": ncu_traffic(cfg.name, "gemv_stream_kernel")},
         }
+        if args.stage_times:
+            st = stage_times_us(step, torch)
+            tens = 1400.0
+            try:
+                with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                    tens = float(json.load(f)["bf16_tflops_sustained"])
+            except (OSError, ValueError, KeyError):
+                pass
+            rf = roofline_times_us(cfg, mean_kv, n_live, peak, tens)
+            line["stages_us"] = {k: round(v, 2) for k, v in st.items()}
+            line["stages_roofline_us"] = {k: round(v, 2) for k, v in rf.items()}
+            line["stages_frac"] = {k: round(rf[k] / st[k], 3) for k in rf}
+        if args.chain > 0 and world == 1:
+            line["chain"] = chain_tokens_per_s(args, cfg, step, inp, seed, torch, to_device, synth)
         if world == 1 and not args.no_cpu_baseline:
             n_or = 10
             sec = time_oracle(cfg, inp, n_or, 1, args.layout)
@@ -405,6 +547,18 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def spawn_ranks(args) -> int:
+    """`--gpus N` without a launcher: start N ranks of this script, one per GPU, the way
+    `python -m torch.distributed.run` would be asked to (rendezvous on 127.0.0.1)."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -418,7 +572,14 @@ def main():
                     help="packed: collapse, then tree (headline); raw: the paper's raw-path tree with masked removed symbols")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every call directly instead of replaying a CUDA graph")
+    ap.add_argument("--force-repeats", action="store_true",
+                    help="draft weights that make neighbouring slots favour the same tokens, so that repeats and merges occur")
+    ap.add_argument("--blank-bias", type=float, default=None, help="blank-logit bias for every sequence (default: the workload's)")
+    ap.add_argument("--stage-times", action="store_true", help="add per-call device times and their roofline times to the line")
+    ap.add_argument("--chain", type=int, default=0, help="also time N chained steps (history update after each); adds tokens/s")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     if args.impl == "reference":
         run_reference(args)
     else:

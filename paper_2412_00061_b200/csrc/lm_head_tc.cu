@@ -20,6 +20,7 @@
 #include "run_state.cuh"
 
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 namespace ctcsd {
@@ -61,6 +62,12 @@ struct TcParams {
     DraftPartial* part;       // [n_tiles][kColSplit][m_tiles*128] per-tile, per-column-share states
     const int* row_seq;       // [M] or null
     const float* blank_bias;  // [B] or null; added to class V-1 of every slot
+    // L2 look-ahead of the weight stream: the K blocks of a tile are asked for in groups of
+    // pf_group (pf_group * 128 contiguous bytes of every weight row in one request), pf_ahead groups
+    // before the tile loads reach them; 0 turns it off
+    const unsigned char* W;   // the weights as plain memory: row r of slot t starts at ((t * V) + r) * row_bytes
+    long long row_bytes;
+    int pf_group, pf_ahead;
 };
 
 struct __align__(8) TcShared {
@@ -154,14 +161,57 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         pre = total_it < p.stages ? total_it : p.stages;
         for (int it = 0; it < pre; ++it) load_stage(it, true, false);
     }
+    // L2 look-ahead (all lanes of warp 0).  A tile load asks DRAM for 128 bytes of every weight row,
+    // rows that lie a whole row pitch apart; the neighbouring 128 bytes of the same rows follow a
+    // stage later.  Here the next pf_group K blocks of every row of the tile are requested as ONE
+    // contiguous piece per row, so that DRAM serves a whole open page at a time; the tile loads
+    // that follow find their data in L2 (or in flight).
+    int pf_next = 0;                                   // first iteration whose group is not yet requested
+    auto prefetch_upto = [&](int it_limit) {
+        if (p.pf_group <= 0) return;
+        if (it_limit > total_it) it_limit = total_it;
+        while (pf_next < it_limit) {
+            const int un = pf_next / p.num_k, kb = pf_next - un * p.num_k;
+            const int u = u_first + un * u_step;
+            const int nt = u / p.m_units;
+            int cnt = p.pf_group - kb % p.pf_group;                    // to the end of this group
+            if (kb + cnt > p.num_k) cnt = p.num_k - kb;
+            int kq = kb + k_start;
+            if (kq >= p.num_k) kq -= p.num_k;
+            if (kq + cnt > p.num_k) cnt = p.num_k - kq;                // the rotated K axis wraps here
+            long long row0;
+            int rows;
+            if constexpr (MODE == 0) {
+                row0 = (long long)nt * p.Nt;
+                rows = p.V - (int)row0 < p.Nt ? p.V - (int)row0 : p.Nt;
+            } else {
+                const int t = nt / p.tiles_per_slot, ntl = nt - t * p.tiles_per_slot;
+                rows = p.V - ntl * p.Nt < p.Nt ? p.V - ntl * p.Nt : p.Nt;
+                row0 = (long long)t * p.V + (long long)ntl * p.Nt;
+            }
+            long long off = (long long)kq * 128;
+            long long len = (long long)cnt * 128;
+            if (off + len > p.row_bytes) len = p.row_bytes - off;       // the last K block may be partial
+            len &= ~15ll;
+            if (len > 0)
+                for (int r = lane; r < rows; r += 32)
+                    tc::bulk_prefetch_l2(p.W + (row0 + r) * p.row_bytes + off, (uint32_t)len);
+            pf_next += cnt;
+        }
+    };
+    if (warp == 0) {
+        pre = __shfl_sync(0xffffffffu, pre, 0);
+        prefetch_upto(pre + p.pf_group * p.pf_ahead);
+    }
     // barriers and tensor memory are set up; the activations may come from the preceding kernel
     pdl_wait();
     pdl_trigger();
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
-        if (lane == 0) {
-            for (int it = 0; it < pre; ++it) load_stage(it, false, true);
+        // ---------------- TMA producer (lane 0; the other lanes help with the L2 look-ahead) ----------------
+        {
+            if (lane == 0)
+                for (int it = 0; it < pre; ++it) load_stage(it, false, true);
             int it = pre;
             bool ok = true;
             // Stages are refilled two at a time: the two weight boxes then ask for adjacent 128-byte
@@ -170,17 +220,23 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int group = p.stages >= 4 ? 2 : 1;
             while (it < total_it && ok) {
                 const int cnt = total_it - it < group ? total_it - it : group;
-                for (int j = 0; j < cnt; ++j) {
-                    const int s = (it + j) % p.stages;
-                    const uint32_t ph = (uint32_t)((it + j) / p.stages) & 1u;
-                    if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                if (lane == 0) {
+                    for (int j = 0; j < cnt; ++j) {
+                        const int s = (it + j) % p.stages;
+                        const uint32_t ph = (uint32_t)((it + j) / p.stages) & 1u;
+                        if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                    }
+                    if (ok) {
+                        for (int j = 0; j < cnt; ++j) load_stage(it + j, true, false);
+                        for (int j = 0; j < cnt; ++j) load_stage(it + j, false, true);
+                    }
                 }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                for (int j = 0; j < cnt; ++j) load_stage(it + j, true, false);
-                for (int j = 0; j < cnt; ++j) load_stage(it + j, false, true);
                 it += cnt;
+                prefetch_upto(it + p.pf_group * p.pf_ahead);
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 1);
                 *abort_flag = 1;
                 // let copies that are still in flight land before the CTA gives its memory back
@@ -473,6 +529,10 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     if (stages < 2) return CTCSD_ERR_UNSUPPORTED;
     p.stages = stages;
     p.part = reinterpret_cast<DraftPartial*>(h->ws + h->lay.tc_part_off);
+    p.W = static_cast<const unsigned char*>(Wd);
+    p.row_bytes = (long long)c.H * 2;
+    p.pf_group = getenv("CTCSD_PF_GROUP") ? atoi(getenv("CTCSD_PF_GROUP")) : 0;
+    p.pf_ahead = getenv("CTCSD_PF_AHEAD") ? atoi(getenv("CTCSD_PF_AHEAD")) : 1;
     p.row_seq = row_seq;
     p.blank_bias = blank_bias;
     p.logits_dbg = out_logits_dbg;
@@ -543,6 +603,10 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     p.out_argmax = out_argmax;
     p.logits_dbg = out_logits_dbg;
     p.status = status_ptr(h);
+    p.W = static_cast<const unsigned char*>(Wl);
+    p.row_bytes = (long long)c.H * 2;
+    p.pf_group = getenv("CTCSD_PF_GROUP") ? atoi(getenv("CTCSD_PF_GROUP")) : 0;
+    p.pf_ahead = getenv("CTCSD_PF_AHEAD") ? atoi(getenv("CTCSD_PF_AHEAD")) : 1;
 
     CUtensorMap tmA, tmW;
     if (!make_map(&tmA, hn, M, c.H, p.a_bytes / 128)) return CTCSD_ERR_CUDA;
