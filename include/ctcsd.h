@@ -230,6 +230,29 @@ int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const voi
                         int* out_next_tok, float* out_logits_dbg);
 
 /*
+ * Sampling acceptance (Sec. 2, second paragraph: a drafted token is accepted with probability
+ * min(1, p/p') - the ratio is printed upside down there - and after a rejection a token is drawn
+ * from norm(max(0, P - P')); Sec. 6 names sampling as the next step).  The tree's tokens are a
+ * deterministic function of the draft head's output, so the proposal P' of a child that is tried
+ * is the point mass on its token: it is accepted with probability P(child), and the rejected
+ * token is removed from P.  Trying a node's children in turn under this rule amounts to one draw
+ * from P that is accepted iff it is a child's token, which is what is computed:
+ *   x[b,i] = argmax_v fma( y[b,i,v], 1/temperature, noise[b, depth[b,i], v] ),  ties to the lower id,
+ * a draw from softmax(y/temperature) when `noise` holds independent standard Gumbel variates
+ * (-log(-log(U))); then the walk of ctcsd_verify_accept with x in place of the arg-max.  Nodes of
+ * equal depth lie on different paths and share a noise row; nodes along a path use different rows.
+ * temperature -> 0 approaches greedy acceptance.  The fused multiply-add is rounded once, to float32.
+ * depth [B,max_nodes] int32 as produced by ctcsd_build_tree;  noise [B,T+1,V] float32;
+ * temperature > 0;  out_token [B,max_nodes] int32 = x;  out_next_tok = x at the last accepted node;
+ * everything else as for ctcsd_verify_accept (out_logits_dbg receives the logits y, without noise).
+ */
+int ctcsd_verify_accept_sampled(ctcsd_handle* h, void* stream, const void* hn, const void* Wl,
+                                const int* node_tok, const int* parent, const int* depth, const int* n_nodes,
+                                const float* noise, float temperature,
+                                int* out_token, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
+                                int* out_next_tok, float* out_logits_dbg);
+
+/*
  * History update after acceptance (Sec. 3.3, last paragraph: the step's output joins the decoding
  * history): the accepted path becomes part of the cached prefix, so that the next step can
  * start without host work.  For sequence b with L = kv_len[b]: the root's key/value row (cache

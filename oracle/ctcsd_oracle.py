@@ -550,3 +550,124 @@ def decode_chain(n_steps: int, x0: np.ndarray, base_tok0: np.ndarray, kv_len0: n
         x = hn[sel_row]                       # the next step drafts from the last accepted node's hidden state
         base_tok = next_tok.copy()            # and its root is this step's bonus token
     return records, K, Vc, kv_len
+
+
+# --------------------------------------------------------------------------------------
+# Sampling acceptance (Sec. 2, second paragraph: a drafted token is accepted with probability
+# min(1, p/p') - the paper typesets the ratio upside down - and on rejection a token is drawn
+# from norm(max(0, P - P')); Sec. 6 names sampling as future work).
+#
+# Reading.  The tree's tokens are a deterministic function of the draft head's output (the k
+# best symbols per place, the N best candidates), so the proposal P' for a child that is tried
+# is the point mass on that child's token: p' = 1, the child is accepted with probability
+# P(child), and after a rejection P - P' clipped at zero and renormalised is P without that
+# token.  Trying the children of a node one after the other under this rule emits child c
+# with probability P(c) and any other token x with probability P(x): exactly one draw from
+# P, accepted iff it is a child.  That is what is computed here, with the draw made by the
+# Gumbel-max rule so that it is a deterministic function of noise the caller passes in:
+#     x[b,i] = argmax_v ( y[b,i,v] / temperature + noise[b, depth(i), v] ),   noise ~ Gumbel(0,1)
+# (nodes of equal depth lie on different paths, at most one of them is reached, so they may
+# share their noise; nodes along one path use independent noise).  The acceptance walk is
+# the greedy one with x in place of the arg-max.  temperature -> 0 gives greedy acceptance.
+# --------------------------------------------------------------------------------------
+def sample_tokens(y: np.ndarray, depth: np.ndarray, n_nodes: np.ndarray, noise: np.ndarray,
+                  inv_temperature: float, fp32: bool = False) -> np.ndarray:
+    """y [B,n_max,V] logits, depth [B,n_max], noise [B,T+1,V] -> x [B,n_max] int64 (dead nodes 0).
+    fp32=True forms y * inv_temperature + noise as one fused multiply-add rounded to float32
+    (the precision in which the CUDA path takes this decision), else in float64."""
+    B, n_max, V = y.shape
+    x = np.zeros((B, n_max), dtype=np.int64)
+    it = np.float64(np.float32(inv_temperature)) if fp32 else np.float64(inv_temperature)
+    for b in range(B):
+        for i in range(int(n_nodes[b])):
+            z = np.asarray(y[b, i], dtype=np.float64) * it + np.asarray(noise[b, int(depth[b, i])], dtype=np.float64)
+            if fp32:
+                z = z.astype(np.float32)
+            x[b, i] = int(np.argmax(z))              # first maximum: lowest id on ties
+    return x
+
+
+def sample_accept(node_tok: np.ndarray, parent: np.ndarray, n_nodes: np.ndarray, depth: np.ndarray,
+                  y: np.ndarray, noise: np.ndarray, inv_temperature: float, T: int, fp32: bool = False):
+    """Returns (x, acc_len, acc_nodes, acc_tok, next_tok): the base model's sampled token after
+    every node and the accepted path (next_tok is the sampled token at the last accepted node)."""
+    x = sample_tokens(y, depth, n_nodes, noise, inv_temperature, fp32)
+    return (x,) + tuple(greedy_accept(node_tok, parent, n_nodes, x, T))
+
+
+# --------------------------------------------------------------------------------------
+# The paper's Attention Draft Module (Sec. 3.1: one transformer layer, built like the base
+# model's layers, on the base model's hidden states; Sec. 3.2: F_hat = DraftModule(F), then the
+# projection to one distribution per place).  The paper gives no further detail.  Reading taken:
+# a LLaMA-style decoder layer with the base model's head shape (pre-norm residual blocks: RMSNorm,
+# rotary self-attention over the hidden states of all positions so far, RMSNorm, SwiGLU MLP), no
+# final norm; the layer's output at the newest position is the state that draft_logits projects
+# to the T places.  Keys and values of earlier positions are cached, as in the base model.
+# --------------------------------------------------------------------------------------
+def rms_norm(x: np.ndarray, gamma: np.ndarray, eps: float) -> np.ndarray:
+    """y = x / sqrt(mean(x^2) + eps) * gamma over the last axis."""
+    x = np.asarray(x, dtype=np.float64)
+    return x / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps) * np.asarray(gamma, dtype=np.float64)
+
+
+def rope_rotate(v: np.ndarray, pos: int, theta: float) -> np.ndarray:
+    """Rotary position embedding of one head vector v [D] at position pos, half-split pairing
+    (element i is paired with i + D/2, frequency theta^(-2i/D)), the LLaMA convention."""
+    v = np.asarray(v, dtype=np.float64)
+    D = v.shape[-1]
+    half = D // 2
+    out = np.empty_like(v)
+    for i in range(half):
+        ang = pos * theta ** (-2.0 * i / D)
+        c, s = math.cos(ang), math.sin(ang)
+        out[i] = v[i] * c - v[i + half] * s
+        out[i + half] = v[i + half] * c + v[i] * s
+    return out
+
+
+def draft_module(F_new: np.ndarray, n_new: np.ndarray, kv_len: np.ndarray, Kd: np.ndarray, Vd: np.ndarray,
+                 w: dict, Hq: int, Hkv: int, D: int, eps: float = 1e-5, theta: float = 10000.0):
+    """One step of the draft layer.  F_new [B,R,H]: the base model's hidden states of the newest
+    n_new[b] <= R positions of each sequence (positions kv_len[b] .. kv_len[b]+n_new[b]-1; the
+    layer's cache Kd, Vd [B,Hkv,Lcap,D] already holds positions < kv_len[b]).  w: g1 [H], Wqkv
+    [(Hq+2Hkv)D, H] (query rows first, then key rows, then value rows), Wo [H, Hq*D], g2 [H],
+    Wgu [2I, H] (gate rows, then up rows), Wdn [H, I].
+    Returns (F_hat [B,H]: the layer's output at each sequence's newest position, Kd', Vd' with the
+    new positions' keys/values appended, kv_len' = kv_len + n_new)."""
+    F_new = np.asarray(F_new, dtype=np.float64)
+    B, R, H = F_new.shape
+    Kd, Vd = np.array(Kd, dtype=np.float64, copy=True), np.array(Vd, dtype=np.float64, copy=True)
+    Wqkv, Wo = np.asarray(w["Wqkv"], dtype=np.float64), np.asarray(w["Wo"], dtype=np.float64)
+    Wgu, Wdn = np.asarray(w["Wgu"], dtype=np.float64), np.asarray(w["Wdn"], dtype=np.float64)
+    I = Wdn.shape[1]
+    grp = Hq // Hkv
+    F_hat = np.zeros((B, H), dtype=np.float64)
+    new_len = np.zeros((B,), dtype=np.int64)
+    for b in range(B):
+        L, r = int(kv_len[b]), int(n_new[b])
+        q_last = None
+        for j in range(r):
+            a = rms_norm(F_new[b, j], w["g1"], eps)
+            qkv = Wqkv @ a
+            q = qkv[:Hq * D].reshape(Hq, D)
+            k = qkv[Hq * D:(Hq + Hkv) * D].reshape(Hkv, D)
+            v = qkv[(Hq + Hkv) * D:].reshape(Hkv, D)
+            for g in range(Hkv):
+                Kd[b, g, L + j] = rope_rotate(k[g], L + j, theta)
+                Vd[b, g, L + j] = v[g]
+            q_last = np.stack([rope_rotate(q[h], L + j, theta) for h in range(Hq)])
+        n_keys = L + r
+        attn = np.zeros((Hq, D))
+        for h in range(Hq):                          # the newest position attends to every position so far
+            s = (Kd[b, h // grp, :n_keys] @ q_last[h]) / math.sqrt(D)
+            p = np.exp(s - s.max())
+            p /= p.sum()
+            attn[h] = p @ Vd[b, h // grp, :n_keys]
+        h1 = F_new[b, r - 1] + Wo @ attn.reshape(-1)
+        m = rms_norm(h1, w["g2"], eps)
+        gu = Wgu @ m
+        gate, up = gu[:I], gu[I:]
+        act = gate / (1.0 + np.exp(-gate)) * up       # SiLU(gate) * up
+        F_hat[b] = h1 + Wdn @ act
+        new_len[b] = n_keys
+    return F_hat, Kd, Vd, new_len

@@ -24,6 +24,7 @@ EXPORTS = [
     "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
     "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static", "ctcsd_draft_logits_rows",
+    "ctcsd_verify_accept_sampled",
     "ctcsd_select_raw_paths", "ctcsd_build_raw_tree", "ctcsd_verify_accept_raw",
 ]
 
@@ -68,6 +69,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_build_tree.argtypes = [vp, vp] + [vp] * 12
     lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
     lib.ctcsd_verify_accept.argtypes = [vp, vp] + [vp] * 11
+    lib.ctcsd_verify_accept_sampled.argtypes = [vp, vp] + [vp] * 7 + [ctypes.c_float] + [vp] * 6
     lib.ctcsd_commit_accepted.argtypes = [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp]
     lib.ctcsd_select_raw_paths.argtypes = [vp, vp, ci] + [vp] * 6
     lib.ctcsd_build_raw_tree.argtypes = [vp, vp] + [vp] * 13
@@ -251,6 +253,24 @@ class Handle:
             _ptr(out_next_tok, i32, c.B, "out_next_tok"),
             _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
         self._check(rc, "verify_accept")
+
+    def verify_accept_sampled(self, hn, Wl, node_tok, parent, depth, n_nodes, noise, temperature, out_token,
+                              out_acc_len, out_acc_nodes, out_acc_tok, out_next_tok, out_logits_dbg=None, stream=None):
+        """Sampling acceptance: noise [B,T+1,V] float32 standard Gumbel variates, temperature > 0."""
+        c = self.cfg
+        i32 = torch.int32
+        nn = c.B * c.max_nodes
+        rc = self.lib.ctcsd_verify_accept_sampled(
+            self._h, _stream_ptr(stream),
+            _ptr(hn, self.act_dtype, nn * c.H, "hn"), _ptr(Wl, self.act_dtype, c.V * c.H, "Wl"),
+            _ptr(node_tok, i32, nn, "node_tok"), _ptr(parent, i32, nn, "parent"), _ptr(depth, i32, nn, "depth"),
+            _ptr(n_nodes, i32, c.B, "n_nodes"), _ptr(noise, torch.float32, c.B * (c.T + 1) * c.V, "noise"),
+            float(temperature),
+            _ptr(out_token, i32, nn, "out_token"), _ptr(out_acc_len, i32, c.B, "out_acc_len"),
+            _ptr(out_acc_nodes, i32, c.B * c.T, "out_acc_nodes"), _ptr(out_acc_tok, i32, c.B * c.T, "out_acc_tok"),
+            _ptr(out_next_tok, i32, c.B, "out_next_tok"),
+            _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
+        self._check(rc, "verify_accept_sampled")
 
     # ---- the paper's raw-tree layout (Sec. 3.3) ----
     def select_raw_paths(self, topk_id, topk_lp, sel_row, out_raw_tok, out_raw_score, out_n_raw, stream=None):

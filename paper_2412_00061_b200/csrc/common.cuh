@@ -56,6 +56,16 @@ struct Handle {
     size_t l2_hint_bytes;
 };
 
+// Sampling acceptance: the token drawn after tree node i of sequence b is
+// argmax_v fma(y[v], inv_temp, noise[(b * rows_per_seq + depth[b,i]) * V + v]).  noise == null: plain arg-max.
+struct SampleNoise {
+    const float* noise;      // [B][rows_per_seq][V] standard Gumbel noise, or null
+    const int* depth;        // [B*max_nodes] tree depth of every node
+    int max_nodes;
+    int rows_per_seq;        // T + 1
+    float inv_temp;
+};
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 Layout make_layout(const ctcsd_config& cfg, int num_sms);

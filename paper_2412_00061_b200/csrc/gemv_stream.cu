@@ -227,6 +227,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                 const int row = p.m0 + own_m;
                 bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
             }
+            // sampling acceptance (LM head only): this thread's activation row is a tree node, whose
+            // depth picks the noise row
+            const float* noise_row = nullptr;
+            if (owner && p.sn.noise != nullptr) {
+                const int row = p.m0 + own_m;
+                int d = p.sn.depth[row];
+                d = d < 0 ? 0 : (d >= p.sn.rows_per_seq ? p.sn.rows_per_seq - 1 : d);
+                noise_row = p.sn.noise + ((size_t)(row / p.sn.max_nodes) * p.sn.rows_per_seq + d) * (size_t)rps;
+            }
             auto push_logit = [&](float z, int i) {          // i: row of the CTA's range
                 const int seg = i >= n_seg0 ? 1 : 0;
                 if (seg != cur_seg) {                         // this thread's rows now belong to the next slot
@@ -238,6 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                 const int v = (int)(r0 + i - (long long)slot * rps);
                 if (v == (int)rps - 1) z += bias;
                 if (p.logits_dbg) p.logits_dbg[((size_t)(p.m0 + own_m) * p.slots + slot) * rps + v] = z;
+                if (noise_row != nullptr) z = __fmaf_rn(z, p.sn.inv_temp, noise_row[v]);
                 st.push(z, v);
             };
 

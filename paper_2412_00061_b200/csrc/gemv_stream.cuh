@@ -36,6 +36,7 @@ struct GemvParams {
     int* out_argmax;          // mode 1: [M]
     float* logits_dbg;        // null or [M,slots,rows_per_slot]
     int* status;              // device status word
+    SampleNoise sn;           // mode 1: noise added to the scaled logit before the arg-max (null: none)
     const void* pf_ptr;       // optional: range the CTAs ask L2 to fetch once their own stream is issued
     unsigned long long pf_bytes;
 };

@@ -65,6 +65,7 @@ struct TcParams {
     // L2 look-ahead of the weight stream: the K blocks of a tile are asked for in groups of
     // pf_group (pf_group * 128 contiguous bytes of every weight row in one request), pf_ahead groups
     // before the tile loads reach them; 0 turns it off
+    SampleNoise sn;           // LM head: noise added to the scaled logit before the arg-max (null: none)
     const unsigned char* W;   // the weights as plain memory: row r of slot t starts at ((t * V) + r) * row_bytes
     long long row_bytes;
     int pf_group, pf_ahead;
@@ -312,6 +313,12 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const uint32_t lane_addr = lane_base + (uint32_t)((p.pair ? h : acc) * kAccCols);
             float best = -INFINITY;
             int best_idx = 0x7fffffff;
+            const float* noise_row = nullptr;                 // sampling acceptance: the row's Gumbel noise
+            if (MODE == 0 && p.sn.noise != nullptr && row < p.M) {
+                int d = p.sn.depth[row];
+                d = d < 0 ? 0 : (d >= p.sn.rows_per_seq ? p.sn.rows_per_seq - 1 : d);
+                noise_row = p.sn.noise + ((size_t)(row / p.sn.max_nodes) * p.sn.rows_per_seq + d) * (size_t)p.V;
+            }
             RunState st;
             if constexpr (MODE == 1) st.init();
             // a warp whose 32 rows lie past the last activation row has nothing to read
@@ -333,8 +340,9 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const int col = n0 + c0 + j;
                     if (col < p.V && c0 + j < p.Nt) {
                         if constexpr (MODE == 0) {
-                            if (v > best) { best = v; best_idx = col; }
                             if (p.logits_dbg != nullptr && row < p.M) p.logits_dbg[(size_t)row * p.V + col] = v;
+                            if (noise_row != nullptr) v = __fmaf_rn(v, p.sn.inv_temp, __ldg(noise_row + col));
+                            if (v > best) { best = v; best_idx = col; }
                         } else {
                             if (col == p.V - 1) v += bias;
                             if (p.logits_dbg != nullptr && row < p.M)
@@ -564,7 +572,7 @@ bool lm_head_tc_supported(const Handle* h) {
 }
 
 int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, const void* Wl,
-                      int* out_argmax, float* out_logits_dbg, const AcceptParams& acc) {
+                      int* out_argmax, float* out_logits_dbg, const AcceptParams& acc, const SampleNoise& sn) {
     const ctcsd_config& c = h->cfg;
     if (!lm_head_tc_supported(h)) return CTCSD_ERR_UNSUPPORTED;
 
@@ -599,6 +607,7 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     p.stages = stages;
     p.keys = reinterpret_cast<unsigned long long*>(h->ws + h->lay.lm_key_off);
     p.acc = acc;
+    p.sn = sn;
     p.counter = counter_ptr(h) + 1;
     p.out_argmax = out_argmax;
     p.logits_dbg = out_logits_dbg;

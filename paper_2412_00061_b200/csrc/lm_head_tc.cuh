@@ -13,7 +13,7 @@ bool lm_head_tc_supported(const Handle* h);
 // epilogue; the CTA that finishes last decodes the arg-max and runs the greedy acceptance walk
 // `acc` over it.  Returns CTCSD_ERR_UNSUPPORTED when the shape is not covered.
 int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, const void* Wl,
-                      int* out_argmax, float* out_logits_dbg, const AcceptParams& acc);
+                      int* out_argmax, float* out_logits_dbg, const AcceptParams& acc, const SampleNoise& sn);
 
 // Draft head on the tensor cores for more than 8 activation rows: the same weight-stream kernel
 // with a per-row online (max, sum of exp, best-8) epilogue per vocabulary tile and a merge

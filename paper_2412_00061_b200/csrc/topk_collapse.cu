@@ -8,8 +8,10 @@
 // alignments is accumulated in 64-bit fixed point relative to the candidate's best
 // alignment, which makes it independent of the order in which threads arrive.
 #include "common.cuh"
+#include "tc_primitives.cuh"
 
 #include <math.h>
+#include <stdlib.h>
 
 namespace ctcsd {
 namespace {
@@ -33,7 +35,31 @@ struct CollapseParams {
     float* out_cand_score;   // [B,topN]
     int* out_n_cand;         // [B]
     int* status;
+    // CTAs beyond the first `nseq` do no collapsing: they ask the L2 cache for [pf_ptr, pf_ptr +
+    // pf_bytes), data that a later kernel of the step streams (see ctcsd_set_l2_prefetch)
+    int nseq;
+    const unsigned char* pf_ptr;
+    unsigned long long pf_bytes;
 };
+
+// The candidate kernels keep one SM per sequence busy for ten to forty microseconds while HBM has
+// nothing to do.  CTAs past the sequences use that time: each asks L2 for its share of a range of
+// constant data (the head of the LM-head weights) in 64 KB pieces and leaves.  They read nothing
+// that a predecessor writes, so they do not wait for it: under programmatic dependent launch they
+// start as soon as an SM has room, i.e. while the slowest CTAs of the draft head are still streaming.
+__device__ __forceinline__ void l2_prefetch_role(const CollapseParams& p) {
+    pdl_trigger();
+    if (threadIdx.x >= 32 || p.pf_bytes == 0) return;
+    const unsigned long long chunk = 64 * 1024;
+    const unsigned long long nchunks = (p.pf_bytes + chunk - 1) / chunk;
+    const unsigned long long me = blockIdx.x - (unsigned)p.nseq, n = gridDim.x - (unsigned)p.nseq;
+    for (unsigned long long c = me + n * threadIdx.x; c < nchunks; c += n * 32) {
+        unsigned long long len = p.pf_bytes - c * chunk;
+        if (len > chunk) len = chunk;
+        len &= ~15ull;
+        if (len) tc::bulk_prefetch_l2(p.pf_ptr + c * chunk, (uint32_t)len);
+    }
+}
 
 __device__ __forceinline__ int key_len(unsigned long long key) { return (int)(key >> 48); }
 __device__ __forceinline__ int key_tok(unsigned long long key, int i) { return (int)((key >> (6 * (7 - i))) & 63ull); }
@@ -379,6 +405,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     __shared__ int s_count, s_has_empty;
 
     const int b = blockIdx.x, tid = threadIdx.x;
+    if (b >= p.nseq) { l2_prefetch_role(p); return; }
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -467,6 +494,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
     const int b = blockIdx.x, tid = threadIdx.x;
+    if (b >= p.nseq) { l2_prefetch_role(p); return; }
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -570,6 +598,7 @@ __global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
     const int b = blockIdx.x, tid = threadIdx.x;
+    if (b >= p.nseq) { l2_prefetch_role(p); return; }
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -608,6 +637,16 @@ __global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
 
 using namespace ctcsd;
 
+// CTAs that the candidate kernels launch on top of one per sequence to carry the L2 hint.
+static int prefetch_ctas(const Handle* h, CollapseParams& p) {
+    p.nseq = h->cfg.B;
+    p.pf_ptr = static_cast<const unsigned char*>(h->l2_hint_ptr);
+    p.pf_bytes = h->l2_hint_bytes;
+    if (getenv("CTCSD_PF_WHERE") && getenv("CTCSD_PF_WHERE")[0] == 'd') p.pf_bytes = 0;
+    if (p.pf_bytes == 0) return 0;
+    return h->num_sms;
+}
+
 static int next_pow2_host(int v) {
     int n = 2;
     while (n < v) n <<= 1;
@@ -641,7 +680,8 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     if (c.beam > 0) {
         const size_t smem = (size_t)kBeamCap * 52;
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_beam_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
+        const int extra = prefetch_ctas(h, p);
+        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B + extra), dim3(kThreads), smem, s, 1, p));
         CTCSD_LAUNCH_CHECK(h);
         return CTCSD_OK;
     }
@@ -654,7 +694,8 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     size_t smem = (size_t)cap * 24 + (size_t)npaths * 2;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_enum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
+    const int extra = prefetch_ctas(h, p);
+    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B + extra), dim3(kThreads), smem, s, 1, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
@@ -686,7 +727,8 @@ extern "C" int ctcsd_select_raw_paths(ctcsd_handle* hh, void* stream, int M, con
     const size_t smem = (size_t)p.cap * 16;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(raw_paths_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B), dim3(kThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
+    const int extra = prefetch_ctas(h, p);
+    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B + extra), dim3(kThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

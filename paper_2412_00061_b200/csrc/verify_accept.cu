@@ -21,7 +21,8 @@ using namespace ctcsd;
 static int verify_accept_common(ctcsd_handle* hh, void* stream, const void* hn, const void* Wl,
                                 const int* node_tok, const int* parent, const int* kept, const int* nka,
                                 const int* n_nodes, int* out_argmax, int* out_acc_len, int* out_acc_nodes,
-                                int* out_acc_tok, int* out_next_tok, float* out_logits_dbg) {
+                                int* out_acc_tok, int* out_next_tok, float* out_logits_dbg,
+                                const float* noise = nullptr, const int* depth = nullptr, float inv_temp = 1.f) {
     Handle* h = &hh->h;
     const ctcsd_config& c = h->cfg;
     if ((reinterpret_cast<uintptr_t>(hn) | reinterpret_cast<uintptr_t>(Wl)) & 15) return CTCSD_ERR_INVALID_ARG;
@@ -33,10 +34,12 @@ static int verify_accept_common(ctcsd_handle* hh, void* stream, const void* hn, 
     a.B = c.B; a.T = c.T; a.max_nodes = c.max_nodes;
     a.acc_len = out_acc_len; a.acc_nodes = out_acc_nodes; a.acc_tok = out_acc_tok; a.next_tok = out_next_tok;
     a.kept = kept; a.nka = nka;
+    SampleNoise sn;
+    sn.noise = noise; sn.depth = depth; sn.max_nodes = c.max_nodes; sn.rows_per_seq = c.T + 1; sn.inv_temp = inv_temp;
 
     // tensor-core path: the acceptance walk runs in the tail of the LM-head kernel
     if (lm_head_tc_supported(h)) {
-        int rc = launch_lm_head_tc(h, s, M, hn, Wl, out_argmax, out_logits_dbg, a);
+        int rc = launch_lm_head_tc(h, s, M, hn, Wl, out_argmax, out_logits_dbg, a, sn);
         if (rc != CTCSD_ERR_UNSUPPORTED) return rc;
     }
     GemvParams g;
@@ -47,6 +50,7 @@ static int verify_accept_common(ctcsd_handle* hh, void* stream, const void* hn, 
     g.out_topk_id = nullptr; g.out_topk_lp = nullptr; g.out_lse = nullptr;
     g.out_argmax = out_argmax;
     g.logits_dbg = out_logits_dbg;
+    g.sn = sn;
     g.pf_ptr = nullptr; g.pf_bytes = 0;
     int rc = launch_gemv_stream(h, s, c.dtype, M, g);
     if (rc != CTCSD_OK) return rc;
@@ -75,4 +79,18 @@ extern "C" int ctcsd_verify_accept_raw(ctcsd_handle* hh, void* stream, const voi
         return CTCSD_ERR_INVALID_ARG;
     return verify_accept_common(hh, stream, hn, Wl, node_tok, nullptr, kept, nka, n_nodes, out_argmax,
                                 out_acc_len, out_acc_nodes, out_acc_tok, out_next_tok, out_logits_dbg);
+}
+
+extern "C" int ctcsd_verify_accept_sampled(ctcsd_handle* hh, void* stream, const void* hn, const void* Wl,
+                                           const int* node_tok, const int* parent, const int* depth, const int* n_nodes,
+                                           const float* noise, float temperature,
+                                           int* out_token, int* out_acc_len, int* out_acc_nodes, int* out_acc_tok,
+                                           int* out_next_tok, float* out_logits_dbg) {
+    if (!hh || !hn || !Wl || !node_tok || !parent || !depth || !n_nodes || !noise || !out_token || !out_acc_len ||
+        !out_acc_nodes || !out_acc_tok || !out_next_tok)
+        return CTCSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f)) return CTCSD_ERR_INVALID_ARG;
+    return verify_accept_common(hh, stream, hn, Wl, node_tok, parent, nullptr, nullptr, n_nodes, out_token,
+                                out_acc_len, out_acc_nodes, out_acc_tok, out_next_tok, out_logits_dbg,
+                                noise, depth, 1.0f / temperature);
 }

@@ -147,6 +147,14 @@ class DraftVerifyStep:
                              o["argmax"], o["acc_len"], o["acc_nodes"], o["acc_tok"], o["next_tok"],
                              o.get("lm_logits_dbg"), stream=stream)
 
+    def verify_sampled(self, noise, temperature, stream=None):
+        """Sampling acceptance in place of the greedy one (packed layout): out["argmax"] then holds
+        the sampled tokens."""
+        i, o = self.inp, self.out
+        self.h.verify_accept_sampled(i["hn"], i["Wl"], o["node_tok"], o["parent"], o["depth"], o["n_nodes"],
+                                     noise, temperature, o["argmax"], o["acc_len"], o["acc_nodes"], o["acc_tok"],
+                                     o["next_tok"], o.get("lm_logits_dbg"), stream=stream)
+
     def commit(self, stream=None):
         """History update (not part of run(): it changes the K/V cache in place)."""
         i, o = self.inp, self.out

@@ -26,7 +26,7 @@ from typing import Dict, Optional, Tuple
 import numpy as np
 
 _TAGS = {"x": 1, "Wd": 2, "bias": 3, "base": 4, "kvlen": 5, "Q": 6, "K": 7, "V": 8,
-         "Wl": 9, "hn_noise": 10, "agree": 11, "repeat": 12}
+         "Wl": 9, "hn_noise": 10, "agree": 11, "repeat": 12, "gumbel": 13}
 
 
 @dataclass(frozen=True)
@@ -222,3 +222,12 @@ def gen_chain_tables(cfg: StepConfig, seed: int, n_steps: int):
 def chain_step_seed(seed: int, step: int) -> int:
     """Seed of gen_node_hidden for step `step` of a chain."""
     return seed * 1009 + 1 + step
+
+
+def gen_gumbel_noise(cfg: StepConfig, seed: int = 0) -> np.ndarray:
+    """Standard Gumbel noise [B, T+1, V] float32 for sampling acceptance: -log(-log(U)) with U
+    uniform on the open interval (0,1).  One row per (sequence, tree depth)."""
+    g = _rng(seed, "gumbel")
+    u = g.random((cfg.B, cfg.T + 1, cfg.V), dtype=np.float64)
+    u = np.clip(u, 1e-300, 1.0 - 1e-16)
+    return (-np.log(-np.log(u))).astype(np.float32)

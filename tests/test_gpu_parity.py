@@ -217,6 +217,58 @@ def test_chained_steps_fp32_and_inside_a_cuda_graph():
     assert r["tokens"] > 4 * SMALL["c3s"].B
 
 
+@pytest.mark.parametrize("name", ["c2s", "c5s", "c1d64", "c1fp32"])
+def test_sampling_acceptance(name):
+    """ctcsd_verify_accept_sampled after a checked step: the sampled token of every node against the
+    oracle fed the kernel's own logits (same float32 fused multiply-add, so bit-exact wherever the two
+    best perturbed logits are not within rounding of each other), against the oracle from the raw
+    inputs in float64 wherever that margin is comfortable, and the acceptance walk over the sampled
+    tokens bit for bit.  Three temperatures; a tiny one must reproduce the greedy result."""
+    import torch
+    from oracle import ctcsd_oracle as orc
+    cfg = SMALL[name] if name in SMALL else C["c1"].replace(name="c1fp32", B=2, kv_lo=3, kv_hi=60)
+    r = _run(cfg, seed=5)
+    step = r["step"]
+    dev = step.device
+    greedy = {k: step.host(k).copy() for k in ("argmax", "acc_len", "acc_nodes", "acc_tok", "next_tok")}
+    node_tok, parent, depth, n_nodes = (step.host(k).astype(np.int64) for k in ("node_tok", "parent", "depth", "n_nodes"))
+    noise = synth.gen_gumbel_noise(cfg, 5)
+    noise_d = torch.from_numpy(noise).to(dev)
+    hn = step.inp["hn"].float().cpu().numpy()
+    Wl = step.inp["Wl"].float().cpu().numpy()
+    y_def, _ = orc.lm_head_argmax(hn, Wl)
+    y_def = y_def.reshape(cfg.B, cfg.max_nodes, cfg.V)
+    accepted = []
+    for temperature in (1.0, 0.05, 1e-6):
+        inv_t = float(np.float32(1.0) / np.float32(temperature))
+        step.verify_sampled(noise_d, temperature)
+        step.check_status()
+        y_gpu = step.host("lm_logits_dbg").reshape(cfg.B, cfg.max_nodes, cfg.V)
+        x_gpu = step.host("argmax").astype(np.int64)
+        want = orc.sample_accept(node_tok, parent, n_nodes, depth, y_gpu, noise, inv_t, cfg.T, fp32=True)
+        for b in range(cfg.B):
+            for i in range(int(n_nodes[b])):
+                z = (y_gpu[b, i].astype(np.float64) * np.float64(np.float32(inv_t)) + noise[b, depth[b, i]]).astype(np.float32)
+                top2 = np.sort(z)[-2:]
+                if top2[1] - top2[0] > 4 * np.spacing(np.float32(abs(top2[1]))):     # not a rounding-level tie
+                    assert x_gpu[b, i] == want[0][b, i], (temperature, b, i)
+                zd = y_def[b, i] * inv_t + noise[b, depth[b, i]]
+                t2 = np.sort(zd)[-2:]
+                if t2[1] - t2[0] > 2 * 2e-2 * inv_t + 1e-3:                          # beyond the logit tolerance
+                    assert x_gpu[b, i] == int(np.argmax(zd)), ("definition mode", temperature, b, i)
+        acc = orc.greedy_accept(node_tok, parent, n_nodes, x_gpu, cfg.T)                 # the walk over the kernel's draws
+        for nm, w in zip(["acc_len", "acc_nodes", "acc_tok", "next_tok"], acc):
+            np.testing.assert_array_equal(step.host(nm), w, err_msg=nm)
+        accepted.append(int(acc[0].sum()))
+    for k, v in greedy.items():                                                      # temperature 1e-6: the greedy result
+        live = np.arange(cfg.max_nodes)[None, :] < n_nodes[:, None]
+        if k == "argmax":
+            np.testing.assert_array_equal(step.host(k)[live], v[live])
+        else:
+            np.testing.assert_array_equal(step.host(k), v, err_msg=k)
+    assert accepted[2] == int(greedy["acc_len"].sum())
+
+
 BIG = {
     # trees above 128 nodes: three and four mask words, two LM-head row tiles per sequence
     "big_enum": C["c2"].replace(name="big_enum", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200,

@@ -715,6 +715,197 @@ def test_commit_accepted_reads_the_cache_as_it_was():
     assert np.array_equal(K2[1], K[1]) and new_len.tolist() == [5, 2] and sel.tolist() == [3, 4]
 
 
+# ------------------------------------------------------------------ sampling acceptance
+def _sequential_rule_distribution(p, children):
+    """Sec. 2's rule written out for a deterministic proposal, with exact probabilities: the
+    children of a node are tried one after the other; a tried child is accepted with probability
+    min(1, P(c) / P'(c)) where P' is the point mass on c; after a rejection P becomes
+    norm(max(0, P - P')), i.e. P without c.  If every child is rejected a token is drawn from what
+    is left.  Returns the probability of every token being the one emitted after this node."""
+    p = np.asarray(p, dtype=np.float64).copy()
+    out = np.zeros_like(p)
+    reach = 1.0                                   # probability that the trials get this far
+    for c in children:
+        a = min(1.0, p[c] / 1.0)
+        out[c] += reach * a
+        reach *= 1.0 - a
+        resid = np.maximum(0.0, p - np.eye(len(p))[c])
+        p = resid / resid.sum()
+    out += reach * p
+    return out
+
+
+def test_sequential_acceptance_with_point_mass_proposals_emits_the_target_distribution():
+    rng = np.random.default_rng(21)
+    for _ in range(20):
+        V = int(rng.integers(3, 8))
+        p = rng.dirichlet(np.ones(V))
+        kids = list(rng.permutation(V)[:int(rng.integers(1, V))])
+        np.testing.assert_allclose(_sequential_rule_distribution(p, kids), p, atol=1e-12)
+
+
+def test_sample_tokens_draws_from_the_softmax_and_a_chain_accepts_with_the_product_rule():
+    """The oracle's rule (one Gumbel-max draw per node, accepted iff it is a child) against the
+    distribution the sequential rule emits (= the target distribution, test above): frequencies
+    over many noise draws, and the accepted length on a chain against prod_d P_d(child_d)."""
+    from paper_2412_00061_b200 import synth
+    V, T, n = 5, 3, 4
+    cfg = synth.CONFIGS["c1"].replace(name="samp", B=1, V=V, T=T, max_nodes=n)
+    rng = np.random.default_rng(5)
+    y = rng.normal(size=(1, n, V)) * 1.5
+    inv_temp = 1.0 / 0.7
+    tok, ln, nc = _pack([(2, 0, 3)], 1, T)
+    node_tok, parent, depth, pos, mask, retrieve, nn = orc.build_tree(np.array([1]), np.array([0]), tok, ln, nc, n_max=n)
+    probs = torch.softmax(torch.tensor(y[0]) * inv_temp, -1).numpy()          # [n,V] target distributions
+    trials = 20000
+    first = np.zeros(V)
+    lens = np.zeros(T + 1)
+    for s in range(trials):
+        g = synth.gen_gumbel_noise(cfg, s)
+        x, acc_len, acc_nodes, acc_tok, next_tok = orc.sample_accept(node_tok, parent, nn, depth, y, g, inv_temp, T)
+        first[x[0, 0]] += 1
+        lens[acc_len[0]] += 1
+    want_first = probs[0]
+    assert np.all(np.abs(first / trials - want_first) <= 4 * np.sqrt(want_first * (1 - want_first) / trials) + 1e-3)
+    a = [probs[0, 2], probs[1, 0], probs[2, 3]]                                # P_d(child_d) along the chain
+    want_len = [1 - a[0], a[0] * (1 - a[1]), a[0] * a[1] * (1 - a[2]), a[0] * a[1] * a[2]]
+    for d in range(T + 1):
+        q = want_len[d]
+        assert abs(lens[d] / trials - q) <= 4 * math.sqrt(q * (1 - q) / trials) + 1e-3
+
+
+def test_sampling_acceptance_special_cases():
+    from paper_2412_00061_b200 import synth
+    rng = np.random.default_rng(6)
+    V, T, n = 9, 4, 16
+    cfg = synth.CONFIGS["c1"].replace(name="samp2", B=2, V=V, T=T, max_nodes=n)
+    cands = [(1, 2, 3), (1, 4), (5,)]
+    tok, ln, nc = _pack(cands, 3, T)
+    tok, ln, nc = np.repeat(tok, 2, 0), np.repeat(ln, 2, 0), np.repeat(nc, 2, 0)
+    node_tok, parent, depth, pos, mask, retrieve, nn = orc.build_tree(np.array([0, 0]), np.array([0, 0]), tok, ln, nc, n_max=n)
+    y = rng.normal(size=(2, n, V))
+    g = synth.gen_gumbel_noise(cfg, 3)
+    # temperature -> 0: the draw is the arg-max, acceptance is the greedy one
+    cold = orc.sample_accept(node_tok, parent, nn, depth, y, g, 1e9, T)
+    am = np.argmax(y, axis=-1)
+    for got, want in zip(cold[1:], orc.greedy_accept(node_tok, parent, nn, am, T)):
+        np.testing.assert_array_equal(got, want)
+    # a target that puts all its mass on a child's token (P = P', the point mass): always accepted
+    y2 = np.full((2, n, V), -50.0)
+    for b in range(2):
+        y2[b, 0, 1] = y2[b, 1, 2] = y2[b, 2, 3] = 50.0
+    for s in range(10):
+        out = orc.sample_accept(node_tok, parent, nn, depth, y2, synth.gen_gumbel_noise(cfg, s), 1.0, T)
+        assert out[1].tolist() == [3, 3] and out[3][0].tolist() == [1, 2, 3, -1]
+    # nodes of equal depth share their noise, nodes along a path do not; the float32 decision differs
+    # from the float64 one only through rounding
+    x64 = orc.sample_tokens(y, depth, nn, g, 1.3)
+    x32 = orc.sample_tokens(y, depth, nn, g, 1.3, fp32=True)
+    assert np.mean(x64 == x32) > 0.9
+    i, j = 2, 4                                              # nodes (1,2) and (1,4): both depth 2
+    assert depth[0, i] == depth[0, j] == 2
+    same_logits = y.copy()
+    same_logits[0, j] = same_logits[0, i]
+    xs = orc.sample_tokens(same_logits, depth, nn, g, 1.3)
+    assert xs[0, i] == xs[0, j]
+
+
+# ------------------------------------------------------------------ the attention draft module
+def _draft_module_case(rng, B=2, R=3, H=32, Hq=4, Hkv=2, D=8, I=48, Lcap=24, zero=False):
+    sc = 0.0 if zero else 0.3
+    w = dict(g1=rng.normal(size=H) * 0.2 + 1.0, g2=rng.normal(size=H) * 0.2 + 1.0,
+             Wqkv=rng.normal(size=((Hq + 2 * Hkv) * D, H)) * 0.3, Wo=rng.normal(size=(H, Hq * D)) * sc,
+             Wgu=rng.normal(size=(2 * I, H)) * 0.3, Wdn=rng.normal(size=(H, I)) * sc)
+    F = rng.normal(size=(B, R, H))
+    n_new = rng.integers(1, R + 1, size=B)
+    kv_len = rng.integers(0, 9, size=B)
+    Kd = rng.normal(size=(B, Hkv, Lcap, D))
+    Vd = rng.normal(size=(B, Hkv, Lcap, D))
+    return w, F, n_new, kv_len, Kd, Vd, (Hq, Hkv, D, I)
+
+
+def _torch_layer_reference(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D, eps, theta):
+    """The same layer out of library pieces: F.rms_norm, rotary embedding as complex multiplication
+    on (x_i, x_{i+D/2}) pairs, scaled_dot_product_attention, F.silu."""
+    import torch.nn.functional as Fn
+    t = lambda a: torch.tensor(np.asarray(a), dtype=torch.float64)
+    B, R, H = F.shape
+    I = w["Wdn"].shape[1]
+    out = np.zeros((B, H))
+    Kd, Vd = t(Kd).clone(), t(Vd).clone()
+
+    def rope(x, pos):                                  # x [heads, D]
+        half = D // 2
+        freqs = theta ** (-2.0 * torch.arange(half, dtype=torch.float64) / D)
+        rot = torch.polar(torch.ones(half, dtype=torch.float64), pos * freqs)
+        z = torch.complex(x[:, :half], x[:, half:]) * rot
+        return torch.cat([z.real, z.imag], dim=1)
+
+    for b in range(B):
+        L, r = int(kv_len[b]), int(n_new[b])
+        for j in range(r):
+            a = Fn.rms_norm(t(F[b, j]), (H,), t(w["g1"]), eps)
+            qkv = t(w["Wqkv"]) @ a
+            q = rope(qkv[:Hq * D].reshape(Hq, D), L + j)
+            Kd[b, :, L + j] = rope(qkv[Hq * D:(Hq + Hkv) * D].reshape(Hkv, D), L + j)
+            Vd[b, :, L + j] = qkv[(Hq + Hkv) * D:].reshape(Hkv, D)
+        n = L + r
+        k = Kd[b, :, :n].repeat_interleave(Hq // Hkv, 0)
+        v = Vd[b, :, :n].repeat_interleave(Hq // Hkv, 0)
+        o = Fn.scaled_dot_product_attention(q[:, None, :], k, v)[:, 0, :]
+        h1 = t(F[b, r - 1]) + t(w["Wo"]) @ o.reshape(-1)
+        m = Fn.rms_norm(h1, (H,), t(w["g2"]), eps)
+        gu = t(w["Wgu"]) @ m
+        out[b] = (h1 + t(w["Wdn"]) @ (Fn.silu(gu[:I]) * gu[I:])).numpy()
+    return out, Kd.numpy(), Vd.numpy()
+
+
+def test_draft_module_against_library_pieces():
+    rng = np.random.default_rng(31)
+    for trial in range(4):
+        w, F, n_new, kv_len, Kd, Vd, (Hq, Hkv, D, I) = _draft_module_case(rng)
+        got = orc.draft_module(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D, eps=1e-5, theta=10000.0)
+        want = _torch_layer_reference(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D, 1e-5, 10000.0)
+        np.testing.assert_allclose(got[0], want[0], atol=1e-11)
+        np.testing.assert_allclose(got[1], want[1], atol=1e-12)
+        np.testing.assert_allclose(got[2], want[2], atol=1e-12)
+        np.testing.assert_array_equal(got[3], kv_len + n_new)
+        for b in range(F.shape[0]):                    # nothing but the new rows of the cache changes
+            L, r = int(kv_len[b]), int(n_new[b])
+            assert np.array_equal(got[1][b, :, :L], Kd[b, :, :L]) and np.array_equal(got[1][b, :, L + r:], Kd[b, :, L + r:])
+
+
+def test_draft_module_special_cases():
+    rng = np.random.default_rng(32)
+    # output projections at zero: both residual branches vanish, the layer is the identity on the
+    # newest hidden state, so drafting from its output equals drafting from the hidden state itself
+    w, F, n_new, kv_len, Kd, Vd, (Hq, Hkv, D, I) = _draft_module_case(rng, zero=True)
+    F_hat, _, _, _ = orc.draft_module(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D)
+    last = np.stack([F[b, n_new[b] - 1] for b in range(F.shape[0])])
+    np.testing.assert_allclose(F_hat, last, atol=1e-15)
+    Wd = rng.normal(size=(3, 11, F.shape[2]))
+    np.testing.assert_allclose(orc.draft_logits(F_hat, Wd), orc.draft_logits(last, Wd), atol=1e-12)
+    # the attention inside the layer is the (separately pinned) tree attention of a one-node tree
+    w, F, n_new, kv_len, Kd, Vd, (Hq, Hkv, D, I) = _draft_module_case(rng, B=1, R=2)
+    w["Wdn"] = np.zeros_like(w["Wdn"])                 # MLP off: F_hat = h + Wo attn
+    F_hat, K2, V2, L2 = orc.draft_module(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D)
+    r, L = int(n_new[0]), int(kv_len[0])
+    a = orc.rms_norm(F[0, r - 1], w["g1"], 1e-5)
+    q = (w["Wqkv"] @ a)[:Hq * D].reshape(Hq, D)
+    Q = np.zeros((1, 4, Hq, D))
+    Q[0, 0] = np.stack([orc.rope_rotate(q[h], L + r - 1, 10000.0) for h in range(Hq)])
+    one = orc.tree_attention(Q, K2, V2, np.array([L + r - 1]), np.array([1]), np.ones((1, 4, 1), dtype=np.uint64),
+                             1.0 / math.sqrt(D))
+    np.testing.assert_allclose(F_hat[0], F[0, r - 1] + w["Wo"] @ one[0, 0].reshape(-1), atol=1e-12)
+    # rotary embedding: a rotation (norm kept), position 0 is the identity, relative-position property
+    v, u = rng.normal(size=D), rng.normal(size=D)
+    np.testing.assert_allclose(orc.rope_rotate(v, 0, 10000.0), v, atol=0)
+    assert abs(np.linalg.norm(orc.rope_rotate(v, 17, 10000.0)) - np.linalg.norm(v)) < 1e-12
+    d1 = orc.rope_rotate(v, 9, 10000.0) @ orc.rope_rotate(u, 4, 10000.0)
+    d2 = orc.rope_rotate(v, 25, 10000.0) @ orc.rope_rotate(u, 20, 10000.0)
+    assert abs(d1 - d2) < 1e-10
+
+
 # ------------------------------------------------------------------ chained steps
 def _chain_case(seed, n_steps, p=0.8):
     from paper_2412_00061_b200 import synth
