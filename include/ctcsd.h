@@ -319,6 +319,53 @@ int ctcsd_verify_accept_raw(ctcsd_handle* h, void* stream, const void* hn, const
                             int* out_next_tok, float* out_logits_dbg);
 
 /*
+ * The paper's Attention Draft Module (Sec. 3.1: one transformer layer, built like the base model's, on
+ * the base model's hidden states; Sec. 3.2: F_hat = DraftModule(F), whose projection gives one
+ * distribution per place; Sec. 4.3: it takes 14.93 % of the paper's decoding time).  The paper gives
+ * no further detail; the layer built here is a LLaMA-style decoder layer with the handle's head
+ * shape (Hq, Hkv, D):
+ *   a = RMSNorm(F; g1);  q,k,v = a Wqkv^T;  rotary embedding of q and k at the row's position;
+ *   attention of the newest position over all positions so far (scale 1/sqrt(D));
+ *   h1 = F + Wo attn;  m = RMSNorm(h1; g2);  F_hat = h1 + Wdn ( SiLU(Wg m) * (Wu m) ).
+ * No final norm.  Per step the caller hands over the hidden states of the newest n_new[b] <= R
+ * positions of every sequence (what the previous step accepted); keys and values are made for all
+ * of them and appended to the layer's own cache, the rest of the layer runs for the newest one,
+ * and its output F_hat [B,H] is what ctcsd_draft_logits projects to the T places.
+ *
+ * ctcsd_draft_layer: weights, all device pointers, the matrices in the handle's dtype with the
+ *   input axis contiguous: Wqkv [(Hq+2Hkv)*D, H] (query rows, then key rows, then value rows),
+ *   Wo [H, Hq*D], Wgu [2I, H] (gate rows, then up rows), Wdn [H, I]; g1, g2 [H] float32;
+ *   I the MLP width (multiple of 8), eps the RMSNorm epsilon, rope_theta the rotary base (the
+ *   rotation pairs element i with i + D/2, frequency rope_theta^(-2i/D)).
+ * workspace: device memory of ctcsd_draft_module_workspace_bytes(cfg, R, I) bytes, 256-byte aligned,
+ *   owned by the caller, used only during the call.
+ * F_new [B,R,H] dtype;  n_new [B] int32 in 1..R;  kv_len [B] int32: positions already in the cache;
+ * Kd, Vd [B,Hkv,Lcap,D] dtype, updated in place at rows kv_len[b] .. kv_len[b]+n_new[b]-1;
+ * out_F [B,H] dtype;  out_kv_len [B] int32 = kv_len + n_new (must not be the array kv_len);
+ * out_F_dbg NULL or [B,H] float32: F_hat before it is rounded to dtype.
+ * A sequence with n_new outside 1..R or kv_len + n_new > Lcap records CTCSD_ERR_INVALID_ARG in the
+ * device status word; its cache is left alone and its output row is not meaningful.
+ */
+typedef struct ctcsd_draft_layer {
+    const float* g1;
+    const void*  Wqkv;
+    const void*  Wo;
+    const float* g2;
+    const void*  Wgu;
+    const void*  Wdn;
+    int   I;
+    float eps;
+    float rope_theta;
+} ctcsd_draft_layer;
+
+int ctcsd_draft_module_workspace_bytes(const ctcsd_config* cfg, int R, int I, size_t* out_bytes);
+int ctcsd_draft_module(ctcsd_handle* h, void* stream, const ctcsd_draft_layer* layer,
+                       void* workspace, size_t workspace_bytes,
+                       int R, const void* F_new, const int* n_new, const int* kv_len,
+                       void* Kd, void* Vd, int Lcap,
+                       void* out_F, int* out_kv_len, float* out_F_dbg);
+
+/*
  * Tree attention without a handle and without any allocation (the paper has no counterpart:
  * this is a packaging variant of ctcsd_tree_attention, same arithmetic, same kernels).
  *

@@ -24,7 +24,7 @@ EXPORTS = [
     "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
     "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static", "ctcsd_draft_logits_rows",
-    "ctcsd_verify_accept_sampled",
+    "ctcsd_verify_accept_sampled", "ctcsd_draft_module_workspace_bytes", "ctcsd_draft_module",
     "ctcsd_select_raw_paths", "ctcsd_build_raw_tree", "ctcsd_verify_accept_raw",
 ]
 
@@ -37,6 +37,12 @@ class CConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "B", "H", "V", "T", "k", "beam", "topN", "max_nodes", "Hq", "Hkv", "D", "dtype", "score_mode",
         "max_draft_rows")]
+
+
+class CDraftLayer(ctypes.Structure):
+    _fields_ = [("g1", ctypes.c_void_p), ("Wqkv", ctypes.c_void_p), ("Wo", ctypes.c_void_p), ("g2", ctypes.c_void_p),
+                ("Wgu", ctypes.c_void_p), ("Wdn", ctypes.c_void_p), ("I", ctypes.c_int), ("eps", ctypes.c_float),
+                ("rope_theta", ctypes.c_float)]
 
 
 _lib = None
@@ -70,6 +76,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_tree_attention.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp, vp, ctypes.c_float, vp]
     lib.ctcsd_verify_accept.argtypes = [vp, vp] + [vp] * 11
     lib.ctcsd_verify_accept_sampled.argtypes = [vp, vp] + [vp] * 7 + [ctypes.c_float] + [vp] * 6
+    lib.ctcsd_draft_module_workspace_bytes.argtypes = [ctypes.POINTER(CConfig), ci, ci, ctypes.POINTER(cs)]
+    lib.ctcsd_draft_module.argtypes = [vp, vp, ctypes.POINTER(CDraftLayer), vp, cs, ci, vp, vp, vp, vp, vp, ci, vp, vp, vp]
     lib.ctcsd_commit_accepted.argtypes = [vp, vp, vp, vp, ci, vp, vp, vp, vp, vp]
     lib.ctcsd_select_raw_paths.argtypes = [vp, vp, ci] + [vp] * 6
     lib.ctcsd_build_raw_tree.argtypes = [vp, vp] + [vp] * 13
@@ -271,6 +279,38 @@ class Handle:
             _ptr(out_next_tok, i32, c.B, "out_next_tok"),
             _ptr(out_logits_dbg, torch.float32, nn * c.V, "out_logits_dbg"))
         self._check(rc, "verify_accept_sampled")
+
+    # ---- the paper's attention draft module (Sec. 3.1) ----
+    def make_draft_layer(self, g1, Wqkv, Wo, g2, Wgu, Wdn, eps=1e-5, rope_theta=10000.0, R=None):
+        """Bundles the layer's weights (device tensors) and allocates the call's workspace."""
+        c = self.cfg
+        I = Wdn.shape[1]
+        f32 = torch.float32
+        layer = CDraftLayer(_ptr(g1, f32, c.H, "g1"), _ptr(Wqkv, self.act_dtype, (c.Hq + 2 * c.Hkv) * c.D * c.H, "Wqkv"),
+                            _ptr(Wo, self.act_dtype, c.H * c.Hq * c.D, "Wo"), _ptr(g2, f32, c.H, "g2"),
+                            _ptr(Wgu, self.act_dtype, 2 * I * c.H, "Wgu"), _ptr(Wdn, self.act_dtype, c.H * I, "Wdn"),
+                            I, float(eps), float(rope_theta))
+        R = R or (c.T + 1)
+        n = ctypes.c_size_t(0)
+        self._check(self.lib.ctcsd_draft_module_workspace_bytes(ctypes.byref(self.cfg), R, I, ctypes.byref(n)),
+                    "draft_module_workspace_bytes")
+        ws = torch.empty(n.value + 256, dtype=torch.uint8, device=self.device)
+        keep = (g1, Wqkv, Wo, g2, Wgu, Wdn)
+        return dict(layer=layer, ws=ws, ws_ptr=(ws.data_ptr() + 255) // 256 * 256, ws_bytes=n.value, R=R, keep=keep)
+
+    def draft_module(self, dl, F_new, n_new, kv_len, Kd, Vd, out_F, out_kv_len, out_F_dbg=None, stream=None):
+        c = self.cfg
+        i32 = torch.int32
+        R = F_new.shape[1]
+        Lcap = Kd.shape[2]
+        rc = self.lib.ctcsd_draft_module(
+            self._h, _stream_ptr(stream), ctypes.byref(dl["layer"]), dl["ws_ptr"], dl["ws_bytes"], R,
+            _ptr(F_new, self.act_dtype, c.B * R * c.H, "F_new"), _ptr(n_new, i32, c.B, "n_new"),
+            _ptr(kv_len, i32, c.B, "kv_len"),
+            _ptr(Kd, self.act_dtype, c.B * c.Hkv * Lcap * c.D, "Kd"), _ptr(Vd, self.act_dtype, c.B * c.Hkv * Lcap * c.D, "Vd"),
+            Lcap, _ptr(out_F, self.act_dtype, c.B * c.H, "out_F"), _ptr(out_kv_len, i32, c.B, "out_kv_len"),
+            _ptr(out_F_dbg, torch.float32, c.B * c.H, "out_F_dbg"))
+        self._check(rc, "draft_module")
 
     # ---- the paper's raw-tree layout (Sec. 3.3) ----
     def select_raw_paths(self, topk_id, topk_lp, sel_row, out_raw_tok, out_raw_score, out_n_raw, stream=None):

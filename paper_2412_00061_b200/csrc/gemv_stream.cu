@@ -247,6 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                 const int v = (int)(r0 + i - (long long)slot * rps);
                 if (v == (int)rps - 1) z += bias;
                 if (p.logits_dbg) p.logits_dbg[((size_t)(p.m0 + own_m) * p.slots + slot) * rps + v] = z;
+                if (p.mode == 2) return;                       // plain product: the value written above is the output
                 if (noise_row != nullptr) z = __fmaf_rn(z, p.sn.inv_temp, noise_row[v]);
                 st.push(z, v);
             };
@@ -363,6 +364,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
         }
     }
     __syncthreads();
+    if (p.mode == 2) return;                                         // no selection, nothing to merge
 
     // fold the CTA's states per segment: warp m merges activation row m's states, one per lane
     for (int seg = 0; seg < 2; ++seg) {
@@ -474,9 +476,13 @@ int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
 // bfloat16 rows go through the tensor-core consumer, up to 8 activation rows per pass over the
 // weights; float32 rows through the fused-multiply-add consumer, up to 4 per pass.
 int launch_typed_bf16(Handle* h, cudaStream_t stream, int M, GemvParams& p) {
-    for (int m0 = 0; m0 < M; m0 += 8) {
+    // the activation rows of a pass sit in shared memory beside the weight ring: with a long inner
+    // dimension fewer rows go into a pass, so that the ring keeps at least two slots of useful size
+    int per_pass = 8;
+    while (per_pass > 1 && (size_t)per_pass * p.H * 2 > 96 * 1024) per_pass >>= 1;
+    for (int m0 = 0; m0 < M; m0 += per_pass) {
         p.m0 = m0;
-        p.mcount = (M - m0 < 8) ? (M - m0) : 8;
+        p.mcount = (M - m0 < per_pass) ? (M - m0) : per_pass;
         int rc;
         if (p.mcount == 1) rc = launch_one<__nv_bfloat16, 1>(h, stream, p);
         else if (p.mcount == 2) rc = launch_one<__nv_bfloat16, 2>(h, stream, p);
@@ -488,9 +494,11 @@ int launch_typed_bf16(Handle* h, cudaStream_t stream, int M, GemvParams& p) {
 }
 
 int launch_typed_f32(Handle* h, cudaStream_t stream, int M, GemvParams& p) {
-    for (int m0 = 0; m0 < M; m0 += 4) {
+    int per_pass = 4;
+    while (per_pass > 1 && (size_t)per_pass * p.H * 4 > 96 * 1024) per_pass >>= 1;
+    for (int m0 = 0; m0 < M; m0 += per_pass) {
         p.m0 = m0;
-        p.mcount = (M - m0 < 4) ? (M - m0) : 4;
+        p.mcount = (M - m0 < per_pass) ? (M - m0) : per_pass;
         int rc;
         if (p.mcount == 1) rc = launch_one<float, 1>(h, stream, p);
         else if (p.mcount == 2) rc = launch_one<float, 2>(h, stream, p);

@@ -28,7 +28,7 @@ struct GemvParams {
     DraftPartial* part;       // [MROWS][grid][2]
     int* part_slot;           // [grid][2] slot id of each partial (-1 = unused)
     unsigned* counter;        // ticket counter, zero on entry, zero again on exit
-    int mode;                 // 0: top-k + lse outputs, 1: arg-max output
+    int mode;                 // 0: top-k + lse outputs, 1: arg-max output, 2: the products themselves (to logits_dbg)
     int k;
     int* out_topk_id;         // mode 0: [M,slots,k]
     float* out_topk_lp;       // mode 0: [M,slots,k]

@@ -48,7 +48,11 @@ struct TcParams {
                       //    (both accumulators in use, one per row tile); 0: one row tile per stage,
                       //    the accumulators alternate between consecutive tiles
     int m_units;      // row tiles (pair = 0) or pairs of row tiles (pair = 1)
-    int a_bytes;      // bytes of the activation tile a stage holds: 128 rows, or 64 when M <= 64
+    int a_bytes;      // bytes of one K block of an activation tile: 128 rows, or 64 when M <= 64
+    int atoms;        // K blocks (of 64 elements, one 128-byte swizzle row each) per stage: 1, or more when
+                      // the hidden size is a multiple of 64 - one copy instruction then brings `atoms`
+                      // blocks of a tile (a box over a [rows][K blocks][64] view of the tensor)
+    int num_ks;       // stages per unit = ceil(num_k / atoms)
     unsigned long long* keys; // [m_tiles*128] packed (logit, id) maxima, zero between calls
     AcceptParams acc;
     unsigned* counter;
@@ -62,13 +66,7 @@ struct TcParams {
     DraftPartial* part;       // [n_tiles][kColSplit][m_tiles*128] per-tile, per-column-share states
     const int* row_seq;       // [M] or null
     const float* blank_bias;  // [B] or null; added to class V-1 of every slot
-    // L2 look-ahead of the weight stream: the K blocks of a tile are asked for in groups of
-    // pf_group (pf_group * 128 contiguous bytes of every weight row in one request), pf_ahead groups
-    // before the tile loads reach them; 0 turns it off
     SampleNoise sn;           // LM head: noise added to the scaled logit before the arg-max (null: none)
-    const unsigned char* W;   // the weights as plain memory: row r of slot t starts at ((t * V) + r) * row_bytes
-    long long row_bytes;
-    int pf_group, pf_ahead;
 };
 
 struct __align__(8) TcShared {
@@ -93,8 +91,11 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
     const uint32_t raw_addr = tc::smem_u32(dyn_raw);
     unsigned char* dyn = dyn_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-    const int a_all = p.a_bytes * (1 + p.pair);             // activation bytes of a stage
-    const int stage_bytes = a_all + p.Nt * 128;
+    // a stage: activations [K block][row tile (two in pair mode)][a_bytes], then weights [K block][Nt x 128 bytes]
+    const int a_blk = p.a_bytes * (1 + p.pair);             // one K block of the stage's activations
+    const int a_all = a_blk * p.atoms;                      // activation bytes of a stage
+    const int w_atom = p.Nt * 128;                          // one K block of the weight tile
+    const int stage_bytes = a_all + w_atom * p.atoms;
     TcShared* sh = reinterpret_cast<TcShared*>(dyn + (size_t)p.stages * stage_bytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -123,34 +124,40 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int u_first = (int)blockIdx.x, u_step = (int)gridDim.x;
     const int n_units = units > u_first ? (int)((units - u_first + u_step - 1) / u_step) : 0;
 
-    // producer state (lane 0 of warp 0 only).  Stage `it` holds K block it % num_k of unit
-    // u_first + (it / num_k) * u_step; every CTA walks the K axis from its own starting block (and wraps), so that
-    // at any moment the CTAs ask L2 for different parts of the shared activations.
-    const int total_it = n_units * p.num_k;
-    const int k_start = (int)(((long long)blockIdx.x * p.num_k) / gridDim.x);
+    // producer state (lane 0 of warp 0 only).  Stage `it` holds K blocks [ks * atoms, (ks+1) * atoms),
+    // ks = it % num_ks, of unit u_first + (it / num_ks) * u_step; every CTA walks the K axis from its
+    // own starting stage (and wraps), so that at any moment the CTAs ask L2 for different parts of
+    // the shared activations.
+    const int total_it = n_units * p.num_ks;
+    const int k_start = (int)(((long long)blockIdx.x * p.num_ks) / gridDim.x);
     const uint64_t pol_w = tc::policy_evict_first();
     const uint64_t pol_a = tc::policy_evict_last();
     auto load_stage = [&](int it, bool do_w, bool do_a) {
-        const int u = u_first + (it / p.num_k) * u_step, kb = it - (it / p.num_k) * p.num_k;
+        const int u = u_first + (it / p.num_ks) * u_step, kb = it - (it / p.num_ks) * p.num_ks;
         const int nt = u / p.m_units, mu = u - nt * p.m_units;
         const int s = it % p.stages;
         unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
         int kq = kb + k_start;
-        if (kq >= p.num_k) kq -= p.num_k;
+        if (kq >= p.num_ks) kq -= p.num_ks;
+        // K blocks past the end of the hidden axis (the last stage when atoms does not divide num_k)
+        // lie outside the tensor and arrive as zeros
         if (do_w) {
             tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)stage_bytes);
             if constexpr (MODE == 0) {
-                tc::tma_load_2d(a_dst + a_all, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
+                if (p.atoms == 1) tc::tma_load_2d(a_dst + a_all, &tmW, &sh->full[s], kq * kBlockK, nt * p.Nt, pol_w);
+                else tc::tma_load_3d(a_dst + a_all, &tmW, &sh->full[s], 0, nt * p.Nt, kq * p.atoms, pol_w);
             } else {
                 const int t = nt / p.tiles_per_slot, ntl = nt - t * p.tiles_per_slot;
-                tc::tma_load_3d(a_dst + a_all, &tmW, &sh->full[s], kq * kBlockK, ntl * p.Nt, t, pol_w);
+                if (p.atoms == 1) tc::tma_load_3d(a_dst + a_all, &tmW, &sh->full[s], kq * kBlockK, ntl * p.Nt, t, pol_w);
+                else tc::tma_load_4d(a_dst + a_all, &tmW, &sh->full[s], 0, ntl * p.Nt, kq * p.atoms, t, pol_w);
             }
         }
         if (do_a) {
-            // a row tile past the last one (odd tile count in pair mode) reads as zeros
-            for (int h = 0; h <= p.pair; ++h)
-                tc::tma_load_2d(a_dst + h * p.a_bytes, &tmA, &sh->full[s], kq * kBlockK,
-                                ((p.pair ? 2 * mu : mu) + h) * kTileM, pol_a);
+            // one box: in pair mode it is 256 rows high and brings both row tiles (rows past the last
+            // activation row read as zeros)
+            const int row0 = (p.pair ? 2 * mu : mu) * kTileM;
+            if (p.atoms == 1) tc::tma_load_2d(a_dst, &tmA, &sh->full[s], kq * kBlockK, row0, pol_a);
+            else tc::tma_load_3d(a_dst, &tmA, &sh->full[s], 0, row0, kq * p.atoms, pol_a);
         }
     };
     // The weights are never written by any kernel: their tiles of the first stages are requested
@@ -162,57 +169,14 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         pre = total_it < p.stages ? total_it : p.stages;
         for (int it = 0; it < pre; ++it) load_stage(it, true, false);
     }
-    // L2 look-ahead (all lanes of warp 0).  A tile load asks DRAM for 128 bytes of every weight row,
-    // rows that lie a whole row pitch apart; the neighbouring 128 bytes of the same rows follow a
-    // stage later.  Here the next pf_group K blocks of every row of the tile are requested as ONE
-    // contiguous piece per row, so that DRAM serves a whole open page at a time; the tile loads
-    // that follow find their data in L2 (or in flight).
-    int pf_next = 0;                                   // first iteration whose group is not yet requested
-    auto prefetch_upto = [&](int it_limit) {
-        if (p.pf_group <= 0) return;
-        if (it_limit > total_it) it_limit = total_it;
-        while (pf_next < it_limit) {
-            const int un = pf_next / p.num_k, kb = pf_next - un * p.num_k;
-            const int u = u_first + un * u_step;
-            const int nt = u / p.m_units;
-            int cnt = p.pf_group - kb % p.pf_group;                    // to the end of this group
-            if (kb + cnt > p.num_k) cnt = p.num_k - kb;
-            int kq = kb + k_start;
-            if (kq >= p.num_k) kq -= p.num_k;
-            if (kq + cnt > p.num_k) cnt = p.num_k - kq;                // the rotated K axis wraps here
-            long long row0;
-            int rows;
-            if constexpr (MODE == 0) {
-                row0 = (long long)nt * p.Nt;
-                rows = p.V - (int)row0 < p.Nt ? p.V - (int)row0 : p.Nt;
-            } else {
-                const int t = nt / p.tiles_per_slot, ntl = nt - t * p.tiles_per_slot;
-                rows = p.V - ntl * p.Nt < p.Nt ? p.V - ntl * p.Nt : p.Nt;
-                row0 = (long long)t * p.V + (long long)ntl * p.Nt;
-            }
-            long long off = (long long)kq * 128;
-            long long len = (long long)cnt * 128;
-            if (off + len > p.row_bytes) len = p.row_bytes - off;       // the last K block may be partial
-            len &= ~15ll;
-            if (len > 0)
-                for (int r = lane; r < rows; r += 32)
-                    tc::bulk_prefetch_l2(p.W + (row0 + r) * p.row_bytes + off, (uint32_t)len);
-            pf_next += cnt;
-        }
-    };
-    if (warp == 0) {
-        pre = __shfl_sync(0xffffffffu, pre, 0);
-        prefetch_upto(pre + p.pf_group * p.pf_ahead);
-    }
     // barriers and tensor memory are set up; the activations may come from the preceding kernel
     pdl_wait();
     pdl_trigger();
 
     if (warp == 0) {
-        // ---------------- TMA producer (lane 0; the other lanes help with the L2 look-ahead) ----------------
-        {
-            if (lane == 0)
-                for (int it = 0; it < pre; ++it) load_stage(it, false, true);
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            for (int it = 0; it < pre; ++it) load_stage(it, false, true);
             int it = pre;
             bool ok = true;
             // Stages are refilled two at a time: the two weight boxes then ask for adjacent 128-byte
@@ -221,23 +185,17 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int group = p.stages >= 4 ? 2 : 1;
             while (it < total_it && ok) {
                 const int cnt = total_it - it < group ? total_it - it : group;
-                if (lane == 0) {
-                    for (int j = 0; j < cnt; ++j) {
-                        const int s = (it + j) % p.stages;
-                        const uint32_t ph = (uint32_t)((it + j) / p.stages) & 1u;
-                        if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-                    }
-                    if (ok) {
-                        for (int j = 0; j < cnt; ++j) load_stage(it + j, true, false);
-                        for (int j = 0; j < cnt; ++j) load_stage(it + j, false, true);
-                    }
+                for (int j = 0; j < cnt; ++j) {
+                    const int s = (it + j) % p.stages;
+                    const uint32_t ph = (uint32_t)((it + j) / p.stages) & 1u;
+                    if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                 }
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                for (int j = 0; j < cnt; ++j) load_stage(it + j, true, false);
+                for (int j = 0; j < cnt; ++j) load_stage(it + j, false, true);
                 it += cnt;
-                prefetch_upto(it + p.pf_group * p.pf_ahead);
             }
-            if (!ok && lane == 0) {
+            if (!ok) {
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 1);
                 *abort_flag = 1;
                 // let copies that are still in flight land before the CTA gives its memory back
@@ -259,24 +217,31 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
                 if (!tc::mbar_wait(&sh->tmem_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after_sync();
-                for (int kb = 0; kb < p.num_k; ++kb, ++it) {
+                for (int kb = 0; kb < p.num_ks; ++kb, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
                     if (!tc::mbar_wait(&sh->full[s], ph, abort_flag)) { ok = false; break; }
                     tc::tc_fence_after_sync();
                     const uint32_t a_addr = tc::smem_u32(dyn + (size_t)s * stage_bytes);
-                    const uint64_t adesc = tc::smem_desc_k_sw128(a_addr);
-                    const uint64_t bdesc = tc::smem_desc_k_sw128(a_addr + a_all);
+                    // which K blocks the stage holds decides nothing here except how many are real:
+                    // the rotated order only permutes the terms of the sum
+                    int kq = kb + k_start;
+                    if (kq >= p.num_ks) kq -= p.num_ks;
+                    for (int j = 0; j < p.atoms; ++j) {
+                        if (kq * p.atoms + j >= p.num_k) break;          // zero blocks past the hidden axis
+                        const uint64_t adesc = tc::smem_desc_k_sw128(a_addr + (uint32_t)(j * a_blk));
+                        const uint64_t bdesc = tc::smem_desc_k_sw128(a_addr + (uint32_t)(a_all + j * w_atom));
 #pragma unroll
-                    for (int k = 0; k < kBlockK / 16; ++k) {
-                        // advancing 16 bf16 along K = 32 bytes = 2 descriptor address units
-                        tc::mma_bf16_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
-                    if (p.pair) {                            // the second row tile against the same weights
-                        const uint64_t adesc1 = tc::smem_desc_k_sw128(a_addr + p.a_bytes);
+                        for (int k = 0; k < kBlockK / 16; ++k) {
+                            // advancing 16 bf16 along K = 32 bytes = 2 descriptor address units
+                            tc::mma_bf16_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | j | k) != 0 ? 1u : 0u);
+                        }
+                        if (p.pair) {                        // the second row tile against the same weights
+                            const uint64_t adesc1 = tc::smem_desc_k_sw128(a_addr + (uint32_t)(j * a_blk + p.a_bytes));
 #pragma unroll
-                        for (int k = 0; k < kBlockK / 16; ++k)
-                            tc::mma_bf16_ss(d_tmem + kAccCols, adesc1 + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < kBlockK / 16; ++k)
+                                tc::mma_bf16_ss(d_tmem + kAccCols, adesc1 + 2 * k, bdesc + 2 * k, idesc, (kb | j | k) != 0 ? 1u : 0u);
+                        }
                     }
                     tc::mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
                 }
@@ -456,6 +421,51 @@ bool make_map3(CUtensorMap* map, const void* base, long long slots, long long ro
     return r == CUDA_SUCCESS;
 }
 
+// The same tensors seen as [rows][K blocks][64 elements] (and [slots][rows][K blocks][64]), which
+// needs the hidden size to be a multiple of 64: a box of `atoms` K blocks x box_rows rows x 64
+// elements lands in shared memory as `atoms` consecutive 128-byte-swizzled K-major tiles, so one
+// copy instruction does the work of `atoms` (each instruction costs the copy engine a fixed few
+// hundred nanoseconds whatever its size, which is what bounds a stream of small boxes), and DRAM
+// is asked for atoms x 128 contiguous bytes of every row at once.
+bool make_map_kblocks(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows, int atoms) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || cols % kBlockK != 0) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kBlockK, (cuuint64_t)rows, (cuuint64_t)(cols / kBlockK)};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)kBlockK * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows, (cuuint32_t)atoms};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool make_map3_kblocks(CUtensorMap* map, const void* base, long long slots, long long rows, long long cols, int box_rows,
+                       int atoms) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || cols % kBlockK != 0) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)kBlockK, (cuuint64_t)rows, (cuuint64_t)(cols / kBlockK), (cuuint64_t)slots};
+    cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)kBlockK * 2, (cuuint64_t)cols * 2 * (cuuint64_t)rows};
+    cuuint32_t box[4] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows, (cuuint32_t)atoms, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// K blocks per stage: as many (up to 4) as still leave `min_stages` stages in shared memory; 1
+// when the hidden size is not a multiple of 64 (the last K block is then partial and only the
+// plain 2-D view reads it correctly).
+int choose_atoms(int H, int num_k, int one_block_bytes, int min_stages) {
+    if (H % kBlockK != 0) return 1;
+    if (getenv("CTCSD_ATOMS")) { int a = atoi(getenv("CTCSD_ATOMS")); if (a >= 1 && a <= 4 && a <= num_k) return a; }
+    const int budget = 220 * 1024 - (int)sizeof(TcShared) - 1024;
+    int atoms = 1;
+    while (atoms < 4 && atoms * 2 <= num_k && budget / (one_block_bytes * atoms * 2) >= min_stages) atoms *= 2;
+    return atoms;
+}
+
 struct DraftMergeParams {
     const DraftPartial* part;     // [slots * tiles_per_slot * kColSplit][mpad]
     int M, mpad, slots, tiles_per_slot, k;
@@ -528,27 +538,31 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     p.n_tiles = p.slots * p.tiles_per_slot;
     const size_t need = sizeof(DraftPartial) * (size_t)p.n_tiles * kColSplit * p.m_tiles * kTileM;
     if (need > h->lay.tc_part_bytes) return CTCSD_ERR_WORKSPACE;
-    p.a_bytes = kABytes;
+    // up to 64 rows: only the lower half of the activation tile is loaded (see launch_lm_head_tc)
+    p.a_bytes = (M <= 64 && p.Nt * 128 >= kABytes / 2) ? kABytes / 2 : kABytes;
     p.pair = 0;                                      // the heavy epilogue needs the other accumulator for overlap
     p.m_units = p.m_tiles;
-    const int stage_bytes = p.a_bytes + p.Nt * 128;
+    p.atoms = choose_atoms(c.H, p.num_k, p.a_bytes + p.Nt * 128, 3);
+    p.num_ks = (p.num_k + p.atoms - 1) / p.atoms;
+    const int stage_bytes = (p.a_bytes + p.Nt * 128) * p.atoms;
     int stages = (int)((220 * 1024 - (int)sizeof(TcShared) - 1024) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return CTCSD_ERR_UNSUPPORTED;
     p.stages = stages;
     p.part = reinterpret_cast<DraftPartial*>(h->ws + h->lay.tc_part_off);
-    p.W = static_cast<const unsigned char*>(Wd);
-    p.row_bytes = (long long)c.H * 2;
-    p.pf_group = getenv("CTCSD_PF_GROUP") ? atoi(getenv("CTCSD_PF_GROUP")) : 0;
-    p.pf_ahead = getenv("CTCSD_PF_AHEAD") ? atoi(getenv("CTCSD_PF_AHEAD")) : 1;
     p.row_seq = row_seq;
     p.blank_bias = blank_bias;
     p.logits_dbg = out_logits_dbg;
     p.status = status_ptr(h);
 
     CUtensorMap tmA, tmW;
-    if (!make_map(&tmA, x, M, c.H, kTileM)) return CTCSD_ERR_CUDA;
-    if (!make_map3(&tmW, Wd, p.slots, p.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
+    if (p.atoms == 1) {
+        if (!make_map(&tmA, x, M, c.H, p.a_bytes / 128)) return CTCSD_ERR_CUDA;
+        if (!make_map3(&tmW, Wd, p.slots, p.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
+    } else {
+        if (!make_map_kblocks(&tmA, x, M, c.H, p.a_bytes / 128, p.atoms)) return CTCSD_ERR_CUDA;
+        if (!make_map3_kblocks(&tmW, Wd, p.slots, p.V, c.H, p.Nt, p.atoms)) return CTCSD_ERR_CUDA;
+    }
     const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     long long units = (long long)p.n_tiles * p.m_tiles;
@@ -588,6 +602,9 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     int rounds = (per_sm + 15) / 16;
     int g_per_tile = (per_sm + rounds - 1) / rounds;
     p.Nt = 16 * g_per_tile;
+    // Two or more row tiles: there are many more units than SMs, so the tiles need not be cut to
+    // the SM count; the widest tile gives the most flops per copy instruction and per weight byte.
+    if (p.m_tiles >= 2 && c.V >= 256 && getenv("CTCSD_NT256") == nullptr) p.Nt = 256;
     p.n_tiles = (c.V + p.Nt - 1) / p.Nt;
     if (p.m_tiles * kTileM > h->lay.lm_key_count) return CTCSD_ERR_WORKSPACE;
     // With at most 64 rows only the lower half of the 128-row activation tile is loaded.  The
@@ -600,7 +617,9 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     // per flop (with one row tile per 28 KB weight stage the tensor core waits for L2).
     p.pair = p.m_tiles >= 2 ? 1 : 0;
     p.m_units = p.pair ? (p.m_tiles + 1) / 2 : p.m_tiles;
-    const int stage_bytes = p.a_bytes * (1 + p.pair) + p.Nt * 128;
+    p.atoms = choose_atoms(c.H, p.num_k, p.a_bytes * (1 + p.pair) + p.Nt * 128, 3);
+    p.num_ks = (p.num_k + p.atoms - 1) / p.atoms;
+    const int stage_bytes = (p.a_bytes * (1 + p.pair) + p.Nt * 128) * p.atoms;
     int stages = (int)((220 * 1024 - (int)sizeof(TcShared) - 1024) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return CTCSD_ERR_UNSUPPORTED;
@@ -612,14 +631,16 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     p.out_argmax = out_argmax;
     p.logits_dbg = out_logits_dbg;
     p.status = status_ptr(h);
-    p.W = static_cast<const unsigned char*>(Wl);
-    p.row_bytes = (long long)c.H * 2;
-    p.pf_group = getenv("CTCSD_PF_GROUP") ? atoi(getenv("CTCSD_PF_GROUP")) : 0;
-    p.pf_ahead = getenv("CTCSD_PF_AHEAD") ? atoi(getenv("CTCSD_PF_AHEAD")) : 1;
 
     CUtensorMap tmA, tmW;
-    if (!make_map(&tmA, hn, M, c.H, p.a_bytes / 128)) return CTCSD_ERR_CUDA;
-    if (!make_map(&tmW, Wl, c.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
+    const int a_box_rows = p.a_bytes / 128 * (1 + p.pair);
+    if (p.atoms == 1) {
+        if (!make_map(&tmA, hn, M, c.H, a_box_rows)) return CTCSD_ERR_CUDA;
+        if (!make_map(&tmW, Wl, c.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
+    } else {
+        if (!make_map_kblocks(&tmA, hn, M, c.H, a_box_rows, p.atoms)) return CTCSD_ERR_CUDA;
+        if (!make_map_kblocks(&tmW, Wl, c.V, c.H, p.Nt, p.atoms)) return CTCSD_ERR_CUDA;
+    }
 
     const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(lm_head_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -100,6 +100,17 @@ int launch_simple(Handle* h, cudaStream_t s, const AttnParams& p) {
 }  // namespace
 }  // namespace ctcsd
 
+namespace ctcsd {
+// The attention kernel that serves the handle's dtype and head grouping.
+int tree_attention_dispatch(Handle* h, cudaStream_t s, const AttnParams& p) {
+    if (h->cfg.dtype == CTCSD_DTYPE_BF16) {
+        if (tree_attention_tc_supported(p)) return launch_tree_attention_tc(h, s, p);
+        return launch_tree_attention_mma(h, s, p);
+    }
+    return launch_simple<float>(h, s, p);
+}
+}  // namespace ctcsd
+
 using namespace ctcsd;
 
 extern "C" int ctcsd_tree_attention(ctcsd_handle* hh, void* stream, const void* Q, const void* K, const void* V,
@@ -115,10 +126,5 @@ extern "C" int ctcsd_tree_attention(ctcsd_handle* hh, void* stream, const void* 
     p.B = c.B; p.Hq = c.Hq; p.Hkv = c.Hkv; p.D = c.D; p.max_nodes = c.max_nodes; p.Lcap = Lcap;
     p.scale = scale;
     p.status = status_ptr(h);
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (c.dtype == CTCSD_DTYPE_BF16) {
-        if (tree_attention_tc_supported(p)) return launch_tree_attention_tc(h, s, p);
-        return launch_tree_attention_mma(h, s, p);
-    }
-    return launch_simple<float>(h, s, p);
+    return tree_attention_dispatch(h, static_cast<cudaStream_t>(stream), p);
 }

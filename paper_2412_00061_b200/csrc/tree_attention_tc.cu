@@ -161,10 +161,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 if (!tc::mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag)) { failed = true; break; }
                 unsigned char* kd = KV + (size_t)s * 2 * kTileBytes;
                 tc::mbar_arrive_expect_tx(&sh->full[s], (uint32_t)(2 * kTileBytes));
-                for (int hh = 0; hh < DH; ++hh) {
-                    tc::tma_load_4d(kd + hh * (kKeys * 128), &tmK, &sh->full[s], hh * 64, blk * kKeys, g, b, pol);
-                    tc::tma_load_4d(kd + kTileBytes + hh * (kKeys * 128), &tmV, &sh->full[s], hh * 64, blk * kKeys, g, b, pol);
-                }
+                // one copy per tile and tensor: the box spans both 64-column halves of the head dimension
+                // and lands as [half][key][128 bytes] (every copy instruction costs the copy engine a fixed
+                // few hundred nanoseconds, whatever its size)
+                tc::tma_load_5d(kd, &tmK, &sh->full[s], 0, blk * kKeys, 0, g, b, pol);
+                tc::tma_load_5d(kd + kTileBytes, &tmV, &sh->full[s], 0, blk * kKeys, 0, g, b, pol);
             }
             if (failed) {
                 if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 21);
@@ -544,12 +545,12 @@ int launch_tc(Handle* h, cudaStream_t s, const AttnParams& p) {
         cuuint32_t box[5] = {64, (cuuint32_t)grp, 1, (cuuint32_t)(kRows / grp), 1};
         if (!make_map_nd(&tmQ, p.Q, 5, dims, str, box)) return CTCSD_ERR_CUDA;
     }
-    {   // K, V [B][Hkv][Lcap][D]: box = 64 columns x 128 keys
-        cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)p.Lcap, (cuuint64_t)p.Hkv, (cuuint64_t)p.B};
-        cuuint64_t str[3] = {(cuuint64_t)D * 2, (cuuint64_t)p.Lcap * D * 2, (cuuint64_t)p.Hkv * p.Lcap * D * 2};
-        cuuint32_t box[4] = {64, (cuuint32_t)kKeys, 1, 1};
-        if (!make_map_nd(&tmK, p.K, 4, dims, str, box)) return CTCSD_ERR_CUDA;
-        if (!make_map_nd(&tmV, p.V, 4, dims, str, box)) return CTCSD_ERR_CUDA;
+    {   // K, V [B][Hkv][Lcap][D] seen as [B][Hkv][D/64][Lcap][64]: box = 64 columns x 128 keys x all D/64 halves
+        cuuint64_t dims[5] = {64, (cuuint64_t)p.Lcap, (cuuint64_t)(D / 64), (cuuint64_t)p.Hkv, (cuuint64_t)p.B};
+        cuuint64_t str[4] = {(cuuint64_t)D * 2, 128, (cuuint64_t)p.Lcap * D * 2, (cuuint64_t)p.Hkv * p.Lcap * D * 2};
+        cuuint32_t box[5] = {64, (cuuint32_t)kKeys, (cuuint32_t)(D / 64), 1, 1};
+        if (!make_map_nd(&tmK, p.K, 5, dims, str, box)) return CTCSD_ERR_CUDA;
+        if (!make_map_nd(&tmV, p.V, 5, dims, str, box)) return CTCSD_ERR_CUDA;
     }
     const size_t smem = (size_t)kRows * D * 2 + (size_t)kStages * 2 * kKeys * D * 2 + (size_t)kRows * kKeys * 2 +
                         sizeof(AttnShared) + 1024;

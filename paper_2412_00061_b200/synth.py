@@ -26,7 +26,9 @@ from typing import Dict, Optional, Tuple
 import numpy as np
 
 _TAGS = {"x": 1, "Wd": 2, "bias": 3, "base": 4, "kvlen": 5, "Q": 6, "K": 7, "V": 8,
-         "Wl": 9, "hn_noise": 10, "agree": 11, "repeat": 12, "gumbel": 13}
+         "Wl": 9, "hn_noise": 10, "agree": 11, "repeat": 12, "gumbel": 13,
+         "dm_g1": 14, "dm_g2": 15, "dm_qkv": 16, "dm_o": 17, "dm_gu": 18, "dm_dn": 19, "dm_F": 20, "dm_K": 21,
+         "dm_V": 22, "dm_n": 23, "dm_len": 24}
 
 
 @dataclass(frozen=True)
@@ -231,3 +233,25 @@ def gen_gumbel_noise(cfg: StepConfig, seed: int = 0) -> np.ndarray:
     u = g.random((cfg.B, cfg.T + 1, cfg.V), dtype=np.float64)
     u = np.clip(u, 1e-300, 1.0 - 1e-16)
     return (-np.log(-np.log(u))).astype(np.float32)
+
+
+def gen_draft_layer(cfg: StepConfig, seed: int, I: int, R: int, kv_lo: int, kv_hi: int):
+    """Random-init weights and inputs of one step of the attention draft module (Sec. 3.1): norm
+    gains ~ 1 + 0.1 N(0,1), projection weights ~ N(0, 0.02^2) like the other weights, hidden states
+    of the R newest positions ~ N(0,1), n_new uniform in 1..R, the layer's own key/value cache
+    ~ N(0,1) with kv_lo..kv_hi positions already in it.  Returns (weights dict, F_new [B,R,H],
+    n_new [B], kv_len [B], Kd, Vd [B,Hkv,Lcap,D])."""
+    H, Hq, Hkv, D = cfg.H, cfg.Hq, cfg.Hkv, cfg.D
+    w = dict(g1=(1.0 + 0.1 * _rng(seed, "dm_g1").standard_normal(H)).astype(np.float32),
+             g2=(1.0 + 0.1 * _rng(seed, "dm_g2").standard_normal(H)).astype(np.float32),
+             Wqkv=_normal(seed, "dm_qkv", ((Hq + 2 * Hkv) * D, H), 0.02, cfg.dtype),
+             Wo=_normal(seed, "dm_o", (H, Hq * D), 0.02, cfg.dtype),
+             Wgu=_normal(seed, "dm_gu", (2 * I, H), 0.02, cfg.dtype),
+             Wdn=_normal(seed, "dm_dn", (H, I), 0.02, cfg.dtype))
+    F_new = _normal(seed, "dm_F", (cfg.B, R, H), 1.0, cfg.dtype)
+    n_new = _rng(seed, "dm_n").integers(1, R + 1, size=cfg.B).astype(np.int32)
+    kv_len = _rng(seed, "dm_len").integers(kv_lo, kv_hi + 1, size=cfg.B).astype(np.int32)
+    Lcap = ((kv_hi + R + 63) // 64) * 64
+    Kd = _normal(seed, "dm_K", (cfg.B, Hkv, Lcap, D), 1.0, cfg.dtype)
+    Vd = _normal(seed, "dm_V", (cfg.B, Hkv, Lcap, D), 1.0, cfg.dtype)
+    return w, F_new, n_new, kv_len, Kd, Vd

@@ -269,6 +269,80 @@ def test_sampling_acceptance(name):
     assert accepted[2] == int(greedy["acc_len"].sum())
 
 
+DM = {
+    # (workload, MLP width I, new rows R, positions already cached)
+    "dm_mha": (C["c2"].replace(name="dm_mha", H=512, V=999, Hq=4, Hkv=4, D=128), 1368, 6, (100, 300)),
+    "dm_gqa": (C["c5"].replace(name="dm_gqa", B=3, H=768, V=999, Hq=12, Hkv=4, D=64), 2048, 7, (0, 200)),
+    "dm_fp32": (C["c1"].replace(name="dm_fp32", B=2, H=256, V=999, Hq=4, Hkv=2, D=64), 688, 5, (3, 90)),
+    "dm_long_inner": (C["c2"].replace(name="dm_long_inner", B=3, H=256, V=999, Hq=2, Hkv=2, D=128), 11008, 3, (10, 50)),
+}
+
+
+@pytest.mark.parametrize("name", sorted(DM))
+def test_attention_draft_module(name):
+    """ctcsd_draft_module against the oracle's layer (fp64, from the same dtype-rounded inputs): the
+    layer's output within 2e-2 (bf16: plus half a unit in the last place of the rounded output), the
+    appended key/value rows within the rounding of one bf16 (their inputs pass through one
+    matrix-vector product), every other cache row untouched, the new lengths exact; then the draft
+    head runs on the layer's output and its top-k lists are checked against the oracle fed its logits."""
+    import torch
+    from oracle import ctcsd_oracle as orc
+    from paper_2412_00061_b200 import binding
+    from paper_2412_00061_b200.step import to_device
+    from tests.parity_util import check_topk, tolerances
+    cfg, I, R, (lo, hi) = DM[name]
+    seed = 8
+    dev = torch.device("cuda:0")
+    w, F_new, n_new, kv_len, Kd, Vd = synth.gen_draft_layer(cfg, seed, I, R, lo, hi)
+    want_F, want_K, want_V, want_len = orc.draft_module(F_new, n_new, kv_len, Kd, Vd, w, cfg.Hq, cfg.Hkv, cfg.D)
+    h = binding.Handle(cfg.B, cfg.H, cfg.V, cfg.T, cfg.k, cfg.beam, cfg.topN, cfg.max_nodes, cfg.Hq, cfg.Hkv, cfg.D,
+                       binding.DTYPE_BF16 if cfg.dtype == "bf16" else binding.DTYPE_F32)
+    td = lambda a: to_device(a, cfg.dtype, dev)
+    f32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float32)).to(dev)
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    dl = h.make_draft_layer(f32(w["g1"]), td(w["Wqkv"]), td(w["Wo"]), f32(w["g2"]), td(w["Wgu"]), td(w["Wdn"]), R=R)
+    Kd_d, Vd_d = td(Kd), td(Vd)
+    act = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    out_F = torch.zeros(cfg.B, cfg.H, dtype=act, device=dev)
+    out_dbg = torch.zeros(cfg.B, cfg.H, dtype=torch.float32, device=dev)
+    out_len = torch.zeros(cfg.B, dtype=torch.int32, device=dev)
+    for rep in range(2):                                   # twice: the workspace carries nothing over
+        Kd_d.copy_(td(Kd)); Vd_d.copy_(td(Vd))
+        h.draft_module(dl, td(F_new), i32(n_new), i32(kv_len), Kd_d, Vd_d, out_F, out_len, out_dbg)
+        assert h.poll_status() == 0
+        logit_tol, rel = tolerances(cfg.dtype)
+        assert np.max(np.abs(out_dbg.cpu().numpy() - want_F)) <= logit_tol
+        got_F = out_F.float().cpu().numpy()
+        ulp = 2.0 ** -8 if cfg.dtype == "bf16" else 0.0
+        assert np.all(np.abs(got_F - want_F) <= logit_tol + ulp * np.abs(want_F))
+        np.testing.assert_array_equal(out_len.cpu().numpy(), want_len)
+        gK, gV = Kd_d.float().cpu().numpy(), Vd_d.float().cpu().numpy()
+        for b in range(cfg.B):
+            L, r = int(kv_len[b]), int(n_new[b])
+            assert np.array_equal(gK[b, :, :L], Kd[b, :, :L]) and np.array_equal(gK[b, :, L + r:], Kd[b, :, L + r:])
+            assert np.array_equal(gV[b, :, :L], Vd[b, :, :L]) and np.array_equal(gV[b, :, L + r:], Vd[b, :, L + r:])
+            assert np.all(np.abs(gK[b, :, L:L + r] - want_K[b, :, L:L + r]) <= logit_tol + ulp * np.abs(want_K[b, :, L:L + r]))
+            assert np.all(np.abs(gV[b, :, L:L + r] - want_V[b, :, L:L + r]) <= logit_tol + ulp * np.abs(want_V[b, :, L:L + r]))
+    # the per-place projection on the layer's output
+    x, Wd, bb = synth.gen_draft(cfg, seed)
+    topk_id = torch.zeros(cfg.B, cfg.T, cfg.k, dtype=torch.int32, device=dev)
+    topk_lp = torch.zeros(cfg.B, cfg.T, cfg.k, dtype=torch.float32, device=dev)
+    lse = torch.zeros(cfg.B, cfg.T, dtype=torch.float32, device=dev)
+    zdbg = torch.zeros(cfg.B, cfg.T, cfg.V + 1, dtype=torch.float32, device=dev)
+    h.draft_logits(out_F, td(Wd), None, torch.from_numpy(bb).to(dev), topk_id, topk_lp, lse, zdbg)
+    assert h.poll_status() == 0
+    z_def = orc.draft_logits(got_F, Wd, bb)
+    assert np.max(np.abs(zdbg.cpu().numpy() - z_def)) <= logit_tol
+    check_topk(zdbg.cpu().numpy(), topk_id.cpu().numpy(), topk_lp.cpu().numpy(), lse.cpu().numpy(), cfg.k, rel)
+    # a sequence whose new rows would leave the cache is reported and its cache left alone
+    bad_len = i32(np.full(cfg.B, Kd.shape[2], dtype=np.int32))
+    Kd_d.copy_(td(Kd))
+    h.draft_module(dl, td(F_new), i32(n_new), bad_len, Kd_d, Vd_d, out_F, out_len)
+    assert h.poll_status() == -1
+    assert np.array_equal(Kd_d.float().cpu().numpy(), Kd)
+    h.close()
+
+
 BIG = {
     # trees above 128 nodes: three and four mask words, two LM-head row tiles per sequence
     "big_enum": C["c2"].replace(name="big_enum", H=520, V=2999, Hq=8, Hkv=8, kv_lo=200, kv_hi=200,
