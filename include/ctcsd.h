@@ -111,12 +111,13 @@ int ctcsd_last_cuda_error(const ctcsd_handle* h);
 long long ctcsd_launch_count(const ctcsd_handle* h);
 
 /*
- * Optional hint.  Names a range of device memory, owned by the caller and never written while
- * the handle is in use, that ctcsd_draft_logits asks the L2 cache to fetch as soon as its own
- * weight stream has been requested.  Meant for the first part of the LM-head weights (what
- * ctcsd_verify_accept streams next): the kernels between the two (collapse, tree, attention)
- * are small and leave HBM idle, so the fetch is free.  Keep `bytes` below the L2 size (about
- * 96 MB works on a B200); 0 turns the hint off.  [host] call; `ptr` 16-byte aligned.
+ * Optional hint, off unless set.  Names a range of device memory, owned by the caller and never
+ * written while the handle is in use, that ctcsd_draft_logits asks the L2 cache to fetch as soon
+ * as its own weight stream has been requested (meant for data that a later call of the step
+ * streams, while the small kernels in between leave HBM idle).  Measured on a B200 at the 7B
+ * shape with the head of the LM-head weights: no gain up to 48 MB, a loss beyond (the requests
+ * lengthen the draft head's tail and compete with the attention's reads), so the step does not
+ * use it.  0 turns the hint off.  [host] call; `ptr` 16-byte aligned.
  */
 int ctcsd_set_l2_prefetch(ctcsd_handle* h, const void* ptr, size_t bytes);
 

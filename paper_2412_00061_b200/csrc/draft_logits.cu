@@ -2,8 +2,6 @@
 #include "gemv_stream.cuh"
 #include "lm_head_tc.cuh"
 
-#include <stdlib.h>
-
 using namespace ctcsd;
 
 namespace {
@@ -52,7 +50,6 @@ int draft_logits_impl(ctcsd_handle* hh, void* stream, int M, const void* x, int 
     p.sn.noise = nullptr; p.sn.depth = nullptr; p.sn.max_nodes = 1; p.sn.rows_per_seq = 1; p.sn.inv_temp = 1.f;
     p.pf_ptr = h->l2_hint_ptr;
     p.pf_bytes = h->l2_hint_bytes;
-    if (!(getenv("CTCSD_PF_WHERE") && getenv("CTCSD_PF_WHERE")[0] == 'd')) p.pf_bytes = 0;
     return launch_gemv_stream(h, static_cast<cudaStream_t>(stream), c.dtype, M, p);
 }
 

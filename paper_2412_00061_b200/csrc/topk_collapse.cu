@@ -8,10 +8,8 @@
 // alignments is accumulated in 64-bit fixed point relative to the candidate's best
 // alignment, which makes it independent of the order in which threads arrive.
 #include "common.cuh"
-#include "tc_primitives.cuh"
 
 #include <math.h>
-#include <stdlib.h>
 
 namespace ctcsd {
 namespace {
@@ -35,31 +33,7 @@ struct CollapseParams {
     float* out_cand_score;   // [B,topN]
     int* out_n_cand;         // [B]
     int* status;
-    // CTAs beyond the first `nseq` do no collapsing: they ask the L2 cache for [pf_ptr, pf_ptr +
-    // pf_bytes), data that a later kernel of the step streams (see ctcsd_set_l2_prefetch)
-    int nseq;
-    const unsigned char* pf_ptr;
-    unsigned long long pf_bytes;
 };
-
-// The candidate kernels keep one SM per sequence busy for ten to forty microseconds while HBM has
-// nothing to do.  CTAs past the sequences use that time: each asks L2 for its share of a range of
-// constant data (the head of the LM-head weights) in 64 KB pieces and leaves.  They read nothing
-// that a predecessor writes, so they do not wait for it: under programmatic dependent launch they
-// start as soon as an SM has room, i.e. while the slowest CTAs of the draft head are still streaming.
-__device__ __forceinline__ void l2_prefetch_role(const CollapseParams& p) {
-    pdl_trigger();
-    if (threadIdx.x >= 32 || p.pf_bytes == 0) return;
-    const unsigned long long chunk = 64 * 1024;
-    const unsigned long long nchunks = (p.pf_bytes + chunk - 1) / chunk;
-    const unsigned long long me = blockIdx.x - (unsigned)p.nseq, n = gridDim.x - (unsigned)p.nseq;
-    for (unsigned long long c = me + n * threadIdx.x; c < nchunks; c += n * 32) {
-        unsigned long long len = p.pf_bytes - c * chunk;
-        if (len > chunk) len = chunk;
-        len &= ~15ull;
-        if (len) tc::bulk_prefetch_l2(p.pf_ptr + c * chunk, (uint32_t)len);
-    }
-}
 
 __device__ __forceinline__ int key_len(unsigned long long key) { return (int)(key >> 48); }
 __device__ __forceinline__ int key_tok(unsigned long long key, int i) { return (int)((key >> (6 * (7 - i))) & 63ull); }
@@ -75,14 +49,16 @@ __device__ __forceinline__ unsigned hash_key(unsigned long long key, int cap) {
 }
 
 // Finds or claims the slot of `key`.  The table never fills (capacity >= 2x the entries).
-__device__ __forceinline__ int table_insert(unsigned long long* keys, int cap, unsigned long long key) {
+__device__ __forceinline__ int table_insert(unsigned long long* keys, int cap, unsigned long long key,
+                                            bool* was_there = nullptr) {
     unsigned s = hash_key(key, cap);
     for (int probe = 0; probe < cap; ++probe) {
         unsigned long long cur = keys[s];
-        if (cur == key) return (int)s;
+        if (cur == key) { if (was_there) *was_there = true; return (int)s; }
         if (cur == kEmpty) {
             unsigned long long old = atomicCAS(&keys[s], kEmpty, key);
-            if (old == kEmpty || old == key) return (int)s;
+            if (old == kEmpty) return (int)s;
+            if (old == key) { if (was_there) *was_there = true; return (int)s; }
         }
         s = (s + 1) & (unsigned)(cap - 1);
     }
@@ -187,6 +163,14 @@ __device__ __forceinline__ unsigned sortable_f32(double v) {
     unsigned u = __float_as_uint((float)v);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
+// 32-bit image used by the radix select.  MASS = false: the score is a logarithm (any sign), its
+// float32 value is used.  MASS = true: the score is a non-negative probability mass that may be
+// far below the float32 range; the upper word of the float64 (exponent and 20 mantissa bits) is
+// monotone for non-negative values.
+template <bool MASS> __device__ __forceinline__ unsigned select_image(double v) {
+    if constexpr (MASS) return (unsigned)__double2hiint(v);
+    else return sortable_f32(v);
+}
 
 __device__ __forceinline__ int next_pow2(int v) {
     int n = 2;
@@ -200,6 +184,7 @@ __device__ __forceinline__ int next_pow2(int v) {
 // exactly (float64 score, then key).  If more than kSelMax entries sit on the threshold the
 // arrays (padded to a power of two, capacity >= next_pow2(count)) are sorted in place instead
 // and sel[] becomes the identity.
+template <bool MASS = false>
 __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int count, int need, int* sel,
                                 SelectScratch& S, bool ordered = true) {
     const int tid = threadIdx.x, lane = tid & 31;
@@ -209,7 +194,7 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
     if (count > need) {
         unsigned lmax = 0u, lmin = 0xffffffffu;
         for (int i = tid; i < count; i += kThreads) {
-            const unsigned f = sortable_f32(sc[i]);
+            const unsigned f = select_image<MASS>(sc[i]);
             lmax = max(lmax, f);
             lmin = min(lmin, f);
         }
@@ -229,7 +214,7 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
             if (tid < 256) S.hist[tid] = 0u;
             __syncthreads();
             for (int i = tid; i < count; i += kThreads) {
-                const unsigned f = sortable_f32(sc[i]);
+                const unsigned f = select_image<MASS>(sc[i]);
                 const unsigned top = lo < 32 ? (f >> lo) : 0u;
                 if (top == thr) atomicAdd(&S.hist[(f >> nlo) & ((1u << width) - 1u)], 1u);
             }
@@ -268,7 +253,7 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
         if (ncand > remaining && ncand > kSelMax) {
             // too many entries share the threshold even at full float32 resolution: sort everything
             const int n2 = next_pow2(count);
-            for (int i = count + tid; i < n2; i += kThreads) { sc[i] = -INFINITY; ky[i] = kEmpty; if (ix) ix[i] = 0; }
+            for (int i = count + tid; i < n2; i += kThreads) { sc[i] = MASS ? -1.0 : -INFINITY; ky[i] = kEmpty; if (ix) ix[i] = 0; }
             __syncthreads();
             bitonic_sort_best_first(sc, ky, ix, n2);
             for (int r = tid; r < need; r += kThreads) sel[r] = r;
@@ -277,7 +262,7 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
         }
         // gather definite winners (above the threshold) and the entries on it
         for (int i = tid; i < count; i += kThreads) {
-            const unsigned f = sortable_f32(sc[i]);
+            const unsigned f = select_image<MASS>(sc[i]);
             const unsigned top = lo < 32 ? (f >> lo) : 0u;
             if (top > thr) S.win[atomicAdd(&S.nwin, 1)] = i;
             else if (top == thr) S.cand[atomicAdd(&S.ccnt, 1)] = i;
@@ -402,10 +387,9 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     __shared__ SlotLists sl;
     __shared__ SelectScratch S;
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
-    __shared__ int s_count, s_has_empty;
+    __shared__ int s_count, s_has_empty, s_merged;
 
     const int b = blockIdx.x, tid = threadIdx.x;
-    if (b >= p.nseq) { l2_prefetch_role(p); return; }
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -416,14 +400,16 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     load_slot_lists(p, row, sl);
     const long long neg_inf_sortable = dbl_sortable(-INFINITY);
     for (int i = tid; i < p.cap; i += kThreads) { keys[i] = kEmpty; best[i] = neg_inf_sortable; fsum[i] = 0ull; }
-    if (tid == 0) { s_count = 0; s_has_empty = 0; }
+    if (tid == 0) { s_count = 0; s_has_empty = 0; s_merged = 0; }
     __syncthreads();
 
     // pass 1: collapse every path, claim a table slot, track the best alignment
     for (int path = tid; path < p.npaths; path += kThreads) {
         double s;
         const unsigned long long key = path_key_and_score(p, sl, path, s);
-        int slot = table_insert(keys, p.cap, key);
+        bool was_there = false;
+        int slot = table_insert(keys, p.cap, key, &was_there);
+        if (was_there) s_merged = 1;                     // some candidate has more than one alignment
         if (slot < 0) { report_error(p.status, CTCSD_ERR_INTERNAL, 1); slot = 0; }
         path_slot[path] = (unsigned short)slot;
         atomicMax(&best[slot], dbl_sortable(s));
@@ -431,8 +417,10 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     __syncthreads();
 
     // pass 2: sum exp(s - best) per candidate in fixed point (order independent).  The best
-    // alignment itself contributes exp(0) = 1 exactly, so it needs no call to exp.
-    if (p.score_mode == CTCSD_SCORE_SUM) {
+    // alignment itself contributes exp(0) = 1 exactly, so it needs no call to exp.  When no two
+    // paths collapsed to the same sequence every sum is that single 1 and the pass is skipped.
+    const bool sums = p.score_mode == CTCSD_SCORE_SUM && s_merged != 0;
+    if (sums) {
         for (int path = tid; path < p.npaths; path += kThreads) {
             double s;
             path_key_and_score(p, sl, path, s);
@@ -450,7 +438,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
         const double mx = sortable_dbl(best[i]);
         double sc = mx;
         // a single alignment sums to exactly 1: log(1) = 0
-        if (p.score_mode == CTCSD_SCORE_SUM && fsum[i] != (1ull << 50)) sc = mx + log((double)fsum[i] * (1.0 / kFix));
+        if (sums && fsum[i] != (1ull << 50)) sc = mx + log((double)fsum[i] * (1.0 / kFix));
         score[i] = sc;
     }
     __syncthreads();
@@ -479,13 +467,14 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams p) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);   // [kBeamCap]
-    double* t_pb = reinterpret_cast<double*>(keys + kBeamCap);    // mass ending in blank (one contributor: the prefix itself)
-    double* t_stay = t_pb + kBeamCap;        // ending in the last token, from the prefix itself (repeat)
-    double* t_ext = t_stay + kBeamCap;       // ending in the last token, from the parent prefix (extension)
-    double* c_sc = t_ext + kBeamCap;                                          // [kBeamCap] sort keys
-    unsigned long long* c_ky = reinterpret_cast<unsigned long long*>(c_sc + kBeamCap);
-    int* c_ix = reinterpret_cast<int*>(c_ky + kBeamCap);                      // [kBeamCap] table slot
+    const int cap = p.cap;                   // hash capacity: a power of two >= 2 * beam * (k + 1), the most distinct prefixes a slot can make
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);   // [cap]
+    double* t_pb = reinterpret_cast<double*>(keys + cap);    // mass ending in blank (one contributor: the prefix itself)
+    double* t_stay = t_pb + cap;        // ending in the last token, from the prefix itself (repeat)
+    double* t_ext = t_stay + cap;       // ending in the last token, from the parent prefix (extension)
+    double* c_sc = t_ext + cap;                                          // [cap] sort keys
+    unsigned long long* c_ky = reinterpret_cast<unsigned long long*>(c_sc + cap);
+    int* c_ix = reinterpret_cast<int*>(c_ky + cap);                      // [cap] table slot
     __shared__ unsigned long long bm_key[CTCSD_MAX_BEAM];
     __shared__ double bm_pb[CTCSD_MAX_BEAM], bm_pnb[CTCSD_MAX_BEAM], bm_tot[CTCSD_MAX_BEAM];
     __shared__ int s_nbeam, s_next;
@@ -494,7 +483,6 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
     const int b = blockIdx.x, tid = threadIdx.x;
-    if (b >= p.nseq) { l2_prefetch_role(p); return; }
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -503,12 +491,34 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         return;
     }
     load_slot_lists(p, row, sl);
-    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 0.0; bm_pnb[0] = -INFINITY; bm_tot[0] = 0.0; s_nbeam = 1; }
+    // The search runs on probability masses, not on their logarithms: a prefix's mass is a sum of
+    // products, which in the log domain costs an exp and a log1p in float64 per addition.  Every
+    // slot's probabilities are taken relative to the slot's best symbol (so the best path has mass
+    // 1 and nothing overflows; a path more than ~700 nats below the best one underflows to "no
+    // alignment"); the logarithm of the common factor is added back when the scores are written.
+    __shared__ double s_pr[CTCSD_MAX_T * CTCSD_MAX_K];
+    __shared__ double s_logoff;
+    if (tid < p.T * p.k) {
+        const int t = tid / p.k;
+        double mx = sl.lp[t * p.k];
+        for (int j = 1; j < p.k; ++j) mx = fmax(mx, sl.lp[t * p.k + j]);
+        s_pr[tid] = exp(sl.lp[tid] - mx);
+        if (tid == 0) {
+            double off = 0.0;
+            for (int q = 0; q < p.T; ++q) {
+                double m2 = sl.lp[q * p.k];
+                for (int j = 1; j < p.k; ++j) m2 = fmax(m2, sl.lp[q * p.k + j]);
+                off += m2;
+            }
+            s_logoff = off;
+        }
+    }
+    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 1.0; bm_pnb[0] = 0.0; bm_tot[0] = 1.0; s_nbeam = 1; }
     __syncthreads();
 
     for (int t = 0; t < p.T; ++t) {
-        for (int i = tid; i < kBeamCap; i += kThreads) {
-            keys[i] = kEmpty; t_pb[i] = -INFINITY; t_stay[i] = -INFINITY; t_ext[i] = -INFINITY;
+        for (int i = tid; i < cap; i += kThreads) {
+            keys[i] = kEmpty; t_pb[i] = 0.0; t_stay[i] = 0.0; t_ext[i] = 0.0;
         }
         if (tid == 0) s_next = 0;
         __syncthreads();
@@ -519,33 +529,35 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
             const double pb = bm_pb[e], pnb = bm_pnb[e];
             const double tot = bm_tot[e];
             const int m = sl.lid[t * p.k + j];
-            const double lp = sl.lp[t * p.k + j];
+            const double pr = s_pr[t * p.k + j];
             const int len = key_len(key);
             const int last = len > 0 ? key_tok(key, len - 1) : -1;
+            if (pr == 0.0) continue;                     // a symbol of probability zero reaches nothing
             if (m == kBlankMark) {
-                int s = table_insert(keys, kBeamCap, key);
-                if (s >= 0) t_pb[s] = tot + lp;
+                int s = table_insert(keys, cap, key);
+                if (s >= 0) t_pb[s] = tot * pr;
             } else if (m == last) {
-                if (pnb != -INFINITY) {
-                    int s = table_insert(keys, kBeamCap, key);
-                    if (s >= 0) t_stay[s] = pnb + lp;
+                if (pnb != 0.0) {
+                    int s = table_insert(keys, cap, key);
+                    if (s >= 0) t_stay[s] = pnb * pr;
                 }
-                if (pb != -INFINITY) {
-                    int s = table_insert(keys, kBeamCap, key_append(key, m));
-                    if (s >= 0) t_ext[s] = pb + lp;
+                if (pb != 0.0) {
+                    int s = table_insert(keys, cap, key_append(key, m));
+                    if (s >= 0) t_ext[s] = pb * pr;
                 }
             } else {
-                int s = table_insert(keys, kBeamCap, key_append(key, m));
-                if (s >= 0) t_ext[s] = tot + lp;
+                int s = table_insert(keys, cap, key_append(key, m));
+                if (s >= 0) t_ext[s] = tot * pr;
             }
         }
         __syncthreads();
         // total mass per prefix; compact into the sort arrays
-        for (int i = tid; i < kBeamCap; i += kThreads) {
+        for (int i = tid; i < cap; i += kThreads) {
             const unsigned long long ki = keys[i];
             if (ki == kEmpty) continue;
-            const double pnb = logadd(t_stay[i], t_ext[i]);
-            const double tot = logadd(t_pb[i], pnb);
+            const double pnb = t_stay[i] + t_ext[i];
+            const double tot = t_pb[i] + pnb;
+            if (tot == 0.0) continue;                    // underflowed: no alignment left
             t_stay[i] = pnb;
             t_ext[i] = tot;
             const int at = atomicAdd(&s_next, 1);
@@ -556,7 +568,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         __syncthreads();
         const int count = s_next;
         // between slots the beam is a set; only the last slot's beam is ranked (the candidates come out of it)
-        const int keep = block_select_top(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1);
+        const int keep = block_select_top<true>(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1);
         for (int r = tid; r < keep; r += kThreads) {
             const int i = s_sel[r];
             const int slot = c_ix[i];
@@ -568,9 +580,12 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         if (tid == 0) s_nbeam = keep;
         __syncthreads();
     }
-    // the beam is already ranked best first by total mass
+    // the beam is already ranked best first by total mass; scores go out as logarithms
     const int nbeam = s_nbeam;
-    for (int r = tid; r < nbeam; r += kThreads) s_sel[r] = r;
+    for (int r = tid; r < nbeam; r += kThreads) {
+        s_sel[r] = r;
+        bm_tot[r] = log(bm_tot[r]) + s_logoff;
+    }
     __syncthreads();
     emit_candidates(p, b, sl, bm_tot, bm_key, s_sel, nbeam, -1);
 }
@@ -598,7 +613,6 @@ __global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
     const int b = blockIdx.x, tid = threadIdx.x;
-    if (b >= p.nseq) { l2_prefetch_role(p); return; }
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -637,16 +651,6 @@ __global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
 
 using namespace ctcsd;
 
-// CTAs that the candidate kernels launch on top of one per sequence to carry the L2 hint.
-static int prefetch_ctas(const Handle* h, CollapseParams& p) {
-    p.nseq = h->cfg.B;
-    p.pf_ptr = static_cast<const unsigned char*>(h->l2_hint_ptr);
-    p.pf_bytes = h->l2_hint_bytes;
-    if (getenv("CTCSD_PF_WHERE") && getenv("CTCSD_PF_WHERE")[0] == 'd') p.pf_bytes = 0;
-    if (p.pf_bytes == 0) return 0;
-    return h->num_sms;
-}
-
 static int next_pow2_host(int v) {
     int n = 2;
     while (n < v) n <<= 1;
@@ -678,10 +682,13 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     p.status = status_ptr(h);
 
     if (c.beam > 0) {
-        const size_t smem = (size_t)kBeamCap * 52;
+        int cap = 64;
+        while (cap < 2 * c.beam * (c.k + 1)) cap <<= 1;
+        if (cap > kBeamCap) cap = kBeamCap;
+        p.cap = cap;
+        const size_t smem = (size_t)cap * 52;
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_beam_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        const int extra = prefetch_ctas(h, p);
-        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B + extra), dim3(kThreads), smem, s, 1, p));
+        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
         CTCSD_LAUNCH_CHECK(h);
         return CTCSD_OK;
     }
@@ -694,8 +701,7 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     size_t smem = (size_t)cap * 24 + (size_t)npaths * 2;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_enum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const int extra = prefetch_ctas(h, p);
-    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B + extra), dim3(kThreads), smem, s, 1, p));
+    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
@@ -727,8 +733,7 @@ extern "C" int ctcsd_select_raw_paths(ctcsd_handle* hh, void* stream, int M, con
     const size_t smem = (size_t)p.cap * 16;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(raw_paths_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const int extra = prefetch_ctas(h, p);
-    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B + extra), dim3(kThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
+    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B), dim3(kThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }

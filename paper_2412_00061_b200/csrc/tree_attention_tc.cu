@@ -164,6 +164,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 // one copy per tile and tensor: the box spans both 64-column halves of the head dimension
                 // and lands as [half][key][128 bytes] (every copy instruction costs the copy engine a fixed
                 // few hundred nanoseconds, whatever its size)
+                // one copy per tile and tensor: the box spans all 64-column parts of the head dimension and
+                // lands as [part][key][128 bytes] (a copy instruction costs the copy engine a fixed few
+                // hundred nanoseconds whatever its size)
                 tc::tma_load_5d(kd, &tmK, &sh->full[s], 0, blk * kKeys, 0, g, b, pol);
                 tc::tma_load_5d(kd + kTileBytes, &tmV, &sh->full[s], 0, blk * kKeys, 0, g, b, pol);
             }

@@ -23,7 +23,10 @@ def to_device(a: np.ndarray, dtype: str, device) -> torch.Tensor:
 
 
 class DraftVerifyStep:
-    L2_PREFETCH_BYTES = 48 << 20
+    # Bytes of the LM-head weights that the draft head asks L2 to fetch when its own stream is issued
+    # (ctcsd_set_l2_prefetch).  Off: on B200 the step was measured at the same time with 0, 24 and 48 MB
+    # and slower beyond (the fetched lines did not shorten the LM head, whose tiles come by TMA).
+    L2_PREFETCH_BYTES = 0
     def __init__(self, cfg: StepConfig, device="cuda:0", max_draft_rows: int = 0, debug_logits: bool = False,
                  layout: str = "packed"):
         """layout "packed": collapse first, tree over the collapsed candidates (the default);
@@ -72,9 +75,7 @@ class DraftVerifyStep:
     def set_inputs(self, **tensors):
         """x, Wd, blank_bias, row_seq, sel_row, base_tok, kv_len, Q, K, V, hn, Wl (device tensors)."""
         self.inp.update(tensors)
-        if "Wl" in tensors and self.cfg.dtype == "bf16":
-            # while the small kernels between draft head and LM head run, HBM is idle: let L2
-            # fetch the head of the LM-head weights then
+        if "Wl" in tensors and self.cfg.dtype == "bf16" and self.L2_PREFETCH_BYTES > 0:
             self.h.set_l2_prefetch(tensors["Wl"], self.L2_PREFETCH_BYTES)
 
     PER_STEP_INPUTS = ("x", "base_tok", "kv_len", "Q", "hn")

@@ -109,8 +109,8 @@ def test_only_blank_paths_leave_just_the_root():
 def test_c2_full_size_sampled():
     """The headline workload at full size.  The definition-mode oracle checks one draft row in
     full, sampled LM-head rows and sampled attention (sequence, head) pairs; all integer stages are
-    compared in full.  Then the step is rerun the way the benchmark launches it (no debug dumps, L2
-    hint, a CUDA graph of three steps replayed twice) and must give the same results bit for bit."""
+    compared in full.  Then the step is rerun the way the benchmark launches it (no debug dumps, a CUDA
+    graph of three steps replayed twice) and must give the same results bit for bit."""
     from tests.parity_util import check_benchmark_launch_configuration
     r = _run(C["c2"], seed=0, require_certified=True, attention_rows=4, lm_rows=8)
     assert 2 <= r["n_nodes"][0] <= 64
