@@ -461,18 +461,14 @@ def run_ours(args):
         # one graph per step: the copy in from pinned memory, the five calls, the copy out
         with torch.cuda.stream(side):
             with torch.cuda.graph(graph1, stream=side):
-                step.upload(h_in)
-                step.run()
-                step.download(h_out)
+                step.run_from_host(h_in, h_out)
         torch.cuda.synchronize()
 
     def e2e_step():
         if graph1 is not None:
             graph1.replay()
         else:
-            step.upload(h_in)
-            step.run()
-            step.download(h_out)
+            step.run_from_host(h_in, h_out)
         torch.cuda.synchronize()
 
     for _ in range(3):

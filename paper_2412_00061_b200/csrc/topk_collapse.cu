@@ -65,6 +65,19 @@ __device__ __forceinline__ int table_insert(unsigned long long* keys, int cap, u
     return -1;
 }
 
+// Appends to a list whose length is one shared counter: the lanes of a warp that have something
+// to append are counted with one ballot and claim their places with ONE atomic (hundreds of
+// threads incrementing the same shared word one by one is what a list build otherwise costs).
+// Every lane of the warp must call it; returns the place of this lane's item (if `has`).
+__device__ __forceinline__ int warp_append(int* counter, bool has) {
+    const unsigned m = __ballot_sync(0xffffffffu, has);
+    const int lane = threadIdx.x & 31;
+    int base = 0;
+    if (lane == 0 && m != 0u) base = atomicAdd(counter, __popc(m));
+    base = __shfl_sync(0xffffffffu, base, 0);
+    return base + __popc(m & ((1u << lane) - 1u));
+}
+
 __device__ __forceinline__ long long dbl_sortable(double d) {
     long long v = __double_as_longlong(d);
     return v ^ ((v >> 63) & 0x7fffffffffffffffll);
@@ -261,11 +274,19 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
             return need;
         }
         // gather definite winners (above the threshold) and the entries on it
-        for (int i = tid; i < count; i += kThreads) {
-            const unsigned f = select_image<MASS>(sc[i]);
-            const unsigned top = lo < 32 ? (f >> lo) : 0u;
-            if (top > thr) S.win[atomicAdd(&S.nwin, 1)] = i;
-            else if (top == thr) S.cand[atomicAdd(&S.ccnt, 1)] = i;
+        for (int i0 = 0; i0 < count; i0 += kThreads) {          // the same trip count for every thread
+            const int i = i0 + tid;
+            bool is_win = false, is_cand = false;
+            if (i < count) {
+                const unsigned f = select_image<MASS>(sc[i]);
+                const unsigned top = lo < 32 ? (f >> lo) : 0u;
+                is_win = top > thr;
+                is_cand = top == thr;
+            }
+            const int aw = warp_append(&S.nwin, is_win);
+            const int ac = warp_append(&S.ccnt, is_cand);
+            if (is_win) S.win[aw] = i;
+            if (is_cand) S.cand[ac] = i;
         }
         __syncthreads();
         // exact ranking among the threshold entries: one warp per entry, its lanes share the
@@ -447,11 +468,13 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     // because the empty sequence may be among them) and write them out
     double* c_sc = reinterpret_cast<double*>(fsum);                     // [cap/2]
     unsigned long long* c_ky = fsum + (p.cap >> 1);                     // [cap/2]
-    for (int i = tid; i < p.cap; i += kThreads) {
-        const unsigned long long ki = keys[i];
-        if (ki == kEmpty) continue;
-        const double si = score[i];
-        const int at = atomicAdd(&s_count, 1);
+    for (int i0 = 0; i0 < p.cap; i0 += kThreads) {
+        const int i = i0 + tid;
+        const unsigned long long ki = i < p.cap ? keys[i] : kEmpty;
+        const bool has = ki != kEmpty;
+        const double si = has ? score[i] : 0.0;
+        const int at = warp_append(&s_count, has);
+        if (!has) continue;
         if (ki == 0ull) s_has_empty = 1;
         c_sc[at] = si;
         c_ky[at] = ki;
@@ -552,15 +575,19 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         }
         __syncthreads();
         // total mass per prefix; compact into the sort arrays
-        for (int i = tid; i < cap; i += kThreads) {
-            const unsigned long long ki = keys[i];
-            if (ki == kEmpty) continue;
-            const double pnb = t_stay[i] + t_ext[i];
-            const double tot = t_pb[i] + pnb;
-            if (tot == 0.0) continue;                    // underflowed: no alignment left
+        for (int i0 = 0; i0 < cap; i0 += kThreads) {
+            const int i = i0 + tid;
+            const unsigned long long ki = i < cap ? keys[i] : kEmpty;
+            double pnb = 0.0, tot = 0.0;
+            if (ki != kEmpty) {
+                pnb = t_stay[i] + t_ext[i];
+                tot = t_pb[i] + pnb;
+            }
+            const bool has = tot != 0.0;                 // (a mass that underflowed has no alignment left)
+            const int at = warp_append(&s_next, has);
+            if (!has) continue;
             t_stay[i] = pnb;
             t_ext[i] = tot;
-            const int at = atomicAdd(&s_next, 1);
             c_sc[at] = tot;
             c_ky[at] = ki;
             c_ix[at] = i;

@@ -97,11 +97,38 @@ class DraftVerifyStep:
             view.copy_(t)
             self.inp[k] = view
             off += sz
+        # x, base_tok and kv_len come first: the draft head and the tree need them; Q and hn are
+        # needed only from the attention on
+        self.early_bytes = sum(sz for k, _, sz in sizes if k in ("x", "base_tok", "kv_len"))
         torch.cuda.synchronize(self.device)
         return self.input_arena.cpu().pin_memory()
 
     def upload(self, host_arena: torch.Tensor):
         self.input_arena.copy_(host_arena, non_blocking=True)
+
+    def run_from_host(self, host_arena: torch.Tensor, host_result: torch.Tensor):
+        """One step end to end on the current stream: every per-step input is copied from the pinned
+        host mirror, the five calls run, the result goes back to pinned host memory.  The copy of
+        the tree queries and tree-node hidden states (the bulk of the bytes) runs on a second stream
+        beside the draft head, which does not read them, and joins before the attention."""
+        cur = torch.cuda.current_stream(self.device)
+        if not hasattr(self, "_copy_stream"):
+            self._copy_stream = torch.cuda.Stream(device=self.device)
+        e = self.early_bytes
+        fork, join = torch.cuda.Event(), torch.cuda.Event()
+        fork.record(cur)
+        self._copy_stream.wait_event(fork)
+        with torch.cuda.stream(self._copy_stream):
+            self.input_arena[e:].copy_(host_arena[e:], non_blocking=True)
+            join.record(self._copy_stream)
+        self.input_arena[:e].copy_(host_arena[:e], non_blocking=True)
+        self.draft()
+        self.collapse()
+        self.tree()
+        cur.wait_event(join)
+        self.attention()
+        self.verify()
+        self.download(host_result)
 
     def download(self, host_result: torch.Tensor):
         host_result.copy_(self.result, non_blocking=True)
