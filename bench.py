@@ -320,6 +320,47 @@ def chain_tokens_per_s(args, cfg, step, inp, seed, torch, to_device, synth):
             "us_per_step": sec * 1e6 / n, "includes": "torch scatter standing in for the base model's K/V write of the tree rows"}
 
 
+def draft_module_time(args, cfg, step, seed, torch, to_device, synth):
+    """--draft-module: the paper's attention draft module (one decoder layer before the draft head,
+    Sec. 3.1) at the workload's shape with a LLaMA-style MLP width, timed alone (20 calls per CUDA
+    graph).  Reports its time, the weight bytes it streams and its share of (layer + step), the
+    figure the paper gives for its own drafter (Sec. 4.3)."""
+    dev = step.device
+    I = {4096: 11008, 5120: 13824, 8192: 28672}.get(cfg.H, (cfg.H * 8 // 3 + 255) // 256 * 256)
+    R = cfg.T + 1
+    w, F_new, n_new, kv_len, Kd, Vd = synth.gen_draft_layer(cfg, seed, I, R, cfg.kv_lo, cfg.kv_hi)
+    td = lambda a: to_device(a, cfg.dtype, dev)
+    f32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float32)).to(dev)
+    i32 = lambda a: torch.from_numpy(np.asarray(a, dtype=np.int32)).to(dev)
+    dl = step.h.make_draft_layer(f32(w["g1"]), td(w["Wqkv"]), td(w["Wo"]), f32(w["g2"]), td(w["Wgu"]), td(w["Wdn"]), R=R)
+    act = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    args_d = (dl, td(F_new), i32(n_new), i32(kv_len), td(Kd), td(Vd), torch.zeros(cfg.B, cfg.H, dtype=act, device=dev),
+              torch.zeros(cfg.B, dtype=torch.int32, device=dev))
+    fn = lambda: step.h.draft_module(*args_d)
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(20):
+                fn()
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+    step.check_status()
+    us = e0.elapsed_time(e1) * 1e3 / 200
+    esz = 2 if cfg.dtype == "bf16" else 4
+    wbytes = esz * (((cfg.Hq + 2 * cfg.Hkv) * cfg.D + cfg.Hq * cfg.D) * cfg.H + 3 * I * cfg.H)
+    return {"us": us, "mlp_width": I, "new_rows": R, "weight_bytes": wbytes, "GBps": wbytes / us / 1e3}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -533,6 +574,11 @@ def run_ours(args):
             line["stages_us"] = {k: round(v, 2) for k, v in st.items()}
             line["stages_roofline_us"] = {k: round(v, 2) for k, v in rf.items()}
             line["stages_frac"] = {k: round(rf[k] / st[k], 3) for k in rf}
+        if args.draft_module and world == 1:
+            dm = draft_module_time(args, cfg, step, seed, torch, to_device, synth)
+            dm["share_of_layer_plus_step"] = dm["us"] / (dm["us"] + ms / K * 1e3)
+            dm["frac_of_%s_hbm_peak" % peak_kind] = dm["GBps"] / peak
+            line["draft_module"] = dm
         if args.chain > 0 and world == 1:
             line["chain"] = chain_tokens_per_s(args, cfg, step, inp, seed, torch, to_device, synth)
         if world == 1 and not args.no_cpu_baseline:
@@ -572,6 +618,8 @@ def main():
                     help="draft weights that make neighbouring slots favour the same tokens, so that repeats and merges occur")
     ap.add_argument("--blank-bias", type=float, default=None, help="blank-logit bias for every sequence (default: the workload's)")
     ap.add_argument("--stage-times", action="store_true", help="add per-call device times and their roofline times to the line")
+    ap.add_argument("--draft-module", action="store_true",
+                    help="also time the paper's attention draft module (one decoder layer before the draft head)")
     ap.add_argument("--chain", type=int, default=0, help="also time N chained steps (history update after each); adds tokens/s")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:

@@ -107,6 +107,11 @@ const char* ctcsd_strerror(int status);
 /* cudaError_t value of the most recent failing CUDA call made through handle `h` (0 if none). */
 int ctcsd_last_cuda_error(const ctcsd_handle* h);
 
+/* 1 when the library was built with -DCTCSD_DEBUG_BOUNDS (the kernels then check the index of
+ * every store into a caller's array or an internal list, record CTCSD_ERR_INTERNAL with
+ * 1000 + the site number in the device status word and skip the store), else 0. */
+int ctcsd_debug_bounds_enabled(void);
+
 /* Number of kernels this handle has launched since creation (for launch accounting). */
 long long ctcsd_launch_count(const ctcsd_handle* h);
 

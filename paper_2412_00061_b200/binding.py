@@ -21,7 +21,7 @@ SCORE_SUM, SCORE_MAX = 0, 1
 
 EXPORTS = [
     "ctcsd_workspace_bytes", "ctcsd_create", "ctcsd_destroy", "ctcsd_poll_status", "ctcsd_strerror",
-    "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
+    "ctcsd_last_cuda_error", "ctcsd_launch_count", "ctcsd_debug_bounds_enabled", "ctcsd_set_l2_prefetch", "ctcsd_selftest_timeout",
     "ctcsd_draft_logits", "ctcsd_topk_collapse", "ctcsd_build_tree", "ctcsd_tree_attention",
     "ctcsd_verify_accept", "ctcsd_commit_accepted", "ctcsd_tree_attention_static", "ctcsd_draft_logits_rows",
     "ctcsd_verify_accept_sampled", "ctcsd_draft_module_workspace_bytes", "ctcsd_draft_module",
@@ -67,6 +67,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ctcsd_last_cuda_error.argtypes = [vp]
     lib.ctcsd_set_l2_prefetch.argtypes = [vp, vp, cs]
     lib.ctcsd_selftest_timeout.argtypes = [vp, vp]
+    lib.ctcsd_debug_bounds_enabled.argtypes = []
     lib.ctcsd_launch_count.argtypes = [vp]
     lib.ctcsd_launch_count.restype = ctypes.c_longlong
     lib.ctcsd_draft_logits.argtypes = [vp, vp, ci] + [vp] * 8
@@ -90,6 +91,17 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     if path is None:
         _lib = lib
     return lib
+
+
+def use_library(path: Optional[str]) -> ctypes.CDLL:
+    """Makes `path` (for example the debug-bounds build) the library that new handles use; None goes
+    back to the regular build."""
+    global _lib
+    _lib = None
+    if path is None:
+        return load_library()
+    _lib = load_library(path)
+    return _lib
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, numel: Optional[int] = None, name: str = "") -> Optional[int]:

@@ -34,14 +34,23 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(f) for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compiles every .cu under csrc/ and links libctcsd.so next to this file.
-    Returns the library path.  Rebuilds only when a source is newer than the library."""
+LIB_DEBUG = os.path.join(PKG, "libctcsd_dbg.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """Compiles every .cu under csrc/ and links libctcsd.so next to this file (with
+    debug_bounds=True: libctcsd_dbg.so, the same code with -DCTCSD_DEBUG_BOUNDS, whose kernels check
+    every output index).  Returns the library path.  Rebuilds only when a source is newer than
+    the library."""
+    LIB = LIB_DEBUG if debug_bounds else globals()["LIB"]
+    OBJ = globals()["OBJ"] + ("_dbg" if debug_bounds else "")
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
         return LIB
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
+    if debug_bounds:
+        extra.append("-DCTCSD_DEBUG_BOUNDS")
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
@@ -63,4 +72,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

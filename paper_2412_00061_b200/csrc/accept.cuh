@@ -14,6 +14,7 @@ struct AcceptParams {
     // kept[b,i] != 0 marks the survivors, nka[b,i] is the nearest kept proper ancestor.  Null for
     // the packed tree.
     const int* kept; const int* nka;
+    int* status;             // device status word
 };
 
 #ifdef __CUDACC__
@@ -99,7 +100,7 @@ __device__ __forceinline__ void accept_warp(const AcceptParams& p, int b, int la
         const unsigned e = s_best[cur];
         if ((e >> 16) == 0u) break;
         const int nxt = (int)(0xffffu - (e & 0xffffu));
-        if (lane == 0) {
+        if (lane == 0 && CTCSD_IN_BOUNDS(p.status, 20, nxt, n_max)) {
             p.acc_nodes[(size_t)b * p.T + len] = nxt;
             p.acc_tok[(size_t)b * p.T + len] = s_am[cur];      // an agreeing node's token is the arg-max before it
         }

@@ -24,6 +24,7 @@ struct TreeParams {
     // raw layout (Sec. 3.3): candidates are full-length slot paths (cand_len null), the blank is
     // a symbol like any other in the trie, and kept/nka/mask/pos describe the CTC transform
     int* kept; int* nka; int blank;
+    int* status;
 };
 
 __device__ __forceinline__ int warp_excl_scan(int v, int lane, int& total) {
@@ -165,7 +166,7 @@ __global__ void __launch_bounds__(32) build_tree_kernel(TreeParams p) {
                     if (node >= n_max) node = -1;
                 }
                 if (c < N) p.retrieve[((size_t)b * N + c) * T + l] = node;
-                if (node >= 0) {
+                if (node >= 0 && CTCSD_IN_BOUNDS(p.status, 10, node, n_max)) {
                     anc.add(node);
                     if (o == c) {                          // this candidate creates the node
                         o_tok[node] = tok[h][l];
@@ -243,6 +244,7 @@ extern "C" int ctcsd_build_tree(ctcsd_handle* hh, void* stream, const int* base_
     p.base_tok = base_tok; p.kv_len = kv_len;
     p.cand_tok = cand_tok; p.cand_len = cand_len; p.n_cand = n_cand;
     p.T = c.T; p.topN = c.topN; p.max_nodes = c.max_nodes;
+    p.status = status_ptr(h);
     p.node_tok = out_node_tok; p.parent = out_parent; p.depth = out_depth; p.pos = out_pos;
     p.mask = out_mask; p.retrieve = out_retrieve; p.n_nodes = out_n_nodes;
     p.kept = nullptr; p.nka = nullptr; p.blank = c.V;
@@ -265,6 +267,7 @@ extern "C" int ctcsd_build_raw_tree(ctcsd_handle* hh, void* stream, const int* b
     p.base_tok = base_tok; p.kv_len = kv_len;
     p.cand_tok = raw_tok; p.cand_len = nullptr; p.n_cand = n_raw;
     p.T = c.T; p.topN = c.topN; p.max_nodes = c.max_nodes;
+    p.status = status_ptr(h);
     p.node_tok = out_node_tok; p.parent = out_parent; p.depth = out_depth; p.pos = out_pos;
     p.mask = out_mask; p.retrieve = out_retrieve; p.n_nodes = out_n_nodes;
     p.kept = out_kept; p.nka = out_nka; p.blank = c.V;

@@ -205,6 +205,22 @@ __device__ __forceinline__ void report_error(int* status, int code, int detail) 
     if (atomicCAS(status, 0, code) == 0) status[1] = detail;
 }
 
+// Debug build (-DCTCSD_DEBUG_BOUNDS): an index check at the places where a kernel forms the index
+// of a store into a caller's array or into a list in shared memory.  A check that fails records
+// CTCSD_ERR_INTERNAL and 1000 + the site number in the device status word and the store is
+// skipped; nothing traps.  In the normal build the checks compile to nothing (the production
+// guards - clamped counts, `row < M` tests and the like - are always there).
+#ifdef CTCSD_DEBUG_BOUNDS
+__device__ __forceinline__ bool debug_in_bounds(int* status, int site, long long idx, long long n) {
+    if (idx >= 0 && idx < n) return true;
+    if (status != nullptr) report_error(status, CTCSD_ERR_INTERNAL, 1000 + site);
+    return false;
+}
+#define CTCSD_IN_BOUNDS(status, site, idx, n) ctcsd::debug_in_bounds((status), (site), (long long)(idx), (long long)(n))
+#else
+#define CTCSD_IN_BOUNDS(status, site, idx, n) true
+#endif
+
 #endif  // __CUDACC__
 
 }  // namespace ctcsd

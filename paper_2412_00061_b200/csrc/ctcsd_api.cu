@@ -147,6 +147,14 @@ extern "C" const char* ctcsd_strerror(int status) {
     }
 }
 
+extern "C" int ctcsd_debug_bounds_enabled(void) {
+#ifdef CTCSD_DEBUG_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 extern "C" int ctcsd_last_cuda_error(const ctcsd_handle* h) { return h ? h->h.last_cuda_error : 0; }
 
 extern "C" long long ctcsd_launch_count(const ctcsd_handle* h) { return h ? h->h.launches : 0; }

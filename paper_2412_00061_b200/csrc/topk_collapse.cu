@@ -199,7 +199,7 @@ __device__ __forceinline__ int next_pow2(int v) {
 // and sel[] becomes the identity.
 template <bool MASS = false>
 __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int count, int need, int* sel,
-                                SelectScratch& S, bool ordered = true) {
+                                SelectScratch& S, bool ordered = true, int* status = nullptr) {
     const int tid = threadIdx.x, lane = tid & 31;
     if (need > count) need = count;
     if (tid == 0) { S.fmax = 0u; S.fmin = 0xffffffffu; S.nwin = 0; S.ncand = 0; S.ccnt = 0; }
@@ -285,8 +285,8 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
             }
             const int aw = warp_append(&S.nwin, is_win);
             const int ac = warp_append(&S.ccnt, is_cand);
-            if (is_win) S.win[aw] = i;
-            if (is_cand) S.cand[ac] = i;
+            if (is_win && CTCSD_IN_BOUNDS(status, 5, aw, CTCSD_MAX_BEAM + 8)) S.win[aw] = i;
+            if (is_cand && CTCSD_IN_BOUNDS(status, 6, ac, kSelMax)) S.cand[ac] = i;
         }
         __syncthreads();
         // exact ranking among the threshold entries: one warp per entry, its lanes share the
@@ -353,6 +353,7 @@ __device__ void emit_candidates(const CollapseParams& p, int b, const SlotLists&
         if (rank >= p.topN) continue;
         const unsigned long long key = ky[sel[e]];
         const int len = key_len(key);
+        if (!CTCSD_IN_BOUNDS(p.status, 1, rank, p.topN) || !CTCSD_IN_BOUNDS(p.status, 2, len, p.T + 1)) continue;
         clen[rank] = len;
         cscore[rank] = (float)sc[sel[e]];
         for (int l = 0; l < len; ++l) ctok[rank * p.T + l] = sl.sorted_tok[key_tok(key, l)];
@@ -474,14 +475,14 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
         const bool has = ki != kEmpty;
         const double si = has ? score[i] : 0.0;
         const int at = warp_append(&s_count, has);
-        if (!has) continue;
+        if (!has || !CTCSD_IN_BOUNDS(p.status, 4, at, p.cap >> 1)) continue;
         if (ki == 0ull) s_has_empty = 1;
         c_sc[at] = si;
         c_ky[at] = ki;
     }
     __syncthreads();
     const int count = s_count;
-    const int nsel = block_select_top(c_sc, c_ky, nullptr, count, p.topN + 1, s_sel, S);
+    const int nsel = block_select_top(c_sc, c_ky, nullptr, count, p.topN + 1, s_sel, S, true, p.status);
     emit_candidates(p, b, sl, c_sc, c_ky, s_sel, nsel, count - s_has_empty);
 }
 
@@ -585,7 +586,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
             }
             const bool has = tot != 0.0;                 // (a mass that underflowed has no alignment left)
             const int at = warp_append(&s_next, has);
-            if (!has) continue;
+            if (!has || !CTCSD_IN_BOUNDS(p.status, 3, at, cap)) continue;
             t_stay[i] = pnb;
             t_ext[i] = tot;
             c_sc[at] = tot;
@@ -595,7 +596,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
         __syncthreads();
         const int count = s_next;
         // between slots the beam is a set; only the last slot's beam is ranked (the candidates come out of it)
-        const int keep = block_select_top<true>(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1);
+        const int keep = block_select_top<true>(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1, p.status);
         for (int r = tid; r < keep; r += kThreads) {
             const int i = s_sel[r];
             const int slot = c_ix[i];
@@ -659,7 +660,7 @@ __global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
     for (int i = tid; i < p.topN * p.T; i += kThreads) rtok[i] = -1;
     for (int i = tid; i < p.topN; i += kThreads) rscore[i] = -INFINITY;
     __syncthreads();
-    const int nsel = block_select_top(sc, ky, nullptr, p.npaths, p.topN, s_sel, S);
+    const int nsel = block_select_top(sc, ky, nullptr, p.npaths, p.topN, s_sel, S, true, p.status);
     for (int e = tid; e < nsel; e += kThreads) {
         const int at = s_sel[e];
         unsigned rem = (unsigned)ky[at];

@@ -28,7 +28,7 @@ constexpr int kSoftmaxWarps = 8;     // two per quarter of the TMEM lanes
 constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
 constexpr int kRows = 128;         // query rows per CTA
 constexpr int kKeys = 128;         // keys per tile
-constexpr int kStages = 2;         // K/V tile buffers
+constexpr int kStages = 3;         // K/V tile buffers: the tile in use, and two on their way
 constexpr float kSlack = 8.f;      // how far (log2 units) the row maximum may run ahead of the exponent's reference
 
 struct __align__(8) AttnShared {
@@ -41,7 +41,7 @@ struct __align__(8) AttnShared {
     uint32_t tmem_base;
     int abort_flag;
     int never_set;
-    float xch[3][2][kRows];        // row maxima (two tile parities) and row sums exchanged between a row's two threads
+    float xch[2][2][kRows];        // row maxima (two tile parities; the row sums at the end take the free parity) exchanged between a row's two threads
 };
 
 // The two softmax warps that share a quarter of the TMEM lanes (64 threads) meet here.
@@ -89,13 +89,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     constexpr int RS = D + 4;                      // floats per row of the merge buffer
     constexpr int PER = D / 32;
     constexpr int DO = D / 2;                      // O columns per softmax thread
-    extern __shared__ unsigned char dyn_raw[];
-    const uint32_t raw_addr = tc::smem_u32(dyn_raw);
-    unsigned char* dyn = dyn_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+    // The tiles need 1024-byte alignment (128-byte swizzle); with three 64 KB stages there is no room
+    // left for an alignment pad, so the alignment is asked for and checked.
+    extern __shared__ __align__(1024) unsigned char dyn[];
     unsigned char* Qs = dyn;                                           // [DH][128 rows][128 B]
     unsigned char* KV = Qs + kQBytes;                                  // [kStages][K tile | V tile]
-    unsigned char* Ps = KV + kStages * 2 * kTileBytes;                 // [2][128 rows][128 B]
-    AttnShared* sh = reinterpret_cast<AttnShared*>(Ps + kPBytes);
+    // P (128 rows x 128 keys of bf16 = 32 KB) has the shape of a K tile with D = 128, and by the time
+    // it is written the tile's K has served its purpose (S is complete): P takes K's place in the
+    // stage.  With D = 64 a K tile is half that size and P has a buffer of its own.
+    constexpr bool kPInK = (kTileBytes >= kPBytes);
+    unsigned char* Ps_own = KV + kStages * 2 * kTileBytes;             // [2][128 rows][128 B], D = 64 only
+    AttnShared* sh = reinterpret_cast<AttnShared*>(Ps_own + (kPInK ? 0 : kPBytes));
+    auto p_tile = [&](int s) -> unsigned char* { return kPInK ? KV + (size_t)s * 2 * kTileBytes : Ps_own; };
+    if ((tc::smem_u32(dyn) & 1023u) != 0u) {                           // uniform over the CTA (and its cluster)
+        if (threadIdx.x == 0) report_error(p.status, CTCSD_ERR_INTERNAL, 24);
+        return;
+    }
 
     const int grp = p.Hq / p.Hkv;
     const int qtile = blockIdx.x / splits, split = blockIdx.x - qtile * splits;
@@ -212,7 +221,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 tc::tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < kKeys / 16; ++kk) {
-                    const uint64_t adesc = tc::smem_desc_k_sw128(tc::smem_u32(Ps) + (kk / 4) * (kRows * 128)) + 2 * (kk % 4);
+                    const uint64_t adesc = tc::smem_desc_k_sw128(tc::smem_u32(p_tile(s)) + (kk / 4) * (kRows * 128)) + 2 * (kk % 4);
                     // 16 keys further along K = 16 rows of 128 bytes
                     const uint64_t bdesc = tc::smem_desc_mn_sw128(v_addr + kk * (16 * 128), kKeys * 128);
                     tc::mma_bf16_ss(tmem_o, adesc, bdesc, idesc_o, (it | kk) != 0 ? 1u : 0u);   // O accumulates over the tiles
@@ -347,7 +356,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                     pv[j] = ((vm >> j) & 1u) ? e : 0.f;
                     ps4[j & 3] += pv[j];
                 }
-                unsigned char* prow = Ps + (c0 / 64) * (kRows * 128) + rl * 128;
+                unsigned char* prow = p_tile(s) + (c0 / 64) * (kRows * 128) + rl * 128;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint4 w;
@@ -382,9 +391,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             tc::tc_fence_before_sync();
         }
         // the row's sum is the two halves' sums (both were kept against the same running maximum)
-        sh->xch[2][half][rl] = sum;
+        // (the parity the last tile did not use: its previous readers passed a later barrier since)
+        sh->xch[ntile & 1][half][rl] = sum;
         pair_barrier(q);
-        sum += sh->xch[2][half ^ 1][rl];
+        sum += sh->xch[ntile & 1][half ^ 1][rl];
         if (failed && lane == 0) {
             if (*abort_flag == 0) report_error(p.status, CTCSD_ERR_TIMEOUT, 23);
             *abort_flag = 1;
@@ -555,8 +565,8 @@ int launch_tc(Handle* h, cudaStream_t s, const AttnParams& p) {
         if (!make_map_nd(&tmK, p.K, 5, dims, str, box)) return CTCSD_ERR_CUDA;
         if (!make_map_nd(&tmV, p.V, 5, dims, str, box)) return CTCSD_ERR_CUDA;
     }
-    const size_t smem = (size_t)kRows * D * 2 + (size_t)kStages * 2 * kKeys * D * 2 + (size_t)kRows * kKeys * 2 +
-                        sizeof(AttnShared) + 1024;
+    const size_t smem = (size_t)kRows * D * 2 + (size_t)kStages * 2 * kKeys * D * 2 +
+                        ((size_t)kKeys * D * 2 >= (size_t)kRows * kKeys * 2 ? 0 : (size_t)kRows * kKeys * 2) + sizeof(AttnShared);
     auto kern = tree_attention_tc_kernel<D>;
     CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     CTCSD_CUDA_CHECK(h, launch_pdl(kern, dim3(qtiles * splits, p.Hkv, p.B), dim3(kThreads), smem, s, splits,

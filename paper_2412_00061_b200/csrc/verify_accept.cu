@@ -34,6 +34,7 @@ static int verify_accept_common(ctcsd_handle* hh, void* stream, const void* hn, 
     a.B = c.B; a.T = c.T; a.max_nodes = c.max_nodes;
     a.acc_len = out_acc_len; a.acc_nodes = out_acc_nodes; a.acc_tok = out_acc_tok; a.next_tok = out_next_tok;
     a.kept = kept; a.nka = nka;
+    a.status = status_ptr(h);
     SampleNoise sn;
     sn.noise = noise; sn.depth = depth; sn.max_nodes = c.max_nodes; sn.rows_per_seq = c.T + 1; sn.inv_temp = inv_temp;
 

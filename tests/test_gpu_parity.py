@@ -275,6 +275,8 @@ DM = {
     "dm_gqa": (C["c5"].replace(name="dm_gqa", B=3, H=768, V=999, Hq=12, Hkv=4, D=64), 2048, 7, (0, 200)),
     "dm_fp32": (C["c1"].replace(name="dm_fp32", B=2, H=256, V=999, Hq=4, Hkv=2, D=64), 688, 5, (3, 90)),
     "dm_long_inner": (C["c2"].replace(name="dm_long_inner", B=3, H=256, V=999, Hq=2, Hkv=2, D=128), 11008, 3, (10, 50)),
+    # the 7B shape: hidden 4096, 32 heads x 128, MLP width 11008, six new rows on top of ~1000 cached positions
+    "dm_7b": (C["c2"].replace(name="dm_7b", V=999), 11008, 6, (900, 1024)),
 }
 
 
