@@ -626,14 +626,20 @@ def rope_rotate(v: np.ndarray, pos: int, theta: float) -> np.ndarray:
 
 
 def draft_module(F_new: np.ndarray, n_new: np.ndarray, kv_len: np.ndarray, Kd: np.ndarray, Vd: np.ndarray,
-                 w: dict, Hq: int, Hkv: int, D: int, eps: float = 1e-5, theta: float = 10000.0):
+                 w: dict, Hq: int, Hkv: int, D: int, eps: float = 1e-5, theta: float = 10000.0, store=None):
     """One step of the draft layer.  F_new [B,R,H]: the base model's hidden states of the newest
     n_new[b] <= R positions of each sequence (positions kv_len[b] .. kv_len[b]+n_new[b]-1; the
     layer's cache Kd, Vd [B,Hkv,Lcap,D] already holds positions < kv_len[b]).  w: g1 [H], Wqkv
     [(Hq+2Hkv)D, H] (query rows first, then key rows, then value rows), Wo [H, Hq*D], g2 [H],
     Wgu [2I, H] (gate rows, then up rows), Wdn [H, I].
+    store: None, or a function that rounds an array to the storage type of the activations (e.g.
+    to bfloat16).  A mixed-precision implementation keeps the four activation vectors that feed a
+    projection - the normalised input, the attention output, the normalised h1, the SwiGLU product -
+    in that type, as it keeps the cached keys and values; with `store` the same four vectors (and
+    the cached rows) are rounded here too, everything else stays float64.
     Returns (F_hat [B,H]: the layer's output at each sequence's newest position, Kd', Vd' with the
     new positions' keys/values appended, kv_len' = kv_len + n_new)."""
+    st = (lambda a: a) if store is None else (lambda a: np.asarray(store(np.asarray(a, dtype=np.float32)), dtype=np.float64))
     F_new = np.asarray(F_new, dtype=np.float64)
     B, R, H = F_new.shape
     Kd, Vd = np.array(Kd, dtype=np.float64, copy=True), np.array(Vd, dtype=np.float64, copy=True)
@@ -647,15 +653,15 @@ def draft_module(F_new: np.ndarray, n_new: np.ndarray, kv_len: np.ndarray, Kd: n
         L, r = int(kv_len[b]), int(n_new[b])
         q_last = None
         for j in range(r):
-            a = rms_norm(F_new[b, j], w["g1"], eps)
+            a = st(rms_norm(F_new[b, j], w["g1"], eps))
             qkv = Wqkv @ a
             q = qkv[:Hq * D].reshape(Hq, D)
             k = qkv[Hq * D:(Hq + Hkv) * D].reshape(Hkv, D)
             v = qkv[(Hq + Hkv) * D:].reshape(Hkv, D)
             for g in range(Hkv):
-                Kd[b, g, L + j] = rope_rotate(k[g], L + j, theta)
-                Vd[b, g, L + j] = v[g]
-            q_last = np.stack([rope_rotate(q[h], L + j, theta) for h in range(Hq)])
+                Kd[b, g, L + j] = st(rope_rotate(k[g], L + j, theta))
+                Vd[b, g, L + j] = st(v[g])
+            q_last = st(np.stack([rope_rotate(q[h], L + j, theta) for h in range(Hq)]))
         n_keys = L + r
         attn = np.zeros((Hq, D))
         for h in range(Hq):                          # the newest position attends to every position so far
@@ -663,11 +669,11 @@ def draft_module(F_new: np.ndarray, n_new: np.ndarray, kv_len: np.ndarray, Kd: n
             p = np.exp(s - s.max())
             p /= p.sum()
             attn[h] = p @ Vd[b, h // grp, :n_keys]
-        h1 = F_new[b, r - 1] + Wo @ attn.reshape(-1)
-        m = rms_norm(h1, w["g2"], eps)
+        h1 = F_new[b, r - 1] + Wo @ st(attn).reshape(-1)
+        m = st(rms_norm(h1, w["g2"], eps))
         gu = Wgu @ m
         gate, up = gu[:I], gu[I:]
-        act = gate / (1.0 + np.exp(-gate)) * up       # SiLU(gate) * up
+        act = st(gate / (1.0 + np.exp(-gate)) * up)   # SiLU(gate) * up
         F_hat[b] = h1 + Wdn @ act
         new_len[b] = n_keys
     return F_hat, Kd, Vd, new_len

@@ -897,6 +897,15 @@ def test_draft_module_special_cases():
     one = orc.tree_attention(Q, K2, V2, np.array([L + r - 1]), np.array([1]), np.ones((1, 4, 1), dtype=np.uint64),
                              1.0 / math.sqrt(D))
     np.testing.assert_allclose(F_hat[0], F[0, r - 1] + w["Wo"] @ one[0, 0].reshape(-1), atol=1e-12)
+    # the optional storage rounding: the identity changes nothing, bfloat16 moves the output by a few 1e-3
+    from paper_2412_00061_b200 import synth
+    w, F, n_new, kv_len, Kd, Vd, (Hq, Hkv, D, I) = _draft_module_case(rng)
+    plain = orc.draft_module(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D)
+    same = orc.draft_module(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D, store=lambda a: a.astype(np.float64))
+    np.testing.assert_allclose(same[0], plain[0], atol=1e-5)            # (float32 round trip of the stored vectors)
+    rounded = orc.draft_module(F, n_new, kv_len, Kd, Vd, w, Hq, Hkv, D, store=synth.round_bf16)
+    assert 0 < np.max(np.abs(rounded[0] - plain[0])) < 0.2
+    np.testing.assert_array_equal(rounded[1][0, :, int(kv_len[0])], synth.round_bf16(rounded[1][0, :, int(kv_len[0])].astype(np.float32)))
     # rotary embedding: a rotation (norm kept), position 0 is the identity, relative-position property
     v, u = rng.normal(size=D), rng.normal(size=D)
     np.testing.assert_allclose(orc.rope_rotate(v, 0, 10000.0), v, atol=0)
