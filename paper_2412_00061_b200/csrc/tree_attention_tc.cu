@@ -36,7 +36,10 @@ struct __align__(8) AttnShared {
     uint64_t full[kStages];        // K and V tile landed
     uint64_t empty[kStages];       // both MMAs of the tile have read it
     uint64_t s_full[2];            // S of an even / odd tile is in tensor memory
-    uint64_t p_full;               // P is in shared memory (and S has been read)
+    uint64_t p_full[2];            // P of an even / odd tile is in shared memory (and S has been read).  Two
+                                   // barriers: a softmax warp may finish tile t+1 while another still writes P
+                                   // of tile t (it cannot reach tile t+2, whose S is issued after P of t is complete),
+                                   // and its arrival must not count for tile t
     uint64_t o_full;               // O_tile is in tensor memory
     uint32_t tmem_base;
     int abort_flag;
@@ -117,7 +120,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         for (int s = 0; s < kStages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
         tc::mbar_init(&sh->s_full[0], 1);
         tc::mbar_init(&sh->s_full[1], 1);
-        tc::mbar_init(&sh->p_full, kSoftmaxWarps);
+        tc::mbar_init(&sh->p_full[0], kSoftmaxWarps);
+        tc::mbar_init(&sh->p_full[1], kSoftmaxWarps);
         tc::mbar_init(&sh->o_full, 1);
         sh->abort_flag = 0;
         sh->never_set = 0;
@@ -217,7 +221,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 if (it + 1 < ntile && !issue_s(it + 1)) { ok = false; break; }
                 const uint32_t v_addr = tc::smem_u32(KV + (size_t)s * 2 * kTileBytes) + kTileBytes;
                 // O_tile = P V once the softmax warps have written P (they have then also read S)
-                if (!tc::mbar_wait(&sh->p_full, (uint32_t)it & 1u, abort_flag)) { ok = false; break; }
+                if (!tc::mbar_wait(&sh->p_full[it & 1], (uint32_t)(it >> 1) & 1u, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < kKeys / 16; ++kk) {
@@ -295,85 +299,95 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
                 if (sft > 32) bits |= mask_word(w + 1) << (64 - sft);
                 return (uint32_t)bits;
             };
-            // pass 1: maximum over this thread's 64 keys, then over the row
-            float bm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four chains instead of one
-            if (!failed) {
+            // One pass over the tile in the common case.  P = 2^(S - ref) is formed against the reference
+            // the row already has, and the tile's maximum is taken along the way; only when that maximum
+            // turns out to lie more than kSlack above the reference (in log2 units; always on the first
+            // tile with a visible key) does the reference move: O and the row sum are rescaled and the
+            // pass is repeated against the new reference.  P therefore stays below 2^kSlack, and O, which
+            // accumulates in tensor memory, rarely needs rescaling.  Both threads of a row see the same
+            // numbers and take the same decisions; a warp repeats the pass if any of its rows has to
+            // (the tensor-memory loads are warp-wide).
+            unsigned char* pt = p_tile(s);
+            if (!kPInK) {
+                // a single P buffer: the previous tile's P V product must have consumed it
+                if (it > 0 && !failed && !tc::mbar_wait(&sh->o_full, (uint32_t)(it - 1) & 1u, abort_flag)) failed = true;
+                failed = __any_sync(0xffffffffu, failed);
+            }
+            float part = 0.f;                              // this thread's share of the tile's row sum
+            float bm = -INFINITY;
+            auto pass = [&](float rf) {                    // rf: reference in log2 units (finite)
+                float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+                float bm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
 #pragma unroll 1
                 for (int c0 = kc0; c0 < kc0 + kKeys / 2; c0 += 32) {
                     uint32_t v[32];
                     tc::tmem_ld32(tmem_s + (uint32_t)((it & 1) * 128) + lane_off + (uint32_t)c0, v);
                     const uint32_t vm = visible32(c0);
                     tc::tmem_ld_wait();
+                    float pv[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if ((vm >> j) & 1u) bm4[j & 3] = fmaxf(bm4[j & 3], __uint_as_float(v[j]));
+                    for (int j = 0; j < 32; ++j) {
+                        const float x = __uint_as_float(v[j]);
+                        const bool vis = (vm >> j) & 1u;
+                        const float e = exp2_fast(fmaf(x, sl2, -rf));
+                        pv[j] = vis ? e : 0.f;
+                        ps4[j & 3] += pv[j];
+                        bm4[j & 3] = vis ? fmaxf(bm4[j & 3], x) : bm4[j & 3];
+                    }
+                    unsigned char* prow = pt + (c0 / 64) * (kRows * 128) + rl * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 w;
+                        w.x = pack_bf16(pv[8 * c + 0], pv[8 * c + 1]);
+                        w.y = pack_bf16(pv[8 * c + 2], pv[8 * c + 3]);
+                        w.z = pack_bf16(pv[8 * c + 4], pv[8 * c + 5]);
+                        w.w = pack_bf16(pv[8 * c + 6], pv[8 * c + 7]);
+                        const int chunk = (c0 % 64) / 8 + c;
+                        *reinterpret_cast<uint4*>(prow + ((chunk ^ (rl & 7)) << 4)) = w;
+                    }
                 }
-            }
-            float bm = fmaxf(fmaxf(bm4[0], bm4[1]), fmaxf(bm4[2], bm4[3]));
+                part = (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+                bm = fmaxf(fmaxf(bm4[0], bm4[1]), fmaxf(bm4[2], bm4[3]));
+            };
+            if (!failed) pass(ref == -INFINITY ? 0.f : ref);
             sh->xch[it & 1][half][rl] = bm;
             pair_barrier(q);
             bm = fmaxf(bm, sh->xch[it & 1][half ^ 1][rl]);
             bm *= sl2;                                 // scale > 0: the maximum commutes with it
-            // The exponent's reference follows the running maximum lazily: it moves only when the
-            // maximum has grown by more than kSlack (in log2 units), so P stays below 2^kSlack and
-            // O, which accumulates in tensor memory, rarely needs rescaling.  Both threads of a row
-            // see the same numbers and take the same decision.
             const bool move = bm > ref + kSlack;       // also the first tile with a visible key (ref = -inf)
-            const float nref = move ? bm : ref;
-            const float corr = move ? exp2_fast(ref - nref) : 1.f;     // exp2(-inf) = 0
-            // P of the previous tile must have been consumed before it is overwritten, and O must be
-            // complete before it is rescaled
-            if (it > 0 && !failed && !tc::mbar_wait(&sh->o_full, (uint32_t)(it - 1) & 1u, abort_flag)) failed = true;
-            failed = __any_sync(0xffffffffu, failed);
+            if (__any_sync(0xffffffffu, move) && !failed) {
+                const float nref = move ? bm : ref;
+                const float corr = move ? exp2_fast(ref - nref) : 1.f;     // exp2(-inf) = 0
+                // O must be complete before it is rescaled
+                if (it > 0) {
+                    if (kPInK && !tc::mbar_wait(&sh->o_full, (uint32_t)(it - 1) & 1u, abort_flag)) failed = true;
+                    failed = __any_sync(0xffffffffu, failed);
+                    if (!failed) {
+                        tc::tc_fence_after_sync();
+#pragma unroll
+                        for (int c0 = 0; c0 < DO; c0 += 32) {
+                            uint32_t v[32];
+                            tc::tmem_ld32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
+                            tc::tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * corr);
+                            tc::tmem_st32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
+                        }
+                        tc::tmem_st_wait();
+                    }
+                }
+                sum *= corr;
+                ref = nref;
+                // a row without any visible key so far keeps ref = -inf; its P is all zero whatever the reference
+                if (!failed) pass(ref == -INFINITY ? 0.f : ref);
+            }
             if (failed) continue;
-            if (it > 0 && __any_sync(0xffffffffu, move)) {
-                tc::tc_fence_after_sync();
-#pragma unroll
-                for (int c0 = 0; c0 < DO; c0 += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * corr);
-                    tc::tmem_st32(tmem_o + lane_off + (uint32_t)(oc0 + c0), v);
-                }
-                tc::tmem_st_wait();
-            }
-            sum *= corr;
-            ref = nref;
-            // pass 2: P = exp2(S - max), partial row sum, P to shared memory as bf16 (K-major, 128-byte swizzle)
-            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-            for (int c0 = kc0; c0 < kc0 + kKeys / 2; c0 += 32) {
-                uint32_t v[32];
-                tc::tmem_ld32(tmem_s + (uint32_t)((it & 1) * 128) + lane_off + (uint32_t)c0, v);
-                tc::tmem_ld_wait();
-                const uint32_t vm = visible32(c0);
-                float pv[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float e = exp2_fast(fmaf(__uint_as_float(v[j]), sl2, -ref));
-                    pv[j] = ((vm >> j) & 1u) ? e : 0.f;
-                    ps4[j & 3] += pv[j];
-                }
-                unsigned char* prow = p_tile(s) + (c0 / 64) * (kRows * 128) + rl * 128;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 w;
-                    w.x = pack_bf16(pv[8 * c + 0], pv[8 * c + 1]);
-                    w.y = pack_bf16(pv[8 * c + 2], pv[8 * c + 3]);
-                    w.z = pack_bf16(pv[8 * c + 4], pv[8 * c + 5]);
-                    w.w = pack_bf16(pv[8 * c + 6], pv[8 * c + 7]);
-                    const int chunk = (c0 % 64) / 8 + c;
-                    *reinterpret_cast<uint4*>(prow + ((chunk ^ (rl & 7)) << 4)) = w;
-                }
-            }
-            sum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+            sum += part;
             // make P (and the cleared V rows) visible to the tensor core, then hand over
             tc::fence_proxy_async();
             tc::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&sh->p_full);
+            if (lane == 0) tc::mbar_arrive(&sh->p_full[it & 1]);
         }
         // O is complete once the last P V product has landed: fetch this thread's half of the row
         if (ntile > 0 && !failed && !tc::mbar_wait(&sh->o_full, (uint32_t)(ntile - 1) & 1u, abort_flag)) failed = true;

@@ -124,6 +124,33 @@ def test_c2_raw_layout_and_c3_in_the_benchmark_launch_configuration():
     check_benchmark_launch_configuration(_run(SMALL["c5s"], seed=2))
 
 
+def test_attention_is_reproducible_while_the_lm_head_streams_beside_it():
+    """Attention and LM head alternating inside one CUDA graph: under programmatic dependent launch
+    the LM head of one pair streams its weights while the last attention CTAs of the same pair still
+    run, which slows their K/V loads and shifts the relative timing of the warps inside them.  The
+    attention output must not depend on that: every replay must reproduce, bit for bit, the output of
+    the stand-alone call that the oracle has checked.  (An earlier version whose softmax warps
+    shared one P-ready barrier between consecutive tiles failed exactly here.)"""
+    import torch
+    r = _run(C["c3"], seed=1, attention_rows=3, lm_rows=6, draft_rows=[0])
+    step = r["step"]
+    want = step.out["O"].clone()
+    side = torch.cuda.Stream(device=step.device)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step.attention(); step.verify()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(4):
+                step.attention()
+                step.verify()
+    for _ in range(6):
+        step.out["O"].zero_()
+        g.replay()
+        step.check_status()
+        assert torch.equal(step.out["O"], want)
+
+
 @pytest.mark.parametrize("name", ["c3", "c4", "c5", "c6"])
 def test_batched_workloads_full_size_sampled(name):
     """The batched workloads at full size (prefix beam, ragged KV lengths, 128-node trees, GQA):
@@ -284,12 +311,16 @@ DM = {
 def test_attention_draft_module(name):
     """ctcsd_draft_module against the oracle's layer.  The CUDA path keeps the four activation vectors
     that feed a projection (and the cached keys/values) in the run dtype; the oracle, float64 otherwise,
-    rounds the same vectors (its `store` argument), and the layer's output must then agree within 2e-2
-    (bf16 output: plus half a unit in the last place).  Against the oracle without any rounding the
-    bound is 6e-2: four chained projections of up to 11008 terms each carry the 2^-9 relative rounding
-    of their bf16 inputs, about 5e-3 r.m.s. at the 7B shape, 4-5 sigma over 4096 outputs.  The appended
-    key/value rows, every other cache row untouched, the new lengths exact; then the draft head runs
-    on the layer's output and its top-k lists are checked against the oracle fed its logits."""
+    can round the same vectors (its `store` argument).  Tolerance, derived for bf16: every rounded vector
+    carries a relative error of 2^-9 / sqrt(3) r.m.s. into a projection of up to 11008 terms with
+    weights of 0.02 r.m.s.; chained through the layer that is 6.5e-3 r.m.s. on an output of 2.4 r.m.s.
+    at the 7B shape (the float64 oracle with and without `store` differ by exactly that: 6.5e-3 r.m.s.,
+    2.4e-2 maximum over 4096 outputs), and two implementations that round at the same places still
+    differ by as much, because a 1e-3 difference in the attention output (P is bf16 inside the kernel)
+    moves many values across a rounding boundary.  Hence: r.m.s. error <= 1.2e-2 and maximum <= 6e-2
+    against both oracles (float32: 6e-4).  The appended key/value rows pass through one projection only
+    and keep the 2e-2 bound; every other cache row must be untouched, the new lengths exact; then the
+    draft head runs on the layer's output and its top-k lists are checked against the oracle fed its logits."""
     import torch
     from oracle import ctcsd_oracle as orc
     from paper_2412_00061_b200 import binding
@@ -318,11 +349,13 @@ def test_attention_draft_module(name):
         h.draft_module(dl, td(F_new), i32(n_new), i32(kv_len), Kd_d, Vd_d, out_F, out_len, out_dbg)
         assert h.poll_status() == 0
         logit_tol, rel = tolerances(cfg.dtype)
-        assert np.max(np.abs(out_dbg.cpu().numpy() - want_F)) <= logit_tol
-        assert np.max(np.abs(out_dbg.cpu().numpy() - exact_F)) <= 3 * logit_tol
+        for ref_F in (want_F, exact_F):
+            err = out_dbg.cpu().numpy() - ref_F
+            assert np.max(np.abs(err)) <= 3 * logit_tol
+            assert np.sqrt(np.mean(err ** 2)) <= 0.6 * logit_tol
         got_F = out_F.float().cpu().numpy()
         ulp = 2.0 ** -8 if cfg.dtype == "bf16" else 0.0
-        assert np.all(np.abs(got_F - want_F) <= logit_tol + ulp * np.abs(want_F))
+        assert np.all(np.abs(got_F - want_F) <= 3 * logit_tol + ulp * np.abs(want_F))
         np.testing.assert_array_equal(out_len.cpu().numpy(), want_len)
         gK, gV = Kd_d.float().cpu().numpy(), Vd_d.float().cpu().numpy()
         for b in range(cfg.B):
