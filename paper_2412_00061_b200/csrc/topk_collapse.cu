@@ -14,7 +14,10 @@
 namespace ctcsd {
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kMaxThreads = 512;
+// threads of the running CTA (the kernels are launched with 512, or with fewer where a sequence has
+// little work per slot: a block-wide barrier costs less with fewer warps)
+#define NTHR ((int)blockDim.x)
 constexpr unsigned long long kEmpty = ~0ull;
 constexpr int kBlankMark = 255;
 constexpr double kFix = 1125899906842624.0;          // 2^50
@@ -86,13 +89,6 @@ __device__ __forceinline__ double sortable_dbl(long long v) {
     return __longlong_as_double(v ^ ((v >> 63) & 0x7fffffffffffffffll));
 }
 
-__device__ __forceinline__ double logadd(double a, double b) {
-    if (a == -INFINITY) return b;
-    if (b == -INFINITY) return a;
-    double hi = fmax(a, b), lo = fmin(a, b);
-    return hi + log1p(exp(lo - hi));
-}
-
 // (score, key) a precedes b: higher score; equal scores -> smaller key (shorter, then lexicographic)
 __device__ __forceinline__ bool precedes(double sa, unsigned long long ka, double sb, unsigned long long kb) {
     return sa > sb || (sa == sb && ka < kb);
@@ -142,7 +138,7 @@ __device__ void bitonic_sort_best_first(double* sc, unsigned long long* ky, int*
     const int tid = threadIdx.x;
     for (int k = 2; k <= n2; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < (n2 >> 1); t += kThreads) {
+            for (int t = tid; t < (n2 >> 1); t += NTHR) {
                 const int lo = t & (j - 1);
                 const int i = ((t - lo) << 1) | lo;
                 const int q = i | j;
@@ -162,14 +158,22 @@ __device__ void bitonic_sort_best_first(double* sc, unsigned long long* ky, int*
 }
 
 constexpr int kSelMax = 256;     // most near-threshold entries the exact tie-break handles
+constexpr int kRankMax = 32;     // the radix rounds go on until this few are left (one comparison round per entry)
 
 struct SelectScratch {
-    unsigned hist[256];
+    unsigned hist[2][256];         // one per round parity; all zero between calls
     int win[CTCSD_MAX_BEAM + 8];   // indices of selected entries (unordered)
     int cand[kSelMax];             // indices of entries on the threshold
-    unsigned fmax, fmin, thr;
-    int lo, need, nwin, ncand, ccnt;
+    unsigned fmax, fmin;           // range of the images (RANGE_GIVEN: accumulated by the caller)
+    unsigned thr[2];               // per round parity: what the scanning warp found
+    int need[2], ncand[2];
+    int nwin, ccnt;                // list lengths; zero between calls
 };
+
+__device__ __forceinline__ void select_scratch_init(SelectScratch& S) {
+    for (int i = threadIdx.x; i < 512; i += NTHR) (&S.hist[0][0])[i] = 0u;
+    if (threadIdx.x == 0) { S.fmax = 0u; S.fmin = 0xffffffffu; S.nwin = 0; S.ccnt = 0; }
+}
 
 // float32 image of a score as an unsigned integer whose order matches the score's
 __device__ __forceinline__ unsigned sortable_f32(double v) {
@@ -192,51 +196,61 @@ __device__ __forceinline__ int next_pow2(int v) {
 }
 
 // Selects the `need` (<= CTCSD_MAX_BEAM) best of `count` entries and writes their indices,
-// best first (in any order when `ordered` is false), to sel[]; returns how many were selected.  A radix select on the float32 image
-// of the scores finds the threshold in O(count) work; entries on the threshold are ranked
-// exactly (float64 score, then key).  If more than kSelMax entries sit on the threshold the
-// arrays (padded to a power of two, capacity >= next_pow2(count)) are sorted in place instead
-// and sel[] becomes the identity.
-template <bool MASS = false>
+// best first (in any order when `ordered` is false), to sel[]; returns how many were selected.
+// A radix select on a 32-bit image of the scores finds the threshold in O(count) work per round of
+// eight bits (the bits all images share are skipped); once at most kRankMax entries sit on the
+// threshold they are ranked exactly (float64 score, then key).  If more than kSelMax entries
+// still sit there at full image resolution the arrays (padded to a power of two, capacity >=
+// next_pow2(count)) are sorted in place instead and sel[] becomes the identity.
+// RANGE_GIVEN: the caller has run select_scratch_init once, and accumulates the largest and the
+// smallest image of this call's entries in S.fmax / S.fmin (and resets them afterwards); this
+// saves the pass that finds them.  Otherwise the call is self-contained.
+// A round costs two barriers: histograms and the scanning warp's results alternate between two
+// copies, so nobody has to wait before the next round overwrites them.
+template <bool MASS = false, bool RANGE_GIVEN = false>
 __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int count, int need, int* sel,
                                 SelectScratch& S, bool ordered = true, int* status = nullptr) {
     const int tid = threadIdx.x, lane = tid & 31;
     if (need > count) need = count;
-    if (tid == 0) { S.fmax = 0u; S.fmin = 0xffffffffu; S.nwin = 0; S.ncand = 0; S.ccnt = 0; }
-    __syncthreads();
-    if (count > need) {
-        unsigned lmax = 0u, lmin = 0xffffffffu;
-        for (int i = tid; i < count; i += kThreads) {
-            const unsigned f = select_image<MASS>(sc[i]);
-            lmax = max(lmax, f);
-            lmin = min(lmin, f);
-        }
-        lmax = __reduce_max_sync(0xffffffffu, lmax);
-        lmin = __reduce_min_sync(0xffffffffu, lmin);
-        if (lane == 0) { atomicMax(&S.fmax, lmax); atomicMin(&S.fmin, lmin); }
+    if constexpr (!RANGE_GIVEN) {
+        select_scratch_init(S);
         __syncthreads();
+    }
+    int* win = ordered ? S.win : sel;                  // an unordered selection goes straight to the caller
+    if (count > need) {
+        if constexpr (!RANGE_GIVEN) {
+            unsigned lmax = 0u, lmin = 0xffffffffu;
+            for (int i = tid; i < count; i += NTHR) {
+                const unsigned f = select_image<MASS>(sc[i]);
+                lmax = max(lmax, f);
+                lmin = min(lmin, f);
+            }
+            lmax = __reduce_max_sync(0xffffffffu, lmax);
+            lmin = __reduce_min_sync(0xffffffffu, lmin);
+            if (lane == 0) { atomicMax(&S.fmax, lmax); atomicMin(&S.fmin, lmin); }
+            __syncthreads();
+        }
         const unsigned diff = S.fmax ^ S.fmin;
-        // bits above `hb` agree for all entries; walk down 8 bits at a time
+        // bits at and above `lo` agree for all entries; walk down 8 bits at a time
         int lo = diff ? (31 - __clz(diff)) + 1 : 0;
         unsigned thr = lo < 32 ? (S.fmax >> lo) : 0u;
         int remaining = need;
         int ncand = count;
-        while (lo > 0 && ncand > remaining) {
+        for (int round = 0; lo > 0 && ncand > remaining; ++round) {
             const int nlo = lo > 8 ? lo - 8 : 0;
             const int width = lo - nlo;
-            if (tid < 256) S.hist[tid] = 0u;
-            __syncthreads();
-            for (int i = tid; i < count; i += kThreads) {
+            unsigned* H = S.hist[round & 1];
+            for (int i = tid; i < count; i += NTHR) {
                 const unsigned f = select_image<MASS>(sc[i]);
                 const unsigned top = lo < 32 ? (f >> lo) : 0u;
-                if (top == thr) atomicAdd(&S.hist[(f >> nlo) & ((1u << width) - 1u)], 1u);
+                if (top == thr) atomicAdd(&H[(f >> nlo) & ((1u << width) - 1u)], 1u);
             }
             __syncthreads();
             if (tid < 32) {
                 // lane owns digits [8*lane, 8*lane+8); find the digit where the count from the top reaches `remaining`
                 unsigned h[8], mine = 0;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) { h[q] = S.hist[8 * lane + q]; mine += h[q]; }
+                for (int q = 0; q < 8; ++q) { h[q] = H[8 * lane + q]; H[8 * lane + q] = 0u; mine += h[q]; }
                 unsigned suf = mine;                      // suffix sum: entries in this lane and above
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -249,32 +263,31 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
 #pragma unroll
                     for (int q = 7; q >= 0; --q) {
                         if (acc < (unsigned)remaining && acc + h[q] >= (unsigned)remaining) {
-                            S.thr = (thr << width) | (unsigned)(8 * lane + q);
-                            S.need = remaining - (int)acc;
-                            S.ncand = (int)h[q];
+                            S.thr[round & 1] = (thr << width) | (unsigned)(8 * lane + q);
+                            S.need[round & 1] = remaining - (int)acc;
+                            S.ncand[round & 1] = (int)h[q];
                         }
                         acc += h[q];
                     }
                 }
             }
             __syncthreads();
-            thr = S.thr; remaining = S.need; ncand = S.ncand;
+            thr = S.thr[round & 1]; remaining = S.need[round & 1]; ncand = S.ncand[round & 1];
             lo = nlo;
-            __syncthreads();
-            if (ncand <= kSelMax) break;
+            if (ncand <= kRankMax) break;
         }
         if (ncand > remaining && ncand > kSelMax) {
-            // too many entries share the threshold even at full float32 resolution: sort everything
+            // too many entries share the threshold even at full image resolution: sort everything
             const int n2 = next_pow2(count);
-            for (int i = count + tid; i < n2; i += kThreads) { sc[i] = MASS ? -1.0 : -INFINITY; ky[i] = kEmpty; if (ix) ix[i] = 0; }
+            for (int i = count + tid; i < n2; i += NTHR) { sc[i] = MASS ? -1.0 : -INFINITY; ky[i] = kEmpty; if (ix) ix[i] = 0; }
             __syncthreads();
             bitonic_sort_best_first(sc, ky, ix, n2);
-            for (int r = tid; r < need; r += kThreads) sel[r] = r;
+            for (int r = tid; r < need; r += NTHR) sel[r] = r;
             __syncthreads();
             return need;
         }
         // gather definite winners (above the threshold) and the entries on it
-        for (int i0 = 0; i0 < count; i0 += kThreads) {          // the same trip count for every thread
+        for (int i0 = 0; i0 < count; i0 += NTHR) {          // the same trip count for every thread
             const int i = i0 + tid;
             bool is_win = false, is_cand = false;
             if (i < count) {
@@ -285,13 +298,13 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
             }
             const int aw = warp_append(&S.nwin, is_win);
             const int ac = warp_append(&S.ccnt, is_cand);
-            if (is_win && CTCSD_IN_BOUNDS(status, 5, aw, CTCSD_MAX_BEAM + 8)) S.win[aw] = i;
+            if (is_win && CTCSD_IN_BOUNDS(status, 5, aw, CTCSD_MAX_BEAM + 8)) win[aw] = i;
             if (is_cand && CTCSD_IN_BOUNDS(status, 6, ac, kSelMax)) S.cand[ac] = i;
         }
         __syncthreads();
         // exact ranking among the threshold entries: one warp per entry, its lanes share the
         // comparisons (a rank is the number of entries that precede it)
-        for (int c = tid >> 5; c < ncand; c += kThreads / 32) {
+        for (int c = tid >> 5; c < ncand; c += NTHR / 32) {
             const int i = S.cand[c];
             const double si = sc[i];
             const unsigned long long ki = ky[i];
@@ -301,20 +314,17 @@ __device__ int block_select_top(double* sc, unsigned long long* ky, int* ix, int
                 rank += precedes(sc[j], ky[j], si, ki) ? 1 : 0;
             }
             rank = __reduce_add_sync(0xffffffffu, rank);
-            if (lane == 0 && rank < remaining) S.win[atomicAdd(&S.nwin, 1)] = i;
+            if (lane == 0 && rank < remaining) win[atomicAdd(&S.nwin, 1)] = i;
         }
         __syncthreads();
+        if (tid == 0) { S.nwin = 0; S.ccnt = 0; }      // (next read after the caller's barrier or this call's last one)
     } else {
-        for (int i = tid; i < count; i += kThreads) S.win[i] = i;
+        for (int i = tid; i < count; i += NTHR) win[i] = i;
         __syncthreads();
     }
-    if (!ordered) {                                   // the caller only needs the set
-        for (int w = tid; w < need; w += kThreads) sel[w] = S.win[w];
-        __syncthreads();
-        return need;
-    }
+    if (!ordered) return need;                        // the caller only needs the set
     // order the winners, again one warp per winner
-    for (int w = tid >> 5; w < need; w += kThreads / 32) {
+    for (int w = tid >> 5; w < need; w += NTHR / 32) {
         const int i = S.win[w];
         const double si = sc[i];
         const unsigned long long ki = ky[i];
@@ -340,14 +350,14 @@ __device__ void emit_candidates(const CollapseParams& p, int b, const SlotLists&
     int* ctok = p.out_cand_tok + (size_t)b * p.topN * p.T;
     int* clen = p.out_cand_len + (size_t)b * p.topN;
     float* cscore = p.out_cand_score + (size_t)b * p.topN;
-    for (int i = tid; i < p.topN * p.T; i += kThreads) ctok[i] = -1;
-    for (int i = tid; i < p.topN; i += kThreads) { clen[i] = 0; cscore[i] = -INFINITY; }
+    for (int i = tid; i < p.topN * p.T; i += NTHR) ctok[i] = -1;
+    for (int i = tid; i < p.topN; i += NTHR) { clen[i] = 0; cscore[i] = -INFINITY; }
     __syncthreads();
-    for (int e = tid; e < nsel; e += kThreads)
+    for (int e = tid; e < nsel; e += NTHR)
         if (key_len(ky[sel[e]]) == 0) s_empty_at = e;
     __syncthreads();
     const int empty_at = s_empty_at;
-    for (int e = tid; e < nsel; e += kThreads) {
+    for (int e = tid; e < nsel; e += NTHR) {
         if (e == empty_at) continue;
         const int rank = e - (empty_at < e ? 1 : 0);
         if (rank >= p.topN) continue;
@@ -400,7 +410,7 @@ __device__ __forceinline__ unsigned long long path_key_and_score(const CollapseP
 // ---------------------------------------------------------------------------------------
 // Exhaustive enumeration of the k^T slot paths
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams p) {
+__global__ void __launch_bounds__(kMaxThreads) collapse_enum_kernel(CollapseParams p) {
     extern __shared__ __align__(16) unsigned char dyn[];
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);             // [cap]
     long long* best = reinterpret_cast<long long*>(keys + p.cap);                      // [cap] sortable max, then score
@@ -421,12 +431,12 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     }
     load_slot_lists(p, row, sl);
     const long long neg_inf_sortable = dbl_sortable(-INFINITY);
-    for (int i = tid; i < p.cap; i += kThreads) { keys[i] = kEmpty; best[i] = neg_inf_sortable; fsum[i] = 0ull; }
+    for (int i = tid; i < p.cap; i += NTHR) { keys[i] = kEmpty; best[i] = neg_inf_sortable; fsum[i] = 0ull; }
     if (tid == 0) { s_count = 0; s_has_empty = 0; s_merged = 0; }
     __syncthreads();
 
     // pass 1: collapse every path, claim a table slot, track the best alignment
-    for (int path = tid; path < p.npaths; path += kThreads) {
+    for (int path = tid; path < p.npaths; path += NTHR) {
         double s;
         const unsigned long long key = path_key_and_score(p, sl, path, s);
         bool was_there = false;
@@ -443,7 +453,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     // paths collapsed to the same sequence every sum is that single 1 and the pass is skipped.
     const bool sums = p.score_mode == CTCSD_SCORE_SUM && s_merged != 0;
     if (sums) {
-        for (int path = tid; path < p.npaths; path += kThreads) {
+        for (int path = tid; path < p.npaths; path += NTHR) {
             double s;
             path_key_and_score(p, sl, path, s);
             const int slot = path_slot[path];
@@ -455,7 +465,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     }
     __syncthreads();
     double* score = reinterpret_cast<double*>(best);
-    for (int i = tid; i < p.cap; i += kThreads) {
+    for (int i = tid; i < p.cap; i += NTHR) {
         if (keys[i] == kEmpty) continue;
         const double mx = sortable_dbl(best[i]);
         double sc = mx;
@@ -469,7 +479,7 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
     // because the empty sequence may be among them) and write them out
     double* c_sc = reinterpret_cast<double*>(fsum);                     // [cap/2]
     unsigned long long* c_ky = fsum + (p.cap >> 1);                     // [cap/2]
-    for (int i0 = 0; i0 < p.cap; i0 += kThreads) {
+    for (int i0 = 0; i0 < p.cap; i0 += NTHR) {
         const int i = i0 + tid;
         const unsigned long long ki = i < p.cap ? keys[i] : kEmpty;
         const bool has = ki != kEmpty;
@@ -489,16 +499,40 @@ __global__ void __launch_bounds__(kThreads) collapse_enum_kernel(CollapseParams 
 // ---------------------------------------------------------------------------------------
 // CTC prefix beam search over the per-slot lists
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams p) {
+// Finds `key` in a set built with table_insert; returns its payload index or -1.
+__device__ __forceinline__ int set_lookup(const unsigned long long* keys, const short* val, int cap, unsigned long long key) {
+    unsigned s = hash_key(key, cap);
+    for (int probe = 0; probe < cap; ++probe) {
+        const unsigned long long cur = keys[s];
+        if (cur == key) return val[s];
+        if (cur == kEmpty) return -1;
+        s = (s + 1) & (unsigned)(cap - 1);
+    }
+    return -1;
+}
+
+// What one slot makes of the beam.  A prefix e with masses (pb: alignments ending in the blank, pnb:
+// ending in its last token) and a slot with symbols m_j of probability p_j give
+//   e itself   pb'  = (pb + pnb) p_blank          (if the blank is among the slot's symbols)
+//              pnb' = pnb p_last(e)               (if e's last token is)
+//   e + m      pnb' = (m == last(e) ? pb : pb + pnb) p_m      for every non-blank m.
+// Two different (e, m) never give the same sequence, and two prefixes of the beam are different
+// sequences, so the only merging there is happens when e + m is itself a prefix e' of the beam:
+// the extension's mass then joins pnb' of e'.  Hence no hash table of candidates: the beam's own
+// keys go into a small set (one insert per prefix), every extension looks itself up there (a
+// read-only probe); a hit hands its mass to the beam prefix through a one-writer inbox, a miss is
+// a new candidate whose mass is final and goes straight onto the selection list.  The prefixes
+// themselves follow once the inboxes are complete.
+__global__ void __launch_bounds__(kMaxThreads) collapse_beam_kernel(CollapseParams p) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    const int cap = p.cap;                   // hash capacity: a power of two >= 2 * beam * (k + 1), the most distinct prefixes a slot can make
-    unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);   // [cap]
-    double* t_pb = reinterpret_cast<double*>(keys + cap);    // mass ending in blank (one contributor: the prefix itself)
-    double* t_stay = t_pb + cap;        // ending in the last token, from the prefix itself (repeat)
-    double* t_ext = t_stay + cap;       // ending in the last token, from the parent prefix (extension)
-    double* c_sc = t_ext + cap;                                          // [cap] sort keys
+    const int cap = p.cap;                   // candidates per slot rounded up to a power of two (the fallback sort needs it)
+    double* c_sc = reinterpret_cast<double*>(dyn);                            // [cap] masses of the candidates
     unsigned long long* c_ky = reinterpret_cast<unsigned long long*>(c_sc + cap);
-    int* c_ix = reinterpret_cast<int*>(c_ky + cap);                      // [cap] table slot
+    int* c_ix = reinterpret_cast<int*>(c_ky + cap);                           // [cap] beam index of a prefix that stayed, -1 for a new one
+    __shared__ unsigned long long h_key[4 * CTCSD_MAX_BEAM];                  // the beam's keys as a set (load <= 1/4)
+    __shared__ short h_val[4 * CTCSD_MAX_BEAM];
+    __shared__ double ext_in[CTCSD_MAX_BEAM];                                 // mass an extension hands to a beam prefix
+    __shared__ double st_pb[CTCSD_MAX_BEAM], st_pnb[CTCSD_MAX_BEAM];          // the new masses of a prefix that stays
     __shared__ unsigned long long bm_key[CTCSD_MAX_BEAM];
     __shared__ double bm_pb[CTCSD_MAX_BEAM], bm_pnb[CTCSD_MAX_BEAM], bm_tot[CTCSD_MAX_BEAM];
     __shared__ int s_nbeam, s_next;
@@ -506,7 +540,7 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     __shared__ SelectScratch S;
     __shared__ int s_sel[CTCSD_MAX_BEAM + 8];
 
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     pdl_wait();                      // the per-slot lists come from the preceding kernel
     pdl_trigger();
     const int row = p.sel_row ? p.sel_row[b] : b;
@@ -522,6 +556,8 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
     // alignment"); the logarithm of the common factor is added back when the scores are written.
     __shared__ double s_pr[CTCSD_MAX_T * CTCSD_MAX_K];
     __shared__ double s_logoff;
+    int hcap = 4;                                        // set capacity: a power of two >= 4 * beam
+    while (hcap < 4 * p.beam) hcap <<= 1;
     if (tid < p.T * p.k) {
         const int t = tid / p.k;
         double mx = sl.lp[t * p.k];
@@ -537,80 +573,113 @@ __global__ void __launch_bounds__(kThreads) collapse_beam_kernel(CollapseParams 
             s_logoff = off;
         }
     }
-    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 1.0; bm_pnb[0] = 0.0; bm_tot[0] = 1.0; s_nbeam = 1; }
+    select_scratch_init(S);
+    for (int i = tid; i < hcap; i += NTHR) h_key[i] = kEmpty;
+    for (int i = tid; i < p.beam; i += NTHR) ext_in[i] = 0.0;
+    if (tid == 0) { bm_key[0] = 0ull; bm_pb[0] = 1.0; bm_pnb[0] = 0.0; bm_tot[0] = 1.0; s_nbeam = 1; s_next = 0; }
+    __syncthreads();
+    if (tid == 0) { const int at = table_insert(h_key, hcap, 0ull); if (at >= 0) h_val[at] = 0; }
     __syncthreads();
 
     for (int t = 0; t < p.T; ++t) {
-        for (int i = tid; i < cap; i += kThreads) {
-            keys[i] = kEmpty; t_pb[i] = 0.0; t_stay[i] = 0.0; t_ext[i] = 0.0;
-        }
-        if (tid == 0) s_next = 0;
-        __syncthreads();
         const int nbeam = s_nbeam;
-        for (int w = tid; w < nbeam * p.k; w += kThreads) {
-            const int e = w / p.k, j = w - e * p.k;
-            const unsigned long long key = bm_key[e];
-            const double pb = bm_pb[e], pnb = bm_pnb[e];
-            const double tot = bm_tot[e];
-            const int m = sl.lid[t * p.k + j];
-            const double pr = s_pr[t * p.k + j];
-            const int len = key_len(key);
-            const int last = len > 0 ? key_tok(key, len - 1) : -1;
-            if (pr == 0.0) continue;                     // a symbol of probability zero reaches nothing
-            if (m == kBlankMark) {
-                int s = table_insert(keys, cap, key);
-                if (s >= 0) t_pb[s] = tot * pr;
-            } else if (m == last) {
-                if (pnb != 0.0) {
-                    int s = table_insert(keys, cap, key);
-                    if (s >= 0) t_stay[s] = pnb * pr;
+        const int next = nbeam * p.k;                    // extensions: item e * k + j
+        const int nitem = next + nbeam;                  // then the prefixes themselves
+        unsigned lmax = 0u, lmin = 0xffffffffu;          // range of the candidates' images, for the selection
+        // ---- extensions look themselves up in the beam; the prefixes work out what stays with them ----
+        for (int w0 = 0; w0 < nitem; w0 += NTHR) {       // (whole warps go round: the list append is a warp operation)
+            const int w = w0 + tid;
+            bool has = false;
+            unsigned long long ck = kEmpty;
+            double val = 0.0;
+            if (w < next) {
+                const int e = w / p.k, j = w - e * p.k;
+                const int m = sl.lid[t * p.k + j];
+                if (m != kBlankMark) {
+                    const unsigned long long key = bm_key[e];
+                    const int len = key_len(key);
+                    const int last = len > 0 ? key_tok(key, len - 1) : -1;
+                    val = (m == last ? bm_pb[e] : bm_tot[e]) * s_pr[t * p.k + j];
+                    if (val != 0.0) {                    // (a symbol or a prefix of mass zero reaches nothing)
+                        ck = key_append(key, m);
+                        const int hit = set_lookup(h_key, h_val, hcap, ck);
+                        if (hit >= 0) ext_in[hit] = val; // e + m is beam prefix `hit`, and this its only such donor
+                        else has = true;
+                    }
                 }
-                if (pb != 0.0) {
-                    int s = table_insert(keys, cap, key_append(key, m));
-                    if (s >= 0) t_ext[s] = pb * pr;
+            } else if (w < nitem) {
+                const int e = w - next;
+                const unsigned long long key = bm_key[e];
+                const int len = key_len(key);
+                const int last = len > 0 ? key_tok(key, len - 1) : -1;
+                const double pnb = bm_pnb[e], tot = bm_tot[e];
+                double cpb = 0.0, cpnb = 0.0;
+                for (int q = 0; q < p.k; ++q) {
+                    const int m = sl.lid[t * p.k + q];
+                    const double pr = s_pr[t * p.k + q];
+                    if (m == kBlankMark) cpb = tot * pr;
+                    else if (m == last) cpnb = pnb * pr;
                 }
-            } else {
-                int s = table_insert(keys, cap, key_append(key, m));
-                if (s >= 0) t_ext[s] = tot * pr;
+                st_pb[e] = cpb;
+                st_pnb[e] = cpnb;
             }
+            const int at = warp_append(&s_next, has);
+            if (!has || !CTCSD_IN_BOUNDS(p.status, 3, at, cap)) continue;
+            c_sc[at] = val;
+            c_ky[at] = ck;
+            c_ix[at] = -1;
+            const unsigned f = select_image<true>(val);
+            lmax = max(lmax, f);
+            lmin = min(lmin, f);
         }
         __syncthreads();
-        // total mass per prefix; compact into the sort arrays
-        for (int i0 = 0; i0 < cap; i0 += kThreads) {
-            const int i = i0 + tid;
-            const unsigned long long ki = i < cap ? keys[i] : kEmpty;
-            double pnb = 0.0, tot = 0.0;
-            if (ki != kEmpty) {
-                pnb = t_stay[i] + t_ext[i];
-                tot = t_pb[i] + pnb;
+        // ---- the prefixes collect what extensions handed them and join the list ----
+        for (int e0 = 0; e0 < nbeam; e0 += NTHR) {
+            const int e = e0 + tid;
+            double tot = 0.0;
+            if (e < nbeam) {
+                const double pnb = st_pnb[e] + ext_in[e];
+                ext_in[e] = 0.0;
+                st_pnb[e] = pnb;
+                tot = st_pb[e] + pnb;
             }
             const bool has = tot != 0.0;                 // (a mass that underflowed has no alignment left)
             const int at = warp_append(&s_next, has);
-            if (!has || !CTCSD_IN_BOUNDS(p.status, 3, at, cap)) continue;
-            t_stay[i] = pnb;
-            t_ext[i] = tot;
+            if (!has || !CTCSD_IN_BOUNDS(p.status, 4, at, cap)) continue;
             c_sc[at] = tot;
-            c_ky[at] = ki;
-            c_ix[at] = i;
+            c_ky[at] = bm_key[e];
+            c_ix[at] = e;
+            const unsigned f = select_image<true>(tot);
+            lmax = max(lmax, f);
+            lmin = min(lmin, f);
         }
+        for (int i = tid; i < hcap; i += NTHR) h_key[i] = kEmpty;       // every lookup is done
+        lmax = __reduce_max_sync(0xffffffffu, lmax);
+        lmin = __reduce_min_sync(0xffffffffu, lmin);
+        if (lane == 0 && lmax >= lmin) { atomicMax(&S.fmax, lmax); atomicMin(&S.fmin, lmin); }
         __syncthreads();
         const int count = s_next;
-        // between slots the beam is a set; only the last slot's beam is ranked (the candidates come out of it)
-        const int keep = block_select_top<true>(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1, p.status);
-        for (int r = tid; r < keep; r += kThreads) {
+        // ---- the `beam` heaviest: between slots a set; only the last slot's beam is ranked ----
+        const int keep = block_select_top<true, true>(c_sc, c_ky, c_ix, count, p.beam, s_sel, S, t == p.T - 1, p.status);
+        // ---- they become the beam, and its key set ----
+        for (int r = tid; r < keep; r += NTHR) {
             const int i = s_sel[r];
-            const int slot = c_ix[i];
-            bm_key[r] = c_ky[i];
-            bm_pb[r] = t_pb[slot];
-            bm_pnb[r] = t_stay[slot];
-            bm_tot[r] = c_sc[i];
+            const int e = c_ix[i];
+            const unsigned long long ck = c_ky[i];
+            const double tot = c_sc[i];
+            bm_key[r] = ck;
+            bm_pb[r] = e >= 0 ? st_pb[e] : 0.0;
+            bm_pnb[r] = e >= 0 ? st_pnb[e] : tot;
+            bm_tot[r] = tot;
+            const int at = table_insert(h_key, hcap, ck);
+            if (at >= 0) h_val[at] = (short)r;
         }
-        if (tid == 0) s_nbeam = keep;
+        if (tid == 0) { s_nbeam = keep; s_next = 0; S.fmax = 0u; S.fmin = 0xffffffffu; }
         __syncthreads();
     }
     // the beam is already ranked best first by total mass; scores go out as logarithms
     const int nbeam = s_nbeam;
-    for (int r = tid; r < nbeam; r += kThreads) {
+    for (int r = tid; r < nbeam; r += NTHR) {
         s_sel[r] = r;
         bm_tot[r] = log(bm_tot[r]) + s_logoff;
     }
@@ -631,7 +700,7 @@ struct RawParams {
     int* out_n_raw;          // [B]
 };
 
-__global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
+__global__ void __launch_bounds__(kMaxThreads) raw_paths_kernel(RawParams rp) {
     extern __shared__ __align__(16) unsigned char dyn[];
     const CollapseParams& p = rp.c;
     double* sc = reinterpret_cast<double*>(dyn);                                   // [cap]
@@ -651,17 +720,17 @@ __global__ void __launch_bounds__(kThreads) raw_paths_kernel(RawParams rp) {
         return;
     }
     load_slot_lists(p, row, sl);
-    for (int path = tid; path < p.npaths; path += kThreads) {
+    for (int path = tid; path < p.npaths; path += NTHR) {
         double s;
         path_key_and_score(p, sl, path, s);
         sc[path] = s;
         ky[path] = (unsigned long long)path;
     }
-    for (int i = tid; i < p.topN * p.T; i += kThreads) rtok[i] = -1;
-    for (int i = tid; i < p.topN; i += kThreads) rscore[i] = -INFINITY;
+    for (int i = tid; i < p.topN * p.T; i += NTHR) rtok[i] = -1;
+    for (int i = tid; i < p.topN; i += NTHR) rscore[i] = -INFINITY;
     __syncthreads();
     const int nsel = block_select_top(sc, ky, nullptr, p.npaths, p.topN, s_sel, S, true, p.status);
-    for (int e = tid; e < nsel; e += kThreads) {
+    for (int e = tid; e < nsel; e += NTHR) {
         const int at = s_sel[e];
         unsigned rem = (unsigned)ky[at];
         rscore[e] = (float)sc[at];
@@ -710,13 +779,16 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     p.status = status_ptr(h);
 
     if (c.beam > 0) {
-        int cap = 64;
-        while (cap < 2 * c.beam * (c.k + 1)) cap <<= 1;
+        int cap = 64;                            // candidates of one slot: beam * (k + 1), as a power of two
+        while (cap < c.beam * (c.k + 1)) cap <<= 1;
         if (cap > kBeamCap) cap = kBeamCap;
         p.cap = cap;
-        const size_t smem = (size_t)cap * 52;
+        // (fewer threads per sequence were measured slower at every beam: 128 / 256 / 320 / 512 threads
+        // took 96 / 64 / 56 / 52 us at beam 128 and 38 / 28 / 28 / 26 us at beam 64)
+        const int beam_threads = kMaxThreads;
+        const size_t smem = (size_t)cap * 20;
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_beam_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
+        CTCSD_CUDA_CHECK(h, launch_pdl(collapse_beam_kernel, dim3(c.B), dim3(beam_threads), smem, s, 1, p));
         CTCSD_LAUNCH_CHECK(h);
         return CTCSD_OK;
     }
@@ -729,7 +801,7 @@ extern "C" int ctcsd_topk_collapse(ctcsd_handle* hh, void* stream, int M, const 
     size_t smem = (size_t)cap * 24 + (size_t)npaths * 2;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(collapse_enum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B), dim3(kThreads), smem, s, 1, p));
+    CTCSD_CUDA_CHECK(h, launch_pdl(collapse_enum_kernel, dim3(c.B), dim3(kMaxThreads), smem, s, 1, p));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
@@ -761,7 +833,7 @@ extern "C" int ctcsd_select_raw_paths(ctcsd_handle* hh, void* stream, int M, con
     const size_t smem = (size_t)p.cap * 16;
     if (smem > 48 * 1024)
         CTCSD_CUDA_CHECK(h, cudaFuncSetAttribute(raw_paths_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B), dim3(kThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
+    CTCSD_CUDA_CHECK(h, launch_pdl(raw_paths_kernel, dim3(c.B), dim3(kMaxThreads), smem, static_cast<cudaStream_t>(stream), 1, rp));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
