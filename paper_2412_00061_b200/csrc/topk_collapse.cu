@@ -410,7 +410,7 @@ __device__ __forceinline__ unsigned long long path_key_and_score(const CollapseP
 // ---------------------------------------------------------------------------------------
 // Exhaustive enumeration of the k^T slot paths
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kMaxThreads) collapse_enum_kernel(CollapseParams p) {
+__global__ void __launch_bounds__(kMaxThreads, 1) collapse_enum_kernel(CollapseParams p) {
     extern __shared__ __align__(16) unsigned char dyn[];
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);             // [cap]
     long long* best = reinterpret_cast<long long*>(keys + p.cap);                      // [cap] sortable max, then score
@@ -523,7 +523,7 @@ __device__ __forceinline__ int set_lookup(const unsigned long long* keys, const 
 // read-only probe); a hit hands its mass to the beam prefix through a one-writer inbox, a miss is
 // a new candidate whose mass is final and goes straight onto the selection list.  The prefixes
 // themselves follow once the inboxes are complete.
-__global__ void __launch_bounds__(kMaxThreads) collapse_beam_kernel(CollapseParams p) {
+__global__ void __launch_bounds__(kMaxThreads, 1) collapse_beam_kernel(CollapseParams p) {
     extern __shared__ __align__(16) unsigned char dyn[];
     const int cap = p.cap;                   // candidates per slot rounded up to a power of two (the fallback sort needs it)
     double* c_sc = reinterpret_cast<double*>(dyn);                            // [cap] masses of the candidates
@@ -700,7 +700,7 @@ struct RawParams {
     int* out_n_raw;          // [B]
 };
 
-__global__ void __launch_bounds__(kMaxThreads) raw_paths_kernel(RawParams rp) {
+__global__ void __launch_bounds__(kMaxThreads, 1) raw_paths_kernel(RawParams rp) {
     extern __shared__ __align__(16) unsigned char dyn[];
     const CollapseParams& p = rp.c;
     double* sc = reinterpret_cast<double*>(dyn);                                   // [cap]

@@ -98,7 +98,7 @@ def check_candidates(cfg, topk_id, topk_lp, sel_row, got, require_certified=Fals
 def run_parity(cfg, seed=0, M=None, force_repeats=False, row_seq=None, sel_row=None, device="cuda:0",
                require_certified=False, attention_rows: Optional[int] = None, lm_rows: Optional[int] = None,
                draft_rows=None):
-    """Runs the five calls on the GPU and checks every output against the oracle.
+    """Runs the calls on the GPU one by one and checks every output against the oracle.
     attention_rows / lm_rows / draft_rows bound the work of the definition-mode oracle at
     large shapes by sampling (sequence, head) pairs / node rows / draft rows."""
     logit_tol, rel = tolerances(cfg.dtype)
@@ -187,7 +187,11 @@ def run_parity(cfg, seed=0, M=None, force_repeats=False, row_seq=None, sel_row=N
     assert np.all(acc[0] <= cfg.T)
 
     # ---- the whole step again in one go: same integers (determinism, no stale state) -------
-    before = {k: step.host(k).copy() for k in ["topk_id", "cand_tok", "node_tok", "mask", "argmax", "acc_len", "acc_tok", "next_tok"]}
+    # (every output of the candidate and tree calls checked above must come out the same, from buffers wiped first)
+    fused = ["cand_tok", "cand_len", "cand_score", "n_cand", "node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes"]
+    before = {k: step.host(k).copy() for k in ["topk_id", "argmax", "acc_len", "acc_tok", "next_tok"] + fused}
+    for k in fused:
+        step.out[k].zero_()
     step.run()
     step.check_status()
     for k, v in before.items():
@@ -286,7 +290,10 @@ def run_parity_raw(cfg, seed=0, force_repeats=False, device="cuda:0", attention_
             d = int(acc[1][b, l])
             assert kept[b, d] == 1 and pos[b, d] == inp["kv_len"][b] + l + 1
 
-    before = {k: step.host(k).copy() for k in ["cand_tok", "node_tok", "mask", "kept", "nka", "argmax", "acc_len", "acc_tok", "next_tok"]}
+    fused = ["cand_tok", "cand_score", "n_cand", "node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes", "kept", "nka"]
+    before = {k: step.host(k).copy() for k in ["argmax", "acc_len", "acc_tok", "next_tok"] + fused}
+    for k in fused:                                     # same outputs, from wiped buffers
+        step.out[k].zero_()
     step.run()
     step.check_status()
     for k, v in before.items():

@@ -526,6 +526,36 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
         np.testing.assert_array_equal(step.host(k), v)
 
 
+@pytest.mark.parametrize("layout", ["packed", "raw"])
+def test_a_draft_row_out_of_range_leaves_the_root_alone(layout):
+    """sel_row pointing outside the draft rows: the call that makes the candidates reports the
+    error and gives that sequence none, the tree is the root alone (what the oracle builds
+    from zero candidates), and the handle runs a correct step afterwards."""
+    import torch
+    from paper_2412_00061_b200 import binding
+    from tests import parity_util
+    r = (_run(C["c1"], seed=2) if layout == "packed" else parity_util.run_parity_raw(C["c1"], seed=2))
+    step, cfg = r["step"], C["c1"]
+    good = {k: step.host(k).copy() for k in ("node_tok", "parent", "mask", "n_nodes", "acc_len")}
+    step.set_inputs(sel_row=torch.full((cfg.B,), 10 ** 6, dtype=torch.int32, device=step.device))
+    step.collapse()
+    step.tree()
+    with pytest.raises(binding.CtcsdError):
+        step.check_status()
+    assert (step.host("n_cand") == 0).all() and (step.host("n_nodes") == 1).all()
+    base_tok, kv_len = parity_util.synth.gen_base(cfg, 2)
+    zero = np.zeros((cfg.B, cfg.topN), dtype=np.int64)
+    want = parity_util.orc.build_tree(base_tok, kv_len, np.full((cfg.B, cfg.topN, cfg.T), -1, dtype=np.int64), zero,
+                                      np.zeros(cfg.B, dtype=np.int64), cfg.max_nodes)
+    for name, w in zip(["node_tok", "parent", "depth", "pos"], want):
+        np.testing.assert_array_equal(step.host(name), w, err_msg=name)
+    step.set_inputs(sel_row=torch.arange(cfg.B, dtype=torch.int32, device=step.device))
+    step.run()
+    step.check_status()
+    for k, v in good.items():
+        np.testing.assert_array_equal(step.host(k), v, err_msg=k)
+
+
 def test_invalid_arguments_are_rejected_on_the_host():
     import ctypes
     from paper_2412_00061_b200 import binding
