@@ -24,7 +24,7 @@ int draft_logits_impl(ctcsd_handle* hh, void* stream, int M, const void* x, int 
                                       out_topk_id, out_topk_lp, out_lse, out_logits_dbg);
         if (rc != CTCSD_ERR_UNSUPPORTED) return rc;
     }
-    GemvParams p;
+    GemvParams p = {};
     p.x = x;
     p.x_rows = x_rows;
     p.x_row_count = x_rows ? x_row_count : M;

@@ -9,7 +9,11 @@
 // only, whose output is the state the draft head projects.  At batch 1 every projection is a
 // matrix-vector product bound by HBM: the four weight matrices go through the same
 // weight-streaming kernel as the draft head (plain-output mode); the attention is the
-// tree-attention kernel on a one-node tree; the pieces between them are row-sized kernels.
+// tree-attention kernel on a one-node tree.  The row-sized pieces between them ride along: both
+// RMSNorms (the second with its residual) and the SwiGLU are applied by the projection that
+// follows them while it loads its activation rows, the last residual by the projection before
+// it as it writes its result; only the rotary embedding with the K/V append is a kernel of its
+// own.  Six launches in all.
 #include "gemv_stream.cuh"
 #include "tree_attention.cuh"
 
@@ -22,23 +26,9 @@ int tree_attention_dispatch(Handle* h, cudaStream_t s, const AttnParams& p);
 
 namespace {
 
-template <typename T> __device__ __forceinline__ float ld_f(const T* p, size_t i);
-template <> __device__ __forceinline__ float ld_f<float>(const float* p, size_t i) { return p[i]; }
-template <> __device__ __forceinline__ float ld_f<__nv_bfloat16>(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
 template <typename T> __device__ __forceinline__ void st_f(T* p, size_t i, float v);
 template <> __device__ __forceinline__ void st_f<float>(float* p, size_t i, float v) { p[i] = v; }
 template <> __device__ __forceinline__ void st_f<__nv_bfloat16>(__nv_bfloat16* p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
-
-__device__ __forceinline__ float block_sum(float v, float* red) {
-    v = warp_sum(v);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();
-    if (lane == 0) red[warp] = v;
-    __syncthreads();
-    float t = 0.f;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
-    return t;
-}
 
 struct DmParams {
     const void* F_new;          // [B,R,H] act dtype
@@ -48,52 +38,28 @@ struct DmParams {
     const float* g1; const float* g2;
     int B, R, H, Hq, Hkv, D, I, Lcap, max_nodes;
     float eps, theta;
+    double inv_freq[64];        // theta^(-2i/D), i < D/2, formed on the host in float64
     // scratch
-    void* a;                    // [B*R,H] act: normalised new rows
     float* qkv;                 // [B*R,(Hq+2Hkv)D]
     void* Qbuf;                 // [B,max_nodes,Hq,D] act: node 0 holds the newest position's query
     void* Obuf;                 // [B,max_nodes,Hq,D] act
     int* attn_len;              // [B] keys before the query row = kv_len + n_new - 1
     int* ones;                  // [B] = 1
     int* o_rows;                // [B] = b * max_nodes
+    int* last_rows;             // [B] = b * R + n_new[b] - 1: the newest position's row of F_new
     unsigned long long* mask;   // [B,max_nodes,W], bit 0 of row 0 set
     float* o;                   // [B,H] attention output projection
     float* h1;                  // [B,H] after the first residual
-    void* m;                    // [B,H] act: normalised h1
     float* gu;                  // [B,2I]
-    void* act;                  // [B,I] act: SiLU(gate) * up
-    float* mlp;                 // [B,H]
     void* out_F;                // [B,H] act
     float* out_F_dbg;           // null or [B,H]
     int* out_kv_len;            // [B]
     int* status;
 };
 
-// RMSNorm of every new row; rows past n_new[b] are written as zero.  One CTA per (row j, sequence b).
-template <typename T>
-__global__ void __launch_bounds__(256) dm_norm_rows_kernel(DmParams p) {
-    __shared__ float red[8];
-    const int j = blockIdx.x, b = blockIdx.y;
-    pdl_wait();
-    pdl_trigger();
-    const T* src = static_cast<const T*>(p.F_new) + ((size_t)b * p.R + j) * p.H;
-    T* dst = static_cast<T*>(p.a) + ((size_t)b * p.R + j) * p.H;
-    int r = p.n_new[b];
-    r = r < 0 ? 0 : (r > p.R ? p.R : r);
-    if (j >= r) {
-        for (int i = threadIdx.x; i < p.H; i += blockDim.x) st_f<T>(dst, i, 0.f);
-        return;
-    }
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < p.H; i += blockDim.x) { const float v = ld_f<T>(src, i); ss += v * v; }
-    ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)p.H + p.eps);
-    for (int i = threadIdx.x; i < p.H; i += blockDim.x) st_f<T>(dst, i, ld_f<T>(src, i) * inv * p.g1[i]);
-}
-
 // Rotary embedding and placement: keys/values of every new position go to the layer's cache, the
 // newest position's query to node 0 of the query buffer; also fills the small arrays that describe
-// the one-node "tree" to the attention kernel.  One CTA per (row j, sequence b); thread = (head, pair).
+// the one-node "tree" to the attention kernel.  Eight CTAs per (row j, sequence b); thread = (head, pair).
 template <typename T>
 __global__ void __launch_bounds__(256) dm_rope_scatter_kernel(DmParams p) {
     const int j = blockIdx.x, b = blockIdx.y;
@@ -104,12 +70,13 @@ __global__ void __launch_bounds__(256) dm_rope_scatter_kernel(DmParams p) {
     const bool bad = r < 1 || r > p.R || L < 0 || L + r > p.Lcap;
     if (bad) r = 0;
     const int W = (p.max_nodes + 63) / 64;
-    if (j == 0) {
+    if (j == 0 && blockIdx.z == 0) {
         if (threadIdx.x == 0) {
             if (bad) report_error(p.status, CTCSD_ERR_INVALID_ARG, b);
             p.attn_len[b] = bad ? 0 : L + r - 1;
             p.ones[b] = bad ? 0 : 1;
             p.o_rows[b] = b * p.max_nodes;
+            p.last_rows[b] = b * p.R + (bad ? 0 : r - 1);
             p.out_kv_len[b] = bad ? L : L + r;
         }
         for (int i = threadIdx.x; i < p.max_nodes * W; i += blockDim.x)
@@ -117,6 +84,15 @@ __global__ void __launch_bounds__(256) dm_rope_scatter_kernel(DmParams p) {
     }
     if (j >= r) return;
     const int half = p.D / 2, Nq = p.Hq * p.D, Nk = p.Hkv * p.D;
+    // the position is the CTA's: one sine and cosine per pair index, shared by all heads
+    // (angle = pos * theta^(-2i/D), formed and reduced in float64 so that long positions keep their phase)
+    __shared__ float s_sin[64], s_cos[64];                  // D is 64 or 128
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        const double two_pi = 6.283185307179586476925286766559;
+        const double ang = (double)(L + j) * p.inv_freq[i];
+        sincosf((float)(ang - floor(ang / two_pi) * two_pi), &s_sin[i], &s_cos[i]);   // reduced in float64, then float32
+    }
+    __syncthreads();
     const float* row = p.qkv + ((size_t)b * p.R + j) * (size_t)(Nq + 2 * Nk);
     const int pos = L + j;
     const bool newest = (j == r - 1);
@@ -124,15 +100,14 @@ __global__ void __launch_bounds__(256) dm_rope_scatter_kernel(DmParams p) {
     T* Vd = static_cast<T*>(p.Vd);
     T* Qb = static_cast<T*>(p.Qbuf);
     const int heads = p.Hq + p.Hkv;                       // rotated heads: queries then keys
-    for (int w = threadIdx.x; w < heads * half; w += blockDim.x) {
+    // (the loops are chains of dependent loads from L2: the work of a row is spread over gridDim.z CTAs)
+    const int tz = blockIdx.z * blockDim.x + threadIdx.x, nz = gridDim.z * blockDim.x;
+    for (int w = tz; w < heads * half; w += nz) {
         const int hd = w / half, i = w - hd * half;
         const bool is_q = hd < p.Hq;
         if (is_q && !newest) continue;
         const float* v = row + (is_q ? hd * p.D : Nq + (hd - p.Hq) * p.D);
-        // angle = pos * theta^(-2i/D), formed in float64 so that long positions keep their phase
-        const double ang = (double)pos * exp2(-2.0 * (double)i / (double)p.D * log2((double)p.theta));
-        float sn, cs;
-        sincosf((float)fmod(ang, 6.283185307179586476925286766559), &sn, &cs);
+        const float sn = s_sin[i], cs = s_cos[i];
         const float x0 = v[i], x1 = v[i + half];
         const float y0 = x0 * cs - x1 * sn, y1 = x1 * cs + x0 * sn;
         if (is_q) {
@@ -145,63 +120,14 @@ __global__ void __launch_bounds__(256) dm_rope_scatter_kernel(DmParams p) {
             st_f<T>(dst, i + half, y1);
         }
     }
-    for (int w = threadIdx.x; w < Nk; w += blockDim.x) {
+    for (int w = tz; w < Nk; w += nz) {
         const int g = w / p.D, d = w - g * p.D;
         st_f<T>(Vd + (((size_t)b * p.Hkv + g) * p.Lcap + pos) * p.D, d, row[Nq + Nk + w]);
     }
 }
 
-// h1 = F_last + o;  m = RMSNorm(h1) * g2.  One CTA per sequence.
-template <typename T>
-__global__ void __launch_bounds__(256) dm_residual_norm_kernel(DmParams p) {
-    __shared__ float red[8];
-    const int b = blockIdx.x;
-    pdl_wait();
-    pdl_trigger();
-    int r = p.n_new[b];
-    r = r < 1 ? 1 : (r > p.R ? p.R : r);
-    const T* src = static_cast<const T*>(p.F_new) + ((size_t)b * p.R + (r - 1)) * p.H;
-    float* h1 = p.h1 + (size_t)b * p.H;
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < p.H; i += blockDim.x) {
-        const float v = ld_f<T>(src, i) + p.o[(size_t)b * p.H + i];
-        h1[i] = v;
-        ss += v * v;
-    }
-    ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)p.H + p.eps);
-    T* dst = static_cast<T*>(p.m) + (size_t)b * p.H;
-    for (int i = threadIdx.x; i < p.H; i += blockDim.x) st_f<T>(dst, i, h1[i] * inv * p.g2[i]);
-}
-
-// act = SiLU(gate) * up
-template <typename T>
-__global__ void __launch_bounds__(256) dm_swiglu_kernel(DmParams p) {
-    pdl_wait();
-    pdl_trigger();
-    const size_t n = (size_t)p.B * p.I;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        const size_t b = e / p.I, i = e - b * p.I;
-        const float g = p.gu[b * 2 * p.I + i], u = p.gu[b * 2 * p.I + p.I + i];
-        st_f<T>(static_cast<T*>(p.act), e, g / (1.f + __expf(-g)) * u);
-    }
-}
-
-// F_hat = h1 + mlp
-template <typename T>
-__global__ void __launch_bounds__(256) dm_residual_out_kernel(DmParams p) {
-    pdl_wait();
-    pdl_trigger();
-    const size_t n = (size_t)p.B * p.H;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        const float v = p.h1[e] + p.mlp[e];
-        st_f<T>(static_cast<T*>(p.out_F), e, v);
-        if (p.out_F_dbg) p.out_F_dbg[e] = v;
-    }
-}
-
 struct DmLayout {
-    size_t a, qkv, Qbuf, Obuf, attn_len, ones, o_rows, mask, o, h1, m, gu, act, mlp, total;
+    size_t qkv, Qbuf, Obuf, attn_len, ones, o_rows, last_rows, mask, o, h1, gu, total;
 };
 
 DmLayout dm_layout(const ctcsd_config& c, int R, int I) {
@@ -210,33 +136,32 @@ DmLayout dm_layout(const ctcsd_config& c, int R, int I) {
     const size_t W = (c.max_nodes + 63) / 64;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
-    l.a = take((size_t)c.B * R * c.H * esz);
     l.qkv = take((size_t)c.B * R * (c.Hq + 2 * c.Hkv) * c.D * 4);
     l.Qbuf = take((size_t)c.B * c.max_nodes * c.Hq * c.D * esz);
     l.Obuf = take((size_t)c.B * c.max_nodes * c.Hq * c.D * esz);
     l.attn_len = take((size_t)c.B * 4);
     l.ones = take((size_t)c.B * 4);
     l.o_rows = take((size_t)c.B * 4);
+    l.last_rows = take((size_t)c.B * 4);
     l.mask = take((size_t)c.B * c.max_nodes * W * 8);
     l.o = take((size_t)c.B * c.H * 4);
     l.h1 = take((size_t)c.B * c.H * 4);
-    l.m = take((size_t)c.B * c.H * esz);
     l.gu = take((size_t)c.B * 2 * I * 4);
-    l.act = take((size_t)c.B * I * esz);
-    l.mlp = take((size_t)c.B * c.H * 4);
     l.total = off;
     return l;
 }
 
 // y[M,N] = x[rows picked by x_rows][K] . W[N,K]^T as float32, through the weight-streaming kernel.
+// `act` is applied to the rows of x on the way in; add / y_t: see GemvParams::plain_add, plain_out_t.
 int plain_gemv(Handle* h, cudaStream_t s, int M, const void* x, int x_row_count, const int* x_rows, const void* W,
-               int K, int N, float* y) {
+               int K, int N, float* y, const ActOp& act, const float* add = nullptr, void* y_t = nullptr) {
     GemvParams g;
     memset(&g, 0, sizeof(g));
     g.x = x; g.x_rows = x_rows; g.x_row_count = x_row_count; g.W = W;
     g.H = K; g.slots = 1; g.rows_per_slot = N;
     g.mode = 2; g.k = 1;
     g.logits_dbg = y;
+    g.act = act; g.plain_add = add; g.plain_out_t = y_t;
     g.sn.max_nodes = 1; g.sn.rows_per_seq = 1; g.sn.inv_temp = 1.f;
     return launch_gemv_stream(h, s, h->cfg.dtype, M, g);
 }
@@ -245,12 +170,14 @@ template <typename T>
 int run_draft_module(Handle* h, cudaStream_t s, DmParams& p, const void* Wqkv, const void* Wo, const void* Wgu,
                      const void* Wdn) {
     const ctcsd_config& c = h->cfg;
-    CTCSD_CUDA_CHECK(h, launch_pdl(dm_norm_rows_kernel<T>, dim3(p.R, p.B), dim3(256), 0, s, 1, p));
-    CTCSD_LAUNCH_CHECK(h);
     const int Nqkv = (c.Hq + 2 * c.Hkv) * c.D;
-    int rc = plain_gemv(h, s, p.B * p.R, p.a, p.B * p.R, nullptr, Wqkv, c.H, Nqkv, p.qkv);
+    ActOp none = {};
+    // q, k, v of every new row: RMSNorm(F) * g1 on the way in (rows past n_new[b] count as zero)
+    ActOp norm1 = {};
+    norm1.op = 1; norm1.eps = p.eps; norm1.gain = p.g1; norm1.n_new = p.n_new; norm1.R = p.R;
+    int rc = plain_gemv(h, s, p.B * p.R, p.F_new, p.B * p.R, nullptr, Wqkv, c.H, Nqkv, p.qkv, norm1);
     if (rc != CTCSD_OK) return rc;
-    CTCSD_CUDA_CHECK(h, launch_pdl(dm_rope_scatter_kernel<T>, dim3(p.R, p.B), dim3(256), 0, s, 1, p));
+    CTCSD_CUDA_CHECK(h, launch_pdl(dm_rope_scatter_kernel<T>, dim3(p.R, p.B, 8), dim3(256), 0, s, 1, p));
     CTCSD_LAUNCH_CHECK(h);
     AttnParams ap;
     ap.Q = p.Qbuf; ap.K = p.Kd; ap.V = p.Vd; ap.O = p.Obuf;
@@ -260,21 +187,18 @@ int run_draft_module(Handle* h, cudaStream_t s, DmParams& p, const void* Wqkv, c
     ap.status = p.status;
     rc = tree_attention_dispatch(h, s, ap);
     if (rc != CTCSD_OK) return rc;
-    rc = plain_gemv(h, s, p.B, p.Obuf, p.B * c.max_nodes, p.o_rows, Wo, c.Hq * c.D, c.H, p.o);
+    rc = plain_gemv(h, s, p.B, p.Obuf, p.B * c.max_nodes, p.o_rows, Wo, c.Hq * c.D, c.H, p.o, none);
     if (rc != CTCSD_OK) return rc;
-    CTCSD_CUDA_CHECK(h, launch_pdl(dm_residual_norm_kernel<T>, dim3(p.B), dim3(256), 0, s, 1, p));
-    CTCSD_LAUNCH_CHECK(h);
-    rc = plain_gemv(h, s, p.B, p.m, p.B, nullptr, Wgu, c.H, 2 * p.I, p.gu);
+    // gate and up: h1 = F_last + o (kept for the last residual), RMSNorm(h1) * g2 on the way in
+    ActOp norm2 = {};
+    norm2.op = 2; norm2.eps = p.eps; norm2.gain = p.g2; norm2.add = p.o; norm2.sum_out = p.h1;
+    rc = plain_gemv(h, s, p.B, p.F_new, p.B * p.R, p.last_rows, Wgu, c.H, 2 * p.I, p.gu, norm2);
     if (rc != CTCSD_OK) return rc;
-    const int eb = (int)(((size_t)p.B * p.I + 255) / 256);
-    CTCSD_CUDA_CHECK(h, launch_pdl(dm_swiglu_kernel<T>, dim3(eb < 1184 ? eb : 1184), dim3(256), 0, s, 1, p));
-    CTCSD_LAUNCH_CHECK(h);
-    rc = plain_gemv(h, s, p.B, p.act, p.B, nullptr, Wdn, p.I, c.H, p.mlp);
-    if (rc != CTCSD_OK) return rc;
-    const int ob = (int)(((size_t)p.B * p.H + 255) / 256);
-    CTCSD_CUDA_CHECK(h, launch_pdl(dm_residual_out_kernel<T>, dim3(ob < 1184 ? ob : 1184), dim3(256), 0, s, 1, p));
-    CTCSD_LAUNCH_CHECK(h);
-    return CTCSD_OK;
+    // down: SiLU(gate) * up on the way in, F_hat = h1 + product on the way out
+    ActOp swiglu = {};
+    swiglu.op = 3; swiglu.gu = p.gu;
+    rc = plain_gemv(h, s, p.B, p.gu, p.B, nullptr, Wdn, p.I, c.H, p.out_F_dbg, swiglu, p.h1, p.out_F);
+    return rc;
 }
 
 }  // namespace
@@ -316,12 +240,14 @@ extern "C" int ctcsd_draft_module(ctcsd_handle* hh, void* stream, const ctcsd_dr
     p.g1 = layer->g1; p.g2 = layer->g2;
     p.B = c.B; p.R = R; p.H = c.H; p.Hq = c.Hq; p.Hkv = c.Hkv; p.D = c.D; p.I = I; p.Lcap = Lcap; p.max_nodes = c.max_nodes;
     p.eps = layer->eps; p.theta = layer->rope_theta;
-    p.a = ws + l.a; p.qkv = reinterpret_cast<float*>(ws + l.qkv);
+    for (int i = 0; i < c.D / 2; ++i) p.inv_freq[i] = exp2(-2.0 * (double)i / (double)c.D * log2((double)layer->rope_theta));
+    p.qkv = reinterpret_cast<float*>(ws + l.qkv);
     p.Qbuf = ws + l.Qbuf; p.Obuf = ws + l.Obuf;
     p.attn_len = reinterpret_cast<int*>(ws + l.attn_len); p.ones = reinterpret_cast<int*>(ws + l.ones);
-    p.o_rows = reinterpret_cast<int*>(ws + l.o_rows); p.mask = reinterpret_cast<unsigned long long*>(ws + l.mask);
-    p.o = reinterpret_cast<float*>(ws + l.o); p.h1 = reinterpret_cast<float*>(ws + l.h1); p.m = ws + l.m;
-    p.gu = reinterpret_cast<float*>(ws + l.gu); p.act = ws + l.act; p.mlp = reinterpret_cast<float*>(ws + l.mlp);
+    p.o_rows = reinterpret_cast<int*>(ws + l.o_rows); p.last_rows = reinterpret_cast<int*>(ws + l.last_rows);
+    p.mask = reinterpret_cast<unsigned long long*>(ws + l.mask);
+    p.o = reinterpret_cast<float*>(ws + l.o); p.h1 = reinterpret_cast<float*>(ws + l.h1);
+    p.gu = reinterpret_cast<float*>(ws + l.gu);
     p.out_F = out_F; p.out_F_dbg = out_F_dbg; p.out_kv_len = out_kv_len;
     p.status = status_ptr(h);
     cudaStream_t s = static_cast<cudaStream_t>(stream);

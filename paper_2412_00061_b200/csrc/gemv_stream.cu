@@ -64,6 +64,141 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+template <typename T> __device__ __forceinline__ void store_as(void* dst, size_t i, float v);
+template <> __device__ __forceinline__ void store_as<float>(void* dst, size_t i, float v) { static_cast<float*>(dst)[i] = v; }
+template <> __device__ __forceinline__ void store_as<__nv_bfloat16>(void* dst, size_t i, float v) {
+    static_cast<__nv_bfloat16*>(dst)[i] = __float2bfloat16_rn(v);
+}
+
+// One 16-byte chunk of activation-type values <-> float32.
+template <typename T> struct Chunk;
+template <> struct Chunk<float> {
+    static constexpr int kN = 4;
+    static __device__ __forceinline__ void unpack(const uint4& c, float* v) {
+        v[0] = __uint_as_float(c.x); v[1] = __uint_as_float(c.y); v[2] = __uint_as_float(c.z); v[3] = __uint_as_float(c.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float* v) {
+        return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+    }
+};
+template <> struct Chunk<__nv_bfloat16> {
+    static constexpr int kN = 8;
+    static __device__ __forceinline__ void unpack(const uint4& c, float* v) {
+        const unsigned w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { v[2 * q] = __uint_as_float(w[q] << 16); v[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u); }
+    }
+    static __device__ __forceinline__ uint4 pack(const float* v) {
+        unsigned w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const unsigned lo = __bfloat16_as_ushort(__float2bfloat16_rn(v[2 * q]));
+            const unsigned hi = __bfloat16_as_ushort(__float2bfloat16_rn(v[2 * q + 1]));
+            w[q] = lo | (hi << 16);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// The activation rows of this pass, transformed on the way into shared memory (ActOp).  Called by
+// every thread of the CTA; all of them share each row (with one row per pass, one warp per row
+// would leave the rest of the CTA waiting for it).
+template <typename T, int MROWS>
+__device__ void load_rows_transformed(const GemvParams& p, uint4* xs, int x_stride, int nch) {
+    constexpr int N = Chunk<T>::kN;
+    constexpr int kNW = kThreads / 32;
+    __shared__ float s_ss[MROWS][kNW];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const ActOp& a = p.act;
+    int src[MROWS];                                     // source row of x, -1: the row is all zero
+#pragma unroll
+    for (int m = 0; m < MROWS; ++m) {
+        const int row = p.m0 + m;
+        int sr = -1;
+        if (m < p.mcount) {
+            sr = row;
+            if (p.x_rows != nullptr) {
+                sr = p.x_rows[row];
+                if (sr < 0 || sr >= p.x_row_count) {
+                    if (tid == 0) report_error(p.status, CTCSD_ERR_INVALID_ARG, row);
+                    sr = -1;
+                }
+            }
+            if (a.op == 1 && a.n_new != nullptr && sr >= 0) {
+                int r = a.n_new[sr / a.R];
+                r = r < 0 ? 0 : (r > a.R ? a.R : r);
+                if (sr - (sr / a.R) * a.R >= r) sr = -1;                 // not a live row
+            }
+        }
+        src[m] = sr;
+    }
+    float v[N];
+    if (a.op == 3) {
+        for (int i = tid; i < MROWS * nch; i += kThreads) {
+            const int m = i / nch, ch = i - m * nch;
+            uint4 out = make_uint4(0, 0, 0, 0);
+            if (m < p.mcount) {
+                const float* g = a.gu + (size_t)(p.m0 + m) * 2 * p.H + (size_t)ch * N;
+                const float* u = g + p.H;
+#pragma unroll
+                for (int q = 0; q < N; ++q) v[q] = g[q] / (1.f + __expf(-g[q])) * u[q];
+                out = Chunk<T>::pack(v);
+            }
+            xs[(size_t)m * x_stride + ch] = out;
+        }
+        return;
+    }
+    float ss[MROWS];
+#pragma unroll
+    for (int m = 0; m < MROWS; ++m) {
+        ss[m] = 0.f;
+        if (src[m] < 0) continue;
+        const int row = p.m0 + m;
+        const uint4* xrow = reinterpret_cast<const uint4*>(p.x) + (size_t)src[m] * nch;
+        const float* add = (a.op == 2) ? a.add + (size_t)row * p.H : nullptr;
+        float* sum_out = (a.op == 2 && a.sum_out != nullptr && blockIdx.x == 0) ? a.sum_out + (size_t)row * p.H : nullptr;
+        for (int ch = tid; ch < nch; ch += kThreads) {
+            Chunk<T>::unpack(xrow[ch], v);
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                if (add) v[q] += add[ch * N + q];
+                if (sum_out) sum_out[ch * N + q] = v[q];
+                ss[m] += v[q] * v[q];
+            }
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < MROWS; ++m) {
+        const float w = warp_sum(ss[m]);
+        if (lane == 0) s_ss[m][warp] = w;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int m = 0; m < MROWS; ++m) {
+        uint4* dst = xs + (size_t)m * x_stride;
+        if (src[m] < 0) {
+            for (int ch = tid; ch < nch; ch += kThreads) dst[ch] = make_uint4(0, 0, 0, 0);
+            continue;
+        }
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < kNW; ++w) tot += s_ss[m][w];
+        const float inv = rsqrtf(tot / (float)p.H + a.eps);
+        const int row = p.m0 + m;
+        const uint4* xrow = reinterpret_cast<const uint4*>(p.x) + (size_t)src[m] * nch;
+        const float* add = (a.op == 2) ? a.add + (size_t)row * p.H : nullptr;
+        for (int ch = tid; ch < nch; ch += kThreads) {
+            Chunk<T>::unpack(xrow[ch], v);
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                if (add) v[q] += add[ch * N + q];
+                v[q] = v[q] * inv * a.gain[ch * N + q];
+            }
+            dst[ch] = Chunk<T>::pack(v);
+        }
+    }
+}
+
 // One CTA per SM.  Warp 8 is the producer: it walks the CTA's contiguous range of weight rows
 // and copies G rows (about 64 KB: the copy engine's cost per copy is high) per ring slot with
 // the bulk-copy engine, as far ahead as the ring allows.  Warps 0..7 consume the slots in
@@ -148,7 +283,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
     // below may come from the kernel that precedes this one in the stream
     pdl_wait();
     pdl_trigger();
-    for (int i = tid; i < MROWS * nch; i += kThreads) {
+    if (p.act.op != 0) load_rows_transformed<T, MROWS>(p, xs, x_stride, nch);
+    else for (int i = tid; i < MROWS * nch; i += kThreads) {
         int m = i / nch, ch = i - m * nch;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (m < p.mcount) {
@@ -246,8 +382,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                 const int slot = slot0 + seg;
                 const int v = (int)(r0 + i - (long long)slot * rps);
                 if (v == (int)rps - 1) z += bias;
-                if (p.logits_dbg) p.logits_dbg[((size_t)(p.m0 + own_m) * p.slots + slot) * rps + v] = z;
-                if (p.mode == 2) return;                       // plain product: the value written above is the output
+                const size_t at = ((size_t)(p.m0 + own_m) * p.slots + slot) * rps + v;
+                if (p.mode == 2) {                             // plain product (plus, if asked, a residual): it is the output
+                    if (p.plain_add) z += p.plain_add[at];
+                    if (p.logits_dbg) p.logits_dbg[at] = z;
+                    if (p.plain_out_t) store_as<T>(p.plain_out_t, at, z);
+                    return;
+                }
+                if (p.logits_dbg) p.logits_dbg[at] = z;
                 if (noise_row != nullptr) z = __fmaf_rn(z, p.sn.inv_temp, noise_row[v]);
                 st.push(z, v);
             };
@@ -285,9 +427,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                     // Four blocks are in flight at a time, each with its own accumulators, so that
                     // neither the loads nor the dependent tensor-core instructions serialise.
                     constexpr int kU = 4;
-                    float cc[kU][4];
+                    float cc[kU][4], ce[kU][4];                 // (the two halves of a block accumulate apart: shorter chains)
 #pragma unroll
-                    for (int u = 0; u < kU; ++u) { cc[u][0] = cc[u][1] = cc[u][2] = cc[u][3] = 0.f; }
+                    for (int u = 0; u < kU; ++u) {
+                        cc[u][0] = cc[u][1] = cc[u][2] = cc[u][3] = 0.f;
+                        ce[u][0] = ce[u][1] = ce[u][2] = ce[u][3] = 0.f;
+                    }
                     for (int kb0 = warp; kb0 * 4 < nch; kb0 += kWarps * kU) {      // the same trip count for all lanes
                         uint4 P[kU], Q[kU], X[kU];
 #pragma unroll
@@ -302,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
 #pragma unroll
                         for (int u = 0; u < kU; ++u) {
                             mma_16816(cc[u], P[u].x, Q[u].x, P[u].y, Q[u].y, X[u].x, X[u].y);
-                            mma_16816(cc[u], P[u].z, Q[u].z, P[u].w, Q[u].w, X[u].z, X[u].w);
+                            mma_16816(ce[u], P[u].z, Q[u].z, P[u].w, Q[u].w, X[u].z, X[u].w);
                         }
                     }
                     // the accumulators depend on every load of the slot: it can be refilled
@@ -310,6 +455,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
                     if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
                     // c0,c1: weight row g x activation rows 2t,2t+1;  c2,c3: weight row g+8
                     if (!tc::mbar_wait(&sh->cempty[d], dph ^ 1u, abort_flag)) { failed = true; break; }
+#pragma unroll
+                    for (int u = 0; u < kU; ++u) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) cc[u][q] += ce[u][q];
+                    }
                     float* cp = &s_cpart[d][warp][0][0];
                     *reinterpret_cast<float2*>(cp + g * 8 + 2 * t) =
                         make_float2((cc[0][0] + cc[1][0]) + (cc[2][0] + cc[3][0]), (cc[0][1] + cc[1][1]) + (cc[2][1] + cc[3][1]));
@@ -456,6 +606,9 @@ int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     int G = (int)((64 * 1024) / row_bytes);
     if (G < 1) G = 1;
     if (G > kWarps * kRowsPerWarp) G = kWarps * kRowsPerWarp;
+    // bfloat16: a tensor-core step costs the same for 1 to 16 weight rows, and a slot's steps are a
+    // chain whose length grows with the row: long rows get at least four rows per slot
+    if (sizeof(T) == 2 && G < 4) G = 4;
     while (G > 1 && fixed + 2 * (size_t)G * row_bytes > budget) --G;
     const size_t slot_bytes = (size_t)G * row_bytes;
     if (fixed + slot_bytes > budget) return CTCSD_ERR_UNSUPPORTED;

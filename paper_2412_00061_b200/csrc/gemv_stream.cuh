@@ -12,6 +12,19 @@
 
 namespace ctcsd {
 
+// What the kernel does to the activation rows while it loads them into shared memory (every CTA
+// repeats it on its own copy: a few rows, hidden behind the first weight copies already in flight).
+struct ActOp {
+    int op;               // 0: x as it is; 1: RMSNorm(x) * gain; 2: RMSNorm(x + add) * gain; 3: SiLU(gate) * up
+    float eps;            // ops 1, 2
+    const float* gain;    // ops 1, 2: [H]
+    const float* add;     // op 2: [M,H] float32, added to activation row m before the norm
+    float* sum_out;       // op 2: [M,H] float32 or null: x + add, written by the first CTA
+    const float* gu;      // op 3: [M,2H] float32, gate then up (x is not read)
+    const int* n_new;     // op 1: row m = b * R + j is all zero when j >= n_new[b] (null: every row is live)
+    int R;
+};
+
 struct GemvParams {
     const void* x;            // [x_row_count,H]
     const int* x_rows;        // [M] or null: activation row m is x[x_rows[m]] (null: x[m])
@@ -28,13 +41,16 @@ struct GemvParams {
     DraftPartial* part;       // [MROWS][grid][2]
     int* part_slot;           // [grid][2] slot id of each partial (-1 = unused)
     unsigned* counter;        // ticket counter, zero on entry, zero again on exit
-    int mode;                 // 0: top-k + lse outputs, 1: arg-max output, 2: the products themselves (to logits_dbg)
+    int mode;                 // 0: top-k + lse outputs, 1: arg-max output, 2: the products themselves (to logits_dbg and/or plain_out_t)
     int k;
     int* out_topk_id;         // mode 0: [M,slots,k]
     float* out_topk_lp;       // mode 0: [M,slots,k]
     float* out_lse;           // mode 0: [M,slots]
     int* out_argmax;          // mode 1: [M]
     float* logits_dbg;        // null or [M,slots,rows_per_slot]
+    ActOp act;                // applied to the activation rows as they are loaded
+    const float* plain_add;   // mode 2: null or [M,slots*rows_per_slot] float32 added to the products
+    void* plain_out_t;        // mode 2: null or [M,slots*rows_per_slot] in the activation type: the (summed) products
     int* status;              // device status word
     SampleNoise sn;           // mode 1: noise added to the scaled logit before the arg-max (null: none)
     const void* pf_ptr;       // optional: range the CTAs ask L2 to fetch once their own stream is issued

@@ -43,7 +43,7 @@ static int verify_accept_common(ctcsd_handle* hh, void* stream, const void* hn, 
         int rc = launch_lm_head_tc(h, s, M, hn, Wl, out_argmax, out_logits_dbg, a, sn);
         if (rc != CTCSD_ERR_UNSUPPORTED) return rc;
     }
-    GemvParams g;
+    GemvParams g = {};
     g.x = hn; g.x_rows = nullptr; g.x_row_count = M; g.W = Wl; g.row_seq = nullptr; g.blank_bias = nullptr;
     g.m0 = 0; g.mcount = 0; g.H = c.H; g.slots = 1; g.rows_per_slot = c.V; g.grid = 0;
     g.part = nullptr; g.part_slot = nullptr; g.counter = nullptr;
