@@ -162,7 +162,7 @@ int ctcsd_draft_logits_rows(ctcsd_handle* h, void* stream, int M, const void* x,
 
 /*
  * Slot paths -> collapsed, deduplicated, scored candidates -> the topN best (Sec. 3.3: the
- * slot tokens are combined and only the most valuable combinations go on; Sec. 2.3 /
+ * per-slot tokens are combined into sequences, of which the best-scoring are kept; Sec. 2.3 /
  * Sec. 3.1: beta^{-1} merges adjacent repeats, then removes blanks; Eq. 6: a path's
  * probability is the product over slots; Eq. 1 / Eq. 5: a candidate's probability is the sum
  * over the paths that collapse to it).
