@@ -526,6 +526,75 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
         np.testing.assert_array_equal(step.host(k), v)
 
 
+def _random_slot_lists(rng, M, T, k, V, pool):
+    """Per-slot lists as S3 would hand them over (k distinct ids, log-probabilities descending), drawn
+    from a small pool of tokens plus the blank so that blanks, repeats and merges are the rule."""
+    ids = np.zeros((M, T, k), dtype=np.int32)
+    lp = np.zeros((M, T, k), dtype=np.float32)
+    symbols = np.array(list(range(pool)) + [V])
+    for m in range(M):
+        for t in range(T):
+            pick = rng.choice(symbols, size=k, replace=False)
+            z = np.sort(rng.normal(0.0, 2.0, size=k))[::-1]
+            ids[m, t] = pick
+            lp[m, t] = (z - np.log(np.sum(np.exp(z))) - rng.uniform(0.0, 0.5)).astype(np.float32)
+    return ids, lp
+
+
+@pytest.mark.parametrize("mode", ["beam", "enumerate"])
+def test_random_slot_lists_through_collapse_and_tree(mode):
+    """S4-S8 on many small random shapes (slots, list length, beam, candidates kept, tree budget all
+    drawn at random; a token pool of k + 1 or k + 2 symbols, so nearly every path has blanks or
+    repeats and most candidates have several alignments), fed straight into the candidate call."""
+    import torch
+    from tests import parity_util
+    from paper_2412_00061_b200.step import DraftVerifyStep
+    rng = np.random.default_rng(20241200 + (mode == "beam"))
+    done = 0
+    for case in range(60):
+        T = int(rng.integers(1, 9))
+        k = int(rng.integers(1, 9))
+        if mode == "enumerate":
+            while k ** T > 4096:
+                k -= 1
+        beam = int(rng.choice([1, 2, 3, 5, 8, 16, 33, 64, 128])) if mode == "beam" else 0
+        N = int(rng.integers(1, 65))
+        B = int(rng.integers(1, 5))
+        M = B + int(rng.integers(0, 3))
+        n_max = int(rng.choice([8, 33, 64, 128, 200, 256]))
+        V = 40
+        cfg = C["c1"].replace(name="rnd", B=B, T=T, k=k, beam=beam, topN=N, max_nodes=n_max, V=V,
+                              score_mode=int(rng.integers(0, 2)) if mode == "enumerate" else 0)
+        ids, lp = _random_slot_lists(rng, M, T, k, V, pool=min(k + int(rng.integers(0, 2)), V))
+        sel = rng.permutation(M)[:B].astype(np.int32)
+        st = {}
+        parity_util.orc.topk_collapse(ids.astype(np.int64), lp.astype(np.float64), blank=V, T=T, N=N, beam=beam,
+                                      score_mode=cfg.score_mode, sel_row=sel, B=B, stats=st)
+        if beam > 0 and min(st["margin"]) <= parity_util.TAU:
+            continue                                    # the beam cut falls inside a tie: several answers are right
+        step = DraftVerifyStep(cfg, device="cuda:0", max_draft_rows=M)
+        dev = step.device
+        step.out["topk_id"].copy_(torch.from_numpy(ids).to(dev))
+        step.out["topk_lp"].copy_(torch.from_numpy(lp).to(dev))
+        base_tok, kv_len = parity_util.synth.gen_base(cfg, case)
+        step.set_inputs(sel_row=torch.from_numpy(sel).to(dev), base_tok=torch.from_numpy(base_tok.astype(np.int32)).to(dev),
+                        kv_len=torch.from_numpy(kv_len.astype(np.int32)).to(dev))
+        step.collapse()
+        step.tree()
+        step.check_status()
+        got = (step.host("cand_tok"), step.host("cand_len"), step.host("cand_score"), step.host("n_cand"))
+        parity_util.check_candidates(cfg, ids, lp, sel, got)
+        want = parity_util.orc.build_tree(base_tok, kv_len, got[0].astype(np.int64), got[1].astype(np.int64),
+                                          got[3].astype(np.int64), n_max)
+        for name, w in zip(["node_tok", "parent", "depth", "pos", "mask", "retrieve", "n_nodes"], want):
+            have = step.host(name)
+            if name == "mask":
+                have = have.view(np.uint64)
+            np.testing.assert_array_equal(have, w, err_msg="case %d %s" % (case, name))
+        done += 1
+    assert done >= 45
+
+
 @pytest.mark.parametrize("layout", ["packed", "raw"])
 def test_a_draft_row_out_of_range_leaves_the_root_alone(layout):
     """sel_row pointing outside the draft rows: the call that makes the candidates reports the
