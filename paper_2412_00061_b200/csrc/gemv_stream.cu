@@ -601,9 +601,12 @@ int launch_one(Handle* h, cudaStream_t stream, GemvParams& p) {
     size_t budget = (size_t)optin - fa.sharedSizeBytes - 2048;
     if (budget > 208 * 1024) budget = 208 * 1024;
     const size_t fixed = (size_t)MROWS * (row_bytes + 64) + sizeof(RingShared);
-    // rows per ring slot: copies of about 64 KB keep the copy engine busiest (its cost per copy is
-    // large), as long as at least two slots fit (two 64 KB slots stream as fast as three)
-    int G = (int)((64 * 1024) / row_bytes);
+    // rows per ring slot: copies of 64 KB and more keep the copy engine busiest (its cost per copy is
+    // large), as long as at least two slots fit.  bfloat16: the consumers are bound by the rate at
+    // which the tensor-core instructions issue, and a slot costs the same number of them for 1 to
+    // 16 rows, so slots of 80 KB (two of them) beat three of 64 KB: 10 / 9 / 8 rows of 8 KB per slot
+    // gave 193 / 197 / 200 us for the 7B draft head and 282 / 286 / 297 us for the step; 12 rows no more.
+    int G = (int)(((sizeof(T) == 2 ? 80 : 64) * 1024) / row_bytes);
     if (G < 1) G = 1;
     if (G > kWarps * kRowsPerWarp) G = kWarps * kRowsPerWarp;
     // bfloat16: a tensor-core step costs the same for 1 to 16 weight rows, and a slot's steps are a
