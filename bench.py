@@ -268,7 +268,7 @@ def roofline_times_us(cfg, mean_kv, n_live, hbm_gbs, tensor_tflops):
     """Per heavy call: the slower of (algorithmic bytes / measured copy bandwidth) and
     (flops / measured bf16 matmul rate); the step's roofline time is their sum."""
     draft_b, lm_b, kv_b = algorithmic_bytes(cfg, mean_kv, n_live)
-    M_lm = cfg.B * cfg.max_nodes
+    M_lm = cfg.B * n_live               # rows the LM head must serve: the live tree nodes
     fl = {"draft_logits": 2.0 * cfg.B * cfg.T * (cfg.V + 1) * cfg.H,
           "verify_accept": 2.0 * M_lm * cfg.V * cfg.H,
           "tree_attention": 4.0 * cfg.B * cfg.Hq * n_live * (mean_kv + n_live) * cfg.D}

@@ -223,12 +223,16 @@ int ctcsd_tree_attention(ctcsd_handle* h, void* stream, const void* Q, const voi
  *   Walk: cur = root; while some child c of cur has node_tok[c] == am[cur]: accept c.  Siblings
  *   carry distinct tokens in a tree from ctcsd_build_tree, so at most one child qualifies; in a
  *   hand-made tree with equal siblings the longest agreeing path is taken, lowest id on ties.
- * hn [B*max_nodes,H] dtype (row b*max_nodes+i is node i of sequence b; rows of unused nodes
- *   are computed but ignored);  Wl [V,H] dtype;  node_tok, parent [B,max_nodes], n_nodes [B].
- * out_argmax [B,max_nodes] int32;  out_acc_len [B] int32 (accepted draft tokens, root and
+ * hn [B*max_nodes,H] dtype (row b*max_nodes+i is node i of sequence b; rows of unused nodes,
+ *   i >= n_nodes[b], are never looked at: with bfloat16 and more than 128 tree rows the live
+ *   rows are first packed densely into the workspace, so unused rows cost no arithmetic);
+ *   Wl [V,H] dtype;  node_tok, parent [B,max_nodes], n_nodes [B].
+ * out_argmax [B,max_nodes] int32 (entries of unused nodes: not meaningful, -1 where the rows
+ *   were packed);  out_acc_len [B] int32 (accepted draft tokens, root and
  *   bonus token excluded);  out_acc_nodes, out_acc_tok [B,T] int32 (-1 padded);
  *   out_next_tok [B] int32 = am at the last accepted node (the bonus token);
- * out_logits_dbg  NULL or [B*max_nodes,V] float32 receiving every logit as computed.
+ * out_logits_dbg  NULL or [B*max_nodes,V] float32 receiving every logit as computed (rows of
+ *   unused nodes may be left untouched).
  */
 int ctcsd_verify_accept(ctcsd_handle* h, void* stream, const void* hn, const void* Wl,
                         const int* node_tok, const int* parent, const int* n_nodes,

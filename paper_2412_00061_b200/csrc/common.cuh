@@ -37,6 +37,8 @@ struct Layout {
     size_t seq_ticket_off;    // unsigned[B]: per-sequence "CTAs finished" tickets of the history update, zero between calls
     size_t tc_part_off;       // DraftPartial[T * tiles_per_slot][rows padded to 128]: tensor-core draft head (only if max_draft_rows > 8)
     size_t tc_part_bytes;
+    size_t lm_rows_off;       // act[lm_key_count][H]: the LM head's live activation rows packed densely (bf16, more than 128 tree rows)
+    size_t lm_rowmap_off;     // int[lm_key_count + 1]: packed row -> tree row; the last entry is the number of live rows
     size_t total;
     int gemv_grid_max;        // largest grid the GEMV may use
     int lm_key_count;

@@ -55,6 +55,11 @@ Layout make_layout(const ctcsd_config& c, int num_sms) {
             off = align_up(off + l.tc_part_bytes, 256);
         }
     }
+    l.lm_rows_off = l.lm_rowmap_off = off;
+    if (c.dtype == CTCSD_DTYPE_BF16 && c.B * c.max_nodes > 128) {
+        l.lm_rows_off = off;    off = align_up(off + (size_t)l.lm_key_count * c.H * 2, 256);
+        l.lm_rowmap_off = off;  off = align_up(off + sizeof(int) * ((size_t)l.lm_key_count + 1), 256);
+    }
     l.total = off;
     return l;
 }

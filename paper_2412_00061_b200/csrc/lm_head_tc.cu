@@ -66,6 +66,12 @@ struct TcParams {
     const int* row_seq;       // [M] or null
     const float* blank_bias;  // [B] or null; added to class V-1 of every slot
     SampleNoise sn;           // LM head: noise added to the scaled logit before the arg-max (null: none)
+    // LM head on more than one row tile: the rows of unused tree nodes are left out.  The
+    // activation rows arrive packed (live rows only, sequence by sequence); row_map[r] is the tree
+    // row of packed row r and row_map[row_map_len] the number of live rows, both written by the
+    // kernel that precedes this one in the stream.  Null: every row is live and in place.
+    const int* row_map;
+    int row_map_len;
 };
 
 struct __align__(8) TcShared {
@@ -116,24 +122,25 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
-    const long long units = (long long)p.n_tiles * p.m_units;
+    int M = p.M, m_tiles = p.m_tiles, m_units = p.m_units;
+    long long units = (long long)p.n_tiles * m_units;
     // CTA c takes units c, c + grid, c + 2 grid, ...: at any moment the CTAs then work on
     // neighbouring units, i.e. on the few row tiles of the same few weight tiles, so a weight tile
     // that several row tiles need is fetched from HBM once and found in L2 by the others.
     const int u_first = (int)blockIdx.x, u_step = (int)gridDim.x;
-    const int n_units = units > u_first ? (int)((units - u_first + u_step - 1) / u_step) : 0;
+    int n_units = units > u_first ? (int)((units - u_first + u_step - 1) / u_step) : 0;
 
     // producer state (lane 0 of warp 0 only).  Stage `it` holds K blocks [ks * atoms, (ks+1) * atoms),
     // ks = it % num_ks, of unit u_first + (it / num_ks) * u_step; every CTA walks the K axis from its
     // own starting stage (and wraps), so that at any moment the CTAs ask L2 for different parts of
     // the shared activations.
-    const int total_it = n_units * p.num_ks;
+    int total_it = n_units * p.num_ks;
     const int k_start = (int)(((long long)blockIdx.x * p.num_ks) / gridDim.x);
     const uint64_t pol_w = tc::policy_evict_first();
     const uint64_t pol_a = tc::policy_evict_last();
     auto load_stage = [&](int it, bool do_w, bool do_a) {
         const int u = u_first + (it / p.num_ks) * u_step, kb = it - (it / p.num_ks) * p.num_ks;
-        const int nt = u / p.m_units, mu = u - nt * p.m_units;
+        const int nt = u / m_units, mu = u - nt * m_units;
         const int s = it % p.stages;
         unsigned char* a_dst = dyn + (size_t)s * stage_bytes;
         int kq = kb + k_start;
@@ -165,12 +172,25 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (warp == 0 && lane == 0) {
         tc::prefetch_tensormap(&tmA);
         tc::prefetch_tensormap(&tmW);
-        pre = total_it < p.stages ? total_it : p.stages;
-        for (int it = 0; it < pre; ++it) load_stage(it, true, false);
+        // (with packed rows the units are known only once the live-row count can be read)
+        if (p.row_map == nullptr) {
+            pre = total_it < p.stages ? total_it : p.stages;
+            for (int it = 0; it < pre; ++it) load_stage(it, true, false);
+        }
     }
     // barriers and tensor memory are set up; the activations may come from the preceding kernel
     pdl_wait();
     pdl_trigger();
+    if (p.row_map != nullptr) {
+        // only the row tiles that hold live rows are units of work
+        M = p.row_map[p.row_map_len];
+        M = M < 0 ? 0 : (M > p.M ? p.M : M);
+        m_tiles = (M + kTileM - 1) / kTileM;
+        m_units = p.pair ? (m_tiles + 1) / 2 : m_tiles;
+        units = (long long)p.n_tiles * m_units;
+        n_units = units > u_first ? (int)((units - u_first + u_step - 1) / u_step) : 0;
+        total_it = n_units * p.num_ks;
+    }
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -212,6 +232,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             bool ok = true;
             for (int u = u_first; ucount < n_units && ok; u += u_step, ++ucount) {
                 const int acc = p.pair ? 0 : (ucount & 1);            // barrier pair that guards this unit
+                const bool second = p.pair && 2 * (u % m_units) + 1 < m_tiles;   // the pair's second row tile exists
                 const uint32_t acc_ph = (uint32_t)(p.pair ? ucount : (ucount >> 1)) & 1u;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
                 if (!tc::mbar_wait(&sh->tmem_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -235,7 +256,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                             // advancing 16 bf16 along K = 32 bytes = 2 descriptor address units
                             tc::mma_bf16_ss(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | j | k) != 0 ? 1u : 0u);
                         }
-                        if (p.pair) {                        // the second row tile against the same weights
+                        if (second) {                        // the second row tile against the same weights
                             const uint64_t adesc1 = tc::smem_desc_k_sw128(a_addr + (uint32_t)(j * a_blk + p.a_bytes));
 #pragma unroll
                             for (int k = 0; k < kBlockK / 16; ++k)
@@ -261,7 +282,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int ucount = 0;
         bool ok = true;
         for (int u = u_first; ucount < n_units && ok; u += u_step, ++ucount) {
-            const int nt = u / p.m_units, mu = u - nt * p.m_units;
+            const int nt = u / m_units, mu = u - nt * m_units;
             // draft mode: tile nt is tile ntl of slot t
             const int t = MODE == 1 ? nt / p.tiles_per_slot : 0;
             const int n0 = (MODE == 1 ? nt - t * p.tiles_per_slot : nt) * p.Nt;
@@ -272,21 +293,23 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             for (int h = 0; h <= p.pair; ++h) {               // pair mode: accumulator h holds row tile 2*mu + h
             const int mt = p.pair ? 2 * mu + h : mu;
             const int row = mt * kTileM + row_in_tile;
+            // the tree row this (packed) row stands for: debug logits and noise are addressed by it
+            const int orow = (MODE == 0 && p.row_map != nullptr && row < M) ? p.row_map[row] : row;
             float bias = 0.f;
             if (MODE == 1 && p.blank_bias != nullptr && row < p.M) bias = p.blank_bias[p.row_seq ? p.row_seq[row] : row];
             const uint32_t lane_addr = lane_base + (uint32_t)((p.pair ? h : acc) * kAccCols);
             float best = -INFINITY;
             int best_idx = 0x7fffffff;
             const float* noise_row = nullptr;                 // sampling acceptance: the row's Gumbel noise
-            if (MODE == 0 && p.sn.noise != nullptr && row < p.M) {
-                int d = p.sn.depth[row];
+            if (MODE == 0 && p.sn.noise != nullptr && row < M) {
+                int d = p.sn.depth[orow];
                 d = d < 0 ? 0 : (d >= p.sn.rows_per_seq ? p.sn.rows_per_seq - 1 : d);
-                noise_row = p.sn.noise + ((size_t)(row / p.sn.max_nodes) * p.sn.rows_per_seq + d) * (size_t)p.V;
+                noise_row = p.sn.noise + ((size_t)(orow / p.sn.max_nodes) * p.sn.rows_per_seq + d) * (size_t)p.V;
             }
             RunState st;
             if constexpr (MODE == 1) st.init();
             // a warp whose 32 rows lie past the last activation row has nothing to read
-            const int c_end = (mt * kTileM + q * 32 < p.M) ? p.Nt : 0;
+            const int c_end = (mt * kTileM + q * 32 < M) ? p.Nt : 0;
             for (int c0 = cs * 32; c0 < c_end; c0 += 32 * kColSplit) {
                 uint32_t r[32];
                 if (c0 + 32 <= p.Nt) {
@@ -304,7 +327,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const int col = n0 + c0 + j;
                     if (col < p.V && c0 + j < p.Nt) {
                         if constexpr (MODE == 0) {
-                            if (p.logits_dbg != nullptr && row < p.M) p.logits_dbg[(size_t)row * p.V + col] = v;
+                            if (p.logits_dbg != nullptr && row < M) p.logits_dbg[(size_t)orow * p.V + col] = v;
                             if (noise_row != nullptr) v = __fmaf_rn(v, p.sn.inv_temp, __ldg(noise_row + col));
                             if (v > best) { best = v; best_idx = col; }
                         } else {
@@ -327,7 +350,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             } else {
             // fold this tile's winner into the row's global maximum: larger logit first, equal
             // logits -> lower id (the id is stored complemented in the low word)
-            if (row < p.M && best_idx != 0x7fffffff) {
+            if (row < M && best_idx != 0x7fffffff) {
                 const unsigned u = __float_as_uint(best);
                 const unsigned sortable = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
                 atomicMax(p.keys + row, ((unsigned long long)sortable << 32) | (0xffffffffu - (unsigned)best_idx));
@@ -358,9 +381,10 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (!sh->is_last) return;
     __threadfence();
     const bool good = sh->abort_flag == 0;
-    for (int row = tid; row < p.M; row += kThreads) {
+    for (int row = tid; row < M; row += kThreads) {
         const unsigned long long key = __ldcg(p.keys + row);
-        if (good) p.out_argmax[row] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
+        const int orow = p.row_map != nullptr ? p.row_map[row] : row;
+        if (good) p.out_argmax[orow] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
         p.keys[row] = 0ull;
     }
     __syncthreads();
@@ -374,6 +398,40 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 accept_warp(p.acc, b, lane, reinterpret_cast<int*>(dyn) + warp * kAcceptScratchInts);
     }
     if (tid == 0) *p.counter = 0u;
+}
+
+// Packs the activation rows of the live tree nodes densely, sequence by sequence, for the LM head on
+// more than one row tile: the rows of unused nodes (a tree rarely fills its budget) then cost
+// neither tensor-core work nor an epilogue.  One CTA per tree row (node i of sequence b).  Writes
+// row_map (packed row -> tree row), the live-row count behind it, and -1 as the arg-max of every
+// unused node.
+__global__ void __launch_bounds__(128) lm_pack_rows_kernel(const uint4* hn, const int* n_nodes, int B, int max_nodes,
+                                                           int chunks, uint4* packed, int* row_map, int row_map_len,
+                                                           int* out_argmax) {
+    __shared__ int s_part[4];
+    const int i = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    pdl_wait();                      // the node counts and the activations come from preceding kernels
+    pdl_trigger();
+    auto count = [&](int q) { const int n = n_nodes[q]; return n < 0 ? 0 : (n > max_nodes ? max_nodes : n); };
+    int before = 0;                                   // live rows of the sequences before this one
+    for (int q = tid; q < b; q += 128) before += count(q);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+    if ((tid & 31) == 0) s_part[tid >> 5] = before;
+    __syncthreads();
+    const int off = s_part[0] + s_part[1] + s_part[2] + s_part[3];
+    const int n = count(b);
+    const int orow = b * max_nodes + i;
+    if (b == B - 1 && i == 0 && tid == 0) row_map[row_map_len] = off + n;
+    if (i >= n) {
+        if (tid == 0) out_argmax[orow] = -1;
+        return;
+    }
+    const int prow = off + i;
+    if (tid == 0) row_map[prow] = orow;
+    const uint4* src = hn + (size_t)orow * chunks;
+    uint4* dst = packed + (size_t)prow * chunks;
+    for (int c = tid; c < chunks; c += 128) dst[c] = src[c];
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -637,13 +695,28 @@ int launch_lm_head_tc(Handle* h, cudaStream_t stream, int M, const void* hn, con
     p.logits_dbg = out_logits_dbg;
     p.status = status_ptr(h);
 
+    // More than one row tile: the live rows are packed first (the rows of unused nodes are skipped).
+    const void* a_rows = hn;
+    long long a_row_count = M;
+    if (p.m_tiles >= 2 && h->lay.lm_rowmap_off != h->lay.lm_rows_off && acc.n_nodes != nullptr) {
+        uint4* packed = reinterpret_cast<uint4*>(h->ws + h->lay.lm_rows_off);
+        int* row_map = reinterpret_cast<int*>(h->ws + h->lay.lm_rowmap_off);
+        CTCSD_CUDA_CHECK(h, launch_pdl(lm_pack_rows_kernel, dim3(c.max_nodes, c.B), dim3(128), 0, stream, 1,
+                                       static_cast<const uint4*>(hn), acc.n_nodes, c.B, c.max_nodes, c.H / 8, packed,
+                                       row_map, h->lay.lm_key_count, out_argmax));
+        CTCSD_LAUNCH_CHECK(h);
+        p.row_map = row_map;
+        p.row_map_len = h->lay.lm_key_count;
+        a_rows = packed;
+        a_row_count = h->lay.lm_key_count;
+    }
     CUtensorMap tmA, tmW;
     const int a_box_rows = p.a_bytes / 128 * (1 + p.pair);
     if (p.atoms == 1) {
-        if (!make_map(&tmA, hn, M, c.H, a_box_rows)) return CTCSD_ERR_CUDA;
+        if (!make_map(&tmA, a_rows, a_row_count, c.H, a_box_rows)) return CTCSD_ERR_CUDA;
         if (!make_map(&tmW, Wl, c.V, c.H, p.Nt)) return CTCSD_ERR_CUDA;
     } else {
-        if (!make_map_kblocks(&tmA, hn, M, c.H, a_box_rows, p.atoms)) return CTCSD_ERR_CUDA;
+        if (!make_map_kblocks(&tmA, a_rows, a_row_count, c.H, a_box_rows, p.atoms)) return CTCSD_ERR_CUDA;
         if (!make_map_kblocks(&tmW, Wl, c.V, c.H, p.Nt, p.atoms)) return CTCSD_ERR_CUDA;
     }
 

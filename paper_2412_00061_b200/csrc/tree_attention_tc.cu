@@ -150,7 +150,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     const int nblk = (Ltot + kKeys - 1) / kKeys;
     const int blk0 = (int)((long long)nblk * split / splits);           // key tiles spread evenly over the splits
     const int blk1 = (int)((long long)nblk * (split + 1) / splits);
-    const int ntile = blk1 - blk0;
+    // a query tile whose rows all belong to unused nodes has nothing to attend to: its rows come out zero
+    const int ntile = (qtile * (kRows / grp) >= n) ? 0 : blk1 - blk0;
 
     // softmax state of the row owned by this thread (softmax warps only)
     float acc[DO];

@@ -177,7 +177,7 @@ def run_parity(cfg, seed=0, M=None, force_repeats=False, row_seq=None, sel_row=N
     y_def, am_def = orc.lm_head_argmax(hn[rows], inp["Wl"])
     assert np.max(np.abs(y_gpu[rows] - y_def)) <= logit_tol
     am_gpu = step.host("argmax")
-    np.testing.assert_array_equal(am_gpu.reshape(-1), orc.argmax_rows(y_gpu))           # stage-fed, all rows
+    np.testing.assert_array_equal(am_gpu.reshape(-1)[live], orc.argmax_rows(y_gpu[live]))   # stage-fed, every live row
     np.testing.assert_array_equal(am_gpu.reshape(-1)[rows], am_def)                      # definition mode
     np.testing.assert_array_equal(am_gpu.reshape(-1)[live], target.reshape(-1)[live])    # the planted targets
     acc = orc.greedy_accept(node_tok, parent, n_nodes, am_gpu.astype(np.int64), cfg.T)
@@ -279,7 +279,7 @@ def run_parity_raw(cfg, seed=0, force_repeats=False, device="cuda:0", attention_
     y_def, am_def = orc.lm_head_argmax(hn[rows], inp["Wl"])
     assert np.max(np.abs(y_gpu[rows] - y_def)) <= logit_tol
     am_gpu = step.host("argmax")
-    np.testing.assert_array_equal(am_gpu.reshape(-1), orc.argmax_rows(y_gpu))
+    np.testing.assert_array_equal(am_gpu.reshape(-1)[live], orc.argmax_rows(y_gpu[live]))
     np.testing.assert_array_equal(am_gpu.reshape(-1)[live], target.reshape(-1)[live])
     acc = orc.raw_accept(node_tok, kept, nka, n_nodes, am_gpu.astype(np.int64), cfg.T)
     for name, want in zip(["acc_len", "acc_nodes", "acc_tok", "next_tok"], acc):
@@ -445,8 +445,13 @@ def run_chain_parity(cfg, seed=0, n_steps=4, layout="packed", device="cuda:0", g
         certified = all(min(r["margin"]) > 1e-5 for r in recs_o)
         if certified:
             for s, r in enumerate(recs_o):
-                for name in ("cand_tok", "node_tok", "parent", "n_nodes", "argmax", "acc_len", "acc_nodes", "acc_tok", "next_tok"):
+                for name in ("cand_tok", "node_tok", "parent", "n_nodes", "acc_len", "acc_nodes", "acc_tok", "next_tok"):
                     np.testing.assert_array_equal(rec[name][s], r[name], err_msg="definition mode, %s at step %d" % (name, s))
+                # (the arg-max of an unused node's row is not part of the result)
+                alive = np.arange(r["argmax"].reshape(len(r["n_nodes"]), -1).shape[1])[None, :] < np.asarray(r["n_nodes"])[:, None]
+                np.testing.assert_array_equal(np.asarray(rec["argmax"][s]).reshape(alive.shape)[alive],
+                                              np.asarray(r["argmax"]).reshape(alive.shape)[alive],
+                                              err_msg="definition mode, argmax at step %d" % s)
             np.testing.assert_array_equal(kv_len, kv_o)
             assert np.array_equal(Kc, K_o) and np.array_equal(Vc, V_o)
     return dict(tokens=tokens, certified=certified, step=step)
