@@ -529,11 +529,13 @@ struct DraftMergeParams {
     int* out_topk_id; float* out_topk_lp; float* out_lse;
 };
 
-// One CTA of four warps per (activation row, slot): every thread folds its share of the slot's
-// per-tile states, the warps combine theirs, and the first warp combines the four results into
-// the log-sum-exp and the top-k of the row.
-__global__ void __launch_bounds__(128) draft_tc_merge_kernel(DraftMergeParams p) {
-    __shared__ DraftPartial s_warp[4];
+// One CTA of sixteen warps per (activation row, slot): every thread folds its share of the slot's
+// per-tile states (about one each at a 32000-word vocabulary: folding a state is a chain of list
+// insertions), the warps combine theirs, and the first warp combines the sixteen results into the
+// log-sum-exp and the top-k of the row.
+constexpr int kMergeThreads = 512;
+__global__ void __launch_bounds__(kMergeThreads) draft_tc_merge_kernel(DraftMergeParams p) {
+    __shared__ DraftPartial s_warp[kMergeThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long pair = blockIdx.x;
     pdl_wait();
@@ -542,14 +544,14 @@ __global__ void __launch_bounds__(128) draft_tc_merge_kernel(DraftMergeParams p)
     RunState fs;
     fs.init();
     const int entries = p.tiles_per_slot * kColSplit;          // per tile: one state per column share
-    for (int e = threadIdx.x; e < entries; e += 128)
+    for (int e = threadIdx.x; e < entries; e += kMergeThreads)
         fs.absorb(load_partial_cg(p.part + ((size_t)t * entries + e) * p.mpad + m));
     warp_combine(fs);
     if (lane == 0) fs.store(&s_warp[warp]);
     __syncthreads();
     if (warp != 0) return;
     fs.init();
-    if (lane < 4) fs.absorb(s_warp[lane]);
+    if (lane < kMergeThreads / 32) fs.absorb(s_warp[lane]);
     warp_combine(fs);
     if (lane == 0) {
         const float lse = fs.mx + logf(fs.sum);
@@ -638,7 +640,7 @@ int launch_draft_head_tc(Handle* h, cudaStream_t stream, int M, const void* x, c
     mp.M = M; mp.mpad = p.m_tiles * kTileM; mp.slots = p.slots; mp.tiles_per_slot = p.tiles_per_slot; mp.k = c.k;
     mp.out_topk_id = out_topk_id; mp.out_topk_lp = out_topk_lp; mp.out_lse = out_lse;
     const long long pairs = (long long)M * p.slots;           // one CTA each
-    CTCSD_CUDA_CHECK(h, launch_pdl(draft_tc_merge_kernel, dim3((unsigned)pairs), dim3(128), 0, stream, 1, mp));
+    CTCSD_CUDA_CHECK(h, launch_pdl(draft_tc_merge_kernel, dim3((unsigned)pairs), dim3(kMergeThreads), 0, stream, 1, mp));
     CTCSD_LAUNCH_CHECK(h);
     return CTCSD_OK;
 }
