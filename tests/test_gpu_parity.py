@@ -541,6 +541,42 @@ def _random_slot_lists(rng, M, T, k, V, pool):
     return ids, lp
 
 
+@pytest.mark.parametrize("pattern", [(1, 64, 17, 64, 1), (1, 1, 1, 1, 1), (64, 64, 64, 64, 64), (3, 2, 64, 1, 40)])
+def test_lm_head_serves_live_rows_only(pattern):
+    """More than 128 tree rows: the LM head packs the rows of used nodes and computes nothing else.  After
+    a checked step the node counts are cut to a pattern (a prefix of a tree is a tree), the rows of
+    nodes that are now unused are filled with large values that would win any arg-max, and the call
+    is repeated: arg-max of every live row and the acceptance against the oracle, -1 for unused rows."""
+    import torch
+    from oracle import ctcsd_oracle as orc
+    from paper_2412_00061_b200.step import to_device
+    cfg = SMALL["c5s"]
+    r = _run(cfg, seed=9)
+    step = r["step"]
+    dev = step.device
+    n0 = step.host("n_nodes").astype(np.int64)
+    n_new = np.minimum(n0, np.array(pattern, dtype=np.int64))
+    node_tok, parent = step.host("node_tok").astype(np.int64), step.host("parent").astype(np.int64)
+    hn = step.inp["hn"].float().cpu().numpy().copy()
+    Wl = step.inp["Wl"].float().cpu().numpy()
+    for b in range(cfg.B):
+        hn[b * cfg.max_nodes + int(n_new[b]):(b + 1) * cfg.max_nodes] = 50.0      # must never be looked at
+    step.set_inputs(hn=to_device(hn, cfg.dtype, dev))
+    step.out["n_nodes"].copy_(torch.from_numpy(n_new.astype(np.int32)).to(dev))
+    step.out["argmax"].fill_(-7)
+    step.verify()
+    step.check_status()
+    am = step.host("argmax").astype(np.int64)
+    live = [b * cfg.max_nodes + i for b in range(cfg.B) for i in range(int(n_new[b]))]
+    dead = sorted(set(range(cfg.B * cfg.max_nodes)) - set(live))
+    _, am_def = orc.lm_head_argmax(hn[live].astype(np.float64), Wl.astype(np.float64))
+    np.testing.assert_array_equal(am.reshape(-1)[live], am_def)
+    assert np.all(am.reshape(-1)[dead] == -1)
+    acc = orc.greedy_accept(node_tok, parent, n_new, am, cfg.T)
+    for name, want in zip(["acc_len", "acc_nodes", "acc_tok", "next_tok"], acc):
+        np.testing.assert_array_equal(step.host(name), want, err_msg=name)
+
+
 @pytest.mark.parametrize("mode", ["beam", "enumerate"])
 def test_random_slot_lists_through_collapse_and_tree(mode):
     """S4-S8 on many small random shapes (slots, list length, beam, candidates kept, tree budget all
