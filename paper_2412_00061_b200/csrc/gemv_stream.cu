@@ -227,14 +227,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
     unsigned char* ring = smem_raw + (size_t)MROWS * x_stride * 16;  // [nslots][G][row_bytes]
     RingShared* sh = reinterpret_cast<RingShared*>(ring + (size_t)nslots * slot_bytes);
     __shared__ DraftPartial s_part[2][kStateRows][MROWS];
-    __shared__ float s_cpart[kCDepth][kWarps][16][8];                // per-warp partial sums of a fill (bf16 path)
+    // per-warp partial sums of a fill (bf16 path).  With eight activation rows their copies in shared
+    // memory leave the weight ring the less room: two buffers instead of four buy an eighth row per slot.
+    constexpr int kCD = MROWS == 8 ? 2 : kCDepth;
+    __shared__ float s_cpart[kCD][kWarps][16][8];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     volatile int* abort_flag = &sh->abort_flag;
 
     if (tid == 0) {
         for (int s = 0; s < nslots; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], kWarps); }
-        for (int d = 0; d < kCDepth; ++d) { tc::mbar_init(&sh->cfull[d], kWarps); tc::mbar_init(&sh->cempty[d], kEpiWarps); }
+        for (int d = 0; d < kCD; ++d) { tc::mbar_init(&sh->cfull[d], kWarps); tc::mbar_init(&sh->cempty[d], kEpiWarps); }
         sh->abort_flag = 0;
         sh->never_set = 0;
         sh->is_last = 0;
@@ -397,8 +400,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(GemvParams p, 
             bool failed = false;
             for (int j = 0; j < nfill; ++j) {
                 const int rows = (ntotal - j * G < G) ? ntotal - j * G : G;
-                const int d = j % kCDepth;
-                const uint32_t dph = (uint32_t)(j / kCDepth) & 1u;
+                const int d = j % kCD;
+                const uint32_t dph = (uint32_t)(j / kCD) & 1u;
                 if (kMma && is_epi) {
                     // ---- epilogue: add the eight partial sums, fold the logit into the state ----
                     if (!tc::mbar_wait(&sh->cfull[d], dph, abort_flag)) { failed = true; break; }
