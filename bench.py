@@ -409,7 +409,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     K, Wm = args.steps, max(3, args.warmup)
-    sampler = ClockSampler(local) if rank == 0 else None
+    sampler = ClockSampler(local, args.clock_period_ms) if rank == 0 else None
     for _ in range(Wm):
         step.run()
     step.check_status()
@@ -628,6 +628,7 @@ def main():
     ap.add_argument("--layout", default="packed", choices=["packed", "raw"],
                     help="packed: collapse, then tree (headline); raw: the paper's raw-path tree with masked removed symbols")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--clock-period-ms", type=int, default=10, help="period of the nvidia-smi clock sampler")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every call directly instead of replaying a CUDA graph")
     ap.add_argument("--force-repeats", action="store_true",
                     help="draft weights that make neighbouring slots favour the same tokens, so that repeats and merges occur")
